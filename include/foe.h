@@ -1,0 +1,173 @@
+/*
+ * foe.h -- C ABI of the B200 (sm_100a) forward pass of one Federation-of-Experts (FoE)
+ * transformer block.
+ *
+ * The operation is the per-layer compute of the paper's Table 2 (right column) with the
+ * layer-boundary rules and the group-limited routing rule of Section 3.1:
+ *
+ *     r[h,i]    = x[h,i] + Attn_h(x[h,:])[i]                      attention residual, per cluster h
+ *     r_full[i] = (1/H) sum_h r[h,i]                              cross-cluster sync
+ *     I_h[i], w_h[i] = TopK_{e in E_h}(Router(r_full[i]), k/H)    per-cluster routing
+ *     x'[h,i]   = r_full[i] + sum_{e in I_h[i]} w_h[i,e] FFN_e(r_full[i])
+ *
+ * On one GPU the sync is a local reduction and dispatch/combine are local permutations.
+ *
+ * Conventions
+ *  - Every pointer in foe_weights, foe_kv_cache and the x/out/h/topk arguments is a DEVICE
+ *    pointer unless marked "host".  Structs themselves live in host memory.
+ *  - bf16 tensors are row-major with the last index contiguous.  Tokens of a call are the
+ *    sequences' new tokens concatenated in sequence order (S = sum of q_lens).
+ *  - Cluster h owns query heads h*g..(h+1)*g-1 (g = n_q_heads / n_clusters), KV heads
+ *    h*c..(h+1)*c-1 (c = n_kv_heads / n_clusters), rows h*g*head_dim.. of W_O and experts
+ *    h*E_c..(h+1)*E_c-1.
+ *  - All tensor memory belongs to the caller.  foe_layer_create copies and repacks the weights
+ *    into library-owned device buffers, so the caller may release its copies afterwards.  The
+ *    handle owns a workspace sized by max_tokens / max_seqs / max_context.
+ *  - Calls are asynchronous on the given stream (a cudaStream_t passed as void*).  A handle is
+ *    used from one stream at a time.  Same inputs give bit-identical outputs and maps.
+ *  - Every function returns a foe_status; argument and shape checks happen on the host before
+ *    anything is launched.  Conditions only the device can see (a bounded wait that ran out, an
+ *    out-of-range page id) are recorded in a device status word read by foe_poll_status.
+ *  - There is no CPU fallback: without a CUDA device every compute entry point fails.
+ */
+#ifndef FOE_H_
+#define FOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FOE_OK = 0,
+  FOE_ERR_NULL = -1,         /* a required pointer is NULL */
+  FOE_ERR_CONFIG = -2,       /* foe_config violates a validity rule */
+  FOE_ERR_SHAPE = -3,        /* call sizes exceed what the handle was created for */
+  FOE_ERR_UNSUPPORTED = -4,
+  FOE_ERR_OOM = -5,          /* device allocation failed */
+  FOE_ERR_CUDA = -6,         /* a CUDA runtime/driver call failed */
+  FOE_ERR_TIMEOUT = -7,      /* device status: a bounded wait inside a kernel ran out */
+  FOE_ERR_BOUNDS = -8        /* device status: an index read from device memory was out of range */
+} foe_status;
+
+typedef enum { FOE_MIDDLE = 0, FOE_FIRST = 1, FOE_LAST = 2, FOE_SINGLE = 3 } foe_position;
+typedef enum { FOE_SYNC_MEAN = 0, FOE_SYNC_SUM = 1 } foe_sync;
+
+/* Layer description.  Validity: n_kv_heads % n_clusters == 0, n_q_heads % n_kv_heads == 0,
+ * head_dim in {64, 128}, 1 <= top_k_per_cluster <= experts_per_cluster <= 128, top_k_per_cluster <= 32,
+ * page_size == 64, hidden % 64 == 0, ffn_inter % 128 == 0, max_* > 0.
+ * position: FOE_FIRST/FOE_SINGLE take x as [S, hidden] (one shared attention, its residual used
+ * in place of r_full); FOE_LAST/FOE_SINGLE write out as [S, hidden] (mean over clusters of x').
+ * Otherwise x and out are [n_clusters, S, hidden]. */
+typedef struct {
+  int hidden, n_q_heads, n_kv_heads, n_clusters, head_dim;
+  int experts_per_cluster, top_k_per_cluster, ffn_inter;
+  int page_size;
+  int max_tokens;      /* largest S of a prefill call */
+  int max_seqs;        /* largest n_seqs of any call (= largest S of a decode call) */
+  int max_context;     /* largest context_len + q_len any sequence reaches */
+  float rope_theta, rms_eps;
+  int position;        /* foe_position */
+  int sync;            /* foe_sync */
+} foe_config;
+
+/* Caller's weights (device pointers; bf16 unless stated). */
+typedef struct {
+  const void* attn_norm_g;   /* [hidden] gain of the RMSNorm before attention (shared by clusters) */
+  const void* wq;            /* [H][hidden][g*head_dim] */
+  const void* wk;            /* [H][hidden][c*head_dim] */
+  const void* wv;            /* [H][hidden][c*head_dim] */
+  const void* wo;            /* [n_q_heads*head_dim][hidden] */
+  const void* ffn_norm_g;    /* [hidden] gain of the RMSNorm before router and experts */
+  const void* w_gate;        /* [E][hidden][ffn_inter] */
+  const void* w_up;          /* [E][hidden][ffn_inter] */
+  const void* w_down;        /* [E][ffn_inter][hidden] */
+  const float* router_w;     /* [E][hidden] fp32; rows h*E_c.. are cluster h's router */
+  const float* router_b;     /* [E] fp32 additive score bias, or NULL */
+} foe_weights;
+
+/* Paged KV cache of one layer.  K is stored after RoPE.  The call writes K/V of the new tokens at
+ * logical positions context_lens[s] .. context_lens[s]+q_len-1 through block_table (pages must be
+ * assigned already) and attends over context_lens[s]+q_len entries.  It never changes context_lens. */
+typedef struct {
+  void* k_pages;              /* [num_pages][n_kv_heads][page_size][head_dim] bf16 */
+  void* v_pages;
+  const int* block_table;     /* [n_seqs][max_pages_per_seq] physical page ids */
+  const int* context_lens;    /* [n_seqs] tokens cached before this call */
+  const int* q_lens;          /* [n_seqs] new tokens in this call; NULL means 1 each (decode) */
+  int n_seqs, max_pages_per_seq, num_pages;
+  int n_tokens;               /* host copy of sum(q_lens) (ignored by foe_decode) */
+  int max_q_len;              /* host upper bound of q_lens (ignored by foe_decode) */
+} foe_kv_cache;
+
+/* Device pointers to the intermediates of the last call on a handle (valid until the next call). */
+typedef struct {
+  int n_tokens;
+  const float* r_full;      /* [S][hidden] fp32 synced residual */
+  const void* u;            /* [S][hidden] bf16 FFN-normed r_full (expert input) */
+  const float* logits;      /* [S][E] fp32 router scores */
+  const int* topk_idx;      /* [S][H][k_c] global expert ids */
+  const float* topk_w;      /* [S][H][k_c] gates */
+  const int* counts;        /* [E] rows per expert */
+  const int* offsets;       /* [E+1] exclusive scan of counts */
+  const int* perm;          /* [S*H*k_c] slot -> token */
+  const int* inv;           /* [S][H][k_c] -> slot */
+  const void* qkv;          /* [S][(n_q+2*n_kv)*head_dim] bf16: q (after RoPE) | k | v (before RoPE) */
+  const void* attn_o;       /* [S][n_q*head_dim] bf16 attention output before W_O */
+} foe_aux;
+
+typedef struct foe_layer foe_layer;
+
+/* Table 2 + Section 3.1: build a layer from its description and weights (host structs, device weight
+ * pointers).  Allocates the repacked weights and the workspace; runs a few repack kernels on the
+ * default stream and synchronises.  *out receives the handle. */
+foe_status foe_layer_create(const foe_config* config, const foe_weights* weights, foe_layer** out);
+
+/* Frees everything the handle owns.  NULL is accepted. */
+foe_status foe_layer_destroy(foe_layer* layer);
+
+/* Table 2 (all four rows) for S = kv->n_tokens new tokens of kv->n_seqs sequences: attention over the
+ * paged cache plus the new tokens (causal), sync, routing, experts, combine.  x: [H][S][hidden] bf16
+ * ([S][hidden] on a first layer); out likewise ([S][hidden] on a last layer); out must not alias x.
+ * Errors: FOE_ERR_NULL, FOE_ERR_SHAPE (S > max_tokens, n_seqs > max_seqs, S == 0 is FOE_OK, no work). */
+foe_status foe_prefill(foe_layer* layer, const void* x, const foe_kv_cache* kv, void* out, void* stream);
+
+/* Same computation for one new token per sequence (S = kv->n_seqs, q_lens ignored), built for the
+ * bandwidth-bound regime: split-KV paged attention and weight-streaming expert kernels.
+ * x_step: [H][n_seqs][hidden] bf16 ([n_seqs][hidden] on a first layer). */
+foe_status foe_decode(foe_layer* layer, const void* x_step, const foe_kv_cache* kv, void* out, void* stream);
+
+/* Section 3.1 "Routing": FFN RMSNorm, fp32 router scores, per-cluster top-k (larger score first, equal
+ * scores -> lower expert id) and gates (softmax over the selected scores) for n_tokens rows of
+ * h = r_full given as [n_tokens][hidden] bf16.  topk_idx: [n_tokens][H][k_c] int32 global expert ids;
+ * topk_w: [n_tokens][H][k_c] fp32.  Also refreshes counts/offsets/perm/inv in the aux record. */
+foe_status foe_route(foe_layer* layer, const void* h, int n_tokens, int* topk_idx, float* topk_w, void* stream);
+
+/* Pointers to the last call's intermediates (host struct filled with device pointers). */
+foe_status foe_get_aux(foe_layer* layer, foe_aux* out);
+
+/* Synchronises the handle's last stream and reads the device status word into *device_status
+ * (FOE_OK, FOE_ERR_TIMEOUT or FOE_ERR_BOUNDS); the word is reset to FOE_OK afterwards. */
+foe_status foe_poll_status(foe_layer* layer, int* device_status);
+
+/* Number of kernel launches the last prefill/decode/route call on this handle issued. */
+int foe_last_launch_count(const foe_layer* layer);
+
+/* Per-stage device timing of prefill/decode calls.  When enabled, every call records CUDA events on its
+ * stream between the stages of the block; foe_get_stage_ms waits for the last call and writes the
+ * foe_num_stages() elapsed times (milliseconds) into ms[0..n), n >= foe_num_stages().  foe_stage_name(i)
+ * names stage i.  FOE_ERR_UNSUPPORTED if the last call was not recorded. */
+foe_status foe_set_profiling(foe_layer* layer, int enabled);
+int foe_num_stages(void);
+const char* foe_stage_name(int i);
+foe_status foe_get_stage_ms(foe_layer* layer, float* ms, int n);
+
+/* Static description of a status code. */
+const char* foe_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FOE_H_ */

@@ -1,0 +1,450 @@
+// Attention core of the FoE block ("Attn_h" of Table 2): causal softmax(q k^T / sqrt(d_h)) v per sequence,
+// every query head reading the KV head of its cluster from the paged cache (the paper's KV cache is split
+// across the expert groups; on one GPU that is the head index of the page layout).
+//
+// Both kernels stage K and V through shared memory with TMA: one cache page of one KV head
+// ([64 tokens][d_h] bf16, contiguous) is one or two 64 x 64 boxes written with the 128-byte swizzle, which
+// is exactly the bank-conflict-free layout ldmatrix wants.  Scores and the PV product run on mma.sync
+// (m16n8k16, fp32 accumulate) with an online softmax in the exp2 domain.
+//
+//  * prefill: one CTA per (128 query rows, query head, sequence); 8 warps x 16 rows; key tiles = pages.
+//  * decode : one CTA per (sequence, KV head, split of the context); the g query heads of the KV head are
+//             the MMA rows; each of 4 warps takes 16 keys of every page; partial (m, l, o) per split are
+//             merged by a second kernel.  The KV cache is read exactly once.
+#include <math.h>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace foe {
+
+// byte offset of element (r, c) inside a [rows][DH] bf16 tile stored as 64-column halves, each half
+// rows x 128 bytes with the 16-byte chunk index XOR-ed by (r & 7)  (= TMA SWIZZLE_128B).
+template <int ROWS>
+__device__ __forceinline__ uint32_t tile_off(int r, int c) {
+  return uint32_t((c >> 6) * (ROWS * 128) + r * 128 + ((((c & 63) >> 3) ^ (r & 7)) << 4) + (c & 7) * 2);
+}
+
+template <int DH>
+__device__ __forceinline__ void tma_load_page(uint8_t* k_dst, uint8_t* v_dst, const CUtensorMap* tmK,
+                                              const CUtensorMap* tmV, uint64_t* bar, int row0) {
+  mbar_expect_tx(bar, 2 * 64 * DH * 2);
+#pragma unroll
+  for (int h = 0; h < DH / 64; ++h) {
+    tma_load_2d(k_dst + h * 64 * 128, tmK, bar, h * 64, row0);
+    tma_load_2d(v_dst + h * 64 * 128, tmV, bar, h * 64, row0);
+  }
+}
+
+// ======================================================================================= prefill
+constexpr int kPfRows = 128;
+constexpr int kPfThreads = 256;
+constexpr int kPfStages = 2;
+
+template <int DH>
+__global__ void __launch_bounds__(kPfThreads, 2)
+attn_prefill_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr int kQBytes = kPfRows * DH * 2;
+  constexpr int kTileBytes = 64 * DH * 2;
+  uint8_t* q_s = smem;
+  uint8_t* kv_s = smem + kQBytes;                      // [stage][K | V]
+  uint64_t* full = reinterpret_cast<uint64_t*>(kv_s + kPfStages * 2 * kTileBytes);
+
+  const int b = blockIdx.z, head = blockIdx.y;
+  const int qb = gridDim.x - 1 - blockIdx.x;           // heavy (late) query blocks first
+  const int q_len = a.q_lens ? a.q_lens[b] : 1;
+  const int q0 = qb * kPfRows;
+  if (q0 >= q_len) return;
+  const int ctx = a.context_lens[b];
+  const int tok0 = a.cu_q[b] + q0;
+  const int kvh = head / (a.n_q / a.n_kv);
+  const int rows_here = min(kPfRows, q_len - q0);
+  const int kv_len = ctx + q0 + rows_here;             // keys any row of this block can see
+  const int n_tiles = (kv_len + 63) >> 6;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ld_qkv = (a.n_q + 2 * a.n_kv) * DH;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kPfStages; ++s) mbar_init(&full[s], 1);
+    mbar_fence_init();
+  }
+  // Q tile (zero rows past the sequence end)
+  for (int q = threadIdx.x; q < kPfRows * (DH / 8); q += kPfThreads) {
+    const int r = q / (DH / 8), ch = q - r * (DH / 8);
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (r < rows_here) v = __ldg(reinterpret_cast<const uint4*>(a.qkv + size_t(tok0 + r) * ld_qkv + head * DH + ch * 8));
+    *reinterpret_cast<uint4*>(q_s + tile_off<kPfRows>(r, ch * 8)) = v;
+  }
+  __syncthreads();
+
+  auto page_row0 = [&](int tile) -> int {
+    int page = a.block_table[size_t(b) * a.max_pages_per_seq + min(tile, a.max_pages_per_seq - 1)];
+    if (page < 0 || page >= a.num_pages) { atomicExch(a.status, kStatusBounds); page = 0; }
+    return (page * a.n_kv + kvh) * 64;
+  };
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kPfStages && s < n_tiles; ++s)
+      tma_load_page<DH>(kv_s + s * 2 * kTileBytes, kv_s + s * 2 * kTileBytes + kTileBytes, &tmK, &tmV, &full[s],
+                        page_row0(s));
+  }
+
+  float o[DH / 8][4];
+#pragma unroll
+  for (int n = 0; n < DH / 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+  const int g = lane >> 2, t4 = lane & 3;
+  const int qpos0 = ctx + q0 + warp * 16 + g;          // position of row g; row g+8 is +8
+  const uint32_t q_base = smem_u32(q_s);
+  bool ok = true;
+
+  for (int j = 0; j < n_tiles; ++j) {
+    const int st = j % kPfStages;
+    if (!mbar_wait(&full[st], (j / kPfStages) & 1)) { ok = false; break; }
+    const uint32_t k_base = smem_u32(kv_s + st * 2 * kTileBytes);
+    const uint32_t v_base = k_base + kTileBytes;
+    // warps whose 16 rows all sit before this key tile have nothing to do in it
+    if (j * 64 <= ctx + q0 + warp * 16 + 15) {
+      float s[8][4];
+#pragma unroll
+      for (int n = 0; n < 8; ++n) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f; }
+#pragma unroll
+      for (int ks = 0; ks < DH / 16; ++ks) {
+        uint32_t qa[4];
+        ldmatrix_x4(qa, q_base + tile_off<kPfRows>(warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, ks * 16 + (lane >> 4) * 8));
+#pragma unroll
+        for (int np = 0; np < 4; ++np) {
+          uint32_t kb[4];
+          ldmatrix_x4(kb, k_base + tile_off<64>(np * 16 + (lane & 7) + (lane >> 4) * 8, ks * 16 + ((lane >> 3) & 1) * 8));
+          mma_bf16_16816(s[2 * np], qa, kb[0], kb[1]);
+          mma_bf16_16816(s[2 * np + 1], qa, kb[2], kb[3]);
+        }
+      }
+      // scale, causal mask (only tiles that reach past the first row of the warp), online softmax
+      const bool need_mask = j * 64 + 63 > ctx + q0 + warp * 16;
+      float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+      for (int n = 0; n < 8; ++n) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float v = s[n][e] * a.scale_log2;
+          if (need_mask) {
+            const int kpos = j * 64 + n * 8 + t4 * 2 + (e & 1);
+            const int qpos = qpos0 + (e >> 1) * 8;
+            if (kpos > qpos) v = -INFINITY;
+          }
+          s[n][e] = v;
+          mx[e >> 1] = fmaxf(mx[e >> 1], v);
+        }
+      }
+      float alpha[2], m_use[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+        mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+        const float m_new = fmaxf(m_run[r], mx[r]);
+        m_use[r] = (m_new == -INFINITY) ? 0.f : m_new;
+        alpha[r] = fast_exp2(m_run[r] - m_use[r]);
+        m_run[r] = m_new;
+      }
+      float rs[2] = {0.f, 0.f};
+#pragma unroll
+      for (int n = 0; n < 8; ++n) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float p = fast_exp2(s[n][e] - m_use[e >> 1]);
+          s[n][e] = p;
+          rs[e >> 1] += p;
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        rs[r] += __shfl_xor_sync(0xffffffffu, rs[r], 1);
+        rs[r] += __shfl_xor_sync(0xffffffffu, rs[r], 2);
+        l_run[r] = l_run[r] * alpha[r] + rs[r];
+      }
+#pragma unroll
+      for (int n = 0; n < DH / 8; ++n) {
+        o[n][0] *= alpha[0]; o[n][1] *= alpha[0]; o[n][2] *= alpha[1]; o[n][3] *= alpha[1];
+      }
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        uint32_t pa[4];
+        pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
+        pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
+        pa[2] = pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+        pa[3] = pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+#pragma unroll
+        for (int dp = 0; dp < DH / 16; ++dp) {
+          uint32_t vb[4];
+          ldmatrix_x4_trans(vb, v_base + tile_off<64>(kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, dp * 16 + (lane >> 4) * 8));
+          mma_bf16_16816(o[2 * dp], pa, vb[0], vb[1]);
+          mma_bf16_16816(o[2 * dp + 1], pa, vb[2], vb[3]);
+        }
+      }
+    }
+    __syncthreads();                                   // every warp is done with stage st
+    if (threadIdx.x == 0 && j + kPfStages < n_tiles)
+      tma_load_page<DH>(kv_s + st * 2 * kTileBytes, kv_s + st * 2 * kTileBytes + kTileBytes, &tmK, &tmV, &full[st],
+                        page_row0(j + kPfStages));
+  }
+  if (!ok) {
+    if (lane == 0) atomicExch(a.status, kStatusTimeout);
+    return;
+  }
+
+  // normalise, stage the warp's 16 rows through its own slice of the Q tile, store 16 bytes per lane
+  const float inv_l[2] = {1.f / l_run[0], 1.f / l_run[1]};
+  __syncwarp();
+#pragma unroll
+  for (int n = 0; n < DH / 8; ++n) {
+    *reinterpret_cast<uint32_t*>(q_s + tile_off<kPfRows>(warp * 16 + g, n * 8 + t4 * 2)) =
+        pack_bf16(o[n][0] * inv_l[0], o[n][1] * inv_l[0]);
+    *reinterpret_cast<uint32_t*>(q_s + tile_off<kPfRows>(warp * 16 + g + 8, n * 8 + t4 * 2)) =
+        pack_bf16(o[n][2] * inv_l[1], o[n][3] * inv_l[1]);
+  }
+  __syncwarp();
+  for (int q = lane; q < 16 * (DH / 8); q += 32) {
+    const int r = warp * 16 + q / (DH / 8), ch = q % (DH / 8);
+    if (r < rows_here)
+      *reinterpret_cast<uint4*>(a.out + size_t(tok0 + r) * (a.n_q * DH) + head * DH + ch * 8) =
+          *reinterpret_cast<const uint4*>(q_s + tile_off<kPfRows>(r, ch * 8));
+  }
+}
+
+template <int DH>
+static void launch_prefill_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st) {
+  constexpr size_t smem = kPfRows * DH * 2 + kPfStages * 2 * 64 * DH * 2 + 1024 + 64;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(attn_prefill_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    configured = true;
+  }
+  dim3 grid((a.max_q_len + kPfRows - 1) / kPfRows, a.n_q, a.n_seqs);
+  attn_prefill_kernel<DH><<<grid, kPfThreads, smem, st>>>(tmK, tmV, a);
+}
+
+void launch_attn_prefill(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st) {
+  if (a.n_seqs <= 0 || a.max_q_len <= 0) return;
+  if (a.dh == 128) launch_prefill_t<128>(tmK, tmV, a, st);
+  else launch_prefill_t<64>(tmK, tmV, a, st);
+}
+
+// ======================================================================================= decode
+constexpr int kDcThreads = 128;
+constexpr int kDcStages = 3;
+
+template <int DH>
+__global__ void __launch_bounds__(kDcThreads, 2)
+attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr int kTileBytes = 64 * DH * 2;
+  constexpr int kQBytes = 16 * DH * 2;
+  uint8_t* kv_s = smem;                                            // [stage][K | V]; reused for the merge
+  uint8_t* q_s = smem + kDcStages * 2 * kTileBytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(q_s + kQBytes);
+
+  const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+  const int ctx = a.context_lens[b];
+  const int kv_len = ctx + 1;                                      // cached tokens + the new one
+  const int n_pages = (kv_len + 63) >> 6;
+  const int p_begin = split * a.pages_per_split;
+  if (p_begin >= n_pages) return;
+  const int p_end = min(n_pages, p_begin + a.pages_per_split);
+  const int n_tiles = p_end - p_begin;
+  const int G = a.n_q / a.n_kv;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tok = a.cu_q[b];
+  const int ld_qkv = (a.n_q + 2 * a.n_kv) * DH;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kDcStages; ++s) mbar_init(&full[s], 1);
+    mbar_fence_init();
+  }
+  for (int q = threadIdx.x; q < 16 * (DH / 8); q += kDcThreads) {
+    const int r = q / (DH / 8), ch = q - r * (DH / 8);
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (r < G) v = __ldg(reinterpret_cast<const uint4*>(a.qkv + size_t(tok) * ld_qkv + (kvh * G + r) * DH + ch * 8));
+    *reinterpret_cast<uint4*>(q_s + tile_off<16>(r, ch * 8)) = v;
+  }
+  __syncthreads();
+
+  auto page_row0 = [&](int lp) -> int {
+    int page = a.block_table[size_t(b) * a.max_pages_per_seq + min(lp, a.max_pages_per_seq - 1)];
+    if (page < 0 || page >= a.num_pages) { atomicExch(a.status, kStatusBounds); page = 0; }
+    return (page * a.n_kv + kvh) * 64;
+  };
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kDcStages && s < n_tiles; ++s)
+      tma_load_page<DH>(kv_s + s * 2 * kTileBytes, kv_s + s * 2 * kTileBytes + kTileBytes, &tmK, &tmV, &full[s],
+                        page_row0(p_begin + s));
+  }
+
+  float o[DH / 8][4];
+#pragma unroll
+  for (int n = 0; n < DH / 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+  const int g = lane >> 2, t4 = lane & 3;
+  const uint32_t q_base = smem_u32(q_s);
+  bool ok = true;
+
+  for (int j = 0; j < n_tiles; ++j) {
+    const int st = j % kDcStages;
+    if (!mbar_wait(&full[st], (j / kDcStages) & 1)) { ok = false; break; }
+    const uint32_t k_base = smem_u32(kv_s + st * 2 * kTileBytes);
+    const uint32_t v_base = k_base + kTileBytes;
+    const int key0 = (p_begin + j) * 64 + warp * 16;               // this warp's 16 keys of the page
+    if (key0 < kv_len) {
+      float s[2][4];
+      s[0][0] = s[0][1] = s[0][2] = s[0][3] = s[1][0] = s[1][1] = s[1][2] = s[1][3] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < DH / 16; ++ks) {
+        uint32_t qa[4], kb[4];
+        ldmatrix_x4(qa, q_base + tile_off<16>((lane & 7) + ((lane >> 3) & 1) * 8, ks * 16 + (lane >> 4) * 8));
+        ldmatrix_x4(kb, k_base + tile_off<64>(warp * 16 + (lane & 7) + (lane >> 4) * 8, ks * 16 + ((lane >> 3) & 1) * 8));
+        mma_bf16_16816(s[0], qa, kb[0], kb[1]);
+        mma_bf16_16816(s[1], qa, kb[2], kb[3]);
+      }
+      float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+      for (int n = 0; n < 2; ++n)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float v = s[n][e] * a.scale_log2;
+          if (key0 + n * 8 + t4 * 2 + (e & 1) >= kv_len) v = -INFINITY;
+          s[n][e] = v;
+          mx[e >> 1] = fmaxf(mx[e >> 1], v);
+        }
+      float alpha[2], m_use[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+        mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+        const float m_new = fmaxf(m_run[r], mx[r]);
+        m_use[r] = (m_new == -INFINITY) ? 0.f : m_new;
+        alpha[r] = fast_exp2(m_run[r] - m_use[r]);
+        m_run[r] = m_new;
+      }
+      float rs[2] = {0.f, 0.f};
+#pragma unroll
+      for (int n = 0; n < 2; ++n)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float p = fast_exp2(s[n][e] - m_use[e >> 1]);
+          s[n][e] = p;
+          rs[e >> 1] += p;
+        }
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        rs[r] += __shfl_xor_sync(0xffffffffu, rs[r], 1);
+        rs[r] += __shfl_xor_sync(0xffffffffu, rs[r], 2);
+        l_run[r] = l_run[r] * alpha[r] + rs[r];
+      }
+      uint32_t pa[4];
+      pa[0] = pack_bf16(s[0][0], s[0][1]);
+      pa[1] = pack_bf16(s[0][2], s[0][3]);
+      pa[2] = pack_bf16(s[1][0], s[1][1]);
+      pa[3] = pack_bf16(s[1][2], s[1][3]);
+#pragma unroll
+      for (int dp = 0; dp < DH / 16; ++dp) {
+        uint32_t vb[4];
+        ldmatrix_x4_trans(vb, v_base + tile_off<64>(warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, dp * 16 + (lane >> 4) * 8));
+        o[2 * dp][0] *= alpha[0]; o[2 * dp][1] *= alpha[0]; o[2 * dp][2] *= alpha[1]; o[2 * dp][3] *= alpha[1];
+        o[2 * dp + 1][0] *= alpha[0]; o[2 * dp + 1][1] *= alpha[0]; o[2 * dp + 1][2] *= alpha[1]; o[2 * dp + 1][3] *= alpha[1];
+        mma_bf16_16816(o[2 * dp], pa, vb[0], vb[1]);
+        mma_bf16_16816(o[2 * dp + 1], pa, vb[2], vb[3]);
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && j + kDcStages < n_tiles)
+      tma_load_page<DH>(kv_s + st * 2 * kTileBytes, kv_s + st * 2 * kTileBytes + kTileBytes, &tmK, &tmV, &full[st],
+                        page_row0(p_begin + j + kDcStages));
+  }
+  if (!ok) {
+    if (lane == 0) atomicExch(a.status, kStatusTimeout);
+    return;
+  }
+
+  // merge the four warps' partial states (each saw a different quarter of every page)
+  float* mo = reinterpret_cast<float*>(kv_s);                      // [4][16][DH]
+  float* mm = mo + 4 * 16 * DH;                                    // [4][16] running max
+  float* ml = mm + 64;                                             // [4][16] running sum
+#pragma unroll
+  for (int n = 0; n < DH / 8; ++n) {
+    *reinterpret_cast<float2*>(mo + (warp * 16 + g) * DH + n * 8 + t4 * 2) = make_float2(o[n][0], o[n][1]);
+    *reinterpret_cast<float2*>(mo + (warp * 16 + g + 8) * DH + n * 8 + t4 * 2) = make_float2(o[n][2], o[n][3]);
+  }
+  if (t4 == 0) {
+    mm[warp * 16 + g] = m_run[0]; mm[warp * 16 + g + 8] = m_run[1];
+    ml[warp * 16 + g] = l_run[0]; ml[warp * 16 + g + 8] = l_run[1];
+  }
+  __syncthreads();
+  for (int q = threadIdx.x; q < G * DH; q += kDcThreads) {
+    const int r = q / DH, c = q - r * DH;
+    float m = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) m = fmaxf(m, mm[w * 16 + r]);
+    float acc = 0.f, l = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float f = fast_exp2(mm[w * 16 + r] - m);                   // 0 for a warp that saw no valid key
+      acc += f * mo[(w * 16 + r) * DH + c];
+      l += f * ml[w * 16 + r];
+    }
+    const size_t pidx = (size_t(b) * a.n_q + kvh * G + r) * a.max_splits + split;
+    a.part_o[pidx * DH + c] = acc;
+    if (c == 0) { a.part_ml[pidx * 2] = m; a.part_ml[pidx * 2 + 1] = l; }
+  }
+}
+
+// one warp per (sequence, query head): combine the splits that exist for that sequence
+template <int DH>
+__global__ void attn_decode_merge_kernel(const AttnArgs a) {
+  const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (wid >= a.n_seqs * a.n_q) return;
+  const int b = wid / a.n_q, head = wid - b * a.n_q;
+  const int n_pages = (a.context_lens[b] + 1 + 63) >> 6;
+  const int n_splits = min(a.max_splits, (n_pages + a.pages_per_split - 1) / a.pages_per_split);
+  const size_t base = (size_t(b) * a.n_q + head) * a.max_splits;
+  float m = -INFINITY;
+  for (int s = 0; s < n_splits; ++s) m = fmaxf(m, a.part_ml[(base + s) * 2]);
+  float acc[DH / 32];
+#pragma unroll
+  for (int q = 0; q < DH / 32; ++q) acc[q] = 0.f;
+  float l = 0.f;
+  for (int s = 0; s < n_splits; ++s) {
+    const float f = fast_exp2(a.part_ml[(base + s) * 2] - m);
+    l += f * a.part_ml[(base + s) * 2 + 1];
+#pragma unroll
+    for (int q = 0; q < DH / 32; ++q) acc[q] += f * a.part_o[(base + s) * DH + q * 32 + lane];
+  }
+  const float inv = 1.f / l;
+  bf16* dst = a.out + size_t(a.cu_q[b]) * (a.n_q * DH) + head * DH;
+#pragma unroll
+  for (int q = 0; q < DH / 32; ++q) dst[q * 32 + lane] = __float2bfloat16_rn(acc[q] * inv);
+}
+
+template <int DH>
+static void launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st) {
+  constexpr size_t smem = kDcStages * 2 * 64 * DH * 2 + 16 * DH * 2 + 1024 + 64;
+  static_assert(kDcStages * 2 * 64 * DH * 2 >= (4 * 16 * DH + 128) * 4, "merge buffer must fit in the stages");
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(attn_decode_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    configured = true;
+  }
+  dim3 grid(a.max_splits, a.n_kv, a.n_seqs);
+  attn_decode_kernel<DH><<<grid, kDcThreads, smem, st>>>(tmK, tmV, a);
+  const int warps = a.n_seqs * a.n_q;
+  attn_decode_merge_kernel<DH><<<(warps * 32 + 127) / 128, 128, 0, st>>>(a);
+}
+
+void launch_attn_decode(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st) {
+  if (a.n_seqs <= 0) return;
+  if (a.dh == 128) launch_decode_t<128>(tmK, tmV, a, st);
+  else launch_decode_t<64>(tmK, tmV, a, st);
+}
+
+}  // namespace foe

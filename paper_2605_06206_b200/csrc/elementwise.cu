@@ -1,0 +1,255 @@
+// Streaming (HBM-bound) steps of the FoE block and the create-time weight repacks.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace foe {
+
+// ------------------------------------------------------------------ RMS statistics (pre-attention norm)
+// One warp per row: inv_rms = rsqrt(mean(x^2) + eps).  The gain is folded into the projection weights
+// and the scale is applied in the GEMM epilogue, so the normalised tensor is never written.
+__global__ void row_inv_rms_kernel(const bf16* __restrict__ x, float* __restrict__ inv_rms, int n_rows, int d,
+                                   float eps) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (warp >= n_rows) return;
+  const uint4* row = reinterpret_cast<const uint4*>(x + size_t(warp) * d);
+  float ss = 0.f;
+  for (int c = lane; c < d / 8; c += 32) {
+    const uint4 q = __ldg(row + c);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float a = bf16_lo(w[j]), b = bf16_hi(w[j]);
+      ss += a * a + b * b;
+    }
+  }
+  ss = warp_sum(ss);
+  if (lane == 0) inv_rms[warp] = rsqrtf(ss / float(d) + eps);
+}
+
+void launch_row_inv_rms(const bf16* x, float* inv_rms, int n_rows, int d, float eps, cudaStream_t st) {
+  if (n_rows <= 0) return;
+  const int threads = 256;
+  const int blocks = (n_rows * 32 + threads - 1) / threads;
+  row_inv_rms_kernel<<<blocks, threads, 0, st>>>(x, inv_rms, n_rows, d, eps);
+}
+
+// ------------------------------------------------------------------ token -> (sequence, position, cache slot)
+__global__ void cu_q_kernel(const int* __restrict__ q_lens, int n_seqs, int* __restrict__ cu_q) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    int acc = 0;
+    cu_q[0] = 0;
+    for (int b = 0; b < n_seqs; ++b) { acc += q_lens ? q_lens[b] : 1; cu_q[b + 1] = acc; }
+  }
+}
+
+__global__ void token_map_kernel(const int* __restrict__ cu_q, int has_q_lens, const int* __restrict__ context_lens,
+                                 const int* __restrict__ block_table, int n_seqs, int max_pages_per_seq,
+                                 int num_pages, int page_size, int n_tokens, int max_context,
+                                 int* __restrict__ tok_seq, int* __restrict__ tok_pos, int* __restrict__ tok_slot,
+                                 int* __restrict__ status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_tokens) return;
+  int b;
+  if (!has_q_lens) b = i;
+  else {
+    int lo = 0, hi = n_seqs;                 // largest b with cu_q[b] <= i
+    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (cu_q[mid] <= i) lo = mid; else hi = mid; }
+    b = lo;
+  }
+  const int local = has_q_lens ? i - cu_q[b] : 0;
+  const int pos = context_lens[b] + local;
+  const int lp = pos / page_size;
+  int slot = -1;
+  if (lp < max_pages_per_seq && pos < max_context) {
+    const int page = block_table[size_t(b) * max_pages_per_seq + lp];
+    if (page >= 0 && page < num_pages) slot = page * page_size + (pos - lp * page_size);
+  }
+  if (slot < 0) atomicExch(status, kStatusBounds);
+  tok_seq[i] = b;
+  tok_pos[i] = pos;
+  tok_slot[i] = slot;
+}
+
+void launch_token_map(const int* q_lens, const int* context_lens, const int* block_table, int n_seqs,
+                      int max_pages_per_seq, int num_pages, int page_size, int n_tokens, int max_context, int* cu_q,
+                      int* tok_seq, int* tok_pos, int* tok_slot, int* status, cudaStream_t st) {
+  cu_q_kernel<<<1, 32, 0, st>>>(q_lens, n_seqs, cu_q);
+  if (n_tokens <= 0) return;
+  token_map_kernel<<<(n_tokens + 255) / 256, 256, 0, st>>>(cu_q, q_lens != nullptr, context_lens, block_table, n_seqs,
+                                                         max_pages_per_seq, num_pages, page_size, n_tokens,
+                                                         max_context, tok_seq, tok_pos, tok_slot, status);
+}
+
+// ------------------------------------------------------------------ RoPE + KV page write
+// One thread per (token, head, 8-wide chunk of the first half of the head): it owns elements
+// j..j+7 and j+dh/2..j+dh/2+7, i.e. eight rotation pairs.  q is rotated in place; k is rotated
+// into its page slot; v is copied into its page slot.
+__global__ void rope_kv_write_kernel(bf16* __restrict__ qkv, const float2* __restrict__ rope_tab,
+                                     const int* __restrict__ tok_pos, const int* __restrict__ tok_slot,
+                                     bf16* __restrict__ k_pages, bf16* __restrict__ v_pages, int n_tokens, int n_q,
+                                     int n_kv, int dh, int page_size) {
+  const int chunks = dh / 16;
+  const int heads = n_q + 2 * n_kv;
+  const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long total = (long long)n_tokens * heads * chunks;
+  if (gid >= total) return;
+  const int ch = int(gid % chunks);
+  const int head = int((gid / chunks) % heads);
+  const int tok = int(gid / (chunks * heads));
+  const int half = dh / 2;
+  bf16* src = qkv + size_t(tok) * heads * dh + size_t(head) * dh + ch * 8;
+  uint4 lo = *reinterpret_cast<const uint4*>(src);
+  uint4 hi = *reinterpret_cast<const uint4*>(src + half);
+  const int slot = tok_slot[tok];
+  if (head < n_q + n_kv) {
+    const float2* tab = rope_tab + size_t(tok_pos[tok]) * half + ch * 8;
+    uint32_t a[4] = {lo.x, lo.y, lo.z, lo.w}, b[4] = {hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 cs0 = __ldg(tab + 2 * j), cs1 = __ldg(tab + 2 * j + 1);
+      const float a0 = bf16_lo(a[j]), a1 = bf16_hi(a[j]), b0 = bf16_lo(b[j]), b1 = bf16_hi(b[j]);
+      a[j] = pack_bf16(a0 * cs0.x - b0 * cs0.y, a1 * cs1.x - b1 * cs1.y);
+      b[j] = pack_bf16(b0 * cs0.x + a0 * cs0.y, b1 * cs1.x + a1 * cs1.y);
+    }
+    lo = make_uint4(a[0], a[1], a[2], a[3]);
+    hi = make_uint4(b[0], b[1], b[2], b[3]);
+  }
+  if (head < n_q) {
+    *reinterpret_cast<uint4*>(src) = lo;
+    *reinterpret_cast<uint4*>(src + half) = hi;
+    return;
+  }
+  if (slot < 0) return;
+  const int page = slot / page_size, off = slot - page * page_size;
+  const bool is_k = head < n_q + n_kv;
+  const int kvh = is_k ? head - n_q : head - n_q - n_kv;
+  bf16* dst = (is_k ? k_pages : v_pages) + ((size_t(page) * n_kv + kvh) * page_size + off) * dh + ch * 8;
+  *reinterpret_cast<uint4*>(dst) = lo;
+  *reinterpret_cast<uint4*>(dst + half) = hi;
+}
+
+void launch_rope_kv_write(bf16* qkv, const float2* rope_tab, const int* tok_pos, const int* tok_slot, bf16* k_pages,
+                          bf16* v_pages, int n_tokens, int n_q, int n_kv, int dh, int page_size, cudaStream_t st) {
+  const long long total = (long long)n_tokens * (n_q + 2 * n_kv) * (dh / 16);
+  if (total <= 0) return;
+  rope_kv_write_kernel<<<unsigned((total + 255) / 256), 256, 0, st>>>(qkv, rope_tab, tok_pos, tok_slot, k_pages,
+                                                                     v_pages, n_tokens, n_q, n_kv, dh, page_size);
+}
+
+// ------------------------------------------------------------------ combine (+ residual, + last-layer mean)
+// Block per token; each thread owns 8 consecutive columns.  x'[h,i] = r_full[i] + sum_j w[i,h,j] y[inv[i,h,j]].
+__global__ void combine_kernel(const float* __restrict__ r_full, const bf16* __restrict__ y, const float* __restrict__ w,
+                               const int* __restrict__ inv, bf16* __restrict__ out, int n_tokens, int d, int H, int kc,
+                               int last_mean) {
+  const int i = blockIdx.x;
+  const float inv_h = 1.0f / float(H);
+  for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {
+    float r[8];
+    {
+      const float4 r0 = *reinterpret_cast<const float4*>(r_full + size_t(i) * d + c);
+      const float4 r1 = *reinterpret_cast<const float4*>(r_full + size_t(i) * d + c + 4);
+      r[0] = r0.x; r[1] = r0.y; r[2] = r0.z; r[3] = r0.w; r[4] = r1.x; r[5] = r1.y; r[6] = r1.z; r[7] = r1.w;
+    }
+    float mean[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) mean[t] = 0.f;
+    for (int h = 0; h < H; ++h) {
+      float acc[8];
+#pragma unroll
+      for (int t = 0; t < 8; ++t) acc[t] = r[t];
+      for (int j = 0; j < kc; ++j) {
+        const int sel = (i * H + h) * kc + j;
+        const float g = __ldg(w + sel);
+        const uint4 q = __ldg(reinterpret_cast<const uint4*>(y + size_t(__ldg(inv + sel)) * d + c));
+        const uint32_t v[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          acc[2 * t] += g * bf16_lo(v[t]);
+          acc[2 * t + 1] += g * bf16_hi(v[t]);
+        }
+      }
+      if (last_mean) {
+#pragma unroll
+        for (int t = 0; t < 8; ++t) mean[t] += acc[t];
+      } else {
+        *reinterpret_cast<uint4*>(out + (size_t(h) * n_tokens + i) * d + c) =
+            make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
+                       pack_bf16(acc[6], acc[7]));
+      }
+    }
+    if (last_mean) {
+      *reinterpret_cast<uint4*>(out + size_t(i) * d + c) =
+          make_uint4(pack_bf16(mean[0] * inv_h, mean[1] * inv_h), pack_bf16(mean[2] * inv_h, mean[3] * inv_h),
+                     pack_bf16(mean[4] * inv_h, mean[5] * inv_h), pack_bf16(mean[6] * inv_h, mean[7] * inv_h));
+    }
+  }
+}
+
+void launch_combine(const float* r_full, const bf16* y, const float* w, const int* inv, bf16* out, int n_tokens, int d,
+                    int H, int kc, int last_mean, cudaStream_t st) {
+  if (n_tokens <= 0) return;
+  int threads = d / 8;
+  if (threads > 256) threads = 256;
+  if (threads < 32) threads = 32;
+  combine_kernel<<<n_tokens, threads, 0, st>>>(r_full, y, w, inv, out, n_tokens, d, H, kc, last_mean);
+}
+
+// ------------------------------------------------------------------ create-time repacks
+// dst[b][n][k] = src[b][k][n] * gain[k]   (gain optional): makes the projection weights K-major.
+__global__ void transpose_batched_kernel(const bf16* __restrict__ src, size_t src_batch, int src_ld,
+                                         bf16* __restrict__ dst, size_t dst_batch, int dst_ld, int K, int N,
+                                         const bf16* __restrict__ gain) {
+  __shared__ float tile[32][33];
+  const bf16* s = src + blockIdx.z * src_batch;
+  bf16* d = dst + blockIdx.z * dst_batch;
+  const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int k = k0 + r, n = n0 + threadIdx.x;
+    float v = 0.f;
+    if (k < K && n < N) {
+      v = __bfloat162float(s[size_t(k) * src_ld + n]);
+      if (gain) v *= __bfloat162float(gain[k]);
+    }
+    tile[r][threadIdx.x] = v;
+  }
+  __syncthreads();
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int n = n0 + r, k = k0 + threadIdx.x;
+    if (k < K && n < N) d[size_t(n) * dst_ld + k] = __float2bfloat16_rn(tile[threadIdx.x][r]);
+  }
+}
+
+void launch_transpose_batched(const bf16* src, size_t src_batch, int src_ld, bf16* dst, size_t dst_batch, int dst_ld,
+                              int K, int N, int batch, const bf16* gain, cudaStream_t st) {
+  if (batch <= 0) return;
+  dim3 grid((N + 31) / 32, (K + 31) / 32, batch), block(32, 8);
+  transpose_batched_kernel<<<grid, block, 0, st>>>(src, src_batch, src_ld, dst, dst_batch, dst_ld, K, N, gain);
+}
+
+// dst[e][b*256 + half*128 + j][k] = (half ? w_up : w_gate)[e][k][b*128 + j]: gate and up columns of one
+// 128-wide block share one 256-wide GEMM tile, so SwiGLU is an epilogue.
+__global__ void pack_gate_up_kernel(const bf16* __restrict__ wg, const bf16* __restrict__ wu, bf16* __restrict__ dst,
+                                    int d, int I) {
+  __shared__ bf16 tile[32][34];
+  const int e = blockIdx.z;
+  const int k0 = blockIdx.y * 32, np0 = blockIdx.x * 32;      // np = packed row index in [0, 2I)
+  const int blk = np0 / 256, half = (np0 % 256) / 128, j0 = np0 % 128;
+  const bf16* src = (half ? wu : wg) + size_t(e) * d * I;
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int k = k0 + r;
+    tile[r][threadIdx.x] = (k < d) ? src[size_t(k) * I + blk * 128 + j0 + threadIdx.x] : __float2bfloat16_rn(0.f);
+  }
+  __syncthreads();
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int k = k0 + threadIdx.x;
+    if (k < d) dst[(size_t(e) * 2 * I + np0 + r) * d + k] = tile[threadIdx.x][r];
+  }
+}
+
+void launch_pack_gate_up(const bf16* wg, const bf16* wu, bf16* dst, int E, int d, int I, cudaStream_t st) {
+  dim3 grid(2 * I / 32, (d + 31) / 32, E), block(32, 8);
+  pack_gate_up_kernel<<<grid, block, 0, st>>>(wg, wu, dst, d, I);
+}
+
+}  // namespace foe

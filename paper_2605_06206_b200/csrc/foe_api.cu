@@ -1,0 +1,488 @@
+// C ABI of the FoE block (see include/foe.h): argument checks, weight repacking, workspace, tensor maps and
+// the launch sequences of prefill, decode and route.  No computation happens on the host.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/foe.h"
+#include "kernels.h"
+
+using namespace foe;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor [rows][cols] (cols contiguous), box [box_rows][64 cols], 128-byte swizzle.
+bool make_map_2d(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  if (rows == 0) rows = 1;
+  const cuuint64_t gdim[2] = {cols, rows};
+  const cuuint64_t gstride[1] = {cols * 2};
+  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+enum Stage { kStPrep = 0, kStQkv, kStRope, kStAttn, kStOproj, kStRoute, kStPermute, kStGemm1, kStGemm2, kStCombine, kNumStages };
+const char* kStageNames[kNumStages] = {"prep", "qkv_proj", "rope_kv_write", "attention", "o_proj_sync", "route",
+                                       "permute", "expert_gemm1_swiglu", "expert_gemm2", "combine"};
+
+}  // namespace
+
+struct foe_layer {
+  foe_config cfg;
+  int H, g, c, dh, d, I, E, Ec, kc, n_q, n_kv, qkv_cols, S_max, R_max, n_sms;
+  bool first, last;
+  std::vector<void*> allocs;
+  // repacked weights
+  bf16 *wqkv_t, *wo_t, *wgu_t, *wd_t, *ffn_gain;
+  float *router_w, *router_b;
+  float2* rope_tab;
+  // workspace
+  float *inv_rms, *r_full, *logits, *topk_w, *part_o, *part_ml;
+  bf16 *qkv, *attn_o, *u, *u_perm, *hmid, *y;
+  int *topk_idx, *cu_q, *tok_seq, *tok_pos, *tok_slot, *status;
+  PermuteBuffers pb;
+  int max_splits, pages_per_split;
+  // static tensor maps
+  CUtensorMap tm_wqkv, tm_attn_o, tm_wo, tm_uperm, tm_wgu, tm_hmid, tm_wd;
+  // call state
+  cudaStream_t last_stream;
+  int last_tokens, launches;
+  int profiling;
+  cudaEvent_t ev[kNumStages + 1];
+  bool ev_valid;
+};
+
+namespace {
+
+template <typename T>
+bool dalloc(foe_layer* L, T** p, size_t count) {
+  void* q = nullptr;
+  if (count == 0) count = 1;
+  if (cudaMalloc(&q, count * sizeof(T)) != cudaSuccess) { cudaGetLastError(); return false; }
+  L->allocs.push_back(q);
+  *p = static_cast<T*>(q);
+  return true;
+}
+
+foe_status validate(const foe_config* c) {
+  if (c->hidden <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->n_clusters <= 0) return FOE_ERR_CONFIG;
+  if (c->n_kv_heads % c->n_clusters || c->n_q_heads % c->n_kv_heads) return FOE_ERR_CONFIG;
+  if (c->head_dim != 64 && c->head_dim != 128) return FOE_ERR_CONFIG;
+  if (c->n_q_heads / c->n_kv_heads > 16) return FOE_ERR_CONFIG;
+  if (c->experts_per_cluster < 1 || c->experts_per_cluster > 128) return FOE_ERR_CONFIG;
+  if (c->top_k_per_cluster < 1 || c->top_k_per_cluster > c->experts_per_cluster || c->top_k_per_cluster > 32)
+    return FOE_ERR_CONFIG;
+  if (c->n_clusters * c->experts_per_cluster > 1024) return FOE_ERR_CONFIG;
+  if (c->page_size != 64) return FOE_ERR_CONFIG;
+  if (c->hidden % 64 || c->ffn_inter % 128 || c->ffn_inter <= 0) return FOE_ERR_CONFIG;
+  if (c->max_tokens <= 0 || c->max_seqs <= 0 || c->max_context <= 0) return FOE_ERR_CONFIG;
+  if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f)) return FOE_ERR_CONFIG;
+  if (c->position < 0 || c->position > 3 || c->sync < 0 || c->sync > 1) return FOE_ERR_CONFIG;
+  return FOE_OK;
+}
+
+void stage_mark(foe_layer* L, int i, cudaStream_t st) {
+  if (L->profiling) cudaEventRecord(L->ev[i], st);
+}
+
+foe_status check_launch() { return cudaGetLastError() == cudaSuccess ? FOE_OK : FOE_ERR_CUDA; }
+
+// routing + dispatch maps for n tokens whose synced residual is r (fp32 internal or bf16 from the caller)
+void run_route_and_permute(foe_layer* L, const void* r, int r_is_bf16, int n, cudaStream_t st) {
+  launch_route(r, r_is_bf16, L->ffn_gain, L->router_w, L->router_b, L->u, L->logits, L->topk_idx, L->topk_w, n, L->d,
+               L->H, L->Ec, L->kc, L->cfg.rms_eps, st);
+  L->launches += 1;
+  stage_mark(L, kStPermute, st);
+  launch_permute(L->topk_idx, L->pb, n, L->H * L->kc, L->E, 128, L->status, st);
+  L->launches += 3;
+}
+
+foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* out, cudaStream_t st, bool decode) {
+  const int S = decode ? kv->n_seqs : kv->n_tokens;
+  L->last_stream = st;
+  L->launches = 0;
+  L->last_tokens = S;
+  L->ev_valid = false;
+  if (S == 0) return FOE_OK;
+  const int H = L->H, d = L->d, dh = L->dh;
+  const bf16* xb = static_cast<const bf16*>(x);
+
+  CUtensorMap tmK, tmV, tmX;
+  const uint64_t page_rows = uint64_t(kv->num_pages) * L->n_kv * 64;
+  if (!make_map_2d(&tmK, kv->k_pages, page_rows, dh, 64) || !make_map_2d(&tmV, kv->v_pages, page_rows, dh, 64))
+    return FOE_ERR_CUDA;
+
+  // ---- prep: token map and pre-attention RMS statistics
+  stage_mark(L, kStPrep, st);
+  launch_token_map(decode ? nullptr : kv->q_lens, kv->context_lens, kv->block_table, kv->n_seqs, kv->max_pages_per_seq,
+                   kv->num_pages, 64, S, L->cfg.max_context, L->cu_q, L->tok_seq, L->tok_pos, L->tok_slot, L->status, st);
+  const int x_rows = L->first ? S : H * S;
+  launch_row_inv_rms(xb, L->inv_rms, x_rows, d, L->cfg.rms_eps, st);
+  L->launches += 3;
+
+  // ---- per-cluster QKV projection (norm gain folded into the weights, 1/rms applied in the epilogue)
+  stage_mark(L, kStQkv, st);
+  if (!decode) {
+    if (!make_map_2d(&tmX, x, x_rows, d, kBM)) return FOE_ERR_CUDA;
+    GemmArgs ga;
+    memset(&ga, 0, sizeof(ga));
+    ga.n_groups = H; ga.rows_per_group = S; ga.a_group_stride = L->first ? 0 : S;
+    ga.N = (L->g + 2 * L->c) * dh; ga.K = d; ga.status = L->status;
+    ga.out = L->qkv; ga.ldo = L->qkv_cols;
+    ga.row_scale = L->inv_rms; ga.scale_group_stride = L->first ? 0 : S;
+    ga.q_cols = L->g * dh; ga.kv_cols = L->c * dh; ga.q_total = L->n_q * dh; ga.kv_total = L->n_kv * dh;
+    launch_gemm(kEpiQKV, tmX, L->tm_wqkv, ga, L->n_sms, st);
+  } else {
+    SmallMArgs sa;
+    memset(&sa, 0, sizeof(sa));
+    sa.W = L->wqkv_t; sa.X = xb; sa.ldx = d; sa.n_groups = H; sa.rows_per_group = S; sa.x_group_stride = L->first ? 0 : S;
+    sa.N = (L->g + 2 * L->c) * dh; sa.K = d; sa.epi = kEpiQKV; sa.out = L->qkv; sa.ldo = L->qkv_cols;
+    sa.row_scale = L->inv_rms; sa.scale_group_stride = L->first ? 0 : S;
+    sa.q_cols = L->g * dh; sa.kv_cols = L->c * dh; sa.q_total = L->n_q * dh; sa.kv_total = L->n_kv * dh;
+    launch_smallm(sa, st);
+  }
+  L->launches += 1;
+
+  // ---- RoPE, K/V into the pages
+  stage_mark(L, kStRope, st);
+  launch_rope_kv_write(L->qkv, L->rope_tab, L->tok_pos, L->tok_slot, static_cast<bf16*>(kv->k_pages),
+                       static_cast<bf16*>(kv->v_pages), S, L->n_q, L->n_kv, dh, 64, st);
+  L->launches += 1;
+
+  // ---- attention core over the paged cache
+  stage_mark(L, kStAttn, st);
+  AttnArgs aa;
+  memset(&aa, 0, sizeof(aa));
+  aa.qkv = L->qkv; aa.out = L->attn_o; aa.cu_q = L->cu_q; aa.context_lens = kv->context_lens;
+  aa.q_lens = decode ? nullptr : kv->q_lens; aa.block_table = kv->block_table; aa.n_seqs = kv->n_seqs;
+  aa.max_pages_per_seq = kv->max_pages_per_seq; aa.num_pages = kv->num_pages; aa.n_q = L->n_q; aa.n_kv = L->n_kv;
+  aa.dh = dh; aa.max_q_len = decode ? 1 : kv->max_q_len; aa.scale_log2 = float(1.4426950408889634 / sqrt(double(dh)));
+  aa.status = L->status; aa.part_o = L->part_o; aa.part_ml = L->part_ml; aa.max_splits = L->max_splits;
+  aa.pages_per_split = L->pages_per_split;
+  if (decode) { launch_attn_decode(tmK, tmV, aa, st); L->launches += 2; }
+  else { launch_attn_prefill(tmK, tmV, aa, st); L->launches += 1; }
+
+  // ---- output projection; the cross-cluster sync is its K-reduction plus the sum of x[h] in the epilogue
+  stage_mark(L, kStOproj, st);
+  const float out_scale = (L->first || L->cfg.sync == FOE_SYNC_SUM) ? 1.0f : 1.0f / float(H);
+  if (!decode) {
+    GemmArgs ga;
+    memset(&ga, 0, sizeof(ga));
+    ga.n_groups = 1; ga.rows_per_group = S; ga.a_group_stride = 0; ga.N = d; ga.K = L->n_q * dh; ga.status = L->status;
+    ga.out = L->r_full; ga.ldo = d; ga.xsum = xb; ga.x_count = L->first ? 1 : H; ga.x_stride = size_t(S) * d;
+    ga.out_scale = out_scale;
+    launch_gemm(kEpiOProj, L->tm_attn_o, L->tm_wo, ga, L->n_sms, st);
+  } else {
+    SmallMArgs sa;
+    memset(&sa, 0, sizeof(sa));
+    sa.W = L->wo_t; sa.X = L->attn_o; sa.ldx = L->n_q * dh; sa.n_groups = 1; sa.rows_per_group = S; sa.N = d;
+    sa.K = L->n_q * dh; sa.epi = kEpiOProj; sa.out = L->r_full; sa.ldo = d; sa.xsum = xb; sa.x_count = L->first ? 1 : H;
+    sa.x_stride = size_t(S) * d; sa.out_scale = out_scale;
+    launch_smallm(sa, st);
+  }
+  L->launches += 1;
+
+  // ---- router, top-k, gates, dispatch maps
+  stage_mark(L, kStRoute, st);
+  run_route_and_permute(L, L->r_full, 0, S, st);
+  const int R = S * H * L->kc;
+
+  if (!decode) {
+    launch_gather_rows(L->u, L->pb.perm, L->u_perm, R, d, st);
+    L->launches += 1;
+    stage_mark(L, kStGemm1, st);
+    GemmArgs g1;
+    memset(&g1, 0, sizeof(g1));
+    g1.n_groups = L->E; g1.mt_group = L->pb.mt_group; g1.mt_row0 = L->pb.mt_row0; g1.group_end = L->pb.offsets + 1;
+    g1.n_mtiles = L->pb.n_mtiles; g1.N = 2 * L->I; g1.K = d; g1.status = L->status; g1.out = L->hmid; g1.ldo = L->I;
+    launch_gemm(kEpiSwiGLU, L->tm_uperm, L->tm_wgu, g1, L->n_sms, st);
+    stage_mark(L, kStGemm2, st);
+    GemmArgs g2 = g1;
+    g2.N = d; g2.K = L->I; g2.out = L->y; g2.ldo = d;
+    launch_gemm(kEpiBf16, L->tm_hmid, L->tm_wd, g2, L->n_sms, st);
+    L->launches += 2;
+  } else {
+    stage_mark(L, kStGemm1, st);
+    SmallMArgs s1;
+    memset(&s1, 0, sizeof(s1));
+    s1.W = L->wgu_t; s1.X = L->u; s1.ldx = d; s1.row_index = L->pb.perm; s1.group_offsets = L->pb.offsets;
+    s1.n_groups = L->E; s1.N = 2 * L->I; s1.K = d; s1.epi = kEpiSwiGLU; s1.out = L->hmid; s1.ldo = L->I;
+    launch_smallm(s1, st);
+    stage_mark(L, kStGemm2, st);
+    SmallMArgs s2;
+    memset(&s2, 0, sizeof(s2));
+    s2.W = L->wd_t; s2.X = L->hmid; s2.ldx = L->I; s2.group_offsets = L->pb.offsets; s2.n_groups = L->E; s2.N = d;
+    s2.K = L->I; s2.epi = kEpiBf16; s2.out = L->y; s2.ldo = d;
+    launch_smallm(s2, st);
+    L->launches += 2;
+  }
+
+  // ---- weighted combine, residual, last-layer mean
+  stage_mark(L, kStCombine, st);
+  launch_combine(L->r_full, L->y, L->topk_w, L->pb.inv, static_cast<bf16*>(out), S, d, H, L->kc, L->last ? 1 : 0, st);
+  L->launches += 1;
+  if (L->profiling) { cudaEventRecord(L->ev[kNumStages], st); L->ev_valid = true; }
+  return check_launch();
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* foe_status_string(int s) {
+  switch (s) {
+    case FOE_OK: return "ok";
+    case FOE_ERR_NULL: return "null pointer argument";
+    case FOE_ERR_CONFIG: return "invalid layer configuration";
+    case FOE_ERR_SHAPE: return "call exceeds the sizes the layer was created for";
+    case FOE_ERR_UNSUPPORTED: return "unsupported";
+    case FOE_ERR_OOM: return "device allocation failed";
+    case FOE_ERR_CUDA: return "CUDA call failed";
+    case FOE_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case FOE_ERR_BOUNDS: return "an index read on the device was out of range";
+    default: return "unknown status";
+  }
+}
+
+foe_status foe_layer_destroy(foe_layer* L) {
+  if (!L) return FOE_OK;
+  for (void* p : L->allocs) cudaFree(p);
+  for (int i = 0; i <= kNumStages; ++i)
+    if (L->ev[i]) cudaEventDestroy(L->ev[i]);
+  delete L;
+  return FOE_OK;
+}
+
+foe_status foe_layer_create(const foe_config* cfg, const foe_weights* w, foe_layer** out) {
+  if (!cfg || !w || !out) return FOE_ERR_NULL;
+  *out = nullptr;
+  const foe_status v = validate(cfg);
+  if (v != FOE_OK) return v;
+  if (!w->attn_norm_g || !w->wq || !w->wk || !w->wv || !w->wo || !w->ffn_norm_g || !w->w_gate || !w->w_up ||
+      !w->w_down || !w->router_w)
+    return FOE_ERR_NULL;
+  int dev = 0, n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  if (cudaGetDevice(&dev) != cudaSuccess) return FOE_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return FOE_ERR_CUDA;
+  if (prop.major != 10) return FOE_ERR_UNSUPPORTED;       // tcgen05/TMEM kernels: sm_100 only
+  if (gemm_configure() != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+
+  foe_layer* L = new (std::nothrow) foe_layer();
+  if (!L) return FOE_ERR_OOM;
+  L->cfg = *cfg;
+  L->H = cfg->n_clusters; L->n_q = cfg->n_q_heads; L->n_kv = cfg->n_kv_heads; L->dh = cfg->head_dim;
+  L->g = L->n_q / L->H; L->c = L->n_kv / L->H; L->d = cfg->hidden; L->I = cfg->ffn_inter;
+  L->Ec = cfg->experts_per_cluster; L->E = L->H * L->Ec; L->kc = cfg->top_k_per_cluster;
+  L->qkv_cols = (L->n_q + 2 * L->n_kv) * L->dh;
+  L->first = cfg->position == FOE_FIRST || cfg->position == FOE_SINGLE;
+  L->last = cfg->position == FOE_LAST || cfg->position == FOE_SINGLE;
+  L->S_max = cfg->max_tokens > cfg->max_seqs ? cfg->max_tokens : cfg->max_seqs;
+  L->R_max = L->S_max * L->H * L->kc;
+  L->n_sms = prop.multiProcessorCount;
+  const int H = L->H, d = L->d, dh = L->dh, I = L->I, E = L->E, S = L->S_max, R = L->R_max;
+  const int max_pages = (cfg->max_context + 63) / 64;
+  L->pages_per_split = 16;
+  L->max_splits = (max_pages + L->pages_per_split - 1) / L->pages_per_split;
+  const int n_blocks = (S + kPermuteBlockTokens - 1) / kPermuteBlockTokens;
+  const int qkvN = (L->g + 2 * L->c) * dh;
+
+  bool ok = true;
+  ok = ok && dalloc(L, &L->wqkv_t, size_t(H) * qkvN * d + 256 * size_t(d));
+  ok = ok && dalloc(L, &L->wo_t, size_t(d) * L->n_q * dh + 256 * size_t(L->n_q) * dh);
+  ok = ok && dalloc(L, &L->wgu_t, size_t(E) * 2 * I * d);
+  ok = ok && dalloc(L, &L->wd_t, size_t(E) * d * I + 256 * size_t(I));
+  ok = ok && dalloc(L, &L->ffn_gain, size_t(d));
+  ok = ok && dalloc(L, &L->router_w, size_t(E) * d);
+  ok = ok && dalloc(L, &L->router_b, size_t(E));
+  ok = ok && dalloc(L, &L->rope_tab, size_t(cfg->max_context) * (dh / 2));
+  ok = ok && dalloc(L, &L->inv_rms, size_t(H) * S);
+  ok = ok && dalloc(L, &L->r_full, size_t(S) * d);
+  ok = ok && dalloc(L, &L->logits, size_t(S) * E);
+  ok = ok && dalloc(L, &L->topk_w, size_t(R));
+  ok = ok && dalloc(L, &L->topk_idx, size_t(R));
+  ok = ok && dalloc(L, &L->qkv, size_t(S) * L->qkv_cols);
+  ok = ok && dalloc(L, &L->attn_o, size_t(S + 128) * L->n_q * dh);
+  ok = ok && dalloc(L, &L->u, size_t(S) * d);
+  ok = ok && dalloc(L, &L->u_perm, size_t(R + 128) * d);
+  ok = ok && dalloc(L, &L->hmid, size_t(R + 128) * I);
+  ok = ok && dalloc(L, &L->y, size_t(R) * d);
+  ok = ok && dalloc(L, &L->cu_q, size_t(cfg->max_seqs) + 1);
+  ok = ok && dalloc(L, &L->tok_seq, size_t(S));
+  ok = ok && dalloc(L, &L->tok_pos, size_t(S));
+  ok = ok && dalloc(L, &L->tok_slot, size_t(S));
+  ok = ok && dalloc(L, &L->status, size_t(1));
+  ok = ok && dalloc(L, &L->part_o, size_t(cfg->max_seqs) * L->n_q * L->max_splits * dh);
+  ok = ok && dalloc(L, &L->part_ml, size_t(cfg->max_seqs) * L->n_q * L->max_splits * 2);
+  ok = ok && dalloc(L, &L->pb.counts, size_t(E));
+  ok = ok && dalloc(L, &L->pb.offsets, size_t(E) + 1);
+  ok = ok && dalloc(L, &L->pb.perm, size_t(R));
+  ok = ok && dalloc(L, &L->pb.inv, size_t(R));
+  ok = ok && dalloc(L, &L->pb.rank, size_t(R));
+  ok = ok && dalloc(L, &L->pb.blk_counts, size_t(n_blocks) * E);
+  ok = ok && dalloc(L, &L->pb.mt_group, size_t(R / 128 + E + 1));
+  ok = ok && dalloc(L, &L->pb.mt_row0, size_t(R / 128 + E + 1));
+  ok = ok && dalloc(L, &L->pb.n_mtiles, size_t(1));
+  if (!ok) { foe_layer_destroy(L); return FOE_ERR_OOM; }
+
+  cudaStream_t st = 0;
+  cudaMemsetAsync(L->status, 0, sizeof(int), st);
+  cudaMemsetAsync(L->attn_o, 0, size_t(S + 128) * L->n_q * dh * sizeof(bf16), st);
+  cudaMemsetAsync(L->u_perm, 0, size_t(R + 128) * d * sizeof(bf16), st);
+  cudaMemsetAsync(L->hmid, 0, size_t(R + 128) * I * sizeof(bf16), st);
+  // K-major ("transposed") weights; the attention-norm gain is folded into W_q|k|v.
+  const bf16* gain_a = static_cast<const bf16*>(w->attn_norm_g);
+  const size_t qkv_batch = size_t(qkvN) * d;
+  launch_transpose_batched(static_cast<const bf16*>(w->wq), size_t(d) * L->g * dh, L->g * dh, L->wqkv_t, qkv_batch, d, d,
+                           L->g * dh, H, gain_a, st);
+  launch_transpose_batched(static_cast<const bf16*>(w->wk), size_t(d) * L->c * dh, L->c * dh,
+                           L->wqkv_t + size_t(L->g) * dh * d, qkv_batch, d, d, L->c * dh, H, gain_a, st);
+  launch_transpose_batched(static_cast<const bf16*>(w->wv), size_t(d) * L->c * dh, L->c * dh,
+                           L->wqkv_t + size_t(L->g + L->c) * dh * d, qkv_batch, d, d, L->c * dh, H, gain_a, st);
+  launch_transpose_batched(static_cast<const bf16*>(w->wo), 0, d, L->wo_t, 0, L->n_q * dh, L->n_q * dh, d, 1, nullptr, st);
+  launch_pack_gate_up(static_cast<const bf16*>(w->w_gate), static_cast<const bf16*>(w->w_up), L->wgu_t, E, d, I, st);
+  for (int e0 = 0; e0 < E; e0 += 32768) {
+    const int nb = E - e0 < 32768 ? E - e0 : 32768;
+    launch_transpose_batched(static_cast<const bf16*>(w->w_down) + size_t(e0) * I * d, size_t(I) * d, d,
+                             L->wd_t + size_t(e0) * d * I, size_t(d) * I, I, I, d, nb, nullptr, st);
+  }
+  cudaMemcpyAsync(L->ffn_gain, w->ffn_norm_g, size_t(d) * sizeof(bf16), cudaMemcpyDeviceToDevice, st);
+  cudaMemcpyAsync(L->router_w, w->router_w, size_t(E) * d * sizeof(float), cudaMemcpyDeviceToDevice, st);
+  if (w->router_b) cudaMemcpyAsync(L->router_b, w->router_b, size_t(E) * sizeof(float), cudaMemcpyDeviceToDevice, st);
+  else cudaMemsetAsync(L->router_b, 0, size_t(E) * sizeof(float), st);
+  // rotary table in double precision on the host: (cos, sin)(p * theta^(-2j/dh))
+  {
+    const int half = dh / 2;
+    std::vector<float2> tab(size_t(cfg->max_context) * half);
+    std::vector<double> inv_freq(half);
+    for (int j = 0; j < half; ++j) inv_freq[j] = pow(double(cfg->rope_theta), -2.0 * j / double(dh));
+    for (int p = 0; p < cfg->max_context; ++p)
+      for (int j = 0; j < half; ++j) {
+        const double ang = double(p) * inv_freq[j];
+        tab[size_t(p) * half + j] = make_float2(float(cos(ang)), float(sin(ang)));
+      }
+    cudaMemcpy(L->rope_tab, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice);
+  }
+  if (cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess) {
+    foe_layer_destroy(L);
+    return FOE_ERR_CUDA;
+  }
+  ok = make_map_2d(&L->tm_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, kBN) &&
+       make_map_2d(&L->tm_attn_o, L->attn_o, uint64_t(S), uint64_t(L->n_q) * dh, kBM) &&
+       make_map_2d(&L->tm_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, kBN) &&
+       make_map_2d(&L->tm_uperm, L->u_perm, uint64_t(R), d, kBM) &&
+       make_map_2d(&L->tm_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, kBN) &&
+       make_map_2d(&L->tm_hmid, L->hmid, uint64_t(R), I, kBM) &&
+       make_map_2d(&L->tm_wd, L->wd_t, uint64_t(E) * d, I, kBN);
+  if (!ok) { foe_layer_destroy(L); return FOE_ERR_CUDA; }
+  for (int i = 0; i <= kNumStages; ++i) cudaEventCreate(&L->ev[i]);
+  *out = L;
+  return FOE_OK;
+}
+
+foe_status foe_prefill(foe_layer* L, const void* x, const foe_kv_cache* kv, void* out, void* stream) {
+  if (!L || !x || !kv || !out) return FOE_ERR_NULL;
+  if (kv->n_tokens < 0 || kv->n_seqs < 0) return FOE_ERR_SHAPE;
+  if (kv->n_tokens == 0) { L->launches = 0; L->last_tokens = 0; return FOE_OK; }
+  if (!kv->k_pages || !kv->v_pages || !kv->block_table || !kv->context_lens || !kv->q_lens) return FOE_ERR_NULL;
+  if (kv->n_tokens > L->cfg.max_tokens || kv->n_seqs > L->cfg.max_seqs || kv->n_seqs == 0) return FOE_ERR_SHAPE;
+  if (kv->max_q_len <= 0 || kv->max_q_len > kv->n_tokens || kv->max_pages_per_seq <= 0 || kv->num_pages <= 0)
+    return FOE_ERR_SHAPE;
+  if (x == out) return FOE_ERR_UNSUPPORTED;
+  return run_block(L, x, kv, out, static_cast<cudaStream_t>(stream), false);
+}
+
+foe_status foe_decode(foe_layer* L, const void* x, const foe_kv_cache* kv, void* out, void* stream) {
+  if (!L || !x || !kv || !out) return FOE_ERR_NULL;
+  if (kv->n_seqs < 0) return FOE_ERR_SHAPE;
+  if (kv->n_seqs == 0) { L->launches = 0; L->last_tokens = 0; return FOE_OK; }
+  if (!kv->k_pages || !kv->v_pages || !kv->block_table || !kv->context_lens) return FOE_ERR_NULL;
+  if (kv->n_seqs > L->cfg.max_seqs || kv->max_pages_per_seq <= 0 || kv->num_pages <= 0) return FOE_ERR_SHAPE;
+  if (x == out) return FOE_ERR_UNSUPPORTED;
+  return run_block(L, x, kv, out, static_cast<cudaStream_t>(stream), true);
+}
+
+foe_status foe_route(foe_layer* L, const void* h, int n_tokens, int* topk_idx, float* topk_w, void* stream) {
+  if (!L || !h || !topk_idx || !topk_w) return FOE_ERR_NULL;
+  if (n_tokens < 0 || n_tokens > L->S_max) return FOE_ERR_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  L->last_stream = st;
+  L->launches = 0;
+  L->last_tokens = n_tokens;
+  L->ev_valid = false;
+  if (n_tokens == 0) return FOE_OK;
+  const int saved = L->profiling;
+  L->profiling = 0;
+  run_route_and_permute(L, h, 1, n_tokens, st);
+  L->profiling = saved;
+  const size_t n = size_t(n_tokens) * L->H * L->kc;
+  cudaMemcpyAsync(topk_idx, L->topk_idx, n * sizeof(int), cudaMemcpyDeviceToDevice, st);
+  cudaMemcpyAsync(topk_w, L->topk_w, n * sizeof(float), cudaMemcpyDeviceToDevice, st);
+  return check_launch();
+}
+
+foe_status foe_get_aux(foe_layer* L, foe_aux* a) {
+  if (!L || !a) return FOE_ERR_NULL;
+  a->n_tokens = L->last_tokens;
+  a->r_full = L->r_full; a->u = L->u; a->logits = L->logits; a->topk_idx = L->topk_idx; a->topk_w = L->topk_w;
+  a->counts = L->pb.counts; a->offsets = L->pb.offsets; a->perm = L->pb.perm; a->inv = L->pb.inv;
+  a->qkv = L->qkv; a->attn_o = L->attn_o;
+  return FOE_OK;
+}
+
+foe_status foe_poll_status(foe_layer* L, int* device_status) {
+  if (!L || !device_status) return FOE_ERR_NULL;
+  if (cudaStreamSynchronize(L->last_stream) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  int v = 0;
+  if (cudaMemcpy(&v, L->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FOE_ERR_CUDA;
+  *device_status = v;
+  if (v != 0) cudaMemset(L->status, 0, sizeof(int));
+  return FOE_OK;
+}
+
+int foe_last_launch_count(const foe_layer* L) { return L ? L->launches : 0; }
+
+foe_status foe_set_profiling(foe_layer* L, int enabled) {
+  if (!L) return FOE_ERR_NULL;
+  L->profiling = enabled ? 1 : 0;
+  return FOE_OK;
+}
+
+int foe_num_stages(void) { return kNumStages; }
+
+const char* foe_stage_name(int i) { return (i >= 0 && i < kNumStages) ? kStageNames[i] : ""; }
+
+foe_status foe_get_stage_ms(foe_layer* L, float* ms, int n) {
+  if (!L || !ms) return FOE_ERR_NULL;
+  if (!L->ev_valid || n < kNumStages) return FOE_ERR_UNSUPPORTED;
+  if (cudaEventSynchronize(L->ev[kNumStages]) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  for (int i = 0; i < kNumStages; ++i)
+    if (cudaEventElapsedTime(&ms[i], L->ev[i], L->ev[i + 1]) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  return FOE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,47 @@
+// Argument block and epilogue kinds of the GEMM kernels (plain data, host and device).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <stddef.h>
+
+namespace foe {
+
+constexpr int kBM = 128;   // GEMM tile rows  (UMMA M)
+constexpr int kBN = 256;   // GEMM tile cols  (UMMA N)
+
+enum GemmEpilogue : int {
+  kEpiBf16 = 0,     // C -> bf16 [row][ldo]
+  kEpiSwiGLU = 1,   // columns [0,128) gate, [128,256) up of one 128-wide block: silu(gate)*up -> bf16
+  kEpiQKV = 2,      // row scale (1/rms) and scatter of the cluster's q|k|v columns into [S][(n_q+2n_kv)*dh]
+  kEpiOProj = 3     // r_full = scale * (C + sum_h x[h]) -> fp32 [row][ldo]
+};
+
+struct GemmArgs {
+  // uniform groups
+  int n_groups;
+  int rows_per_group;
+  int a_group_stride;       // first A row of group g = g * a_group_stride
+  // ragged groups (n_mtiles != nullptr)
+  const int* mt_group;      // [n_mtiles] group of each m-tile
+  const int* mt_row0;       // [n_mtiles] first A row of each m-tile
+  const int* group_end;     // [n_groups] one past the last A row of the group
+  const int* n_mtiles;      // device scalar
+  int N;                    // columns per group (rows of B per group)
+  int K;
+  int* status;              // device status word
+  // epilogue
+  void* out;
+  int ldo;                  // elements per output row
+  // kEpiQKV
+  const float* row_scale;   // [n_groups * scale_group_stride]
+  int scale_group_stride;
+  int q_cols, kv_cols;      // g*dh and c*dh of one cluster
+  int q_total, kv_total;    // n_q*dh and n_kv*dh
+  // kEpiOProj
+  const __nv_bfloat16* xsum; // [x_count][x_stride] residual streams added to C
+  int x_count;
+  size_t x_stride;
+  float out_scale;
+};
+
+}  // namespace foe

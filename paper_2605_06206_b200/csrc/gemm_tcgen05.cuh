@@ -1,0 +1,253 @@
+// Grouped bf16 GEMM on the 5th-generation tensor cores (tcgen05 + TMEM), operands staged by TMA.
+//
+//   C_g[m, n] = sum_k A[row_g(m), k] * B_g[n, k]          fp32 accumulation in tensor memory
+//
+// One persistent CTA per SM walks a static round-robin list of 128 x 256 output tiles.  Warp 0 is
+// the TMA producer, warp 1 issues the MMAs and owns the TMEM allocation, warps 2..5 drain the
+// accumulator (tcgen05.ld) and apply the epilogue.  Two accumulator stages (2 x 256 TMEM columns)
+// let the epilogue of one tile overlap the MMAs of the next.  Groups are either uniform (every
+// group has the same row count: the per-cluster QKV projection, the output projection) or ragged
+// (the experts: an m-tile table built on the device by the permute step, so no host sync).
+//
+// Used for steps of the paper's Table 2: Attn_h's projections ("Attn. residual" row), the sync
+// ("Cross-group avg." row, fused into the output-projection epilogue) and FFN_e ("MoE update" row).
+#pragma once
+
+#include "common.cuh"
+#include "gemm_args.h"
+
+namespace foe {
+
+constexpr int kBK = 64;              // k-block: 64 bf16 = one 128-byte swizzle row
+constexpr int kUmmaK = 16;
+constexpr int kStages = 4;
+constexpr int kABytes = kBM * kBK * 2;   // 16 KB
+constexpr int kBBytes = kBN * kBK * 2;   // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kGemmThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr size_t kGemmSmemBytes = size_t(kStages) * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+__device__ __forceinline__ float silu_f(float z) { return z / (1.0f + __expf(-z)); }
+
+template <int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const GemmArgs args) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  uint64_t* empty_bar = full_bar + kStages;
+  uint64_t* acc_full = empty_bar + kStages;
+  uint64_t* acc_empty = acc_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); }
+    mbar_fence_init();
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const bool ragged = args.n_mtiles != nullptr;
+  const int tiles_per_group = (args.rows_per_group + kBM - 1) / kBM;
+  const int n_mtiles = ragged ? *args.n_mtiles : args.n_groups * tiles_per_group;
+  const int n_ntiles = (args.N + kBN - 1) / kBN;
+  const int total_tiles = n_mtiles * n_ntiles;
+  const int kblocks = (args.K + kBK - 1) / kBK;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (one thread)
+    if (elect_one()) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int mt = tile / n_ntiles, nt = tile - mt * n_ntiles;
+        int group, row0;
+        if (ragged) { group = args.mt_group[mt]; row0 = args.mt_row0[mt]; }
+        else { group = mt / tiles_per_group; row0 = group * args.a_group_stride + (mt - group * tiles_per_group) * kBM; }
+        const int brow0 = group * args.N + nt * kBN;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(&empty_bar[stage], phase ^ 1)) { ok = false; break; }
+          uint8_t* sa = smem + stage * kStageBytes;
+          mbar_expect_tx(&full_bar[stage], kStageBytes);
+          tma_load_2d(sa, &tmA, &full_bar[stage], kb * kBK, row0);
+          tma_load_2d(sa + kABytes, &tmB, &full_bar[stage], kb * kBK, brow0);
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) atomicExch(args.status, kStatusTimeout);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (one thread)
+    if (elect_one()) {
+      constexpr uint32_t idesc = umma_idesc_bf16(kBM, kBN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+        const int acc = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1;
+        if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * kBN;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(&full_bar[stage], phase)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + stage * kStageBytes);
+          const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+          for (int k = 0; k < kBK / kUmmaK; ++k) {
+            umma_bf16(d_tmem, umma_desc_sw128(a_addr + k * kUmmaK * 2), umma_desc_sw128(b_addr + k * kUmmaK * 2),
+                      idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(&empty_bar[stage]);
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+        if (ok) umma_commit(&acc_full[acc]);
+      }
+      if (!ok) atomicExch(args.status, kStatusTimeout);
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (4 warps = 128 TMEM lanes)
+    const int quarter = warp & 3;                 // a warp may only touch TMEM lanes 32*(warp%4)..+31
+    const int row_in_tile = quarter * 32 + lane;
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+      const int mt = tile / n_ntiles, nt = tile - mt * n_ntiles;
+      int group, row0, row_end, group_row0;
+      if (ragged) {
+        group = args.mt_group[mt]; row0 = args.mt_row0[mt]; row_end = args.group_end[group]; group_row0 = 0;
+      } else {
+        group = mt / tiles_per_group;
+        group_row0 = group * args.a_group_stride;
+        row0 = group_row0 + (mt - group * tiles_per_group) * kBM;
+        row_end = group_row0 + args.rows_per_group;
+      }
+      const int row = row0 + row_in_tile;          // A row
+      const bool row_ok = row < row_end;
+      const int n0 = nt * kBN;                     // column inside the group
+      const int acc = it & 1;
+      const uint32_t acc_phase = (it >> 1) & 1;
+      if (!mbar_wait(&acc_full[acc], acc_phase)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kBN;
+
+      if constexpr (EPI == kEpiSwiGLU) {
+        __nv_bfloat16* out = static_cast<__nv_bfloat16*>(args.out);
+#pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t gt[32], up[32];
+          __syncwarp();
+          tmem_ld32(taddr + ch * 32, gt);
+          tmem_ld32(taddr + 128 + ch * 32, up);
+          tmem_ld_wait();
+          if (row_ok) {
+            uint4* dst = reinterpret_cast<uint4*>(out + size_t(row) * args.ldo + (n0 >> 1) + ch * 32);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint32_t w[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int c = v * 8 + j * 2;
+                const float h0 = silu_f(__uint_as_float(gt[c])) * __uint_as_float(up[c]);
+                const float h1 = silu_f(__uint_as_float(gt[c + 1])) * __uint_as_float(up[c + 1]);
+                w[j] = pack_bf16(h0, h1);
+              }
+              dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      } else {
+        const int row_local = row - group_row0;
+        float scale = 1.0f;
+        if constexpr (EPI == kEpiQKV) {
+          if (row_ok) scale = args.row_scale[size_t(group) * args.scale_group_stride + row_local];
+        }
+#pragma unroll 1
+        for (int ch = 0; ch < kBN / 32; ++ch) {
+          const int n = n0 + ch * 32;
+          if (n >= args.N) break;                       // warp-uniform
+          uint32_t r[32];
+          __syncwarp();
+          tmem_ld32(taddr + ch * 32, r);
+          tmem_ld_wait();
+          if (row_ok) {
+          if constexpr (EPI == kEpiBf16 || EPI == kEpiQKV) {
+            int col = n;
+            int orow = row;
+            if constexpr (EPI == kEpiQKV) {
+              orow = row_local;
+              if (n < args.q_cols) col = group * args.q_cols + n;
+              else if (n < args.q_cols + args.kv_cols) col = args.q_total + group * args.kv_cols + (n - args.q_cols);
+              else col = args.q_total + args.kv_total + group * args.kv_cols + (n - args.q_cols - args.kv_cols);
+            }
+            uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + size_t(orow) * args.ldo + col);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint32_t w[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int c = v * 8 + j * 2;
+                w[j] = pack_bf16(__uint_as_float(r[c]) * scale, __uint_as_float(r[c + 1]) * scale);
+              }
+              dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          } else {  // kEpiOProj
+            float acc32[32];
+#pragma unroll
+            for (int c = 0; c < 32; ++c) acc32[c] = __uint_as_float(r[c]);
+            for (int h = 0; h < args.x_count; ++h) {
+              const uint4* xs = reinterpret_cast<const uint4*>(args.xsum + h * args.x_stride + size_t(row) * args.ldo + n);
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                const uint4 q = __ldg(xs + v);
+                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  acc32[v * 8 + j * 2] += bf16_lo(w[j]);
+                  acc32[v * 8 + j * 2 + 1] += bf16_hi(w[j]);
+                }
+              }
+            }
+            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(args.out) + size_t(row) * args.ldo + n);
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+              dst[v] = make_float4(acc32[v * 4] * args.out_scale, acc32[v * 4 + 1] * args.out_scale,
+                                   acc32[v * 4 + 2] * args.out_scale, acc32[v * 4 + 3] * args.out_scale);
+          }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[acc]);
+    }
+    if (!ok && lane == 0) atomicExch(args.status, kStatusTimeout);
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace foe

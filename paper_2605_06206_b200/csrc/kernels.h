@@ -1,0 +1,103 @@
+// Host-callable launchers of the FoE kernels (internal to the library).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gemm_args.h"
+
+namespace foe {
+
+typedef __nv_bfloat16 bf16;
+
+// ---- elementwise.cu
+// inv_rms[r] = rsqrt(mean(x[r,:]^2) + eps) for n_rows rows of d bf16 values
+void launch_row_inv_rms(const bf16* x, float* inv_rms, int n_rows, int d, float eps, cudaStream_t st);
+// per-token position / sequence / cache slot from q_lens and context_lens (device arrays)
+void launch_token_map(const int* q_lens, const int* context_lens, const int* block_table, int n_seqs,
+                      int max_pages_per_seq, int num_pages, int page_size, int n_tokens, int max_context, int* cu_q,
+                      int* tok_seq, int* tok_pos, int* tok_slot, int* status, cudaStream_t st);
+// RoPE on q (in place) and k, then K/V of the new tokens into their pages
+void launch_rope_kv_write(bf16* qkv, const float2* rope_tab, const int* tok_pos, const int* tok_slot, bf16* k_pages,
+                          bf16* v_pages, int n_tokens, int n_q, int n_kv, int dh, int page_size, cudaStream_t st);
+// combine: out = r_full + sum_j w * y[inv]  (per cluster), optional mean over clusters
+void launch_combine(const float* r_full, const bf16* y, const float* w, const int* inv, bf16* out, int n_tokens,
+                    int d, int H, int kc, int last_mean, cudaStream_t st);
+// weight repacks (create time)
+void launch_transpose_batched(const bf16* src, size_t src_batch, int src_ld, bf16* dst, size_t dst_batch, int dst_ld,
+                              int K, int N, int batch, const bf16* gain, cudaStream_t st);
+void launch_pack_gate_up(const bf16* wg, const bf16* wu, bf16* dst, int E, int d, int I, cudaStream_t st);
+
+// ---- route.cu
+// FFN norm + fp32 router + per-cluster top-k + gates.  r_in is fp32 or bf16 [S][d].
+void launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const float* br, bf16* u_out,
+                  float* logits, int* idx, float* w, int n_tokens, int d, int H, int Ec, int kc, float eps,
+                  cudaStream_t st);
+
+// ---- permute.cu
+struct PermuteBuffers {
+  int* counts;        // [E]
+  int* offsets;       // [E+1]
+  int* perm;          // [R]
+  int* inv;           // [S*H*kc]
+  int* rank;          // [S*H*kc] rank of the selection inside its token block
+  int* blk_counts;    // [n_blocks][E]
+  int* mt_group;      // [R/128 + E]
+  int* mt_row0;
+  int* n_mtiles;      // scalar
+};
+constexpr int kPermuteBlockTokens = 256;
+void launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int sel_per_token, int E, int tile_rows,
+                    int* status, cudaStream_t st);
+// u_perm[slot, :] = u[perm[slot], :]   (16-byte vector copies)
+void launch_gather_rows(const bf16* u, const int* perm, bf16* u_perm, int n_rows, int d, cudaStream_t st);
+
+// ---- attention.cu
+struct AttnArgs {
+  const bf16* qkv;          // [S][(n_q+2n_kv)*dh]; q after RoPE
+  bf16* out;                // [S][n_q*dh]
+  const int* cu_q;          // [n_seqs+1]
+  const int* context_lens;  // [n_seqs]
+  const int* q_lens;        // [n_seqs] or nullptr (1 each)
+  const int* block_table;   // [n_seqs][max_pages_per_seq]
+  int n_seqs, max_pages_per_seq, num_pages;
+  int n_q, n_kv, dh;
+  int max_q_len;
+  float scale_log2;         // log2(e) / sqrt(dh)
+  int* status;
+  // decode only
+  float* part_o;            // [n_seqs][n_q][max_splits][dh]
+  float* part_ml;           // [n_seqs][n_q][max_splits][2]
+  int max_splits;
+  int pages_per_split;
+};
+void launch_attn_prefill(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st);
+void launch_attn_decode(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st);
+
+// ---- gemm_tcgen05.cu
+void launch_gemm(int epi, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args, int n_sms,
+                 cudaStream_t st);
+cudaError_t gemm_configure();   // opt in to the dynamic shared memory the kernels need
+
+// ---- smallm.cu  (weight-streaming GEMMs for a handful of rows per group)
+struct SmallMArgs {
+  const bf16* W;            // [n_groups][N][K]  K contiguous
+  const bf16* X;            // activation rows, K contiguous, row stride ldx
+  int ldx;
+  const int* row_index;     // optional gather: X row of logical row r is row_index[r]; nullptr = identity
+  const int* group_offsets; // ragged: rows of group g are [off[g], off[g+1]); nullptr = uniform
+  int n_groups;
+  int rows_per_group;       // uniform
+  int x_group_stride;       // uniform: first X row of group g = g * x_group_stride
+  int N, K;
+  int epi;                  // GemmEpilogue
+  void* out; int ldo;
+  const float* row_scale; int scale_group_stride;
+  int q_cols, kv_cols, q_total, kv_total;
+  const bf16* xsum; int x_count; size_t x_stride; float out_scale;
+};
+void launch_smallm(const SmallMArgs& a, cudaStream_t st);
+
+}  // namespace foe

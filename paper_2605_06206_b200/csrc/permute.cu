@@ -1,0 +1,136 @@
+// Dispatch maps of the FoE block: the local form of the token -> expert all-to-all.  Integer work:
+// per-expert counts, an exclusive scan, and a stable scatter (inside an expert, tokens ascend), so
+// the maps are a pure function of the routing decision -- no atomics decide an order.
+//
+//   counts[e]  = number of (token, cluster, j) selections of expert e
+//   offsets    = exclusive scan of counts over the global expert id
+//   perm[slot] = token of the slot,  inv[token, cluster, j] = slot
+//
+// Three launches: (1) every block of 256 tokens builds a token-bitmap per expert in shared memory,
+// from which each selection reads its rank inside the block; (2) one block scans block counts and
+// expert totals and writes the m-tile table the grouped GEMM walks; (3) every selection computes its
+// slot.  A fourth kernel moves activation rows into slot order with 16-byte vector copies.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace foe {
+
+constexpr int kPB = kPermuteBlockTokens;      // 256 tokens per block = 8 bitmap words per expert
+
+__global__ void __launch_bounds__(kPB)
+permute_count_kernel(const int* __restrict__ idx, int* __restrict__ rank, int* __restrict__ blk_counts, int n_tokens,
+                     int sel, int E, int* __restrict__ status) {
+  extern __shared__ uint32_t bm[];            // [E][8]
+  for (int q = threadIdx.x; q < E * 8; q += kPB) bm[q] = 0u;
+  __syncthreads();
+  const int t = threadIdx.x;
+  const int i = blockIdx.x * kPB + t;
+  if (i < n_tokens) {
+    for (int s = 0; s < sel; ++s) {
+      const int e = idx[size_t(i) * sel + s];
+      if (e < 0 || e >= E) { atomicExch(status, kStatusBounds); continue; }
+      atomicOr(&bm[e * 8 + (t >> 5)], 1u << (t & 31));
+    }
+  }
+  __syncthreads();
+  if (i < n_tokens) {
+    for (int s = 0; s < sel; ++s) {
+      const int e = idx[size_t(i) * sel + s];
+      int r = 0;
+      if (e >= 0 && e < E) {
+        const uint32_t* w = bm + e * 8;
+        for (int k = 0; k < (t >> 5); ++k) r += __popc(w[k]);
+        r += __popc(w[t >> 5] & ((1u << (t & 31)) - 1u));
+      }
+      rank[size_t(i) * sel + s] = r;
+    }
+  }
+  for (int e = threadIdx.x; e < E; e += kPB) {
+    int c = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) c += __popc(bm[e * 8 + k]);
+    blk_counts[size_t(blockIdx.x) * E + e] = c;
+  }
+}
+
+// Single block.  blk_counts[b][e] becomes the exclusive prefix over b; counts/offsets and the m-tile table
+// (group and first row of every tile_rows-row tile of every non-empty expert) are written.
+__global__ void __launch_bounds__(1024)
+permute_scan_kernel(int* __restrict__ blk_counts, int n_blocks, int E, int tile_rows, int* __restrict__ counts,
+                    int* __restrict__ offsets, int* __restrict__ mt_group, int* __restrict__ mt_row0,
+                    int* __restrict__ n_mtiles) {
+  __shared__ int s_a[1024], s_b[1024];
+  const int e = threadIdx.x;
+  int total = 0;
+  if (e < E) {
+    for (int b = 0; b < n_blocks; ++b) {
+      const int c = blk_counts[size_t(b) * E + e];
+      blk_counts[size_t(b) * E + e] = total;
+      total += c;
+    }
+    counts[e] = total;
+  }
+  const int tiles = (total + tile_rows - 1) / tile_rows;
+  // two inclusive Hillis-Steele scans over the expert id (rows and tiles)
+  s_a[e] = total;
+  s_b[e] = tiles;
+  __syncthreads();
+  for (int o = 1; o < 1024; o <<= 1) {
+    const int va = e >= o ? s_a[e - o] : 0;
+    const int vb = e >= o ? s_b[e - o] : 0;
+    __syncthreads();
+    s_a[e] += va;
+    s_b[e] += vb;
+    __syncthreads();
+  }
+  if (e < E) {
+    const int row0 = s_a[e] - total, tile0 = s_b[e] - tiles;
+    offsets[e] = row0;
+    if (e == E - 1) { offsets[E] = s_a[e]; *n_mtiles = s_b[e]; }
+    for (int j = 0; j < tiles; ++j) { mt_group[tile0 + j] = e; mt_row0[tile0 + j] = row0 + j * tile_rows; }
+  }
+}
+
+__global__ void permute_scatter_kernel(const int* __restrict__ idx, const int* __restrict__ rank,
+                                       const int* __restrict__ blk_prefix, const int* __restrict__ offsets,
+                                       int* __restrict__ perm, int* __restrict__ inv, int n_tokens, int sel, int E) {
+  const int q = blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= n_tokens * sel) return;
+  const int i = q / sel;
+  const int e = idx[q];
+  if (e < 0 || e >= E) { inv[q] = 0; return; }
+  const int slot = offsets[e] + blk_prefix[size_t(i / kPB) * E + e] + rank[q];
+  inv[q] = slot;
+  perm[slot] = i;
+}
+
+void launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int sel, int E, int tile_rows, int* status,
+                    cudaStream_t st) {
+  if (n_tokens <= 0) return;
+  const int n_blocks = (n_tokens + kPB - 1) / kPB;
+  permute_count_kernel<<<n_blocks, kPB, size_t(E) * 32, st>>>(idx, pb.rank, pb.blk_counts, n_tokens, sel, E, status);
+  permute_scan_kernel<<<1, 1024, 0, st>>>(pb.blk_counts, n_blocks, E, tile_rows, pb.counts, pb.offsets, pb.mt_group,
+                                          pb.mt_row0, pb.n_mtiles);
+  const int total = n_tokens * sel;
+  permute_scatter_kernel<<<(total + 255) / 256, 256, 0, st>>>(idx, pb.rank, pb.blk_counts, pb.offsets, pb.perm, pb.inv,
+                                                            n_tokens, sel, E);
+}
+
+// One warp per slot: u_perm[slot, :] = u[perm[slot], :], 16 bytes per lane per step.
+__global__ void gather_rows_kernel(const bf16* __restrict__ u, const int* __restrict__ perm, bf16* __restrict__ u_perm,
+                                   int n_rows, int d) {
+  const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (row >= n_rows) return;
+  const uint4* src = reinterpret_cast<const uint4*>(u + size_t(perm[row]) * d);
+  uint4* dst = reinterpret_cast<uint4*>(u_perm + size_t(row) * d);
+  for (int c = lane; c < d / 8; c += 32) dst[c] = __ldg(src + c);
+}
+
+void launch_gather_rows(const bf16* u, const int* perm, bf16* u_perm, int n_rows, int d, cudaStream_t st) {
+  if (n_rows <= 0) return;
+  const long long threads = (long long)n_rows * 32;
+  gather_rows_kernel<<<unsigned((threads + 255) / 256), 256, 0, st>>>(u, perm, u_perm, n_rows, d);
+}
+
+}  // namespace foe
