@@ -1,0 +1,393 @@
+#!/usr/bin/env python
+"""Benchmark of the FoE block forward pass on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload prefill|decode] [--impl ours|reference]
+
+A step is one pass of the whole block (every stage: norms, projections, attention, sync, routing,
+dispatch maps, experts, combine) over one batch of seeded synthetic input.  The default workload is the
+single-block prefill (hidden 2048, 16q/4kv heads, 4 clusters x 16 experts, top-2 per cluster, 4 x 4096
+tokens); the decode workload (64 sequences, contexts 4096..16384, paged KV) is measured in the same run and
+reported under "decode".  With N > 1 (torchrun) every rank runs an independent replica of the workload:
+the path has no sharding and no collective, so the aggregate is N x tokens / max-over-ranks time.
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2605_06206_b200 import synth  # noqa: E402
+
+
+# ----------------------------------------------------------------------------------------------
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            m = json.load(f)
+        return dict(hbm_gbs=float(m["hbm_gbs"]), bf16_tflops=float(m["bf16_tflops"]),
+                    bf16_tflops_sustained=float(m.get("bf16_tflops_sustained", m["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+# ----------------------------------------------------------------------------------------------
+def build_workload(kind: str, device, seed_offset: int = 0):
+    """Layer + inputs of the prefill (workload 2) or decode (workload 3) benchmark on `device`."""
+    from paper_2605_06206_b200 import binding
+    n = 2 if kind == "prefill" else 3
+    shape, info = synth.workload(n)
+    seed = info["seed"] + 1000 * seed_offset
+    W = synth.make_weights(shape, seed, device)
+    q_lens, ctx = info["q_lens"], info["context_lens"]
+    S = sum(q_lens)
+    x = synth.make_x(shape, seed, S, device)
+    kv = synth.make_paged_cache(shape, seed, ctx, q_lens, device)
+    layer = binding.FoeLayer(shape, W, max_tokens=S if kind == "prefill" else 1, max_seqs=len(q_lens),
+                             max_context=max(c + q for c, q in zip(ctx, q_lens)))
+    del W
+    torch.cuda.empty_cache()
+    return dict(kind=kind, shape=shape, info=info, layer=layer, x=x, kv=kv, S=S, n=n)
+
+
+def step_fn(wl):
+    layer, x, kv, S = wl["layer"], wl["x"], wl["kv"], wl["S"]
+    out = torch.empty_like(x) if wl["shape"].grouped_output == wl["shape"].grouped_input else None
+    mq = max(wl["info"]["q_lens"])
+    if wl["kind"] == "prefill":
+        return (lambda: layer.prefill(x, kv, n_tokens=S, max_q_len=mq, out=out)), out
+    return (lambda: layer.decode(x, kv, out=out)), out
+
+
+def timed_loop(fn, steps, warmup, dist_on):
+    import torch.distributed as dist
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if dist_on:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    if dist_on:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        ms = float(t.item())
+    return ms
+
+
+def stage_profile(wl, fn, steps):
+    """Average per-stage device time (ms) over `steps` calls with the library's stage events on."""
+    layer = wl["layer"]
+    layer.set_profiling(True)
+    acc = {}
+    for _ in range(steps):
+        fn()
+        for k, v in layer.stage_ms().items():
+            acc[k] = acc.get(k, 0.0) + v
+    layer.set_profiling(False)
+    return {k: v / steps for k, v in acc.items()}
+
+
+def algorithmic_work(wl):
+    """Flops / bytes the method itself must do for this call, from the actual routing of the last call."""
+    s, info, S = wl["shape"], wl["info"], wl["S"]
+    aux = wl["layer"].aux()
+    counts = aux["counts"].cpu()
+    touched = int((counts > 0).sum())
+    R = int(counts.sum())
+    d, I, dh = s.hidden, s.ffn_inter, s.head_dim
+    nq, nkv = s.n_q_heads, s.n_kv_heads
+    w = dict(rows=R, touched_experts=touched)
+    w["gemm1_flops"] = 2.0 * R * d * 2 * I
+    w["gemm2_flops"] = 2.0 * R * I * d
+    w["qkv_flops"] = 2.0 * S * d * (nq + 2 * nkv) * dh
+    w["oproj_flops"] = 2.0 * S * nq * dh * d
+    w["router_flops"] = 2.0 * S * d * s.n_experts
+    if wl["kind"] == "prefill":
+        w["attn_flops"] = sum(2.0 * (c + q) * q * dh * nq * 2 * 0.5 if c == 0 else 4.0 * q * (c + q / 2.0) * dh * nq
+                              for c, q in zip(info["context_lens"], info["q_lens"]))
+    else:
+        w["attn_flops"] = sum(4.0 * (c + 1) * dh * nq for c in info["context_lens"])
+    w["total_flops"] = sum(v for k, v in w.items() if k.endswith("_flops"))
+    # decode bytes: valid KV tokens, touched experts only, attention + router weights, activations in/out
+    kv_bytes = sum((c + 1) for c in info["context_lens"]) * nkv * dh * 2 * 2 if wl["kind"] == "decode" else 0
+    w["kv_bytes"] = kv_bytes
+    w["gemm1_weight_bytes"] = touched * 2 * I * d * 2
+    w["gemm2_weight_bytes"] = touched * I * d * 2
+    w["attn_weight_bytes"] = ((nq + 2 * nkv) * dh * d + nq * dh * d) * 2
+    w["router_bytes"] = s.n_experts * d * 4
+    H = s.n_clusters
+    w["act_bytes"] = (H * S * d * 2) * 2
+    w["total_bytes"] = (kv_bytes + w["gemm1_weight_bytes"] + w["gemm2_weight_bytes"] + w["attn_weight_bytes"] +
+                        w["router_bytes"] + w["act_bytes"])
+    return w
+
+
+def e2e_loop(wl, steps, warmup):
+    """Same call with HOST buffers: H2D of x from pinned memory, the block, D2H of the output."""
+    layer, kv, S = wl["layer"], wl["kv"], wl["S"]
+    x_host = wl["x"].cpu().pin_memory()
+    x_dev = torch.empty_like(wl["x"])
+    fn_dev, out_dev = step_fn(dict(wl, x=x_dev))
+    probe = fn_dev()
+    out_host = torch.empty(probe.shape, dtype=probe.dtype).pin_memory()
+    torch.cuda.synchronize()
+
+    def one():
+        x_dev.copy_(x_host, non_blocking=True)
+        o = fn_dev()
+        out_host.copy_(o, non_blocking=True)
+
+    for _ in range(warmup):
+        one()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return ms, x_host.numel() * 2, out_host.numel() * 2
+
+
+# ----------------------------------------------------------------------------------------------
+def oracle_sample(kind: str, n_tokens: int, seed: int = 0):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload.  Returns (seconds, tokens,
+    threads, description)."""
+    import numpy as np
+    from oracle import adapter, foe_oracle as orc
+    n = 2 if kind == "prefill" else 3
+    shape, info = synth.workload(n)
+    W = adapter.weights_to_numpy(synth.make_weights(shape, info["seed"]))
+    cfg = adapter.cfg_from_shape(shape)
+    threads = os.cpu_count() or 1
+    if kind == "prefill":
+        x = adapter.to_np(synth.make_x(shape, info["seed"] + seed, n_tokens))
+        t0 = time.perf_counter()
+        orc.foe_block(cfg, W, x, [n_tokens])
+        dt = time.perf_counter() - t0
+        return dt, n_tokens, threads, f"one sequence of {n_tokens} tokens, full block, workload-2 layer"
+    n_seqs = n_tokens
+    ctx = info["context_lens"][:n_seqs]
+    kv = synth.make_paged_cache(shape, info["seed"], ctx, [1] * n_seqs)
+    cache = adapter.logical_cache(kv.k_pages, kv.v_pages, kv.block_table, ctx, 64)
+    x = adapter.to_np(synth.make_x(shape, info["seed"] + seed, n_seqs))
+    t0 = time.perf_counter()
+    orc.foe_block(cfg, W, x, [1] * n_seqs, ctx, cache)
+    dt = time.perf_counter() - t0
+    return dt, n_seqs, threads, f"{n_seqs} of the 64 sequences, one decode step, workload-3 layer and contexts"
+
+
+def run_reference(args, rank):
+    """The reference arm: the CPU oracle on host cores, bounded sample per step."""
+    if rank != 0:
+        return
+    kind = args.workload
+    n_tok = 256 if kind == "prefill" else 8
+    for _ in range(args.warmup):
+        oracle_sample(kind, n_tok)
+    tot_s, tot_tok, thr, desc = 0.0, 0, 1, ""
+    for i in range(args.steps):
+        dt, ntk, thr, desc = oracle_sample(kind, n_tok, seed=i)
+        tot_s += dt
+        tot_tok += ntk
+    val = tot_tok / tot_s
+    unit = "tokens/s"
+    line = dict(impl="reference", metric=f"foe_block_{kind}_tokens_per_s", value=val, unit=unit, n_gpus=args.gpus,
+                steps=args.steps, warmup=args.warmup, ms_per_step=1e3 * tot_s / args.steps, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=f"workload {2 if kind == 'prefill' else 3} ({kind}), bounded sample: {desc}"),
+                cpu_baseline=dict(value=val, unit=unit, cores=thr, kind="oracle", sample=desc),
+                e2e=dict(value=val, unit=unit, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+def measure(kind, args, dist_on, rank, world, peaks, with_cpu):
+    dev = torch.device("cuda", torch.cuda.current_device())
+    wl = build_workload(kind, dev, seed_offset=rank)
+    fn, _ = step_fn(wl)
+    fn()
+    torch.cuda.synchronize()
+    st = wl["layer"].poll_status()
+    if st != 0:
+        raise RuntimeError(f"device status {st} after the first {kind} step")
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    ms_total = timed_loop(fn, args.steps, args.warmup, dist_on)
+    clocks = sampler.stop()
+    ms = ms_total / args.steps
+    launches = wl["layer"].last_launch_count()
+    stages = stage_profile(wl, fn, max(3, min(args.steps, 20)))
+    work = algorithmic_work(wl)
+    S = wl["S"]
+    res = dict(ms_per_step=ms, tokens_per_s=world * S / (ms * 1e-3), launches_per_step=launches, stages_ms=stages,
+               clocks=clocks, tokens_per_step=S)
+    if kind == "prefill":
+        t = stages["expert_gemm1_swiglu"] * 1e-3
+        ach = work["gemm1_flops"] / t / 1e12
+        peak = peaks["bf16_tflops_sustained"]
+        res["roofline"] = dict(bound="tensor", kernel="gemm_tcgen05_kernel<SwiGLU> (expert GEMM 1)", achieved=ach,
+                               peak=peak, unit="TFLOP/s", frac=ach / peak, traffic=None,
+                               peak_source=f"{peaks['source']} sustained bf16 (kernel timed inside the step)",
+                               frac_of_nominal_2250=ach / 2250.0,
+                               gemm2_tflops=work["gemm2_flops"] / (stages["expert_gemm2"] * 1e-3) / 1e12,
+                               whole_step_tflops=work["total_flops"] / (ms * 1e-3) / 1e12)
+    else:
+        t = stages["attention"] * 1e-3
+        ach = work["kv_bytes"] / t / 1e9
+        peak = peaks["hbm_gbs"]
+        g1 = work["gemm1_weight_bytes"] / (stages["expert_gemm1_swiglu"] * 1e-3) / 1e9
+        g2 = work["gemm2_weight_bytes"] / (stages["expert_gemm2"] * 1e-3) / 1e9
+        res["roofline"] = dict(bound="hbm", kernel="attn_decode_kernel (paged split-KV attention)", achieved=ach,
+                               peak=peak, unit="GB/s", frac=ach / peak, traffic=None,
+                               peak_source=f"{peaks['source']} copy bandwidth", frac_of_nominal_8000=ach / 8000.0,
+                               gemm1_gbs=g1, gemm2_gbs=g2,
+                               whole_step_gbs=work["total_bytes"] / (ms * 1e-3) / 1e9,
+                               whole_step_frac=work["total_bytes"] / (ms * 1e-3) / 1e9 / peak)
+    res["work"] = {k: v for k, v in work.items()}
+    e_ms, h2d, d2h = e2e_loop(wl, max(2, min(args.steps, 10)), 2)
+    res["e2e"] = dict(value=world * S / (e_ms * 1e-3), unit="tokens/s", ms_per_step=e_ms, h2d_bytes_per_step=h2d,
+                      d2h_bytes_per_step=d2h)
+    wl["layer"].close()
+    del wl
+    torch.cuda.empty_cache()
+    if with_cpu:
+        dt, ntk, thr, desc = oracle_sample(kind, 1024 if kind == "prefill" else 16)
+        res["cpu_baseline"] = dict(value=ntk / dt, unit="tokens/s", cores=thr, kind="oracle", sample=desc,
+                                   seconds=dt)
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", choices=["prefill", "decode"], default="prefill")
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the other workload's measurement")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the block has no CPU path)")
+    torch.cuda.set_device(local)
+    dist_on = world > 1
+    if dist_on:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = measured_peaks()
+
+    main_kind = args.workload
+    other = "decode" if main_kind == "prefill" else "prefill"
+    m = measure(main_kind, args, dist_on, rank, world, peaks, with_cpu=(rank == 0 and world == 1))
+    o = None if args.no_secondary else measure(other, args, dist_on, rank, world, peaks,
+                                               with_cpu=(rank == 0 and world == 1))
+    if rank == 0:
+        wl_n = 2 if main_kind == "prefill" else 3
+        line = dict(metric=f"foe_block_{main_kind}_tokens_per_s", value=m["tokens_per_s"], unit="tokens/s",
+                    n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=m["ms_per_step"],
+                    higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic",
+                    config=dict(workload=f"workload {wl_n}: single FoE block {main_kind}, hidden 2048, 16q/4kv heads, "
+                                         f"4 clusters x 16 experts top-2, inter 1024, "
+                                         + ("4 x 4096 tokens causal" if main_kind == "prefill" else
+                                            "64 sequences x 1 token, paged KV (page 64), contexts U[4096,16384]"),
+                                tokens_per_step=m["tokens_per_step"], replicas=world,
+                                l2="inputs larger than L2: weights 0.8 GB + activations/KV >= 0.5 GB per step"),
+                    clocks=m["clocks"], roofline=m["roofline"], e2e=m["e2e"],
+                    gpu_launches=m["launches_per_step"] * args.steps, stages_ms=m["stages_ms"])
+        if "cpu_baseline" in m:
+            line["cpu_baseline"] = m["cpu_baseline"]
+        if o is not None:
+            line[other] = dict(tokens_per_s=o["tokens_per_s"], ms_per_step=o["ms_per_step"], roofline=o["roofline"],
+                               e2e=o["e2e"], stages_ms=o["stages_ms"], clocks=o["clocks"],
+                               gpu_launches=o["launches_per_step"] * args.steps,
+                               cpu_baseline=o.get("cpu_baseline"))
+        print(json.dumps(line))
+    if dist_on:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
