@@ -338,6 +338,7 @@ def main():
     ap.add_argument("--workload", choices=["prefill", "decode"], default="prefill")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-secondary", action="store_true", help="skip the other workload's measurement")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle (profiler runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
@@ -360,9 +361,9 @@ def main():
 
     main_kind = args.workload
     other = "decode" if main_kind == "prefill" else "prefill"
-    m = measure(main_kind, args, dist_on, rank, world, peaks, with_cpu=(rank == 0 and world == 1))
+    m = measure(main_kind, args, dist_on, rank, world, peaks, with_cpu=(rank == 0 and world == 1 and not args.no_cpu_baseline))
     o = None if args.no_secondary else measure(other, args, dist_on, rank, world, peaks,
-                                               with_cpu=(rank == 0 and world == 1))
+                                               with_cpu=(rank == 0 and world == 1 and not args.no_cpu_baseline))
     if rank == 0:
         wl_n = 2 if main_kind == "prefill" else 3
         line = dict(metric=f"foe_block_{main_kind}_tokens_per_s", value=m["tokens_per_s"], unit="tokens/s",

@@ -405,9 +405,10 @@ foe_status foe_layer_create(const foe_config* cfg, const foe_weights* w, foe_lay
 }
 
 foe_status foe_prefill(foe_layer* L, const void* x, const foe_kv_cache* kv, void* out, void* stream) {
-  if (!L || !x || !kv || !out) return FOE_ERR_NULL;
+  if (!L || !kv) return FOE_ERR_NULL;
   if (kv->n_tokens < 0 || kv->n_seqs < 0) return FOE_ERR_SHAPE;
   if (kv->n_tokens == 0) { L->launches = 0; L->last_tokens = 0; return FOE_OK; }
+  if (!x || !out) return FOE_ERR_NULL;
   if (!kv->k_pages || !kv->v_pages || !kv->block_table || !kv->context_lens || !kv->q_lens) return FOE_ERR_NULL;
   if (kv->n_tokens > L->cfg.max_tokens || kv->n_seqs > L->cfg.max_seqs || kv->n_seqs == 0) return FOE_ERR_SHAPE;
   if (kv->max_q_len <= 0 || kv->max_q_len > kv->n_tokens || kv->max_pages_per_seq <= 0 || kv->num_pages <= 0)
@@ -417,9 +418,10 @@ foe_status foe_prefill(foe_layer* L, const void* x, const foe_kv_cache* kv, void
 }
 
 foe_status foe_decode(foe_layer* L, const void* x, const foe_kv_cache* kv, void* out, void* stream) {
-  if (!L || !x || !kv || !out) return FOE_ERR_NULL;
+  if (!L || !kv) return FOE_ERR_NULL;
   if (kv->n_seqs < 0) return FOE_ERR_SHAPE;
   if (kv->n_seqs == 0) { L->launches = 0; L->last_tokens = 0; return FOE_OK; }
+  if (!x || !out) return FOE_ERR_NULL;
   if (!kv->k_pages || !kv->v_pages || !kv->block_table || !kv->context_lens) return FOE_ERR_NULL;
   if (kv->n_seqs > L->cfg.max_seqs || kv->max_pages_per_seq <= 0 || kv->num_pages <= 0) return FOE_ERR_SHAPE;
   if (x == out) return FOE_ERR_UNSUPPORTED;

@@ -1,0 +1,255 @@
+"""GPU parity tests: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Small cases are compared element by element; the full-size workloads on sampled tokens."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import adapter
+from oracle import foe_oracle as orc
+from paper_2605_06206_b200 import binding, synth
+
+from parity import (assert_close, check_maps, check_routing, run_block_parity, scaled_weights)
+
+pytestmark = pytest.mark.gpu
+
+
+def shape_small(**kw):
+    base = dict(hidden=256, n_q_heads=8, n_kv_heads=4, n_clusters=4, head_dim=64, experts_per_cluster=8,
+                top_k_per_cluster=2, ffn_inter=128)
+    base.update(kw)
+    return synth.LayerShape(**base)
+
+
+# ------------------------------------------------------------------------------------------ routing
+@pytest.mark.parametrize("wl,n_tok,zipf", [(1, 128, False), (2, 3000, False), (4, 2500, True), (4, 64, True)])
+def test_route_bit_exact(wl, n_tok, zipf):
+    shape, info = synth.workload(wl)
+    dev = "cuda"
+    W = synth.make_weights(shape, info["seed"], dev)
+    if zipf:
+        W["router_b"] = synth.zipf_router_bias(shape, info["seed"], 1.0, 1.2, dead_per_cluster=2).to(dev)
+    h = synth.normal_bf16(info["seed"], 77, (n_tok, shape.hidden), 1.5, 0.0, dev)
+    layer = binding.FoeLayer(shape, W, max_tokens=n_tok, max_seqs=1, max_context=64)
+    idx, w = layer.route(h)
+    assert layer.poll_status() == 0
+    aux = layer.aux()
+    layer.close()
+    cfg = adapter.cfg_from_shape(shape)
+    Wn = {k: adapter.to_np(W[k]) for k in ("ffn_norm_g", "router_w", "router_b")}
+    rt = orc.route(cfg, Wn, adapter.to_np(h))
+    idx_g, w_g = idx.cpu().numpy(), w.cpu().numpy().astype(np.float64)
+    exempt = check_routing(shape, idx_g, w_g, rt["logits"], rt["idx"], rt["w"])
+    assert exempt <= max(2, n_tok // 200)
+    # list order: descending score inside every (token, cluster)
+    lg = np.take_along_axis(rt["logits"], idx_g.reshape(n_tok, -1).astype(np.int64), 1).reshape(idx_g.shape)
+    assert (np.diff(lg, axis=-1) <= 1e-5).all()
+    assert np.abs(adapter.to_np(aux["logits"]) - rt["logits"]).max() <= 2e-5 * max(1.0, np.abs(rt["logits"][rt["logits"] > -1e29]).max())
+    mp = check_maps(shape, aux, idx_g)
+    if zipf:
+        dead = adapter.to_np(W["router_b"]) < -1e29
+        assert dead.sum() == 2 * shape.n_clusters and (mp["counts"][dead] == 0).all()      # guaranteed-empty experts
+        live = mp["counts"][~dead]
+        assert live.max() > 4 * max(1, live.min())                                          # skewed load
+
+
+def test_route_is_deterministic():
+    shape, info = synth.workload(1)
+    W = synth.make_weights(shape, 0, "cuda")
+    h = synth.normal_bf16(0, 78, (500, shape.hidden), 1.0, 0.0, "cuda")
+    layer = binding.FoeLayer(shape, W, max_tokens=500, max_seqs=1, max_context=64)
+    a = layer.route(h)
+    auxa = layer.aux()
+    b = layer.route(h)
+    auxb = layer.aux()
+    layer.close()
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    for k in ("perm", "inv", "counts", "offsets"):
+        assert torch.equal(auxa[k], auxb[k])
+
+
+# ------------------------------------------------------------------------------------------ small blocks
+def test_workload1_prefill_elementwise():
+    shape, info = synth.workload(1)
+    r = run_block_parity(shape, info["seed"], info["q_lens"], info["context_lens"])
+    assert r["launches"] > 0
+
+
+@pytest.mark.parametrize("position,sync", [("middle", "mean"), ("middle", "sum"), ("first", "mean"),
+                                           ("last", "mean"), ("single", "mean"), ("last", "sum")])
+def test_positions_and_sync_modes(position, sync):
+    shape = shape_small(position=position, sync=sync)
+    run_block_parity(shape, 11, [100, 29, 1, 200], [0, 0, 0, 0], wscale=4.0)
+
+
+def test_one_cluster_baseline_and_wide_topk():
+    shape = shape_small(n_clusters=1, experts_per_cluster=32, top_k_per_cluster=8)
+    run_block_parity(shape, 12, [150, 70], [0, 0], wscale=4.0)
+    shape = shape_small(n_clusters=2, n_kv_heads=4, experts_per_cluster=128, top_k_per_cluster=16)
+    run_block_parity(shape, 13, [90], [0], wscale=4.0)
+
+
+def test_head_dim_128_and_ragged_tiles():
+    shape = synth.LayerShape(512, 8, 2, 2, 128, 4, 2, 256)
+    run_block_parity(shape, 14, [130, 300, 63, 65], [0, 0, 0, 0], wscale=4.0)       # several 128-row tiles + tails
+
+
+def test_chunked_prefill_over_cached_context():
+    shape = shape_small()
+    run_block_parity(shape, 15, [40, 17, 130], [100, 64, 1], wscale=4.0)
+
+
+def test_empty_and_single_token_calls():
+    shape = shape_small()
+    W = synth.make_weights(shape, 16, "cuda")
+    layer = binding.FoeLayer(shape, W, max_tokens=8, max_seqs=2, max_context=128)
+    kv = synth.make_paged_cache(shape, 16, [0], [0], "cuda")
+    x = torch.empty((4, 0, 256), dtype=torch.bfloat16, device="cuda")
+    out = layer.prefill(x, kv, n_tokens=0, max_q_len=0)
+    assert out.shape == (4, 0, 256) and layer.last_launch_count() == 0
+    layer.close()
+    run_block_parity(shape, 16, [1], [0], wscale=4.0)
+
+
+def test_skewed_router_bias_small():
+    shape = shape_small(experts_per_cluster=16, top_k_per_cluster=4)
+    bias = synth.zipf_router_bias(shape, 17, 1.0, 1.2, dead_per_cluster=3)
+    r = run_block_parity(shape, 17, [300, 212], [0, 0], wscale=4.0, router_bias=bias)
+    assert (r["counts"] == 0).sum() >= 12                                         # dead experts stay empty
+
+
+# ------------------------------------------------------------------------------------------ decode
+def test_decode_small_elementwise():
+    shape = shape_small()
+    run_block_parity(shape, 21, [1] * 7, [0, 1, 63, 64, 65, 200, 1500], decode=True, wscale=4.0)
+
+
+def test_decode_head_dim_128_many_splits():
+    shape = synth.LayerShape(512, 8, 2, 2, 128, 4, 2, 256)
+    run_block_parity(shape, 22, [1] * 4, [10, 1030, 2100, 5000], decode=True, wscale=4.0)
+
+
+@pytest.mark.parametrize("position", ["first", "last"])
+def test_decode_boundary_layers(position):
+    shape = shape_small(position=position)
+    run_block_parity(shape, 23, [1] * 3, [5, 70, 300], decode=True, wscale=4.0)
+
+
+def test_physical_page_order_does_not_matter():
+    shape = shape_small()
+    a = run_block_parity(shape, 24, [1] * 3, [100, 257, 640], decode=True, wscale=4.0, shuffle_pages=True,
+                         return_all=True)
+    # same logical cache laid out in identity page order
+    kv_a = a["kv"]
+    ctx = [100, 257, 640]
+    kv_b = synth.make_paged_cache(shape, 24, ctx, [1] * 3, "cuda", fill_random=False, shuffle=False)
+    for s in range(3):
+        npg = (ctx[s] + 1 + 63) // 64
+        kv_b.k_pages[kv_b.block_table[s, :npg].long()] = kv_a.k_pages[kv_a.block_table[s, :npg].long()]
+        kv_b.v_pages[kv_b.block_table[s, :npg].long()] = kv_a.v_pages[kv_a.block_table[s, :npg].long()]
+    layer = binding.FoeLayer(shape, a["W"], max_tokens=1, max_seqs=3, max_context=700)
+    out_b = layer.decode(a["x"], kv_b)
+    assert layer.poll_status() == 0
+    layer.close()
+    assert torch.equal(out_b, a["out"])                                            # bit-identical
+
+
+def test_prefill_then_decode_matches_longer_prefill():
+    shape = shape_small()
+    T = 150
+    W = scaled_weights(shape, 25, "cuda", 4.0)
+    x = synth.make_x(shape, 25, T + 1, "cuda")
+    kv = synth.make_paged_cache(shape, 25, [0], [T + 1], "cuda", fill_random=False)
+    layer = binding.FoeLayer(shape, W, max_tokens=T + 1, max_seqs=1, max_context=T + 1)
+    full = layer.prefill(x, kv)
+    kv2 = synth.make_paged_cache(shape, 25, [0], [T + 1], "cuda", fill_random=False)
+    kv2.q_lens = torch.tensor([T], dtype=torch.int32, device="cuda")
+    layer.prefill(x[:, :T].contiguous(), kv2)
+    kv2.context_lens = torch.tensor([T], dtype=torch.int32, device="cuda")
+    step = layer.decode(x[:, T:].contiguous(), kv2)
+    assert layer.poll_status() == 0
+    layer.close()
+    assert_close(adapter.to_np(step[:, 0]), adapter.to_np(full[:, T]).astype(np.float64), "decode vs prefill row")
+    # the first T tokens went through the same kernels; the last one through the decode projection
+    assert_close(adapter.to_np(kv2.k_pages), adapter.to_np(kv.k_pages).astype(np.float64), "K pages", 1e-2, 1e-3)
+    assert_close(adapter.to_np(kv2.v_pages), adapter.to_np(kv.v_pages).astype(np.float64), "V pages", 1e-2, 1e-3)
+
+
+def test_same_inputs_give_bit_identical_outputs():
+    shape = shape_small()
+    W = scaled_weights(shape, 26, "cuda", 4.0)
+    x = synth.make_x(shape, 26, 333, "cuda")
+    layer = binding.FoeLayer(shape, W, max_tokens=333, max_seqs=2, max_context=256)
+    outs = []
+    for _ in range(2):
+        kv = synth.make_paged_cache(shape, 26, [0, 0], [200, 133], "cuda", fill_random=False)
+        outs.append(layer.prefill(x, kv).clone())
+    layer.close()
+    assert torch.equal(outs[0], outs[1])
+
+
+# ------------------------------------------------------------------------------------------ error paths (host side)
+def test_host_side_argument_errors():
+    shape = shape_small()
+    W = synth.make_weights(shape, 27, "cuda")
+    bad = shape_small(head_dim=32)
+    with pytest.raises(binding.FoeError) as e:
+        binding.FoeLayer(bad, W, 8, 1, 64)
+    assert e.value.code == -2
+    layer = binding.FoeLayer(shape, W, max_tokens=8, max_seqs=1, max_context=64)
+    kv = synth.make_paged_cache(shape, 27, [0], [16], "cuda")
+    x = synth.make_x(shape, 27, 16, "cuda")
+    with pytest.raises(binding.FoeError) as e:
+        layer.prefill(x, kv)                                                       # 16 tokens > max_tokens
+    assert e.value.code == -3
+    # a block-table entry outside the pool is reported through the device status word, nothing faults
+    kv = synth.make_paged_cache(shape, 27, [0], [8], "cuda")
+    kv.block_table[0, 0] = 10_000
+    layer.prefill(synth.make_x(shape, 27, 8, "cuda"), kv)
+    assert layer.poll_status() == -8
+    assert layer.poll_status() == 0
+    layer.close()
+
+
+# ------------------------------------------------------------------------------------------ full-size workloads
+def _sample_rows(q_lens, per_seq, seed):
+    rows, at = [], 0
+    for b, T in enumerate(q_lens):
+        pick = synth.uniform_int(seed, 500 + b, per_seq, 0, T - 1).tolist()
+        pick += [0, T - 1, 63, 64, 127, 128]
+        rows += sorted({at + p for p in pick if p < T})
+        at += T
+    return np.array(rows, dtype=np.int64)
+
+
+def test_workload2_full_size_prefill_sampled():
+    shape, info = synth.workload(2)
+    rows = _sample_rows(info["q_lens"], 40, 2)
+    r = run_block_parity(shape, info["seed"], info["q_lens"], info["context_lens"], rows=rows)
+    print("workload 2:", {k: r[k] for k in ("max_abs", "rel_l1", "flips", "launches")})
+    c = r["counts"]
+    assert c.min() > 1500 and c.max() < 2700                                       # near-uniform load, ~2048 rows/expert
+
+
+def test_workload3_full_size_decode_all_tokens():
+    shape, info = synth.workload(3)
+    r = run_block_parity(shape, info["seed"], info["q_lens"], info["context_lens"], decode=True)
+    print("workload 3:", {k: r[k] for k in ("max_abs", "rel_l1", "flips", "launches")})
+
+
+def test_workload4_skewed_routing_sampled():
+    shape, info = synth.workload(4)
+    dev = "cuda"
+    W = synth.make_weights(shape, info["seed"], dev)
+    # spread of the unbiased scores, measured with the library on a sample, sets the bias scale
+    h = synth.normal_bf16(info["seed"], 79, (2048, shape.hidden), 1.0, 0.0, dev)
+    layer = binding.FoeLayer(shape, W, max_tokens=2048, max_seqs=1, max_context=64)
+    layer.route(h)
+    sigma = float(layer.aux()["logits"].std())
+    layer.close()
+    bias = synth.zipf_router_bias(shape, info["seed"], sigma, info["zipf"], dead_per_cluster=2)
+    rows = _sample_rows(info["q_lens"], 12, 4)
+    r = run_block_parity(shape, info["seed"], info["q_lens"], info["context_lens"], rows=rows, router_bias=bias,
+                         weights=W)
+    c = r["counts"].reshape(shape.n_clusters, shape.experts_per_cluster)
+    print("workload 4:", {k: r[k] for k in ("max_abs", "rel_l1", "flips")}, "max/mean rows", c.max() / c.mean())
+    assert (c == 0).sum() >= 2 * shape.n_clusters and c.max() > 3 * c.mean()       # empty and overfull experts
