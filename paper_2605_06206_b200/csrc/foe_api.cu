@@ -60,13 +60,14 @@ struct foe_layer {
   float *router_w, *router_b;
   float2* rope_tab;
   // workspace
-  float *inv_rms, *r_full, *logits, *topk_w, *part_o, *part_ml;
+  float *inv_rms, *inv_rms_f, *route_part, *r_full, *logits, *topk_w, *part_o, *part_ml;
   bf16 *qkv, *attn_o, *u, *u_perm, *hmid, *y;
   int *topk_idx, *cu_q, *tok_seq, *tok_pos, *tok_slot, *status;
   PermuteBuffers pb;
   int max_splits, pages_per_split;
   // static tensor maps
   CUtensorMap tm_wqkv, tm_attn_o, tm_wo, tm_uperm, tm_wgu, tm_hmid, tm_wd;
+  CUtensorMap tms_wqkv, tms_wo, tms_wgu, tms_wd;   // same weights, boxes sized for the decode kernels
   // call state
   cudaStream_t last_stream;
   int last_tokens, launches;
@@ -97,7 +98,8 @@ foe_status validate(const foe_config* c) {
     return FOE_ERR_CONFIG;
   if (c->n_clusters * c->experts_per_cluster > 1024) return FOE_ERR_CONFIG;
   if (c->page_size != 64) return FOE_ERR_CONFIG;
-  if (c->hidden % 64 || c->ffn_inter % 128 || c->ffn_inter <= 0) return FOE_ERR_CONFIG;
+  if (c->hidden % 128 || c->ffn_inter % 128 || c->ffn_inter <= 0) return FOE_ERR_CONFIG;
+  if ((c->n_q_heads * c->head_dim) % 128) return FOE_ERR_CONFIG;
   if (c->max_tokens <= 0 || c->max_seqs <= 0 || c->max_context <= 0) return FOE_ERR_CONFIG;
   if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f)) return FOE_ERR_CONFIG;
   if (c->position < 0 || c->position > 3 || c->sync < 0 || c->sync > 1) return FOE_ERR_CONFIG;
@@ -112,9 +114,8 @@ foe_status check_launch() { return cudaGetLastError() == cudaSuccess ? FOE_OK : 
 
 // routing + dispatch maps for n tokens whose synced residual is r (fp32 internal or bf16 from the caller)
 void run_route_and_permute(foe_layer* L, const void* r, int r_is_bf16, int n, cudaStream_t st) {
-  launch_route(r, r_is_bf16, L->ffn_gain, L->router_w, L->router_b, L->u, L->logits, L->topk_idx, L->topk_w, n, L->d,
-               L->H, L->Ec, L->kc, L->cfg.rms_eps, st);
-  L->launches += 1;
+  L->launches += launch_route(r, r_is_bf16, L->ffn_gain, L->router_w, L->router_b, L->u, L->inv_rms_f, L->route_part,
+                              L->logits, L->topk_idx, L->topk_w, n, L->d, L->H, L->Ec, L->kc, L->cfg.rms_eps, L->n_sms, st);
   stage_mark(L, kStPermute, st);
   launch_permute(L->topk_idx, L->pb, n, L->H * L->kc, L->E, 128, L->status, st);
   L->launches += 3;
@@ -162,7 +163,8 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     sa.N = (L->g + 2 * L->c) * dh; sa.K = d; sa.epi = kEpiQKV; sa.out = L->qkv; sa.ldo = L->qkv_cols;
     sa.row_scale = L->inv_rms; sa.scale_group_stride = L->first ? 0 : S;
     sa.q_cols = L->g * dh; sa.kv_cols = L->c * dh; sa.q_total = L->n_q * dh; sa.kv_total = L->n_kv * dh;
-    launch_smallm(sa, st);
+    sa.status = L->status;
+    launch_smallm(L->tms_wqkv, sa, st);
   }
   L->launches += 1;
 
@@ -200,8 +202,8 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     memset(&sa, 0, sizeof(sa));
     sa.W = L->wo_t; sa.X = L->attn_o; sa.ldx = L->n_q * dh; sa.n_groups = 1; sa.rows_per_group = S; sa.N = d;
     sa.K = L->n_q * dh; sa.epi = kEpiOProj; sa.out = L->r_full; sa.ldo = d; sa.xsum = xb; sa.x_count = L->first ? 1 : H;
-    sa.x_stride = size_t(S) * d; sa.out_scale = out_scale;
-    launch_smallm(sa, st);
+    sa.x_stride = size_t(S) * d; sa.out_scale = out_scale; sa.status = L->status;
+    launch_smallm(L->tms_wo, sa, st);
   }
   L->launches += 1;
 
@@ -230,13 +232,15 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     memset(&s1, 0, sizeof(s1));
     s1.W = L->wgu_t; s1.X = L->u; s1.ldx = d; s1.row_index = L->pb.perm; s1.group_offsets = L->pb.offsets;
     s1.n_groups = L->E; s1.N = 2 * L->I; s1.K = d; s1.epi = kEpiSwiGLU; s1.out = L->hmid; s1.ldo = L->I;
-    launch_smallm(s1, st);
+    s1.status = L->status;
+    launch_smallm(L->tms_wgu, s1, st);
     stage_mark(L, kStGemm2, st);
     SmallMArgs s2;
     memset(&s2, 0, sizeof(s2));
     s2.W = L->wd_t; s2.X = L->hmid; s2.ldx = L->I; s2.group_offsets = L->pb.offsets; s2.n_groups = L->E; s2.N = d;
     s2.K = L->I; s2.epi = kEpiBf16; s2.out = L->y; s2.ldo = d;
-    launch_smallm(s2, st);
+    s2.status = L->status;
+    launch_smallm(L->tms_wd, s2, st);
     L->launches += 2;
   }
 
@@ -323,6 +327,8 @@ foe_status foe_layer_create(const foe_config* cfg, const foe_weights* w, foe_lay
   ok = ok && dalloc(L, &L->inv_rms, size_t(H) * S);
   ok = ok && dalloc(L, &L->r_full, size_t(S) * d);
   ok = ok && dalloc(L, &L->logits, size_t(S) * E);
+  ok = ok && dalloc(L, &L->inv_rms_f, size_t(S));
+  ok = ok && dalloc(L, &L->route_part, size_t(S) * E > (size_t(1) << 21) ? size_t(S) * E : (size_t(1) << 21));
   ok = ok && dalloc(L, &L->topk_w, size_t(R));
   ok = ok && dalloc(L, &L->topk_idx, size_t(R));
   ok = ok && dalloc(L, &L->qkv, size_t(S) * L->qkv_cols);
@@ -397,7 +403,11 @@ foe_status foe_layer_create(const foe_config* cfg, const foe_weights* w, foe_lay
        make_map_2d(&L->tm_uperm, L->u_perm, uint64_t(R), d, kBM) &&
        make_map_2d(&L->tm_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, kBN) &&
        make_map_2d(&L->tm_hmid, L->hmid, uint64_t(R), I, kBM) &&
-       make_map_2d(&L->tm_wd, L->wd_t, uint64_t(E) * d, I, kBN);
+       make_map_2d(&L->tm_wd, L->wd_t, uint64_t(E) * d, I, kBN) &&
+       make_map_2d(&L->tms_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, 64) &&
+       make_map_2d(&L->tms_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, 64) &&
+       make_map_2d(&L->tms_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, 32) &&
+       make_map_2d(&L->tms_wd, L->wd_t, uint64_t(E) * d, I, 64);
   if (!ok) { foe_layer_destroy(L); return FOE_ERR_CUDA; }
   for (int i = 0; i <= kNumStages; ++i) cudaEventCreate(&L->ev[i]);
   *out = L;

@@ -32,9 +32,11 @@ void launch_pack_gate_up(const bf16* wg, const bf16* wu, bf16* dst, int E, int d
 
 // ---- route.cu
 // FFN norm + fp32 router + per-cluster top-k + gates.  r_in is fp32 or bf16 [S][d].
-void launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const float* br, bf16* u_out,
-                  float* logits, int* idx, float* w, int n_tokens, int d, int H, int Ec, int kc, float eps,
-                  cudaStream_t st);
+// Returns the number of kernels launched.  inv_rms: [S] scratch; part: scratch for the split-K partial scores
+// (at least max(S*E, 2^21) floats).
+int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const float* br, bf16* u_out,
+                 float* inv_rms, float* part, float* logits, int* idx, float* w, int n_tokens, int d, int H, int Ec,
+                 int kc, float eps, int n_sms, cudaStream_t st);
 
 // ---- permute.cu
 struct PermuteBuffers {
@@ -97,7 +99,9 @@ struct SmallMArgs {
   const float* row_scale; int scale_group_stride;
   int q_cols, kv_cols, q_total, kv_total;
   const bf16* xsum; int x_count; size_t x_stride; float out_scale;
+  int* status;
 };
-void launch_smallm(const SmallMArgs& a, cudaStream_t st);
+// tmW: tensor map of W as [n_groups*N][K] with 64-column boxes of 64 rows (32 rows for the SwiGLU packing)
+void launch_smallm(const CUtensorMap& tmW, const SmallMArgs& a, cudaStream_t st);
 
 }  // namespace foe

@@ -2,6 +2,16 @@
 // per-cluster top-k inside the cluster's contiguous expert block, gates = softmax over the selected
 // scores.  Everything on this path is fp32 on the plain ALUs: the decision it takes (which experts)
 // is an integer result that must agree with a float32 reference, so no reduced-precision tensor path.
+//
+// Three kernels:
+//  1. ffn_norm:     one warp per token: inv_rms and the bf16 expert input u = r * inv_rms * gain.
+//  2. router_gemm:  SIMT fp32 GEMM, 32 tokens x 64 experts per CTA, 4 x 4 register tiles, k-major shared
+//                   tiles, register-staged double buffering; the normalisation is applied while the token
+//                   tile is loaded (u is never rounded to bf16 on this path).  For a handful of tokens the
+//                   reduction dimension is split over gridDim.z so that the grid still fills the GPU; the
+//                   partial scores are summed in a fixed order by kernel 3.
+//  3. topk_gates:   one warp per (token, cluster): bias, top-k by (score descending, expert id ascending),
+//                   softmax over the selected scores.
 #include <float.h>
 
 #include "common.cuh"
@@ -9,196 +19,236 @@
 
 namespace foe {
 
-constexpr int kRouteThreads = 256;
-
-template <int TOK>
-__global__ void __launch_bounds__(kRouteThreads)
-route_kernel(const void* __restrict__ r_in, int r_is_bf16, const bf16* __restrict__ gain,
-             const float* __restrict__ wr, const float* __restrict__ br, bf16* __restrict__ u_out,
-             float* __restrict__ logits_out, int* __restrict__ idx_out, float* __restrict__ w_out, int n_tokens,
-             int d, int H, int Ec, int kc, float eps) {
-  extern __shared__ float smem_f[];
-  float* u_s = smem_f;                       // [TOK][d]
-  float* lg_s = u_s + size_t(TOK) * d;       // [TOK][E]
-  const int E = H * Ec;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_warps = kRouteThreads / 32;
-  const int tok0 = blockIdx.x * TOK;
-
-  // ---- 1. FFN norm: u = r * rsqrt(mean r^2 + eps) * gain   (fp32, kept in shared memory)
-  for (int t = warp; t < TOK; t += n_warps) {
-    const int i = tok0 + t;
-    float* urow = u_s + size_t(t) * d;
-    if (i >= n_tokens) {
-      for (int c = lane; c < d; c += 32) urow[c] = 0.f;
-      continue;
-    }
-    float ss = 0.f;
-    if (r_is_bf16) {
-      const uint4* row = reinterpret_cast<const uint4*>(static_cast<const bf16*>(r_in) + size_t(i) * d);
-      for (int c = lane; c < d / 8; c += 32) {
-        const uint4 q = __ldg(row + c);
-        const uint32_t v[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float a = bf16_lo(v[j]), b = bf16_hi(v[j]);
-          urow[c * 8 + 2 * j] = a;
-          urow[c * 8 + 2 * j + 1] = b;
-          ss += a * a + b * b;
-        }
-      }
-    } else {
-      const float4* row = reinterpret_cast<const float4*>(static_cast<const float*>(r_in) + size_t(i) * d);
-      for (int c = lane; c < d / 4; c += 32) {
-        const float4 q = __ldg(row + c);
-        *reinterpret_cast<float4*>(urow + c * 4) = q;
-        ss += q.x * q.x + q.y * q.y + q.z * q.z + q.w * q.w;
-      }
-    }
-    ss = warp_sum(ss);
-    const float inv = rsqrtf(ss / float(d) + eps);
-    __syncwarp();
+// ------------------------------------------------------------------------------------------------ 1
+__global__ void ffn_norm_kernel(const void* __restrict__ r_in, int r_is_bf16, const bf16* __restrict__ gain,
+                                bf16* __restrict__ u_out, float* __restrict__ inv_out, int n_tokens, int d,
+                                float eps) {
+  const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (i >= n_tokens) return;
+  float ss = 0.f;
+  if (r_is_bf16) {
+    const uint4* row = reinterpret_cast<const uint4*>(static_cast<const bf16*>(r_in) + size_t(i) * d);
     for (int c = lane; c < d / 8; c += 32) {
-      const uint4 gq = __ldg(reinterpret_cast<const uint4*>(gain) + c);
-      const uint32_t g[4] = {gq.x, gq.y, gq.z, gq.w};
-      float v[8];
+      const uint4 q = __ldg(row + c);
+      const uint32_t v[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        v[2 * j] = urow[c * 8 + 2 * j] * inv * bf16_lo(g[j]);
-        v[2 * j + 1] = urow[c * 8 + 2 * j + 1] * inv * bf16_hi(g[j]);
-      }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) urow[c * 8 + j] = v[j];
-      if (u_out)
-        *reinterpret_cast<uint4*>(u_out + size_t(i) * d + c * 8) =
-            make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+      for (int j = 0; j < 4; ++j) { const float a = bf16_lo(v[j]), b = bf16_hi(v[j]); ss += a * a + b * b; }
+    }
+  } else {
+    const float4* row = reinterpret_cast<const float4*>(static_cast<const float*>(r_in) + size_t(i) * d);
+    for (int c = lane; c < d / 4; c += 32) {
+      const float4 q = __ldg(row + c);
+      ss += q.x * q.x + q.y * q.y + q.z * q.z + q.w * q.w;
     }
   }
-  __syncthreads();
+  ss = warp_sum(ss);
+  const float inv = rsqrtf(ss / float(d) + eps);
+  if (lane == 0) inv_out[i] = inv;
+  for (int c = lane; c < d / 8; c += 32) {
+    float v[8];
+    if (r_is_bf16) {
+      const uint4 q = __ldg(reinterpret_cast<const uint4*>(static_cast<const bf16*>(r_in) + size_t(i) * d) + c);
+      const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { v[2 * j] = bf16_lo(w[j]); v[2 * j + 1] = bf16_hi(w[j]); }
+    } else {
+      const float4* row = reinterpret_cast<const float4*>(static_cast<const float*>(r_in) + size_t(i) * d);
+      const float4 a = __ldg(row + 2 * c), b = __ldg(row + 2 * c + 1);
+      v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    }
+    const uint4 gq = __ldg(reinterpret_cast<const uint4*>(gain) + c);
+    const uint32_t g[4] = {gq.x, gq.y, gq.z, gq.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { v[2 * j] = v[2 * j] * inv * bf16_lo(g[j]); v[2 * j + 1] = v[2 * j + 1] * inv * bf16_hi(g[j]); }
+    *reinterpret_cast<uint4*>(u_out + size_t(i) * d + c * 8) =
+        make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+  }
+}
 
-  // ---- 2. scores: register tile of 4 experts x 4 tokens per warp task, K split over the lanes
-  const int e_groups = (E + 3) / 4, t_groups = TOK / 4;
-  for (int task = warp; task < e_groups * t_groups; task += n_warps) {
-    const int eg = task / t_groups, tg = task - eg * t_groups;
-    const float* wrow[4];
+// ------------------------------------------------------------------------------------------------ 2
+constexpr int kRgTM = 32, kRgTN = 64, kRgKC = 32, kRgThreads = 128;
+constexpr int kRgPA = kRgTM + 4, kRgPB = kRgTN + 4;      // padded pitches (floats), multiples of 4
+
+__global__ void __launch_bounds__(kRgThreads)
+router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __restrict__ inv_rms,
+                   const bf16* __restrict__ gain, const float* __restrict__ wr, float* __restrict__ part,
+                   int n_tokens, int d, int E, int k_per_split) {
+  __shared__ __align__(16) float As[2][kRgKC][kRgPA];     // [k][token]
+  __shared__ __align__(16) float Bs[2][kRgKC][kRgPB];     // [k][expert]
+  const int tid = threadIdx.x;
+  const int tok0 = blockIdx.x * kRgTM, exp0 = blockIdx.y * kRgTN;
+  const int kbeg = blockIdx.z * k_per_split, kend = min(d, kbeg + k_per_split);
+  const int ty = tid >> 4, tx = tid & 15;                 // 8 x 16 threads, 4 tokens x 4 experts each
+
+  // loader roles: A = 32 tokens x 8 float4 (2 per thread), B = 64 experts x 8 float4 (4 per thread)
+  const int la_k4 = tid & 7, la_t = tid >> 3;             // tokens la_t and la_t + 16
+  const int lb_k4 = tid & 7, lb_e = tid >> 3;             // experts lb_e + 16 * j
+  float inv_t[2];
 #pragma unroll
-    for (int a = 0; a < 4; ++a) wrow[a] = wr + size_t(min(eg * 4 + a, E - 1)) * d;
-    float acc[4][4];
+  for (int j = 0; j < 2; ++j) {
+    const int t = tok0 + la_t + 16 * j;
+    inv_t[j] = t < n_tokens ? inv_rms[t] : 0.f;
+  }
+  float4 ra[2], rb[4];
+
+  auto load_chunk = [&](int k0) {
+    const int k = k0 + la_k4 * 4;
+    float g4[4];
+    {
+      const uint2 gq = __ldg(reinterpret_cast<const uint2*>(gain + k));
+      g4[0] = bf16_lo(gq.x); g4[1] = bf16_hi(gq.x); g4[2] = bf16_lo(gq.y); g4[3] = bf16_hi(gq.y);
+    }
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+    for (int j = 0; j < 2; ++j) {
+      const int t = tok0 + la_t + 16 * j;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (t < n_tokens) {
+        if (r_is_bf16) {
+          const uint2 q = __ldg(reinterpret_cast<const uint2*>(static_cast<const bf16*>(r_in) + size_t(t) * d + k));
+          v = make_float4(bf16_lo(q.x), bf16_hi(q.x), bf16_lo(q.y), bf16_hi(q.y));
+        } else {
+          v = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(r_in) + size_t(t) * d + k));
+        }
+      }
+      ra[j] = make_float4(v.x * inv_t[j] * g4[0], v.y * inv_t[j] * g4[1], v.z * inv_t[j] * g4[2], v.w * inv_t[j] * g4[3]);
+    }
 #pragma unroll
-      for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
-    for (int k = lane * 4; k < d; k += 128) {
-      float4 wv[4], uv[4];
+    for (int j = 0; j < 4; ++j) {
+      const int e = min(exp0 + lb_e + 16 * j, E - 1);
+      rb[j] = __ldg(reinterpret_cast<const float4*>(wr + size_t(e) * d + k0 + lb_k4 * 4));
+    }
+  };
+  auto store_chunk = [&](int buf) {
 #pragma unroll
-      for (int a = 0; a < 4; ++a) wv[a] = __ldg(reinterpret_cast<const float4*>(wrow[a] + k));
+    for (int j = 0; j < 2; ++j) {
+      const int t = la_t + 16 * j;
+      As[buf][la_k4 * 4 + 0][t] = ra[j].x; As[buf][la_k4 * 4 + 1][t] = ra[j].y;
+      As[buf][la_k4 * 4 + 2][t] = ra[j].z; As[buf][la_k4 * 4 + 3][t] = ra[j].w;
+    }
 #pragma unroll
-      for (int b = 0; b < 4; ++b) uv[b] = *reinterpret_cast<const float4*>(u_s + size_t(tg * 4 + b) * d + k);
+    for (int j = 0; j < 4; ++j) {
+      const int e = lb_e + 16 * j;
+      Bs[buf][lb_k4 * 4 + 0][e] = rb[j].x; Bs[buf][lb_k4 * 4 + 1][e] = rb[j].y;
+      Bs[buf][lb_k4 * 4 + 2][e] = rb[j].z; Bs[buf][lb_k4 * 4 + 3][e] = rb[j].w;
+    }
+  };
+
+  float acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+
+  load_chunk(kbeg);
+  store_chunk(0);
+  __syncthreads();
+  int buf = 0;
+  for (int k0 = kbeg; k0 < kend; k0 += kRgKC) {
+    const bool more = k0 + kRgKC < kend;
+    if (more) load_chunk(k0 + kRgKC);
+#pragma unroll
+    for (int k = 0; k < kRgKC; ++k) {
+      const float4 av = *reinterpret_cast<const float4*>(&As[buf][k][ty * 4]);
+      const float4 bv = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 4]);
+      const float a4[4] = {av.x, av.y, av.z, av.w}, b4[4] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
       for (int a = 0; a < 4; ++a)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          acc[a][b] = fmaf(wv[a].x, uv[b].x, acc[a][b]);
-          acc[a][b] = fmaf(wv[a].y, uv[b].y, acc[a][b]);
-          acc[a][b] = fmaf(wv[a].z, uv[b].z, acc[a][b]);
-          acc[a][b] = fmaf(wv[a].w, uv[b].w, acc[a][b]);
-        }
+        for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(a4[a], b4[b], acc[a][b]);
     }
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-      for (int b = 0; b < 4; ++b) acc[a][b] = warp_sum(acc[a][b]);
-    if (lane < 16) {
-      const int a = lane >> 2, b = lane & 3;
-      const int e = eg * 4 + a, t = tg * 4 + b;
-      float v = 0.f;
-#pragma unroll
-      for (int aa = 0; aa < 4; ++aa)
-#pragma unroll
-        for (int bb = 0; bb < 4; ++bb)
-          if (aa == a && bb == b) v = acc[aa][bb];
-      if (e < E) {
-        if (br) v += __ldg(br + e);
-        lg_s[t * E + e] = v;
-        if (logits_out && tok0 + t < n_tokens) logits_out[size_t(tok0 + t) * E + e] = v;
-      }
-    }
+    if (more) store_chunk(buf ^ 1);
+    __syncthreads();
+    buf ^= 1;
   }
-  __syncthreads();
-
-  // ---- 3. per (token, cluster): top-k_c by (score descending, expert id ascending), then gates
-  for (int task = warp; task < TOK * H; task += n_warps) {
-    const int t = task / H, h = task - t * H;
-    const int i = tok0 + t;
-    if (i >= n_tokens) continue;
-    const float* lg = lg_s + t * E + h * Ec;
-    float cand[4];
-    bool taken[4];
+  float* dst = part + size_t(blockIdx.z) * n_tokens * E;
 #pragma unroll
-    for (int s = 0; s < 4; ++s) {
-      const int e = lane + 32 * s;
-      cand[s] = e < Ec ? lg[e] : -FLT_MAX;
-      taken[s] = e >= Ec;
-    }
-    float my_sel = -FLT_MAX;      // lane j keeps the j-th selected score
-    int my_idx = 0;
-    for (int j = 0; j < kc; ++j) {
-      float bv = -FLT_MAX;
-      int bi = 0x7fffffff;
+  for (int a = 0; a < 4; ++a) {
+    const int t = tok0 + ty * 4 + a;
+    if (t >= n_tokens) continue;
 #pragma unroll
-      for (int s = 0; s < 4; ++s) {
-        const int e = lane + 32 * s;
-        if (!taken[s] && (bi == 0x7fffffff || cand[s] > bv)) { bv = cand[s]; bi = e; }   // ascending e: first wins ties
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        if (oi != 0x7fffffff && (bi == 0x7fffffff || ov > bv || (ov == bv && oi < bi))) { bv = ov; bi = oi; }
-      }
-      if ((bi & 31) == lane) {
-#pragma unroll
-        for (int s = 0; s < 4; ++s)
-          if ((bi >> 5) == s) taken[s] = true;
-      }
-      if (lane == j) { my_sel = bv; my_idx = bi; }
-    }
-    const float m = __shfl_sync(0xffffffffu, my_sel, 0);
-    const float ex = lane < kc ? expf(my_sel - m) : 0.f;
-    const float sum = warp_sum(ex);
-    if (lane < kc) {
-      const size_t o = (size_t(i) * H + h) * kc + lane;
-      idx_out[o] = h * Ec + my_idx;
-      w_out[o] = ex / sum;
+    for (int b = 0; b < 4; ++b) {
+      const int e = exp0 + tx * 4 + b;
+      if (e < E) dst[size_t(t) * E + e] = acc[a][b];
     }
   }
 }
 
-void launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const float* br, bf16* u_out,
-                  float* logits, int* idx, float* w, int n_tokens, int d, int H, int Ec, int kc, float eps,
-                  cudaStream_t st) {
-  if (n_tokens <= 0) return;
+// ------------------------------------------------------------------------------------------------ 3
+__global__ void topk_gates_kernel(const float* __restrict__ part, int k_splits, const float* __restrict__ br,
+                                  float* __restrict__ logits_out, int* __restrict__ idx_out, float* __restrict__ w_out,
+                                  int n_tokens, int H, int Ec, int kc) {
+  const int task = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (task >= n_tokens * H) return;
+  const int i = task / H, h = task - i * H;
   const int E = H * Ec;
-  static bool configured = false;
-  if (!configured) {
-    cudaFuncSetAttribute(route_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    cudaFuncSetAttribute(route_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    cudaFuncSetAttribute(route_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    configured = true;
+  float cand[4];
+  bool taken[4];
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    const int e = lane + 32 * s;
+    float v = -FLT_MAX;
+    if (e < Ec) {
+      const size_t o = size_t(i) * E + h * Ec + e;
+      v = 0.f;
+      for (int z = 0; z < k_splits; ++z) v += part[size_t(z) * n_tokens * E + o];
+      if (br) v += __ldg(br + h * Ec + e);
+      logits_out[o] = v;
+    }
+    cand[s] = v;
+    taken[s] = e >= Ec;
   }
-  int tok = 16;
-  while (tok > 4 && size_t(tok) * (d + E) * 4 > 160 * 1024) tok >>= 1;
-  const size_t smem = size_t(tok) * (d + E) * 4;
-  const int blocks = (n_tokens + tok - 1) / tok;
-  if (tok == 16)
-    route_kernel<16><<<blocks, kRouteThreads, smem, st>>>(r_in, r_is_bf16, gain, wr, br, u_out, logits, idx, w,
-                                                         n_tokens, d, H, Ec, kc, eps);
-  else if (tok == 8)
-    route_kernel<8><<<blocks, kRouteThreads, smem, st>>>(r_in, r_is_bf16, gain, wr, br, u_out, logits, idx, w,
-                                                        n_tokens, d, H, Ec, kc, eps);
-  else
-    route_kernel<4><<<blocks, kRouteThreads, smem, st>>>(r_in, r_is_bf16, gain, wr, br, u_out, logits, idx, w,
-                                                        n_tokens, d, H, Ec, kc, eps);
+  float my_sel = -FLT_MAX;      // lane j keeps the j-th selected score
+  int my_idx = 0;
+  for (int j = 0; j < kc; ++j) {
+    float bv = -FLT_MAX;
+    int bi = 0x7fffffff;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      const int e = lane + 32 * s;
+      if (!taken[s] && (bi == 0x7fffffff || cand[s] > bv)) { bv = cand[s]; bi = e; }   // ascending e: first wins ties
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (oi != 0x7fffffff && (bi == 0x7fffffff || ov > bv || (ov == bv && oi < bi))) { bv = ov; bi = oi; }
+    }
+    if ((bi & 31) == lane) {
+#pragma unroll
+      for (int s = 0; s < 4; ++s)
+        if ((bi >> 5) == s) taken[s] = true;
+    }
+    if (lane == j) { my_sel = bv; my_idx = bi; }
+  }
+  const float m = __shfl_sync(0xffffffffu, my_sel, 0);
+  const float ex = lane < kc ? expf(my_sel - m) : 0.f;
+  const float sum = warp_sum(ex);
+  if (lane < kc) {
+    const size_t o = (size_t(i) * H + h) * kc + lane;
+    idx_out[o] = h * Ec + my_idx;
+    w_out[o] = ex / sum;
+  }
+}
+
+int route_k_splits(int n_tokens, int d, int E, int n_sms) {
+  const int ctas = ((n_tokens + kRgTM - 1) / kRgTM) * ((E + kRgTN - 1) / kRgTN);
+  int ks = 1;
+  while (ctas * ks < 2 * n_sms && ks < 16 && (d / (ks * 2)) % kRgKC == 0 && d / (ks * 2) >= 64) ks *= 2;
+  return ks;
+}
+
+int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const float* br, bf16* u_out,
+                 float* inv_rms, float* part, float* logits, int* idx, float* w, int n_tokens, int d, int H, int Ec,
+                 int kc, float eps, int n_sms, cudaStream_t st) {
+  if (n_tokens <= 0) return 0;
+  const int E = H * Ec;
+  ffn_norm_kernel<<<(n_tokens * 32 + 255) / 256, 256, 0, st>>>(r_in, r_is_bf16, gain, u_out, inv_rms, n_tokens, d, eps);
+  const int ks = route_k_splits(n_tokens, d, E, n_sms);
+  dim3 grid((n_tokens + kRgTM - 1) / kRgTM, (E + kRgTN - 1) / kRgTN, ks);
+  router_gemm_kernel<<<grid, kRgThreads, 0, st>>>(r_in, r_is_bf16, inv_rms, gain, wr, part, n_tokens, d, E, d / ks);
+  const int tasks = n_tokens * H;
+  topk_gates_kernel<<<(tasks * 32 + 255) / 256, 256, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc);
+  return 3;
 }
 
 }  // namespace foe
