@@ -26,7 +26,9 @@ constexpr int kBBytes = kBN * kBK * 2;   // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kGemmThreads = 192;
 constexpr int kTmemCols = 512;
-constexpr size_t kGemmSmemBytes = size_t(kStages) * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kStgPitch = 128 + 16;                 // staging row: 128 bytes of output + bank-spreading pad
+constexpr int kStgWarpBytes = 32 * kStgPitch;        // one epilogue warp stages its 32 rows
+constexpr size_t kGemmSmemBytes = size_t(kStages) * kStageBytes + 4 * kStgWarpBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 __device__ __forceinline__ float silu_f(float z) { return z / (1.0f + __expf(-z)); }
 
@@ -36,7 +38,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const GemmArgs args) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  uint8_t* stg_all = smem + kStages * kStageBytes;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(stg_all + 4 * kStgWarpBytes);
   uint64_t* empty_bar = full_bar + kStages;
   uint64_t* acc_full = empty_bar + kStages;
   uint64_t* acc_empty = acc_full + 2;
@@ -126,6 +129,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // ------------------------------------------------------------ epilogue (4 warps = 128 TMEM lanes)
     const int quarter = warp & 3;                 // a warp may only touch TMEM lanes 32*(warp%4)..+31
     const int row_in_tile = quarter * 32 + lane;
+    uint8_t* stg = stg_all + quarter * kStgWarpBytes;
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
@@ -148,95 +152,114 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kBN;
 
-      if constexpr (EPI == kEpiSwiGLU) {
-        __nv_bfloat16* out = static_cast<__nv_bfloat16*>(args.out);
+      // Every pass turns 128 bytes of output per row into registers (thread = accumulator row), parks them
+      // in the warp's staging tile and writes them out again with 8 lanes per row, so that global stores
+      // are whole 128-byte lines instead of 32 scattered 16-byte pieces.
+      const int row_local = row - group_row0;
+      float scale = 1.0f;
+      if constexpr (EPI == kEpiQKV) {
+        if (row_ok) scale = args.row_scale[size_t(group) * args.scale_group_stride + row_local];
+      }
+      constexpr int kPassCols = (EPI == kEpiOProj) ? 32 : 64;          // output columns per pass
+      constexpr int kTilePasses = (EPI == kEpiSwiGLU) ? 2 : kBN / kPassCols;
+      const int wr_row = lane >> 3, wr_chunk = lane & 7;                // write-out role: row (+4j), 16-byte chunk
 #pragma unroll 1
-        for (int ch = 0; ch < 4; ++ch) {
+      for (int ps = 0; ps < kTilePasses; ++ps) {
+        const int n = (EPI == kEpiSwiGLU) ? (n0 >> 1) + ps * 64 : n0 + ps * kPassCols;   // output column in the group
+        if (EPI != kEpiSwiGLU && n >= args.N) break;                    // warp-uniform
+        uint32_t w[32];                                                // 128 bytes of this row's output
+        __syncwarp();
+        if constexpr (EPI == kEpiSwiGLU) {
           uint32_t gt[32], up[32];
-          __syncwarp();
-          tmem_ld32(taddr + ch * 32, gt);
-          tmem_ld32(taddr + 128 + ch * 32, up);
-          tmem_ld_wait();
-          if (row_ok) {
-            uint4* dst = reinterpret_cast<uint4*>(out + size_t(row) * args.ldo + (n0 >> 1) + ch * 32);
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              uint32_t w[4];
+          for (int hf = 0; hf < 2; ++hf) {
+            tmem_ld32(taddr + ps * 64 + hf * 32, gt);
+            tmem_ld32(taddr + 128 + ps * 64 + hf * 32, up);
+            tmem_ld_wait();
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const int c = v * 8 + j * 2;
-                const float h0 = silu_f(__uint_as_float(gt[c])) * __uint_as_float(up[c]);
-                const float h1 = silu_f(__uint_as_float(gt[c + 1])) * __uint_as_float(up[c + 1]);
-                w[j] = pack_bf16(h0, h1);
-              }
-              dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+            for (int c = 0; c < 16; ++c) {
+              const float h0 = silu_f(__uint_as_float(gt[2 * c])) * __uint_as_float(up[2 * c]);
+              const float h1 = silu_f(__uint_as_float(gt[2 * c + 1])) * __uint_as_float(up[2 * c + 1]);
+              w[hf * 16 + c] = pack_bf16(h0, h1);
             }
           }
-        }
-      } else {
-        const int row_local = row - group_row0;
-        float scale = 1.0f;
-        if constexpr (EPI == kEpiQKV) {
-          if (row_ok) scale = args.row_scale[size_t(group) * args.scale_group_stride + row_local];
-        }
-#pragma unroll 1
-        for (int ch = 0; ch < kBN / 32; ++ch) {
-          const int n = n0 + ch * 32;
-          if (n >= args.N) break;                       // warp-uniform
-          uint32_t r[32];
-          __syncwarp();
-          tmem_ld32(taddr + ch * 32, r);
+        } else if constexpr (EPI == kEpiOProj) {
+          tmem_ld32(taddr + ps * 32, w);
           tmem_ld_wait();
-          if (row_ok) {
-          if constexpr (EPI == kEpiBf16 || EPI == kEpiQKV) {
-            int col = n;
-            int orow = row;
+        } else {
+          uint32_t r[32];
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            tmem_ld32(taddr + ps * 64 + hf * 32, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int c = 0; c < 16; ++c)
+              w[hf * 16 + c] = pack_bf16(__uint_as_float(r[2 * c]) * scale, __uint_as_float(r[2 * c + 1]) * scale);
+          }
+        }
+        if (ps == kTilePasses - 1 || (EPI != kEpiSwiGLU && n + kPassCols >= args.N)) {
+          // last read of this accumulator stage: hand it back to the MMA warp before the stores
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&acc_empty[acc]);
+        }
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          *reinterpret_cast<uint4*>(stg + lane * kStgPitch + c * 16) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+        __syncwarp();
+        if constexpr (EPI == kEpiOProj) {
+          // r_full = scale * (C + sum_h x[h]): the residual streams are read here, 8 lanes x 8 bytes per row
+          // and stream.  All loads of four rows are issued before the first use (the epilogue has to keep
+          // tens of KB in flight per SM: this GEMM moves almost as many bytes as it has flops to hide them).
+#pragma unroll
+          for (int jh = 0; jh < 2; ++jh) {
+            uint2 xq[4][8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int grow = row0 + quarter * 32 + wr_row + 4 * (jh * 4 + j);
+              const size_t off = size_t(grow) * args.ldo + n + wr_chunk * 4;
+#pragma unroll
+              for (int h = 0; h < 8; ++h) {
+                xq[j][h] = make_uint2(0u, 0u);
+                if (h < args.x_count && grow < row_end)
+                  xq[j][h] = __ldg(reinterpret_cast<const uint2*>(args.xsum + h * args.x_stride + off));
+              }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int rr = wr_row + 4 * (jh * 4 + j);
+              const int grow = row0 + quarter * 32 + rr;
+              if (grow >= row_end) continue;
+              const uint4 v = *reinterpret_cast<const uint4*>(stg + rr * kStgPitch + wr_chunk * 16);
+              float a4[4] = {__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w)};
+#pragma unroll
+              for (int h = 0; h < 8; ++h) {
+                a4[0] += bf16_lo(xq[j][h].x); a4[1] += bf16_hi(xq[j][h].x);
+                a4[2] += bf16_lo(xq[j][h].y); a4[3] += bf16_hi(xq[j][h].y);
+              }
+              *reinterpret_cast<float4*>(static_cast<float*>(args.out) + size_t(grow) * args.ldo + n + wr_chunk * 4) =
+                  make_float4(a4[0] * args.out_scale, a4[1] * args.out_scale, a4[2] * args.out_scale, a4[3] * args.out_scale);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int rr = wr_row + 4 * j;                              // row inside the warp's 32
+            const int grow = row0 + quarter * 32 + rr;
+            if (grow >= row_end) continue;
+            const uint4 v = *reinterpret_cast<const uint4*>(stg + rr * kStgPitch + wr_chunk * 16);
+            int col = n, orow = grow;
             if constexpr (EPI == kEpiQKV) {
-              orow = row_local;
+              orow = grow - group_row0;
               if (n < args.q_cols) col = group * args.q_cols + n;
               else if (n < args.q_cols + args.kv_cols) col = args.q_total + group * args.kv_cols + (n - args.q_cols);
               else col = args.q_total + args.kv_total + group * args.kv_cols + (n - args.q_cols - args.kv_cols);
             }
-            uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + size_t(orow) * args.ldo + col);
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              uint32_t w[4];
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const int c = v * 8 + j * 2;
-                w[j] = pack_bf16(__uint_as_float(r[c]) * scale, __uint_as_float(r[c + 1]) * scale);
-              }
-              dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-          } else {  // kEpiOProj
-            float acc32[32];
-#pragma unroll
-            for (int c = 0; c < 32; ++c) acc32[c] = __uint_as_float(r[c]);
-            for (int h = 0; h < args.x_count; ++h) {
-              const uint4* xs = reinterpret_cast<const uint4*>(args.xsum + h * args.x_stride + size_t(row) * args.ldo + n);
-#pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                const uint4 q = __ldg(xs + v);
-                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  acc32[v * 8 + j * 2] += bf16_lo(w[j]);
-                  acc32[v * 8 + j * 2 + 1] += bf16_hi(w[j]);
-                }
-              }
-            }
-            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(args.out) + size_t(row) * args.ldo + n);
-#pragma unroll
-            for (int v = 0; v < 8; ++v)
-              dst[v] = make_float4(acc32[v * 4] * args.out_scale, acc32[v * 4 + 1] * args.out_scale,
-                                   acc32[v * 4 + 2] * args.out_scale, acc32[v * 4 + 3] * args.out_scale);
-          }
+            *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + size_t(orow) * args.ldo + col + wr_chunk * 8) = v;
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&acc_empty[acc]);
+
     }
     if (!ok && lane == 0) atomicExch(args.status, kStatusTimeout);
   }
