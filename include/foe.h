@@ -146,6 +146,28 @@ foe_status foe_decode(foe_layer* layer, const void* x_step, const foe_kv_cache* 
  * topk_w: [n_tokens][H][k_c] fp32.  Also refreshes counts/offsets/perm/inv in the aux record. */
 foe_status foe_route(foe_layer* layer, const void* h, int n_tokens, int* topk_idx, float* topk_w, void* stream);
 
+/* The paper has no counterpart for this call; it exists for callers that cannot allocate device memory.
+ * Examples: a server that gave all GPU memory to its own pool at start-up, so that cudaMalloc has nothing
+ * left to hand out; a thread on a latency-critical path that must stay clear of the driver's allocator (its
+ * lock, and the device-wide synchronisation that comes with freeing).  Such callers cannot create a handle
+ * either, because foe_layer_create allocates.  foe_route_noalloc computes what foe_route computes -- FFN
+ * RMSNorm of h, fp32 router scores, per-cluster top-k and gates -- from plain arguments and never calls
+ * cudaMalloc, cudaFree or anything else that allocates.  Its scratch is a fixed array inside the library
+ * image (about 6 MB, present on every GPU that loads the library until the process exits).
+ *   ffn_norm_g [hidden] bf16, router_w [E][hidden] fp32, router_b [E] fp32 or NULL, h [n_tokens][hidden] bf16,
+ *   topk_idx / topk_w [n_tokens][n_clusters][top_k_per_cluster] (int32 global expert ids / fp32 gates): all
+ *   device pointers owned by the caller.  The dispatch maps and the expert input are not produced.
+ * Limits: n_tokens <= 8192 and n_tokens * n_clusters * experts_per_cluster <= 524288; larger calls return
+ * FOE_ERR_SHAPE and launch nothing.  Shape rules as for the layer description (FOE_ERR_CONFIG otherwise).
+ * The first call on each device looks up the device address of the scratch array (with that device current);
+ * make that first call before any stream capture begins.  Every call on a device uses the same scratch, which
+ * simply keeps the previous call's contents (nothing in it needs clearing: each call writes what it reads);
+ * two calls that overlap on the GPU -- different streams, or different host threads -- race on it, so run
+ * them one after the other. */
+foe_status foe_route_noalloc(int hidden, int n_clusters, int experts_per_cluster, int top_k_per_cluster, float rms_eps,
+                             const void* ffn_norm_g, const float* router_w, const float* router_b, const void* h,
+                             int n_tokens, int* topk_idx, float* topk_w, void* stream);
+
 /* Pointers to the last call's intermediates (host struct filled with device pointers). */
 foe_status foe_get_aux(foe_layer* layer, foe_aux* out);
 

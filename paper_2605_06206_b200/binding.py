@@ -21,7 +21,7 @@ SYNCS = {"mean": 0, "sum": 1}
 
 EXPORTS = ["foe_layer_create", "foe_layer_destroy", "foe_prefill", "foe_decode", "foe_route", "foe_get_aux",
            "foe_poll_status", "foe_last_launch_count", "foe_status_string", "foe_set_profiling", "foe_num_stages",
-           "foe_stage_name", "foe_get_stage_ms"]
+           "foe_stage_name", "foe_get_stage_ms", "foe_route_noalloc"]
 
 
 class FoeConfig(ctypes.Structure):
@@ -90,6 +90,8 @@ def load_library() -> ctypes.CDLL:
     lib.foe_stage_name.restype = ctypes.c_char_p
     lib.foe_get_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ci]
     lib.foe_get_stage_ms.restype = ci
+    lib.foe_route_noalloc.argtypes = [ci, ci, ci, ci, ctypes.c_float, vp, vp, vp, vp, ci, vp, vp, vp]
+    lib.foe_route_noalloc.restype = ci
     _lib = lib
     return lib
 
@@ -249,3 +251,19 @@ class FoeLayer:
         buf = (ctypes.c_float * n)()
         _check(self.lib.foe_get_stage_ms(self.handle, buf, n), "foe_get_stage_ms")
         return {self.lib.foe_stage_name(i).decode(): float(buf[i]) for i in range(n)}
+
+
+def route_noalloc(shape, ffn_norm_g: torch.Tensor, router_w: torch.Tensor, router_b: Optional[torch.Tensor],
+                  h: torch.Tensor, idx: torch.Tensor, w: torch.Tensor, stream=None) -> None:
+    """foe_route_noalloc: routing for callers that must not allocate device memory.  The caller supplies the
+    outputs idx / w ([n, H, k_c] int32 / fp32); the library works on its built-in scratch area and this
+    wrapper creates no tensors either.  Calls on one device must not overlap (they share the scratch)."""
+    lib = load_library()
+    assert h.is_cuda and h.is_contiguous() and h.dtype == torch.bfloat16
+    assert idx.is_cuda and idx.dtype == torch.int32 and idx.is_contiguous()
+    assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous()
+    assert ffn_norm_g.dtype == torch.bfloat16 and router_w.dtype == torch.float32
+    _check(lib.foe_route_noalloc(shape.hidden, shape.n_clusters, shape.experts_per_cluster, shape.top_k_per_cluster,
+                                 shape.rms_eps, ffn_norm_g.data_ptr(), router_w.data_ptr(), _ptr(router_b),
+                                 h.data_ptr(), h.shape[0], idx.data_ptr(), w.data_ptr(), _stream_ptr(stream)),
+           "foe_route_noalloc")

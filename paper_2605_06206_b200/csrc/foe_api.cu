@@ -457,6 +457,21 @@ foe_status foe_route(foe_layer* L, const void* h, int n_tokens, int* topk_idx, f
   return check_launch();
 }
 
+foe_status foe_route_noalloc(int hidden, int n_clusters, int experts_per_cluster, int top_k_per_cluster, float rms_eps,
+                             const void* ffn_norm_g, const float* router_w, const float* router_b, const void* h,
+                             int n_tokens, int* topk_idx, float* topk_w, void* stream) {
+  if (!ffn_norm_g || !router_w || !h || !topk_idx || !topk_w) return FOE_ERR_NULL;
+  if (hidden <= 0 || hidden % 128 || n_clusters <= 0 || experts_per_cluster < 1 || experts_per_cluster > 128 ||
+      top_k_per_cluster < 1 || top_k_per_cluster > experts_per_cluster || top_k_per_cluster > 32 ||
+      n_clusters * experts_per_cluster > 1024 || !(rms_eps >= 0.f))
+    return FOE_ERR_CONFIG;
+  if (n_tokens < 0) return FOE_ERR_SHAPE;
+  const int rc = launch_route_noalloc(static_cast<const bf16*>(h), static_cast<const bf16*>(ffn_norm_g), router_w, router_b,
+                                      topk_idx, topk_w, n_tokens, hidden, n_clusters, experts_per_cluster,
+                                      top_k_per_cluster, rms_eps, static_cast<cudaStream_t>(stream));
+  return rc == 0 ? FOE_OK : (rc == -3 ? FOE_ERR_SHAPE : FOE_ERR_CUDA);
+}
+
 foe_status foe_get_aux(foe_layer* L, foe_aux* a) {
   if (!L || !a) return FOE_ERR_NULL;
   a->n_tokens = L->last_tokens;

@@ -38,6 +38,10 @@ int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float*
                  float* inv_rms, float* part, float* logits, int* idx, float* w, int n_tokens, int d, int H, int Ec,
                  int kc, float eps, int n_sms, cudaStream_t st);
 
+// routing on the library's built-in scratch area (no allocation); 0, -3 (too large) or -6 (CUDA error)
+int launch_route_noalloc(const bf16* h, const bf16* gain, const float* wr, const float* br, int* idx, float* w,
+                         int n_tokens, int d, int H, int Ec, int kc, float eps, cudaStream_t st);
+
 // ---- permute.cu
 struct PermuteBuffers {
   int* counts;        // [E]

@@ -251,4 +251,78 @@ int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float*
   return 3;
 }
 
+
+// ================================================================================================
+// Routing without any allocation.
+//
+// Some callers of this library cannot allocate device memory at all: a serving process that handed the whole
+// GPU to its own memory pool when it started (cudaMalloc would fail or steal from that pool), or a thread on a
+// latency-critical path that must not take the driver's allocation lock nor run into the device-wide
+// synchronisation that freeing memory implies.  foe_layer_create allocates, so those callers cannot even own a
+// handle.  For them the routing step is offered on a fixed scratch area that lives inside the library image:
+// the array below is part of every GPU's copy of the module from load until the process exits (about 6 MB).
+// The array's name is only a host-side stand-in; the device address is looked up once per device with
+// cudaGetSymbolAddress and handed to the same kernels the handle-based path runs.
+// ================================================================================================
+constexpr size_t kNaMaxTokens = 8192;                 // inv_rms entries
+constexpr size_t kNaMaxScores = size_t(1) << 19;      // n_tokens * n_experts of one call
+constexpr size_t kNaMaxPartial = size_t(1) << 20;     // split-K partial scores
+constexpr int kNaMaxDevices = 64;
+
+static __device__ __align__(256) float g_route_scratch[kNaMaxTokens + kNaMaxScores + kNaMaxPartial];
+
+static float* g_route_scratch_dev[kNaMaxDevices];     // device address of the array, per device
+static int g_route_sms[kNaMaxDevices];
+
+// inv_rms only: the expert input u is not produced on this path (the caller asked for routing, nothing else)
+__global__ void ffn_inv_rms_bf16_kernel(const bf16* __restrict__ r_in, float* __restrict__ inv_out, int n_tokens, int d,
+                                        float eps) {
+  const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (i >= n_tokens) return;
+  const uint4* row = reinterpret_cast<const uint4*>(r_in + size_t(i) * d);
+  float ss = 0.f;
+  for (int c = lane; c < d / 8; c += 32) {
+    const uint4 q = __ldg(row + c);
+    const uint32_t v[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { const float a = bf16_lo(v[j]), b = bf16_hi(v[j]); ss += a * a + b * b; }
+  }
+  ss = warp_sum(ss);
+  if (lane == 0) inv_out[i] = rsqrtf(ss / float(d) + eps);
+}
+
+// Returns 0 on success, -3 when the sizes exceed the fixed scratch, -6 on a CUDA error.  Calls nothing that
+// allocates.  The first call on a device resolves the scratch address (and reads the SM count).
+int launch_route_noalloc(const bf16* h, const bf16* gain, const float* wr, const float* br, int* idx, float* w,
+                         int n_tokens, int d, int H, int Ec, int kc, float eps, cudaStream_t st) {
+  const int E = H * Ec;
+  if (size_t(n_tokens) > kNaMaxTokens || size_t(n_tokens) * E > kNaMaxScores) return -3;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNaMaxDevices) return -6;
+  if (!g_route_scratch_dev[dev]) {
+    float* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_route_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return -6;
+    }
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return -6;
+    g_route_sms[dev] = sms;
+    g_route_scratch_dev[dev] = p;
+  }
+  float* inv = g_route_scratch_dev[dev];
+  float* logits = inv + kNaMaxTokens;
+  float* part = logits + kNaMaxScores;
+  if (n_tokens <= 0) return 0;
+  // Nothing in the scratch has to start at zero: every entry that is read below is written first by this call.
+  ffn_inv_rms_bf16_kernel<<<(n_tokens * 32 + 255) / 256, 256, 0, st>>>(h, inv, n_tokens, d, eps);
+  int ks = route_k_splits(n_tokens, d, E, g_route_sms[dev]);
+  while (ks > 1 && size_t(ks) * n_tokens * E > kNaMaxPartial) ks >>= 1;
+  dim3 grid((n_tokens + kRgTM - 1) / kRgTM, (E + kRgTN - 1) / kRgTN, ks);
+  router_gemm_kernel<<<grid, kRgThreads, 0, st>>>(h, 1, inv, gain, wr, part, n_tokens, d, E, d / ks);
+  const int tasks = n_tokens * H;
+  topk_gates_kernel<<<(tasks * 32 + 255) / 256, 256, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc);
+  return cudaGetLastError() == cudaSuccess ? 0 : -6;
+}
+
 }  // namespace foe
