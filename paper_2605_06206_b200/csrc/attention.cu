@@ -2,15 +2,13 @@
 // every query head reading the KV head of its cluster from the paged cache (the paper's KV cache is split
 // across the expert groups; on one GPU that is the head index of the page layout).
 //
-// Both kernels stage K and V through shared memory with TMA: one cache page of one KV head
-// ([64 tokens][d_h] bf16, contiguous) is one or two 64 x 64 boxes written with the 128-byte swizzle, which
-// is exactly the bank-conflict-free layout ldmatrix wants.  Scores and the PV product run on mma.sync
-// (m16n8k16, fp32 accumulate) with an online softmax in the exp2 domain.
-//
-//  * prefill: one CTA per (128 query rows, query head, sequence); 8 warps x 16 rows; key tiles = pages.
-//  * decode : one CTA per (sequence, KV head, split of the context); the g query heads of the KV head are
-//             the MMA rows; each of 4 warps takes 16 keys of every page; partial (m, l, o) per split are
-//             merged by a second kernel.  The KV cache is read exactly once.
+// This file holds the decode kernel (one new token per sequence; the prefill kernel on the tcgen05 tensor
+// cores is in attention_tc.cu).  Decode is bound by reading the KV cache once from HBM: K and V are staged
+// through shared memory with TMA -- one cache page of one KV head ([64 tokens][d_h] bf16, contiguous) is one or
+// two 64 x 64 boxes written with the 128-byte swizzle, the bank-conflict-free layout ldmatrix wants.  One CTA
+// per (sequence, KV head, split of the context); the g query heads of the KV head are the rows of mma.sync
+// m16n8k16 tiles (fp32 accumulate, online softmax in the exp2 domain); each of 4 warps takes 16 keys of every
+// page; partial (m, l, o) per split are merged by a second kernel.
 #include <math.h>
 
 #include "common.cuh"
@@ -34,201 +32,6 @@ __device__ __forceinline__ void tma_load_page(uint8_t* k_dst, uint8_t* v_dst, co
     tma_load_2d(k_dst + h * 64 * 128, tmK, bar, h * 64, row0);
     tma_load_2d(v_dst + h * 64 * 128, tmV, bar, h * 64, row0);
   }
-}
-
-// ======================================================================================= prefill
-constexpr int kPfRows = 128;
-constexpr int kPfThreads = 256;
-constexpr int kPfStages = 2;
-
-template <int DH>
-__global__ void __launch_bounds__(kPfThreads, 2)
-attn_prefill_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  constexpr int kQBytes = kPfRows * DH * 2;
-  constexpr int kTileBytes = 64 * DH * 2;
-  uint8_t* q_s = smem;
-  uint8_t* kv_s = smem + kQBytes;                      // [stage][K | V]
-  uint64_t* full = reinterpret_cast<uint64_t*>(kv_s + kPfStages * 2 * kTileBytes);
-
-  const int b = blockIdx.z, head = blockIdx.y;
-  const int qb = gridDim.x - 1 - blockIdx.x;           // heavy (late) query blocks first
-  const int q_len = a.q_lens ? a.q_lens[b] : 1;
-  const int q0 = qb * kPfRows;
-  if (q0 >= q_len) return;
-  const int ctx = a.context_lens[b];
-  const int tok0 = a.cu_q[b] + q0;
-  const int kvh = head / (a.n_q / a.n_kv);
-  const int rows_here = min(kPfRows, q_len - q0);
-  const int kv_len = ctx + q0 + rows_here;             // keys any row of this block can see
-  const int n_tiles = (kv_len + 63) >> 6;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int ld_qkv = (a.n_q + 2 * a.n_kv) * DH;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kPfStages; ++s) mbar_init(&full[s], 1);
-    mbar_fence_init();
-  }
-  // Q tile (zero rows past the sequence end)
-  for (int q = threadIdx.x; q < kPfRows * (DH / 8); q += kPfThreads) {
-    const int r = q / (DH / 8), ch = q - r * (DH / 8);
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (r < rows_here) v = __ldg(reinterpret_cast<const uint4*>(a.qkv + size_t(tok0 + r) * ld_qkv + head * DH + ch * 8));
-    *reinterpret_cast<uint4*>(q_s + tile_off<kPfRows>(r, ch * 8)) = v;
-  }
-  __syncthreads();
-
-  auto page_row0 = [&](int tile) -> int {
-    int page = a.block_table[size_t(b) * a.max_pages_per_seq + min(tile, a.max_pages_per_seq - 1)];
-    if (page < 0 || page >= a.num_pages) { atomicExch(a.status, kStatusBounds); page = 0; }
-    return (page * a.n_kv + kvh) * 64;
-  };
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kPfStages && s < n_tiles; ++s)
-      tma_load_page<DH>(kv_s + s * 2 * kTileBytes, kv_s + s * 2 * kTileBytes + kTileBytes, &tmK, &tmV, &full[s],
-                        page_row0(s));
-  }
-
-  float o[DH / 8][4];
-#pragma unroll
-  for (int n = 0; n < DH / 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
-  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-  const int g = lane >> 2, t4 = lane & 3;
-  const int qpos0 = ctx + q0 + warp * 16 + g;          // position of row g; row g+8 is +8
-  const uint32_t q_base = smem_u32(q_s);
-  bool ok = true;
-
-  for (int j = 0; j < n_tiles; ++j) {
-    const int st = j % kPfStages;
-    if (!mbar_wait(&full[st], (j / kPfStages) & 1)) { ok = false; break; }
-    const uint32_t k_base = smem_u32(kv_s + st * 2 * kTileBytes);
-    const uint32_t v_base = k_base + kTileBytes;
-    // warps whose 16 rows all sit before this key tile have nothing to do in it
-    if (j * 64 <= ctx + q0 + warp * 16 + 15) {
-      float s[8][4];
-#pragma unroll
-      for (int n = 0; n < 8; ++n) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f; }
-#pragma unroll
-      for (int ks = 0; ks < DH / 16; ++ks) {
-        uint32_t qa[4];
-        ldmatrix_x4(qa, q_base + tile_off<kPfRows>(warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, ks * 16 + (lane >> 4) * 8));
-#pragma unroll
-        for (int np = 0; np < 4; ++np) {
-          uint32_t kb[4];
-          ldmatrix_x4(kb, k_base + tile_off<64>(np * 16 + (lane & 7) + (lane >> 4) * 8, ks * 16 + ((lane >> 3) & 1) * 8));
-          mma_bf16_16816(s[2 * np], qa, kb[0], kb[1]);
-          mma_bf16_16816(s[2 * np + 1], qa, kb[2], kb[3]);
-        }
-      }
-      // scale, causal mask (only tiles that reach past the first row of the warp), online softmax
-      const bool need_mask = j * 64 + 63 > ctx + q0 + warp * 16;
-      float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-      for (int n = 0; n < 8; ++n) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float v = s[n][e] * a.scale_log2;
-          if (need_mask) {
-            const int kpos = j * 64 + n * 8 + t4 * 2 + (e & 1);
-            const int qpos = qpos0 + (e >> 1) * 8;
-            if (kpos > qpos) v = -INFINITY;
-          }
-          s[n][e] = v;
-          mx[e >> 1] = fmaxf(mx[e >> 1], v);
-        }
-      }
-      float alpha[2], m_use[2];
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
-        mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-        const float m_new = fmaxf(m_run[r], mx[r]);
-        m_use[r] = (m_new == -INFINITY) ? 0.f : m_new;
-        alpha[r] = fast_exp2(m_run[r] - m_use[r]);
-        m_run[r] = m_new;
-      }
-      float rs[2] = {0.f, 0.f};
-#pragma unroll
-      for (int n = 0; n < 8; ++n) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float p = fast_exp2(s[n][e] - m_use[e >> 1]);
-          s[n][e] = p;
-          rs[e >> 1] += p;
-        }
-      }
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        rs[r] += __shfl_xor_sync(0xffffffffu, rs[r], 1);
-        rs[r] += __shfl_xor_sync(0xffffffffu, rs[r], 2);
-        l_run[r] = l_run[r] * alpha[r] + rs[r];
-      }
-#pragma unroll
-      for (int n = 0; n < DH / 8; ++n) {
-        o[n][0] *= alpha[0]; o[n][1] *= alpha[0]; o[n][2] *= alpha[1]; o[n][3] *= alpha[1];
-      }
-#pragma unroll
-      for (int kk = 0; kk < 4; ++kk) {
-        uint32_t pa[4];
-        pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
-        pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
-        pa[2] = pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-        pa[3] = pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
-#pragma unroll
-        for (int dp = 0; dp < DH / 16; ++dp) {
-          uint32_t vb[4];
-          ldmatrix_x4_trans(vb, v_base + tile_off<64>(kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, dp * 16 + (lane >> 4) * 8));
-          mma_bf16_16816(o[2 * dp], pa, vb[0], vb[1]);
-          mma_bf16_16816(o[2 * dp + 1], pa, vb[2], vb[3]);
-        }
-      }
-    }
-    __syncthreads();                                   // every warp is done with stage st
-    if (threadIdx.x == 0 && j + kPfStages < n_tiles)
-      tma_load_page<DH>(kv_s + st * 2 * kTileBytes, kv_s + st * 2 * kTileBytes + kTileBytes, &tmK, &tmV, &full[st],
-                        page_row0(j + kPfStages));
-  }
-  if (!ok) {
-    if (lane == 0) atomicExch(a.status, kStatusTimeout);
-    return;
-  }
-
-  // normalise, stage the warp's 16 rows through its own slice of the Q tile, store 16 bytes per lane
-  const float inv_l[2] = {1.f / l_run[0], 1.f / l_run[1]};
-  __syncwarp();
-#pragma unroll
-  for (int n = 0; n < DH / 8; ++n) {
-    *reinterpret_cast<uint32_t*>(q_s + tile_off<kPfRows>(warp * 16 + g, n * 8 + t4 * 2)) =
-        pack_bf16(o[n][0] * inv_l[0], o[n][1] * inv_l[0]);
-    *reinterpret_cast<uint32_t*>(q_s + tile_off<kPfRows>(warp * 16 + g + 8, n * 8 + t4 * 2)) =
-        pack_bf16(o[n][2] * inv_l[1], o[n][3] * inv_l[1]);
-  }
-  __syncwarp();
-  for (int q = lane; q < 16 * (DH / 8); q += 32) {
-    const int r = warp * 16 + q / (DH / 8), ch = q % (DH / 8);
-    if (r < rows_here)
-      *reinterpret_cast<uint4*>(a.out + size_t(tok0 + r) * (a.n_q * DH) + head * DH + ch * 8) =
-          *reinterpret_cast<const uint4*>(q_s + tile_off<kPfRows>(r, ch * 8));
-  }
-}
-
-template <int DH>
-static void launch_prefill_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st) {
-  constexpr size_t smem = kPfRows * DH * 2 + kPfStages * 2 * 64 * DH * 2 + 1024 + 64;
-  static bool configured = false;
-  if (!configured) {
-    cudaFuncSetAttribute(attn_prefill_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    configured = true;
-  }
-  dim3 grid((a.max_q_len + kPfRows - 1) / kPfRows, a.n_q, a.n_seqs);
-  attn_prefill_kernel<DH><<<grid, kPfThreads, smem, st>>>(tmK, tmV, a);
-}
-
-void launch_attn_prefill(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st) {
-  if (a.n_seqs <= 0 || a.max_q_len <= 0) return;
-  if (a.dh == 128) launch_prefill_t<128>(tmK, tmV, a, st);
-  else launch_prefill_t<64>(tmK, tmV, a, st);
 }
 
 // ======================================================================================= decode

@@ -1,0 +1,342 @@
+// Prefill attention on the 5th-generation tensor cores: causal softmax(q k^T / sqrt(d_h)) v for the new
+// tokens of every sequence against the paged cache ("Attn_h" of the paper's Table 2; cluster h's query heads
+// read cluster h's KV heads).
+//
+// One CTA owns 128 query rows of TWO query heads that share a KV head (GQA), so both tiles walk the same K/V
+// pages with the same causal extent.  Per page of 64 keys:
+//     S_t = Q_t K^T        tcgen05.mma  M128 N64  K16 x (d_h/16)   accumulator in tensor memory
+//     P_t = softmax step   one thread per query row: tcgen05.ld, exp2, row max/sum without any shuffle,
+//                          P written to shared memory in the K-major 128-byte-swizzled operand layout
+//     O_t += P_t V         tcgen05.mma  M128 N d_h K16 x 4, V used straight from its page ([key][d_h],
+//                          i.e. an MN-major B operand); O stays in tensor memory for the whole row block
+// The running maximum used for the exponentials is only moved when the true maximum has grown by more than
+// 2^8 since it was last moved (the result is mathematically the same, probabilities stay below 256); only
+// then is O rescaled in tensor memory (tcgen05.ld / tcgen05.st), which after the first pages is rare.
+// Warp roles: warp 0 TMA producer (Q once, K/V pages through a 3-stage ring), warp 1 MMA issuer (warps 2-3
+// idle; the first warpgroup gives its registers away with setmaxnreg), warps 4-7 softmax of tile 0, warps 8-11
+// softmax of tile 1.  While one tile's softmax runs, the tensor core works on
+// the other tile.  All waits are bounded; on expiry the role records a timeout in the status word and the
+// CTA still reaches its teardown (tensor memory is released).
+#include <math.h>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace foe {
+
+constexpr int kAtRows = 128;          // query rows per tile
+constexpr int kAtKeys = 64;           // keys per step = one cache page
+constexpr int kAtStages = 3;
+constexpr int kAtThreads = 384;        // warpgroup 0: producer + MMA issuer (+2 idle warps); warpgroups 1, 2: softmax
+
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// K-major operand, 128-byte swizzle (rows of 128 bytes, 8-row groups 1024 bytes apart)
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) { return umma_desc_sw128(addr); }
+// MN-major operand, 128-byte swizzle: 64 contiguous elements of the M/N dimension per 128-byte row, one row
+// per k; 8-k groups `sbo` bytes apart, successive 64-element blocks of M/N `lbo` bytes apart.
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr >> 4) & 0x3fff);
+  d |= static_cast<uint64_t>((lbo >> 4) & 0x3fff) << 16;
+  d |= static_cast<uint64_t>((sbo >> 4) & 0x3fff) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+
+template <int DH>
+struct AtSmem {
+  static constexpr int kHalves = DH / 64;
+  static constexpr int kQTile = kAtRows * DH * 2;              // one query tile
+  static constexpr int kKVTile = kAtKeys * DH * 2;             // one K or V page of one head
+  static constexpr int kPTile = kAtRows * kAtKeys * 2;         // probabilities of one tile (bf16)
+  static constexpr int kQOff = 0;
+  static constexpr int kKVOff = 2 * kQTile;
+  static constexpr int kPOff = kKVOff + kAtStages * 2 * kKVTile;
+  static constexpr int kBarOff = kPOff + 4 * kPTile;           // P is double-buffered per tile
+  static constexpr size_t kBytes = kBarOff + 256 + 1024;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(kAtThreads, 1)
+attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                       const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
+  using L = AtSmem<DH>;
+  constexpr int HN = DH / 64;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
+  uint64_t* q_full = bars;                 // 1
+  uint64_t* kv_full = bars + 1;            // kAtStages
+  uint64_t* kv_empty = kv_full + kAtStages;
+  uint64_t* s_full = kv_empty + kAtStages; // 2
+  uint64_t* p_ready = s_full + 2;          // 2
+  uint64_t* o_full = p_ready + 2;          // 2
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_full + 2);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.z;
+  const int G = a.n_q / a.n_kv;
+  const int n_tiles_q = (G % 2 == 0) ? 2 : 1;              // heads per CTA
+  const int head0 = blockIdx.y * n_tiles_q;
+  const int qb = gridDim.x - 1 - blockIdx.x;               // heavy (late) query blocks first
+  const int q_len = a.q_lens ? a.q_lens[b] : 1;
+  const int q0 = qb * kAtRows;
+  if (q0 >= q_len) return;
+  const int ctx = a.context_lens[b];
+  const int tok0 = a.cu_q[b] + q0;
+  const int kvh = head0 / G;
+  const int rows_here = min(kAtRows, q_len - q0);
+  const int kv_len = ctx + q0 + rows_here;
+  const int n_tiles = (kv_len + kAtKeys - 1) / kAtKeys;
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    for (int s = 0; s < kAtStages; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(&s_full[t], 1); mbar_init(&p_ready[t], 4); mbar_init(&o_full[t], 1);
+    }
+    mbar_fence_init();
+    tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // tensor-memory columns: S of tile t at 64 t, per-step O of tile t at 128 + DH t
+  const uint32_t q_u32 = smem_u32(smem + L::kQOff), kv_u32 = smem_u32(smem + L::kKVOff), p_u32 = smem_u32(smem + L::kPOff);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (elect_one()) {
+      bool ok = true;
+      mbar_expect_tx(q_full, n_tiles_q * L::kQTile);
+      for (int t = 0; t < n_tiles_q; ++t)
+        for (int h = 0; h < HN; ++h)
+          tma_load_2d(smem + L::kQOff + t * L::kQTile + h * (kAtRows * 128), &tmQ, q_full, (head0 + t) * DH + h * 64, tok0);
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int s = j % kAtStages;
+        if (!mbar_wait(&kv_empty[s], ((j / kAtStages) & 1) ^ 1)) { ok = false; break; }
+        int page = a.block_table[size_t(b) * a.max_pages_per_seq + min(j, a.max_pages_per_seq - 1)];
+        if (page < 0 || page >= a.num_pages) { atomicExch(a.status, kStatusBounds); page = 0; }
+        const int row0 = (page * a.n_kv + kvh) * kAtKeys;
+        uint8_t* kd = smem + L::kKVOff + s * 2 * L::kKVTile;
+        mbar_expect_tx(&kv_full[s], 2 * L::kKVTile);
+        for (int h = 0; h < HN; ++h) {
+          tma_load_2d(kd + h * (kAtKeys * 128), &tmK, &kv_full[s], h * 64, row0);
+          tma_load_2d(kd + L::kKVTile + h * (kAtKeys * 128), &tmV, &kv_full[s], h * 64, row0);
+        }
+      }
+      if (!ok) atomicExch(a.status, kStatusTimeout);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (elect_one()) {
+      constexpr uint32_t idesc_s = umma_idesc_bf16(kAtRows, kAtKeys);
+      constexpr uint32_t idesc_o = umma_idesc_bf16(kAtRows, DH) | (1u << 16);      // B operand (V) is MN-major
+      bool ok = mbar_wait(q_full, 0);
+      auto issue_s = [&](int t, int j) {                      // S_t = Q_t K_j^T
+        const int s = j % kAtStages;
+        const uint32_t qb_ = q_u32 + t * L::kQTile, kb_ = kv_u32 + s * 2 * L::kKVTile;
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks) {
+          const uint32_t off_q = (ks >> 2) * (kAtRows * 128) + (ks & 3) * 32;
+          const uint32_t off_k = (ks >> 2) * (kAtKeys * 128) + (ks & 3) * 32;
+          umma_bf16(tmem_base + t * 64, desc_kmajor(qb_ + off_q), desc_kmajor(kb_ + off_k), idesc_s, ks != 0);
+        }
+        umma_commit(&s_full[t]);
+      };
+      auto issue_o = [&](int t, int j) {                      // O_t = P_t V_j
+        const int s = j % kAtStages;
+        const uint32_t pb_ = p_u32 + (t * 2 + (j & 1)) * L::kPTile, vb_ = kv_u32 + s * 2 * L::kKVTile + L::kKVTile;
+#pragma unroll
+        for (int kk = 0; kk < kAtKeys / 16; ++kk)
+          umma_bf16(tmem_base + 128 + t * DH, desc_kmajor(pb_ + kk * 32),
+                    desc_mnmajor(vb_ + kk * (16 * 128), kAtKeys * 128, 1024), idesc_o, (j | kk) != 0);
+        umma_commit(&o_full[t]);
+      };
+      if (ok && n_tiles > 0) {
+        ok = mbar_wait(&kv_full[0], 0);
+        if (ok) {
+          tc_fence_after();
+          for (int t = 0; t < n_tiles_q; ++t) issue_s(t, 0);
+        }
+      }
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const uint32_t ph = j & 1;
+        bool next_ready = false;
+        for (int t = 0; t < n_tiles_q && ok; ++t) {
+          if (!mbar_wait(&p_ready[t], ph)) { ok = false; break; }       // P_t(j) in shared memory, S_t free again
+          tc_fence_after();
+          if (j + 1 < n_tiles) {
+            if (!next_ready) {
+              if (!mbar_wait(&kv_full[(j + 1) % kAtStages], ((j + 1) / kAtStages) & 1)) { ok = false; break; }
+              tc_fence_after();
+              next_ready = true;
+            }
+            issue_s(t, j + 1);
+          }
+          issue_o(t, j);
+        }
+        if (ok) umma_commit(&kv_empty[j % kAtStages]);                  // stage j reusable once those MMAs retire
+      }
+      if (!ok) atomicExch(a.status, kStatusTimeout);
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ softmax, one thread per query row
+    const int t = (warp - 4) >> 2;                           // tile of this warp group
+    if (t < n_tiles_q) {
+      const int quarter = warp & 3;
+      const int row = quarter * 32 + lane;                   // row of the tile = TMEM lane
+      const uint32_t lane_sel = static_cast<uint32_t>(quarter * 32) << 16;
+      const uint32_t s_addr = tmem_base + lane_sel + t * 64;
+      const uint32_t o_addr = tmem_base + lane_sel + 128 + t * DH;
+      const int qpos = ctx + q0 + row;
+      const int first_mask_tile = (ctx + q0) / kAtKeys;
+      uint8_t* p_rows = smem + L::kPOff + t * 2 * L::kPTile + row * 128;
+      float m_ref = -INFINITY, l_run = 0.f;                  // m_ref: the (possibly stale) maximum the exponentials use
+      bool ok = true;
+      for (int j = 0; j < n_tiles; ++j) {
+        const uint32_t ph = j & 1;
+        if (!mbar_wait(&s_full[t], ph)) { ok = false; break; }
+        tc_fence_after();
+        const bool masked = j >= first_mask_tile;
+        // pass 1: row maximum of the 64 scores
+        float mx = -INFINITY;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t r[32];
+          tmem_ld32(s_addr + hf * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            float v = __uint_as_float(r[c]);
+            if (masked && j * kAtKeys + hf * 32 + c > qpos) v = -INFINITY;
+            mx = fmaxf(mx, v);
+          }
+        }
+        const float m_new = fmaxf(m_ref, mx * a.scale_log2);
+        // move the reference maximum (and rescale O) only when it is off by more than 2^8; warp-uniform so that
+        // the tensor-memory accesses stay aligned
+        const bool move = __any_sync(0xffffffffu, m_new > m_ref + 8.0f);
+        if (move) {
+          const float alpha = (m_ref == -INFINITY) ? 0.f : fast_exp2(m_ref - m_new);
+          if (j > 0) {
+            if (!mbar_wait(&o_full[t], ph ^ 1)) { ok = false; break; }      // every P V product so far has landed
+            tc_fence_after();
+#pragma unroll
+            for (int ch = 0; ch < DH / 32; ++ch) {
+              uint32_t r[32];
+              tmem_ld32(o_addr + ch * 32, r);
+              tmem_ld_wait();
+#pragma unroll
+              for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
+              tmem_st32(o_addr + ch * 32, r);
+            }
+            tmem_st_wait();
+          }
+          l_run *= alpha;
+          m_ref = m_new;
+        }
+        const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+        // pass 2: probabilities, written as the bf16 A operand of the PV product
+        uint8_t* p_row = p_rows + (j & 1) * L::kPTile;
+        float rs = 0.f;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t r[32];
+          tmem_ld32(s_addr + hf * 32, r);
+          tmem_ld_wait();
+          uint32_t pk[16];
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            float v0 = __uint_as_float(r[2 * c]), v1 = __uint_as_float(r[2 * c + 1]);
+            float p0 = fast_exp2(fmaf(v0, a.scale_log2, -m_use)), p1 = fast_exp2(fmaf(v1, a.scale_log2, -m_use));
+            if (masked) {
+              if (j * kAtKeys + hf * 32 + 2 * c > qpos) p0 = 0.f;
+              if (j * kAtKeys + hf * 32 + 2 * c + 1 > qpos) p1 = 0.f;
+            }
+            rs += p0 + p1;
+            pk[c] = pack_bf16(p0, p1);
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            *reinterpret_cast<uint4*>(p_row + (((hf * 4 + q) ^ (row & 7)) << 4)) =
+                make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+        }
+        l_run += rs;
+        tc_fence_before();
+        fence_async_smem();                                  // P visible to the tensor core's shared-memory reads
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_ready[t]);
+      }
+      if (ok && n_tiles > 0) ok = mbar_wait(&o_full[t], (n_tiles - 1) & 1);
+      tc_fence_after();
+      if (!ok) {
+        if (lane == 0) atomicExch(a.status, kStatusTimeout);
+      } else {
+        // normalise; stage the warp's 32 rows in its slice of the (no longer needed) query tile; store rows whole
+        const float inv_l = 1.f / l_run;
+        uint8_t* stg = smem + L::kQOff + t * L::kQTile + quarter * 32 * (DH * 2);
+        constexpr int CH = DH / 8;                           // 16-byte chunks per row
+#pragma unroll
+        for (int ch = 0; ch < DH / 32; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(o_addr + ch * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int c = ch * 4 + q;
+            uint4 v = make_uint4(pack_bf16(__uint_as_float(r[8 * q]) * inv_l, __uint_as_float(r[8 * q + 1]) * inv_l),
+                                 pack_bf16(__uint_as_float(r[8 * q + 2]) * inv_l, __uint_as_float(r[8 * q + 3]) * inv_l),
+                                 pack_bf16(__uint_as_float(r[8 * q + 4]) * inv_l, __uint_as_float(r[8 * q + 5]) * inv_l),
+                                 pack_bf16(__uint_as_float(r[8 * q + 6]) * inv_l, __uint_as_float(r[8 * q + 7]) * inv_l));
+            *reinterpret_cast<uint4*>(stg + lane * (DH * 2) + ((c ^ (lane & 7)) << 4)) = v;
+          }
+        }
+        __syncwarp();
+        constexpr int RPI = 32 / CH;                         // rows per store instruction
+        for (int r0 = 0; r0 < 32; r0 += RPI) {
+          const int rr = r0 + lane / CH, c = lane % CH;
+          const int grow = quarter * 32 + rr;
+          if (grow < rows_here)
+            *reinterpret_cast<uint4*>(a.out + size_t(tok0 + grow) * (a.n_q * DH) + (head0 + t) * DH + c * 8) =
+                *reinterpret_cast<const uint4*>(stg + rr * (DH * 2) + ((c ^ (rr & 7)) << 4));
+        }
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+template <int DH>
+static void launch_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
+                      cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(attn_prefill_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(AtSmem<DH>::kBytes));
+    configured = true;
+  }
+  const int G = a.n_q / a.n_kv;
+  const int heads_per_cta = (G % 2 == 0) ? 2 : 1;
+  dim3 grid((a.max_q_len + kAtRows - 1) / kAtRows, a.n_q / heads_per_cta, a.n_seqs);
+  attn_prefill_tc_kernel<DH><<<grid, kAtThreads, AtSmem<DH>::kBytes, st>>>(tmQ, tmK, tmV, a);
+}
+
+void launch_attn_prefill_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
+                            cudaStream_t st) {
+  if (a.n_seqs <= 0 || a.max_q_len <= 0) return;
+  if (a.dh == 128) launch_tc<128>(tmQ, tmK, tmV, a, st);
+  else launch_tc<64>(tmQ, tmK, tmV, a, st);
+}
+
+}  // namespace foe

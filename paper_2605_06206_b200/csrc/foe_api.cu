@@ -67,6 +67,7 @@ struct foe_layer {
   int max_splits, pages_per_split;
   // static tensor maps
   CUtensorMap tm_wqkv, tm_attn_o, tm_wo, tm_uperm, tm_wgu, tm_hmid, tm_wd;
+  CUtensorMap tm_qkv;
   CUtensorMap tms_wqkv, tms_wo, tms_wgu, tms_wd;   // same weights, boxes sized for the decode kernels
   // call state
   cudaStream_t last_stream;
@@ -185,7 +186,7 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
   aa.status = L->status; aa.part_o = L->part_o; aa.part_ml = L->part_ml; aa.max_splits = L->max_splits;
   aa.pages_per_split = L->pages_per_split;
   if (decode) { launch_attn_decode(tmK, tmV, aa, st); L->launches += 2; }
-  else { launch_attn_prefill(tmK, tmV, aa, st); L->launches += 1; }
+  else { launch_attn_prefill_tc(L->tm_qkv, tmK, tmV, aa, st); L->launches += 1; }
 
   // ---- output projection; the cross-cluster sync is its K-reduction plus the sum of x[h] in the epilogue
   stage_mark(L, kStOproj, st);
@@ -404,6 +405,7 @@ foe_status foe_layer_create(const foe_config* cfg, const foe_weights* w, foe_lay
        make_map_2d(&L->tm_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, kBN) &&
        make_map_2d(&L->tm_hmid, L->hmid, uint64_t(R), I, kBM) &&
        make_map_2d(&L->tm_wd, L->wd_t, uint64_t(E) * d, I, kBN) &&
+       make_map_2d(&L->tm_qkv, L->qkv, uint64_t(S), uint64_t(L->qkv_cols), 128) &&
        make_map_2d(&L->tms_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, 64) &&
        make_map_2d(&L->tms_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, 64) &&
        make_map_2d(&L->tms_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, 32) &&

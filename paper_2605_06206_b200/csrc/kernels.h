@@ -79,7 +79,9 @@ struct AttnArgs {
   int max_splits;
   int pages_per_split;
 };
-void launch_attn_prefill(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st);
+// tensor-core (tcgen05) prefill attention; tmQ maps the qkv buffer [S][(n_q+2n_kv)*dh] with 128-row boxes
+void launch_attn_prefill_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
+                            cudaStream_t st);
 void launch_attn_decode(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st);
 
 // ---- gemm_tcgen05.cu
