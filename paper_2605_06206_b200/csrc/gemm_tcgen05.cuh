@@ -208,38 +208,40 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           *reinterpret_cast<uint4*>(stg + lane * kStgPitch + c * 16) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
         __syncwarp();
         if constexpr (EPI == kEpiOProj) {
-          // r_full = scale * (C + sum_h x[h]): the residual streams are read here, 8 lanes x 8 bytes per row
-          // and stream.  All loads of four rows are issued before the first use (the epilogue has to keep
-          // tens of KB in flight per SM: this GEMM moves almost as many bytes as it has flops to hide them).
+          // r_full = scale * (C + sum_h x[h]): the residual streams are read here.  This GEMM moves almost as many
+          // bytes as it has flops to hide them, so the epilogue has to keep ~256 bytes per thread in flight:
+          // 4 lanes x 16 bytes per row and stream, and all loads of the pass are issued before the first use.
+          const int or_row = lane >> 2, or_cg = lane & 3;           // row (+8j) and group of 8 columns
+          uint4 xq[4][8];
 #pragma unroll
-          for (int jh = 0; jh < 2; ++jh) {
-            uint2 xq[4][8];
+          for (int j = 0; j < 4; ++j) {
+            const int grow = row0 + quarter * 32 + or_row + 8 * j;
+            const size_t off = size_t(grow) * args.ldo + n + or_cg * 8;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const int grow = row0 + quarter * 32 + wr_row + 4 * (jh * 4 + j);
-              const size_t off = size_t(grow) * args.ldo + n + wr_chunk * 4;
-#pragma unroll
-              for (int h = 0; h < 8; ++h) {
-                xq[j][h] = make_uint2(0u, 0u);
-                if (h < args.x_count && grow < row_end)
-                  xq[j][h] = __ldg(reinterpret_cast<const uint2*>(args.xsum + h * args.x_stride + off));
-              }
+            for (int h = 0; h < 8; ++h) {
+              xq[j][h] = make_uint4(0u, 0u, 0u, 0u);
+              if (h < args.x_count && grow < row_end)
+                xq[j][h] = __ldg(reinterpret_cast<const uint4*>(args.xsum + h * args.x_stride + off));
             }
+          }
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const int rr = wr_row + 4 * (jh * 4 + j);
-              const int grow = row0 + quarter * 32 + rr;
-              if (grow >= row_end) continue;
-              const uint4 v = *reinterpret_cast<const uint4*>(stg + rr * kStgPitch + wr_chunk * 16);
-              float a4[4] = {__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w)};
+          for (int j = 0; j < 4; ++j) {
+            const int rr = or_row + 8 * j;
+            const int grow = row0 + quarter * 32 + rr;
+            if (grow >= row_end) continue;
+            const float4 c0 = *reinterpret_cast<const float4*>(stg + rr * kStgPitch + or_cg * 32);
+            const float4 c1 = *reinterpret_cast<const float4*>(stg + rr * kStgPitch + or_cg * 32 + 16);
+            float a8[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
-              for (int h = 0; h < 8; ++h) {
-                a4[0] += bf16_lo(xq[j][h].x); a4[1] += bf16_hi(xq[j][h].x);
-                a4[2] += bf16_lo(xq[j][h].y); a4[3] += bf16_hi(xq[j][h].y);
-              }
-              *reinterpret_cast<float4*>(static_cast<float*>(args.out) + size_t(grow) * args.ldo + n + wr_chunk * 4) =
-                  make_float4(a4[0] * args.out_scale, a4[1] * args.out_scale, a4[2] * args.out_scale, a4[3] * args.out_scale);
+            for (int h = 0; h < 8; ++h) {
+              const uint32_t w4[4] = {xq[j][h].x, xq[j][h].y, xq[j][h].z, xq[j][h].w};
+#pragma unroll
+              for (int q = 0; q < 4; ++q) { a8[2 * q] += bf16_lo(w4[q]); a8[2 * q + 1] += bf16_hi(w4[q]); }
             }
+            float* dst = static_cast<float*>(args.out) + size_t(grow) * args.ldo + n + or_cg * 8;
+            const float sc = args.out_scale;
+            *reinterpret_cast<float4*>(dst) = make_float4(a8[0] * sc, a8[1] * sc, a8[2] * sc, a8[3] * sc);
+            *reinterpret_cast<float4*>(dst + 4) = make_float4(a8[4] * sc, a8[5] * sc, a8[6] * sc, a8[7] * sc);
           }
         } else {
 #pragma unroll

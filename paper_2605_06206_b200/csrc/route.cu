@@ -5,7 +5,7 @@
 //
 // Three kernels:
 //  1. ffn_norm:     one warp per token: inv_rms and the bf16 expert input u = r * inv_rms * gain.
-//  2. router_gemm:  SIMT fp32 GEMM, 32 tokens x 64 experts per CTA, 4 x 4 register tiles, k-major shared
+//  2. router_gemm:  SIMT fp32 GEMM, 64 tokens x 64 experts per CTA, 8 x 8 register tiles, k-major shared
 //                   tiles, register-staged double buffering; the normalisation is applied while the token
 //                   tile is loaded (u is never rounded to bf16 on this path).  For a handful of tokens the
 //                   reduction dimension is split over gridDim.z so that the grid still fills the GPU; the
@@ -66,7 +66,7 @@ __global__ void ffn_norm_kernel(const void* __restrict__ r_in, int r_is_bf16, co
 }
 
 // ------------------------------------------------------------------------------------------------ 2
-constexpr int kRgTM = 32, kRgTN = 64, kRgKC = 32, kRgThreads = 128;
+constexpr int kRgTM = 64, kRgTN = 64, kRgKC = 32, kRgThreads = 64;
 constexpr int kRgPA = kRgTM + 4, kRgPB = kRgTN + 4;      // padded pitches (floats), multiples of 4
 
 __global__ void __launch_bounds__(kRgThreads)
@@ -78,29 +78,28 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
   const int tid = threadIdx.x;
   const int tok0 = blockIdx.x * kRgTM, exp0 = blockIdx.y * kRgTN;
   const int kbeg = blockIdx.z * k_per_split, kend = min(d, kbeg + k_per_split);
-  const int ty = tid >> 4, tx = tid & 15;                 // 8 x 16 threads, 4 tokens x 4 experts each
+  const int ty = tid >> 3, tx = tid & 7;                  // 8 x 8 threads, 8 tokens x 8 experts each
 
-  // loader roles: A = 32 tokens x 8 float4 (2 per thread), B = 64 experts x 8 float4 (4 per thread)
-  const int la_k4 = tid & 7, la_t = tid >> 3;             // tokens la_t and la_t + 16
-  const int lb_k4 = tid & 7, lb_e = tid >> 3;             // experts lb_e + 16 * j
-  float inv_t[2];
+  // loader roles: a tile is 64 rows x 8 float4; thread loads float4 (row = tid/8 + 8 j, k4 = tid%8), j < 8
+  const int l_k4 = tid & 7, l_r = tid >> 3;
+  float inv_t[8];
 #pragma unroll
-  for (int j = 0; j < 2; ++j) {
-    const int t = tok0 + la_t + 16 * j;
+  for (int j = 0; j < 8; ++j) {
+    const int t = tok0 + l_r + 8 * j;
     inv_t[j] = t < n_tokens ? inv_rms[t] : 0.f;
   }
-  float4 ra[2], rb[4];
+  float4 ra[8], rb[8];
 
   auto load_chunk = [&](int k0) {
-    const int k = k0 + la_k4 * 4;
+    const int k = k0 + l_k4 * 4;
     float g4[4];
     {
       const uint2 gq = __ldg(reinterpret_cast<const uint2*>(gain + k));
       g4[0] = bf16_lo(gq.x); g4[1] = bf16_hi(gq.x); g4[2] = bf16_lo(gq.y); g4[3] = bf16_hi(gq.y);
     }
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const int t = tok0 + la_t + 16 * j;
+    for (int j = 0; j < 8; ++j) {
+      const int t = tok0 + l_r + 8 * j;
       float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
       if (t < n_tokens) {
         if (r_is_bf16) {
@@ -113,31 +112,27 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
       ra[j] = make_float4(v.x * inv_t[j] * g4[0], v.y * inv_t[j] * g4[1], v.z * inv_t[j] * g4[2], v.w * inv_t[j] * g4[3]);
     }
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int e = min(exp0 + lb_e + 16 * j, E - 1);
-      rb[j] = __ldg(reinterpret_cast<const float4*>(wr + size_t(e) * d + k0 + lb_k4 * 4));
+    for (int j = 0; j < 8; ++j) {
+      const int e = min(exp0 + l_r + 8 * j, E - 1);
+      rb[j] = __ldg(reinterpret_cast<const float4*>(wr + size_t(e) * d + k));
     }
   };
   auto store_chunk = [&](int buf) {
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const int t = la_t + 16 * j;
-      As[buf][la_k4 * 4 + 0][t] = ra[j].x; As[buf][la_k4 * 4 + 1][t] = ra[j].y;
-      As[buf][la_k4 * 4 + 2][t] = ra[j].z; As[buf][la_k4 * 4 + 3][t] = ra[j].w;
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int e = lb_e + 16 * j;
-      Bs[buf][lb_k4 * 4 + 0][e] = rb[j].x; Bs[buf][lb_k4 * 4 + 1][e] = rb[j].y;
-      Bs[buf][lb_k4 * 4 + 2][e] = rb[j].z; Bs[buf][lb_k4 * 4 + 3][e] = rb[j].w;
+    for (int j = 0; j < 8; ++j) {
+      const int r = l_r + 8 * j;
+      As[buf][l_k4 * 4 + 0][r] = ra[j].x; As[buf][l_k4 * 4 + 1][r] = ra[j].y;
+      As[buf][l_k4 * 4 + 2][r] = ra[j].z; As[buf][l_k4 * 4 + 3][r] = ra[j].w;
+      Bs[buf][l_k4 * 4 + 0][r] = rb[j].x; Bs[buf][l_k4 * 4 + 1][r] = rb[j].y;
+      Bs[buf][l_k4 * 4 + 2][r] = rb[j].z; Bs[buf][l_k4 * 4 + 3][r] = rb[j].w;
     }
   };
 
-  float acc[4][4];
+  float acc[8][8];
 #pragma unroll
-  for (int a = 0; a < 4; ++a)
+  for (int a = 0; a < 8; ++a)
 #pragma unroll
-    for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+    for (int b = 0; b < 8; ++b) acc[a][b] = 0.f;
 
   load_chunk(kbeg);
   store_chunk(0);
@@ -146,15 +141,18 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
   for (int k0 = kbeg; k0 < kend; k0 += kRgKC) {
     const bool more = k0 + kRgKC < kend;
     if (more) load_chunk(k0 + kRgKC);
-#pragma unroll
+#pragma unroll 8
     for (int k = 0; k < kRgKC; ++k) {
-      const float4 av = *reinterpret_cast<const float4*>(&As[buf][k][ty * 4]);
-      const float4 bv = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 4]);
-      const float a4[4] = {av.x, av.y, av.z, av.w}, b4[4] = {bv.x, bv.y, bv.z, bv.w};
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][k][ty * 8]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&As[buf][k][ty * 8 + 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 8]);
+      const float4 b1 = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 8 + 4]);
+      const float a8[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float b8[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
-      for (int a = 0; a < 4; ++a)
+      for (int a = 0; a < 8; ++a)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(a4[a], b4[b], acc[a][b]);
+        for (int b = 0; b < 8; ++b) acc[a][b] = fmaf(a8[a], b8[b], acc[a][b]);
     }
     if (more) store_chunk(buf ^ 1);
     __syncthreads();
@@ -162,12 +160,12 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
   }
   float* dst = part + size_t(blockIdx.z) * n_tokens * E;
 #pragma unroll
-  for (int a = 0; a < 4; ++a) {
-    const int t = tok0 + ty * 4 + a;
+  for (int a = 0; a < 8; ++a) {
+    const int t = tok0 + ty * 8 + a;
     if (t >= n_tokens) continue;
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      const int e = exp0 + tx * 4 + b;
+    for (int b = 0; b < 8; ++b) {
+      const int e = exp0 + tx * 8 + b;
       if (e < E) dst[size_t(t) * E + e] = acc[a][b];
     }
   }
