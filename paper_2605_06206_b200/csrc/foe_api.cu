@@ -61,12 +61,12 @@ struct foe_layer {
   float2* rope_tab;
   // workspace
   float *inv_rms, *inv_rms_f, *route_part, *r_full, *logits, *topk_w, *part_o, *part_ml;
-  bf16 *qkv, *attn_o, *u, *u_perm, *hmid, *y;
+  bf16 *qkv, *attn_o, *u, *hmid, *y;
   int *topk_idx, *cu_q, *tok_seq, *tok_pos, *tok_slot, *status;
   PermuteBuffers pb;
   int max_splits, pages_per_split;
   // static tensor maps
-  CUtensorMap tm_wqkv, tm_attn_o, tm_wo, tm_uperm, tm_wgu, tm_hmid, tm_wd;
+  CUtensorMap tm_wqkv, tm_attn_o, tm_wo, tm_wgu, tm_hmid, tm_wd;
   CUtensorMap tm_qkv;
   CUtensorMap tms_wqkv, tms_wo, tms_wgu, tms_wd;   // same weights, boxes sized for the decode kernels
   // call state
@@ -214,16 +214,16 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
   const int R = S * H * L->kc;
 
   if (!decode) {
-    launch_gather_rows(L->u, L->pb.perm, L->u_perm, R, d, st);
-    L->launches += 1;
     stage_mark(L, kStGemm1, st);
     GemmArgs g1;
     memset(&g1, 0, sizeof(g1));
     g1.n_groups = L->E; g1.mt_group = L->pb.mt_group; g1.mt_row0 = L->pb.mt_row0; g1.group_end = L->pb.offsets + 1;
     g1.n_mtiles = L->pb.n_mtiles; g1.N = 2 * L->I; g1.K = d; g1.status = L->status; g1.out = L->hmid; g1.ldo = L->I;
-    launch_gemm(kEpiSwiGLU, L->tm_uperm, L->tm_wgu, g1, L->n_sms, st);
+    g1.a_gather = L->u; g1.a_row_index = L->pb.perm;      // rows of u gathered through the dispatch map
+    launch_gemm(kEpiSwiGLU, L->tm_hmid, L->tm_wgu, g1, L->n_sms, st);   // the A map is unused with a gathered A
     stage_mark(L, kStGemm2, st);
     GemmArgs g2 = g1;
+    g2.a_gather = nullptr; g2.a_row_index = nullptr;
     g2.N = d; g2.K = L->I; g2.out = L->y; g2.ldo = d;
     launch_gemm(kEpiBf16, L->tm_hmid, L->tm_wd, g2, L->n_sms, st);
     L->launches += 2;
@@ -335,7 +335,6 @@ foe_status foe_layer_create(const foe_config* cfg, const foe_weights* w, foe_lay
   ok = ok && dalloc(L, &L->qkv, size_t(S) * L->qkv_cols);
   ok = ok && dalloc(L, &L->attn_o, size_t(S + 128) * L->n_q * dh);
   ok = ok && dalloc(L, &L->u, size_t(S) * d);
-  ok = ok && dalloc(L, &L->u_perm, size_t(R + 128) * d);
   ok = ok && dalloc(L, &L->hmid, size_t(R + 128) * I);
   ok = ok && dalloc(L, &L->y, size_t(R) * d);
   ok = ok && dalloc(L, &L->cu_q, size_t(cfg->max_seqs) + 1);
@@ -359,7 +358,6 @@ foe_status foe_layer_create(const foe_config* cfg, const foe_weights* w, foe_lay
   cudaStream_t st = 0;
   cudaMemsetAsync(L->status, 0, sizeof(int), st);
   cudaMemsetAsync(L->attn_o, 0, size_t(S + 128) * L->n_q * dh * sizeof(bf16), st);
-  cudaMemsetAsync(L->u_perm, 0, size_t(R + 128) * d * sizeof(bf16), st);
   cudaMemsetAsync(L->hmid, 0, size_t(R + 128) * I * sizeof(bf16), st);
   // K-major ("transposed") weights; the attention-norm gain is folded into W_q|k|v.
   const bf16* gain_a = static_cast<const bf16*>(w->attn_norm_g);
@@ -401,7 +399,6 @@ foe_status foe_layer_create(const foe_config* cfg, const foe_weights* w, foe_lay
   ok = make_map_2d(&L->tm_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, kBN) &&
        make_map_2d(&L->tm_attn_o, L->attn_o, uint64_t(S), uint64_t(L->n_q) * dh, kBM) &&
        make_map_2d(&L->tm_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, kBN) &&
-       make_map_2d(&L->tm_uperm, L->u_perm, uint64_t(R), d, kBM) &&
        make_map_2d(&L->tm_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, kBN) &&
        make_map_2d(&L->tm_hmid, L->hmid, uint64_t(R), I, kBM) &&
        make_map_2d(&L->tm_wd, L->wd_t, uint64_t(E) * d, I, kBN) &&

@@ -29,6 +29,9 @@ struct GemmArgs {
   int N;                    // columns per group (rows of B per group)
   int K;
   int* status;              // device status word
+  // gathered A operand (expert GEMM 1): A row r of a tile is a_gather[a_row_index[r]][:]; nullptr = A through tmA
+  const __nv_bfloat16* a_gather;
+  const int* a_row_index;
   // epilogue
   void* out;
   int ldo;                  // elements per output row

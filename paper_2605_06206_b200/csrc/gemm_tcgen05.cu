@@ -6,13 +6,13 @@ namespace foe {
 
 cudaError_t gemm_configure() {
   cudaError_t e;
-  e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kEpiBf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmemBytes));
+  e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kEpiBf16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmemBytes));
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kEpiSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmemBytes));
+  e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kEpiSwiGLU, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmemBytes));
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kEpiQKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmemBytes));
+  e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kEpiQKV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmemBytes));
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kEpiOProj>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmemBytes));
+  e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kEpiOProj, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmemBytes));
   return e;
 }
 
@@ -25,10 +25,12 @@ void launch_gemm(int epi, const CUtensorMap& tmA, const CUtensorMap& tmB, const 
     if (grid <= 0) return;
   }
   switch (epi) {
-    case kEpiBf16: gemm_tcgen05_kernel<kEpiBf16><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(tmA, tmB, args); break;
-    case kEpiSwiGLU: gemm_tcgen05_kernel<kEpiSwiGLU><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(tmA, tmB, args); break;
-    case kEpiQKV: gemm_tcgen05_kernel<kEpiQKV><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(tmA, tmB, args); break;
-    default: gemm_tcgen05_kernel<kEpiOProj><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(tmA, tmB, args); break;
+    case kEpiBf16: gemm_tcgen05_kernel<kEpiBf16, false><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(tmA, tmB, args); break;
+    case kEpiSwiGLU:   // expert GEMM 1: always fed through the dispatch permutation
+      gemm_tcgen05_kernel<kEpiSwiGLU, true><<<grid, kGemmThreads + kGatherThreads, kGemmSmemBytes, st>>>(tmA, tmB, args);
+      break;
+    case kEpiQKV: gemm_tcgen05_kernel<kEpiQKV, false><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(tmA, tmB, args); break;
+    default: gemm_tcgen05_kernel<kEpiOProj, false><<<grid, kGemmThreads, kGemmSmemBytes, st>>>(tmA, tmB, args); break;
   }
 }
 

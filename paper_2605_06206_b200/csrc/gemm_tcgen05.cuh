@@ -25,6 +25,8 @@ constexpr int kABytes = kBM * kBK * 2;   // 16 KB
 constexpr int kBBytes = kBN * kBK * 2;   // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kGemmThreads = 192;
+constexpr int kGatherThreads = 128;   // extra producer warps when the A rows are gathered
+constexpr int kGatherAhead = 2;       // cp.async groups a gather thread keeps in flight
 constexpr int kTmemCols = 512;
 constexpr int kStgPitch = 128 + 16;                 // staging row: 128 bytes of output + bank-spreading pad
 constexpr int kStgWarpBytes = 32 * kStgPitch;        // one epilogue warp stages its 32 rows
@@ -32,8 +34,8 @@ constexpr size_t kGemmSmemBytes = size_t(kStages) * kStageBytes + 4 * kStgWarpBy
 
 __device__ __forceinline__ float silu_f(float z) { return z / (1.0f + __expf(-z)); }
 
-template <int EPI>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+template <int EPI, bool GATHER>
+__global__ void __launch_bounds__(kGemmThreads + (GATHER ? kGatherThreads : 0), 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const GemmArgs args) {
   extern __shared__ uint8_t smem_raw[];
@@ -49,7 +51,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], GATHER ? 1 + kGatherThreads / 32 : 1); mbar_init(&empty_bar[s], 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); }
     mbar_fence_init();
     tma_prefetch_desc(&tmA);
@@ -86,8 +88,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1)) { ok = false; break; }
           uint8_t* sa = smem + stage * kStageBytes;
-          mbar_expect_tx(&full_bar[stage], kStageBytes);
-          tma_load_2d(sa, &tmA, &full_bar[stage], kb * kBK, row0);
+          if constexpr (GATHER) {
+            mbar_expect_tx(&full_bar[stage], kBBytes);       // the A half arrives through the gather warps
+          } else {
+            mbar_expect_tx(&full_bar[stage], kStageBytes);
+            tma_load_2d(sa, &tmA, &full_bar[stage], kb * kBK, row0);
+          }
           tma_load_2d(sa + kABytes, &tmB, &full_bar[stage], kb * kBK, brow0);
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
@@ -125,7 +131,60 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
       if (!ok) atomicExch(args.status, kStatusTimeout);
     }
-  } else {
+  } else if (GATHER && warp >= 6) {
+    // ------------------------------------------------------------ A-gather producers (4 warps, one tile row each)
+    // Row r of the tile is row a_row_index[row0 + r] of a_gather: the dispatch permutation is applied while
+    // the operand is staged, so the permuted activations are never written to memory.  Each thread copies one
+    // 16-byte chunk of eight rows per k-block with cp.async into the 128-byte-swizzled operand layout, keeps
+    // kGatherAhead groups in flight, and makes a finished group visible to the tensor core (async proxy
+    // fence) before its warp arrives on the stage's barrier.
+    const int gt = threadIdx.x - kGemmThreads;            // 0..127
+    const int gc = gt & 7, gr = gt >> 3;                  // 16-byte chunk of a row; rows gr + 16 j, j < 8:
+                                                          // 8 lanes read one row's 128 bytes as a whole line
+    int stage = 0, arr_stage = 0;
+    uint32_t phase = 0;
+    int issued = 0;
+    bool ok = true;
+    auto retire = [&](int pending) {                       // arrive for the oldest un-signalled group
+      if (pending == 2) asm volatile("cp.async.wait_group 2;" ::: "memory");
+      else if (pending == 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
+      else asm volatile("cp.async.wait_group 0;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&full_bar[arr_stage]);
+      if (++arr_stage == kStages) arr_stage = 0;
+    };
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int mt = tile / n_ntiles;
+      const int group = args.mt_group[mt], row0 = args.mt_row0[mt], row_end = args.group_end[group];
+      const uint8_t* src[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int src_row = args.a_row_index[min(row0 + gr + 16 * j, row_end - 1)];
+        src[j] = reinterpret_cast<const uint8_t*>(args.a_gather) + size_t(src_row) * args.K * 2 + gc * 16;
+      }
+      for (int kb = 0; kb < kblocks; ++kb) {
+        if (!mbar_wait(&empty_bar[stage], phase ^ 1)) { ok = false; break; }
+        const uint32_t dst = smem_u32(smem + stage * kStageBytes);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int r = gr + 16 * j;
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + r * 128 + ((gc ^ (r & 7)) << 4)),
+                       "l"(src[j] + size_t(kb) * 128) : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        ++issued;
+        if (issued > kGatherAhead) retire(kGatherAhead);
+        if (++stage == kStages) { stage = 0; phase ^= 1; }
+      }
+    }
+    if (ok) {
+      int left = issued < kGatherAhead ? issued : kGatherAhead;
+      while (left > 0) { retire(left - 1); --left; }
+    } else if (lane == 0) {
+      atomicExch(args.status, kStatusTimeout);
+    }
+  } else if (warp >= 2 && warp < 6) {
     // ------------------------------------------------------------ epilogue (4 warps = 128 TMEM lanes)
     const int quarter = warp & 3;                 // a warp may only touch TMEM lanes 32*(warp%4)..+31
     const int row_in_tile = quarter * 32 + lane;

@@ -57,8 +57,6 @@ struct PermuteBuffers {
 constexpr int kPermuteBlockTokens = 256;
 void launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int sel_per_token, int E, int tile_rows,
                     int* status, cudaStream_t st);
-// u_perm[slot, :] = u[perm[slot], :]   (16-byte vector copies)
-void launch_gather_rows(const bf16* u, const int* perm, bf16* u_perm, int n_rows, int d, cudaStream_t st);
 
 // ---- attention.cu
 struct AttnArgs {

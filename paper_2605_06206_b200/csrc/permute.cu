@@ -6,10 +6,11 @@
 //   offsets    = exclusive scan of counts over the global expert id
 //   perm[slot] = token of the slot,  inv[token, cluster, j] = slot
 //
-// Three launches: (1) every block of 256 tokens builds a token-bitmap per expert in shared memory,
+// The activation rows themselves are not moved here: expert GEMM 1 gathers them through perm while it stages
+// its A operand.  Three launches: (1) every block of 256 tokens builds a token-bitmap per expert in shared memory,
 // from which each selection reads its rank inside the block; (2) one block scans block counts and
 // expert totals and writes the m-tile table the grouped GEMM walks; (3) every selection computes its
-// slot.  A fourth kernel moves activation rows into slot order with 16-byte vector copies.
+// slot.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -114,23 +115,6 @@ void launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int 
   const int total = n_tokens * sel;
   permute_scatter_kernel<<<(total + 255) / 256, 256, 0, st>>>(idx, pb.rank, pb.blk_counts, pb.offsets, pb.perm, pb.inv,
                                                             n_tokens, sel, E);
-}
-
-// One warp per slot: u_perm[slot, :] = u[perm[slot], :], 16 bytes per lane per step.
-__global__ void gather_rows_kernel(const bf16* __restrict__ u, const int* __restrict__ perm, bf16* __restrict__ u_perm,
-                                   int n_rows, int d) {
-  const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (row >= n_rows) return;
-  const uint4* src = reinterpret_cast<const uint4*>(u + size_t(perm[row]) * d);
-  uint4* dst = reinterpret_cast<uint4*>(u_perm + size_t(row) * d);
-  for (int c = lane; c < d / 8; c += 32) dst[c] = __ldg(src + c);
-}
-
-void launch_gather_rows(const bf16* u, const int* perm, bf16* u_perm, int n_rows, int d, cudaStream_t st) {
-  if (n_rows <= 0) return;
-  const long long threads = (long long)n_rows * 32;
-  gather_rows_kernel<<<unsigned((threads + 255) / 256), 256, 0, st>>>(u, perm, u_perm, n_rows, d);
 }
 
 }  // namespace foe
