@@ -126,6 +126,14 @@ typedef struct foe_layer foe_layer;
  * default stream and synchronises.  *out receives the handle. */
 foe_status foe_layer_create(const foe_config* config, const foe_weights* weights, foe_layer** out);
 
+/* Same as foe_layer_create, but the new layer borrows the workspace of `donor` instead of allocating its own
+ * (a 16-layer stack needs one workspace, not sixteen).  The two layers must agree in every shape field and in
+ * max_tokens / max_seqs / max_context (FOE_ERR_SHAPE otherwise); position, sync, rope_theta and rms_eps may differ.
+ * Layers that share a workspace must not run concurrently; foe_get_aux of any of them shows the intermediates of
+ * whichever ran last.  The workspace is released when its last user is destroyed.  donor == NULL allocates. */
+foe_status foe_layer_create_shared(const foe_config* config, const foe_weights* weights, foe_layer* donor,
+                                   foe_layer** out);
+
 /* Frees everything the handle owns.  NULL is accepted. */
 foe_status foe_layer_destroy(foe_layer* layer);
 

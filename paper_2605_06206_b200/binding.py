@@ -21,7 +21,7 @@ SYNCS = {"mean": 0, "sum": 1}
 
 EXPORTS = ["foe_layer_create", "foe_layer_destroy", "foe_prefill", "foe_decode", "foe_route", "foe_get_aux",
            "foe_poll_status", "foe_last_launch_count", "foe_status_string", "foe_set_profiling", "foe_num_stages",
-           "foe_stage_name", "foe_get_stage_ms", "foe_route_noalloc"]
+           "foe_stage_name", "foe_get_stage_ms", "foe_route_noalloc", "foe_layer_create_shared"]
 
 
 class FoeConfig(ctypes.Structure):
@@ -66,6 +66,8 @@ def load_library() -> ctypes.CDLL:
     vp, ci = ctypes.c_void_p, ctypes.c_int
     lib.foe_layer_create.argtypes = [ctypes.POINTER(FoeConfig), ctypes.POINTER(FoeWeights), ctypes.POINTER(vp)]
     lib.foe_layer_create.restype = ci
+    lib.foe_layer_create_shared.argtypes = [ctypes.POINTER(FoeConfig), ctypes.POINTER(FoeWeights), vp, ctypes.POINTER(vp)]
+    lib.foe_layer_create_shared.restype = ci
     lib.foe_layer_destroy.argtypes = [vp]
     lib.foe_layer_destroy.restype = ci
     for name in ("foe_prefill", "foe_decode"):
@@ -135,7 +137,8 @@ def _stream_ptr(stream) -> int:
 class FoeLayer:
     """One FoE block on the current CUDA device (foe_layer_create / foe_prefill / foe_decode / foe_route)."""
 
-    def __init__(self, shape, weights: Dict[str, torch.Tensor], max_tokens: int, max_seqs: int, max_context: int):
+    def __init__(self, shape, weights: Dict[str, torch.Tensor], max_tokens: int, max_seqs: int, max_context: int,
+                 share_workspace_with: Optional["FoeLayer"] = None):
         if not torch.cuda.is_available():
             raise RuntimeError("FoeLayer needs a CUDA device: the block has no CPU path")
         self.lib = load_library()
@@ -153,7 +156,9 @@ class FoeLayer:
             setattr(w, name, _ptr(t))
         h = ctypes.c_void_p()
         torch.cuda.synchronize()
-        _check(self.lib.foe_layer_create(ctypes.byref(cfg), ctypes.byref(w), ctypes.byref(h)), "foe_layer_create")
+        donor = share_workspace_with.handle if share_workspace_with is not None else None
+        _check(self.lib.foe_layer_create_shared(ctypes.byref(cfg), ctypes.byref(w), donor, ctypes.byref(h)),
+               "foe_layer_create")
         self.handle = h
         self.max_tokens, self.max_seqs, self.max_context = max_tokens, max_seqs, max_context
 

@@ -50,6 +50,18 @@ const char* kStageNames[kNumStages] = {"prep", "qkv_proj", "rope_kv_write", "att
 
 }  // namespace
 
+// Per-call scratch.  Layers of one stack run one after the other on a stream, so they can share one workspace
+// (foe_layer_create_shared); it is freed with its last user.
+struct foe_workspace {
+  int refs;
+  std::vector<void*> allocs;
+  float *inv_rms, *inv_rms_f, *route_part, *r_full, *logits, *topk_w, *part_o, *part_ml;
+  bf16 *qkv, *attn_o, *u, *hmid, *y;
+  int *topk_idx, *cu_q, *tok_seq, *tok_pos, *tok_slot, *status;
+  PermuteBuffers pb;
+  CUtensorMap tm_attn_o, tm_hmid, tm_qkv;       // maps of workspace buffers (A operands, attention Q)
+};
+
 struct foe_layer {
   foe_config cfg;
   int H, g, c, dh, d, I, E, Ec, kc, n_q, n_kv, qkv_cols, S_max, R_max, n_sms;
@@ -59,15 +71,10 @@ struct foe_layer {
   bf16 *wqkv_t, *wo_t, *wgu_t, *wd_t, *ffn_gain;
   float *router_w, *router_b;
   float2* rope_tab;
-  // workspace
-  float *inv_rms, *inv_rms_f, *route_part, *r_full, *logits, *topk_w, *part_o, *part_ml;
-  bf16 *qkv, *attn_o, *u, *hmid, *y;
-  int *topk_idx, *cu_q, *tok_seq, *tok_pos, *tok_slot, *status;
-  PermuteBuffers pb;
+  foe_workspace* ws;
   int max_splits, pages_per_split;
-  // static tensor maps
-  CUtensorMap tm_wqkv, tm_attn_o, tm_wo, tm_wgu, tm_hmid, tm_wd;
-  CUtensorMap tm_qkv;
+  // tensor maps of the weights
+  CUtensorMap tm_wqkv, tm_wo, tm_wgu, tm_wd;
   CUtensorMap tms_wqkv, tms_wo, tms_wgu, tms_wd;   // same weights, boxes sized for the decode kernels
   // call state
   cudaStream_t last_stream;
@@ -87,6 +94,23 @@ bool dalloc(foe_layer* L, T** p, size_t count) {
   L->allocs.push_back(q);
   *p = static_cast<T*>(q);
   return true;
+}
+
+template <typename T>
+bool walloc(foe_workspace* W, T** p, size_t count) {
+  void* q = nullptr;
+  if (count == 0) count = 1;
+  if (cudaMalloc(&q, count * sizeof(T)) != cudaSuccess) { cudaGetLastError(); return false; }
+  W->allocs.push_back(q);
+  *p = static_cast<T*>(q);
+  return true;
+}
+
+void ws_release(foe_workspace* W) {
+  if (!W) return;
+  if (--W->refs > 0) return;
+  for (void* p : W->allocs) cudaFree(p);
+  delete W;
 }
 
 foe_status validate(const foe_config* c) {
@@ -115,10 +139,10 @@ foe_status check_launch() { return cudaGetLastError() == cudaSuccess ? FOE_OK : 
 
 // routing + dispatch maps for n tokens whose synced residual is r (fp32 internal or bf16 from the caller)
 void run_route_and_permute(foe_layer* L, const void* r, int r_is_bf16, int n, cudaStream_t st) {
-  L->launches += launch_route(r, r_is_bf16, L->ffn_gain, L->router_w, L->router_b, L->u, L->inv_rms_f, L->route_part,
-                              L->logits, L->topk_idx, L->topk_w, n, L->d, L->H, L->Ec, L->kc, L->cfg.rms_eps, L->n_sms, st);
+  L->launches += launch_route(r, r_is_bf16, L->ffn_gain, L->router_w, L->router_b, L->ws->u, L->ws->inv_rms_f, L->ws->route_part,
+                              L->ws->logits, L->ws->topk_idx, L->ws->topk_w, n, L->d, L->H, L->Ec, L->kc, L->cfg.rms_eps, L->n_sms, st);
   stage_mark(L, kStPermute, st);
-  launch_permute(L->topk_idx, L->pb, n, L->H * L->kc, L->E, 128, L->status, st);
+  launch_permute(L->ws->topk_idx, L->ws->pb, n, L->H * L->kc, L->E, 128, L->ws->status, st);
   L->launches += 3;
 }
 
@@ -140,9 +164,9 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
   // ---- prep: token map and pre-attention RMS statistics
   stage_mark(L, kStPrep, st);
   launch_token_map(decode ? nullptr : kv->q_lens, kv->context_lens, kv->block_table, kv->n_seqs, kv->max_pages_per_seq,
-                   kv->num_pages, 64, S, L->cfg.max_context, L->cu_q, L->tok_seq, L->tok_pos, L->tok_slot, L->status, st);
+                   kv->num_pages, 64, S, L->cfg.max_context, L->ws->cu_q, L->ws->tok_seq, L->ws->tok_pos, L->ws->tok_slot, L->ws->status, st);
   const int x_rows = L->first ? S : H * S;
-  launch_row_inv_rms(xb, L->inv_rms, x_rows, d, L->cfg.rms_eps, st);
+  launch_row_inv_rms(xb, L->ws->inv_rms, x_rows, d, L->cfg.rms_eps, st);
   L->launches += 3;
 
   // ---- per-cluster QKV projection (norm gain folded into the weights, 1/rms applied in the epilogue)
@@ -152,26 +176,26 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     GemmArgs ga;
     memset(&ga, 0, sizeof(ga));
     ga.n_groups = H; ga.rows_per_group = S; ga.a_group_stride = L->first ? 0 : S;
-    ga.N = (L->g + 2 * L->c) * dh; ga.K = d; ga.status = L->status;
-    ga.out = L->qkv; ga.ldo = L->qkv_cols;
-    ga.row_scale = L->inv_rms; ga.scale_group_stride = L->first ? 0 : S;
+    ga.N = (L->g + 2 * L->c) * dh; ga.K = d; ga.status = L->ws->status;
+    ga.out = L->ws->qkv; ga.ldo = L->qkv_cols;
+    ga.row_scale = L->ws->inv_rms; ga.scale_group_stride = L->first ? 0 : S;
     ga.q_cols = L->g * dh; ga.kv_cols = L->c * dh; ga.q_total = L->n_q * dh; ga.kv_total = L->n_kv * dh;
     launch_gemm(kEpiQKV, tmX, L->tm_wqkv, ga, L->n_sms, st);
   } else {
     SmallMArgs sa;
     memset(&sa, 0, sizeof(sa));
     sa.W = L->wqkv_t; sa.X = xb; sa.ldx = d; sa.n_groups = H; sa.rows_per_group = S; sa.x_group_stride = L->first ? 0 : S;
-    sa.N = (L->g + 2 * L->c) * dh; sa.K = d; sa.epi = kEpiQKV; sa.out = L->qkv; sa.ldo = L->qkv_cols;
-    sa.row_scale = L->inv_rms; sa.scale_group_stride = L->first ? 0 : S;
+    sa.N = (L->g + 2 * L->c) * dh; sa.K = d; sa.epi = kEpiQKV; sa.out = L->ws->qkv; sa.ldo = L->qkv_cols;
+    sa.row_scale = L->ws->inv_rms; sa.scale_group_stride = L->first ? 0 : S;
     sa.q_cols = L->g * dh; sa.kv_cols = L->c * dh; sa.q_total = L->n_q * dh; sa.kv_total = L->n_kv * dh;
-    sa.status = L->status;
+    sa.status = L->ws->status;
     launch_smallm(L->tms_wqkv, sa, st);
   }
   L->launches += 1;
 
   // ---- RoPE, K/V into the pages
   stage_mark(L, kStRope, st);
-  launch_rope_kv_write(L->qkv, L->rope_tab, L->tok_pos, L->tok_slot, static_cast<bf16*>(kv->k_pages),
+  launch_rope_kv_write(L->ws->qkv, L->rope_tab, L->ws->tok_pos, L->ws->tok_slot, static_cast<bf16*>(kv->k_pages),
                        static_cast<bf16*>(kv->v_pages), S, L->n_q, L->n_kv, dh, 64, st);
   L->launches += 1;
 
@@ -179,14 +203,14 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
   stage_mark(L, kStAttn, st);
   AttnArgs aa;
   memset(&aa, 0, sizeof(aa));
-  aa.qkv = L->qkv; aa.out = L->attn_o; aa.cu_q = L->cu_q; aa.context_lens = kv->context_lens;
+  aa.qkv = L->ws->qkv; aa.out = L->ws->attn_o; aa.cu_q = L->ws->cu_q; aa.context_lens = kv->context_lens;
   aa.q_lens = decode ? nullptr : kv->q_lens; aa.block_table = kv->block_table; aa.n_seqs = kv->n_seqs;
   aa.max_pages_per_seq = kv->max_pages_per_seq; aa.num_pages = kv->num_pages; aa.n_q = L->n_q; aa.n_kv = L->n_kv;
   aa.dh = dh; aa.max_q_len = decode ? 1 : kv->max_q_len; aa.scale_log2 = float(1.4426950408889634 / sqrt(double(dh)));
-  aa.status = L->status; aa.part_o = L->part_o; aa.part_ml = L->part_ml; aa.max_splits = L->max_splits;
+  aa.status = L->ws->status; aa.part_o = L->ws->part_o; aa.part_ml = L->ws->part_ml; aa.max_splits = L->max_splits;
   aa.pages_per_split = L->pages_per_split;
   if (decode) { launch_attn_decode(tmK, tmV, aa, st); L->launches += 2; }
-  else { launch_attn_prefill_tc(L->tm_qkv, tmK, tmV, aa, st); L->launches += 1; }
+  else { launch_attn_prefill_tc(L->ws->tm_qkv, tmK, tmV, aa, st); L->launches += 1; }
 
   // ---- output projection; the cross-cluster sync is its K-reduction plus the sum of x[h] in the epilogue
   stage_mark(L, kStOproj, st);
@@ -194,60 +218,60 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
   if (!decode) {
     GemmArgs ga;
     memset(&ga, 0, sizeof(ga));
-    ga.n_groups = 1; ga.rows_per_group = S; ga.a_group_stride = 0; ga.N = d; ga.K = L->n_q * dh; ga.status = L->status;
-    ga.out = L->r_full; ga.ldo = d; ga.xsum = xb; ga.x_count = L->first ? 1 : H; ga.x_stride = size_t(S) * d;
+    ga.n_groups = 1; ga.rows_per_group = S; ga.a_group_stride = 0; ga.N = d; ga.K = L->n_q * dh; ga.status = L->ws->status;
+    ga.out = L->ws->r_full; ga.ldo = d; ga.xsum = xb; ga.x_count = L->first ? 1 : H; ga.x_stride = size_t(S) * d;
     ga.out_scale = out_scale;
-    launch_gemm(kEpiOProj, L->tm_attn_o, L->tm_wo, ga, L->n_sms, st);
+    launch_gemm(kEpiOProj, L->ws->tm_attn_o, L->tm_wo, ga, L->n_sms, st);
   } else {
     SmallMArgs sa;
     memset(&sa, 0, sizeof(sa));
-    sa.W = L->wo_t; sa.X = L->attn_o; sa.ldx = L->n_q * dh; sa.n_groups = 1; sa.rows_per_group = S; sa.N = d;
-    sa.K = L->n_q * dh; sa.epi = kEpiOProj; sa.out = L->r_full; sa.ldo = d; sa.xsum = xb; sa.x_count = L->first ? 1 : H;
-    sa.x_stride = size_t(S) * d; sa.out_scale = out_scale; sa.status = L->status;
+    sa.W = L->wo_t; sa.X = L->ws->attn_o; sa.ldx = L->n_q * dh; sa.n_groups = 1; sa.rows_per_group = S; sa.N = d;
+    sa.K = L->n_q * dh; sa.epi = kEpiOProj; sa.out = L->ws->r_full; sa.ldo = d; sa.xsum = xb; sa.x_count = L->first ? 1 : H;
+    sa.x_stride = size_t(S) * d; sa.out_scale = out_scale; sa.status = L->ws->status;
     launch_smallm(L->tms_wo, sa, st);
   }
   L->launches += 1;
 
   // ---- router, top-k, gates, dispatch maps
   stage_mark(L, kStRoute, st);
-  run_route_and_permute(L, L->r_full, 0, S, st);
+  run_route_and_permute(L, L->ws->r_full, 0, S, st);
   const int R = S * H * L->kc;
 
   if (!decode) {
     stage_mark(L, kStGemm1, st);
     GemmArgs g1;
     memset(&g1, 0, sizeof(g1));
-    g1.n_groups = L->E; g1.mt_group = L->pb.mt_group; g1.mt_row0 = L->pb.mt_row0; g1.group_end = L->pb.offsets + 1;
-    g1.n_mtiles = L->pb.n_mtiles; g1.N = 2 * L->I; g1.K = d; g1.status = L->status; g1.out = L->hmid; g1.ldo = L->I;
-    g1.a_gather = L->u; g1.a_row_index = L->pb.perm;      // rows of u gathered through the dispatch map
-    launch_gemm(kEpiSwiGLU, L->tm_hmid, L->tm_wgu, g1, L->n_sms, st);   // the A map is unused with a gathered A
+    g1.n_groups = L->E; g1.mt_group = L->ws->pb.mt_group; g1.mt_row0 = L->ws->pb.mt_row0; g1.group_end = L->ws->pb.offsets + 1;
+    g1.n_mtiles = L->ws->pb.n_mtiles; g1.N = 2 * L->I; g1.K = d; g1.status = L->ws->status; g1.out = L->ws->hmid; g1.ldo = L->I;
+    g1.a_gather = L->ws->u; g1.a_row_index = L->ws->pb.perm;      // rows of u gathered through the dispatch map
+    launch_gemm(kEpiSwiGLU, L->ws->tm_hmid, L->tm_wgu, g1, L->n_sms, st);   // the A map is unused with a gathered A
     stage_mark(L, kStGemm2, st);
     GemmArgs g2 = g1;
     g2.a_gather = nullptr; g2.a_row_index = nullptr;
-    g2.N = d; g2.K = L->I; g2.out = L->y; g2.ldo = d;
-    launch_gemm(kEpiBf16, L->tm_hmid, L->tm_wd, g2, L->n_sms, st);
+    g2.N = d; g2.K = L->I; g2.out = L->ws->y; g2.ldo = d;
+    launch_gemm(kEpiBf16, L->ws->tm_hmid, L->tm_wd, g2, L->n_sms, st);
     L->launches += 2;
   } else {
     stage_mark(L, kStGemm1, st);
     SmallMArgs s1;
     memset(&s1, 0, sizeof(s1));
-    s1.W = L->wgu_t; s1.X = L->u; s1.ldx = d; s1.row_index = L->pb.perm; s1.group_offsets = L->pb.offsets;
-    s1.n_groups = L->E; s1.N = 2 * L->I; s1.K = d; s1.epi = kEpiSwiGLU; s1.out = L->hmid; s1.ldo = L->I;
-    s1.status = L->status;
+    s1.W = L->wgu_t; s1.X = L->ws->u; s1.ldx = d; s1.row_index = L->ws->pb.perm; s1.group_offsets = L->ws->pb.offsets;
+    s1.n_groups = L->E; s1.N = 2 * L->I; s1.K = d; s1.epi = kEpiSwiGLU; s1.out = L->ws->hmid; s1.ldo = L->I;
+    s1.status = L->ws->status;
     launch_smallm(L->tms_wgu, s1, st);
     stage_mark(L, kStGemm2, st);
     SmallMArgs s2;
     memset(&s2, 0, sizeof(s2));
-    s2.W = L->wd_t; s2.X = L->hmid; s2.ldx = L->I; s2.group_offsets = L->pb.offsets; s2.n_groups = L->E; s2.N = d;
-    s2.K = L->I; s2.epi = kEpiBf16; s2.out = L->y; s2.ldo = d;
-    s2.status = L->status;
+    s2.W = L->wd_t; s2.X = L->ws->hmid; s2.ldx = L->I; s2.group_offsets = L->ws->pb.offsets; s2.n_groups = L->E; s2.N = d;
+    s2.K = L->I; s2.epi = kEpiBf16; s2.out = L->ws->y; s2.ldo = d;
+    s2.status = L->ws->status;
     launch_smallm(L->tms_wd, s2, st);
     L->launches += 2;
   }
 
   // ---- weighted combine, residual, last-layer mean
   stage_mark(L, kStCombine, st);
-  launch_combine(L->r_full, L->y, L->topk_w, L->pb.inv, static_cast<bf16*>(out), S, d, H, L->kc, L->last ? 1 : 0, st);
+  launch_combine(L->ws->r_full, L->ws->y, L->ws->topk_w, L->ws->pb.inv, static_cast<bf16*>(out), S, d, H, L->kc, L->last ? 1 : 0, st);
   L->launches += 1;
   if (L->profiling) { cudaEventRecord(L->ev[kNumStages], st); L->ev_valid = true; }
   return check_launch();
@@ -275,6 +299,7 @@ const char* foe_status_string(int s) {
 foe_status foe_layer_destroy(foe_layer* L) {
   if (!L) return FOE_OK;
   for (void* p : L->allocs) cudaFree(p);
+  ws_release(L->ws);
   for (int i = 0; i <= kNumStages; ++i)
     if (L->ev[i]) cudaEventDestroy(L->ev[i]);
   delete L;
@@ -282,6 +307,10 @@ foe_status foe_layer_destroy(foe_layer* L) {
 }
 
 foe_status foe_layer_create(const foe_config* cfg, const foe_weights* w, foe_layer** out) {
+  return foe_layer_create_shared(cfg, w, nullptr, out);
+}
+
+foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, foe_layer* donor, foe_layer** out) {
   if (!cfg || !w || !out) return FOE_ERR_NULL;
   *out = nullptr;
   const foe_status v = validate(cfg);
@@ -296,6 +325,15 @@ foe_status foe_layer_create(const foe_config* cfg, const foe_weights* w, foe_lay
   if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return FOE_ERR_CUDA;
   if (prop.major != 10) return FOE_ERR_UNSUPPORTED;       // tcgen05/TMEM kernels: sm_100 only
   if (gemm_configure() != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  if (donor) {   // a shared workspace must have been sized for exactly these shapes
+    const foe_config& a = donor->cfg;
+    if (a.hidden != cfg->hidden || a.n_q_heads != cfg->n_q_heads || a.n_kv_heads != cfg->n_kv_heads ||
+        a.n_clusters != cfg->n_clusters || a.head_dim != cfg->head_dim ||
+        a.experts_per_cluster != cfg->experts_per_cluster || a.top_k_per_cluster != cfg->top_k_per_cluster ||
+        a.ffn_inter != cfg->ffn_inter || a.max_tokens != cfg->max_tokens || a.max_seqs != cfg->max_seqs ||
+        a.max_context != cfg->max_context)
+      return FOE_ERR_SHAPE;
+  }
 
   foe_layer* L = new (std::nothrow) foe_layer();
   if (!L) return FOE_ERR_OOM;
@@ -325,40 +363,54 @@ foe_status foe_layer_create(const foe_config* cfg, const foe_weights* w, foe_lay
   ok = ok && dalloc(L, &L->router_w, size_t(E) * d);
   ok = ok && dalloc(L, &L->router_b, size_t(E));
   ok = ok && dalloc(L, &L->rope_tab, size_t(cfg->max_context) * (dh / 2));
-  ok = ok && dalloc(L, &L->inv_rms, size_t(H) * S);
-  ok = ok && dalloc(L, &L->r_full, size_t(S) * d);
-  ok = ok && dalloc(L, &L->logits, size_t(S) * E);
-  ok = ok && dalloc(L, &L->inv_rms_f, size_t(S));
-  ok = ok && dalloc(L, &L->route_part, size_t(S) * E > (size_t(1) << 21) ? size_t(S) * E : (size_t(1) << 21));
-  ok = ok && dalloc(L, &L->topk_w, size_t(R));
-  ok = ok && dalloc(L, &L->topk_idx, size_t(R));
-  ok = ok && dalloc(L, &L->qkv, size_t(S) * L->qkv_cols);
-  ok = ok && dalloc(L, &L->attn_o, size_t(S + 128) * L->n_q * dh);
-  ok = ok && dalloc(L, &L->u, size_t(S) * d);
-  ok = ok && dalloc(L, &L->hmid, size_t(R + 128) * I);
-  ok = ok && dalloc(L, &L->y, size_t(R) * d);
-  ok = ok && dalloc(L, &L->cu_q, size_t(cfg->max_seqs) + 1);
-  ok = ok && dalloc(L, &L->tok_seq, size_t(S));
-  ok = ok && dalloc(L, &L->tok_pos, size_t(S));
-  ok = ok && dalloc(L, &L->tok_slot, size_t(S));
-  ok = ok && dalloc(L, &L->status, size_t(1));
-  ok = ok && dalloc(L, &L->part_o, size_t(cfg->max_seqs) * L->n_q * L->max_splits * dh);
-  ok = ok && dalloc(L, &L->part_ml, size_t(cfg->max_seqs) * L->n_q * L->max_splits * 2);
-  ok = ok && dalloc(L, &L->pb.counts, size_t(E));
-  ok = ok && dalloc(L, &L->pb.offsets, size_t(E) + 1);
-  ok = ok && dalloc(L, &L->pb.perm, size_t(R));
-  ok = ok && dalloc(L, &L->pb.inv, size_t(R));
-  ok = ok && dalloc(L, &L->pb.rank, size_t(R));
-  ok = ok && dalloc(L, &L->pb.blk_counts, size_t(n_blocks) * E);
-  ok = ok && dalloc(L, &L->pb.mt_group, size_t(R / 128 + E + 1));
-  ok = ok && dalloc(L, &L->pb.mt_row0, size_t(R / 128 + E + 1));
-  ok = ok && dalloc(L, &L->pb.n_mtiles, size_t(1));
   if (!ok) { foe_layer_destroy(L); return FOE_ERR_OOM; }
-
   cudaStream_t st = 0;
-  cudaMemsetAsync(L->status, 0, sizeof(int), st);
-  cudaMemsetAsync(L->attn_o, 0, size_t(S + 128) * L->n_q * dh * sizeof(bf16), st);
-  cudaMemsetAsync(L->hmid, 0, size_t(R + 128) * I * sizeof(bf16), st);
+  if (donor) {
+    L->ws = donor->ws;
+    L->ws->refs += 1;
+  } else {
+    foe_workspace* W = new (std::nothrow) foe_workspace();
+    if (!W) { foe_layer_destroy(L); return FOE_ERR_OOM; }
+    W->refs = 1;
+    L->ws = W;
+    ok = ok && walloc(W, &W->inv_rms, size_t(H) * S);
+    ok = ok && walloc(W, &W->r_full, size_t(S) * d);
+    ok = ok && walloc(W, &W->logits, size_t(S) * E);
+    ok = ok && walloc(W, &W->inv_rms_f, size_t(S));
+    ok = ok && walloc(W, &W->route_part, size_t(S) * E > (size_t(1) << 21) ? size_t(S) * E : (size_t(1) << 21));
+    ok = ok && walloc(W, &W->topk_w, size_t(R));
+    ok = ok && walloc(W, &W->topk_idx, size_t(R));
+    ok = ok && walloc(W, &W->qkv, size_t(S) * L->qkv_cols);
+    ok = ok && walloc(W, &W->attn_o, size_t(S + 128) * L->n_q * dh);
+    ok = ok && walloc(W, &W->u, size_t(S) * d);
+    ok = ok && walloc(W, &W->hmid, size_t(R + 128) * I);
+    ok = ok && walloc(W, &W->y, size_t(R) * d);
+    ok = ok && walloc(W, &W->cu_q, size_t(cfg->max_seqs) + 1);
+    ok = ok && walloc(W, &W->tok_seq, size_t(S));
+    ok = ok && walloc(W, &W->tok_pos, size_t(S));
+    ok = ok && walloc(W, &W->tok_slot, size_t(S));
+    ok = ok && walloc(W, &W->status, size_t(1));
+    ok = ok && walloc(W, &W->part_o, size_t(cfg->max_seqs) * L->n_q * L->max_splits * dh);
+    ok = ok && walloc(W, &W->part_ml, size_t(cfg->max_seqs) * L->n_q * L->max_splits * 2);
+    ok = ok && walloc(W, &W->pb.counts, size_t(E));
+    ok = ok && walloc(W, &W->pb.offsets, size_t(E) + 1);
+    ok = ok && walloc(W, &W->pb.perm, size_t(R));
+    ok = ok && walloc(W, &W->pb.inv, size_t(R));
+    ok = ok && walloc(W, &W->pb.rank, size_t(R));
+    ok = ok && walloc(W, &W->pb.blk_counts, size_t(n_blocks) * E);
+    ok = ok && walloc(W, &W->pb.mt_group, size_t(R / 128 + E + 1));
+    ok = ok && walloc(W, &W->pb.mt_row0, size_t(R / 128 + E + 1));
+    ok = ok && walloc(W, &W->pb.n_mtiles, size_t(1));
+    if (!ok) { foe_layer_destroy(L); return FOE_ERR_OOM; }
+    cudaMemsetAsync(W->status, 0, sizeof(int), st);
+    cudaMemsetAsync(W->attn_o, 0, size_t(S + 128) * L->n_q * dh * sizeof(bf16), st);
+    cudaMemsetAsync(W->hmid, 0, size_t(R + 128) * I * sizeof(bf16), st);
+    ok = make_map_2d(&W->tm_attn_o, W->attn_o, uint64_t(S), uint64_t(L->n_q) * dh, kBM) &&
+         make_map_2d(&W->tm_hmid, W->hmid, uint64_t(R), I, kBM) &&
+         make_map_2d(&W->tm_qkv, W->qkv, uint64_t(S), uint64_t(L->qkv_cols), 128);
+    if (!ok) { foe_layer_destroy(L); return FOE_ERR_CUDA; }
+  }
+
   // K-major ("transposed") weights; the attention-norm gain is folded into W_q|k|v.
   const bf16* gain_a = static_cast<const bf16*>(w->attn_norm_g);
   const size_t qkv_batch = size_t(qkvN) * d;
@@ -397,12 +449,9 @@ foe_status foe_layer_create(const foe_config* cfg, const foe_weights* w, foe_lay
     return FOE_ERR_CUDA;
   }
   ok = make_map_2d(&L->tm_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, kBN) &&
-       make_map_2d(&L->tm_attn_o, L->attn_o, uint64_t(S), uint64_t(L->n_q) * dh, kBM) &&
        make_map_2d(&L->tm_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, kBN) &&
        make_map_2d(&L->tm_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, kBN) &&
-       make_map_2d(&L->tm_hmid, L->hmid, uint64_t(R), I, kBM) &&
        make_map_2d(&L->tm_wd, L->wd_t, uint64_t(E) * d, I, kBN) &&
-       make_map_2d(&L->tm_qkv, L->qkv, uint64_t(S), uint64_t(L->qkv_cols), 128) &&
        make_map_2d(&L->tms_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, 64) &&
        make_map_2d(&L->tms_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, 64) &&
        make_map_2d(&L->tms_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, 32) &&
@@ -451,8 +500,8 @@ foe_status foe_route(foe_layer* L, const void* h, int n_tokens, int* topk_idx, f
   run_route_and_permute(L, h, 1, n_tokens, st);
   L->profiling = saved;
   const size_t n = size_t(n_tokens) * L->H * L->kc;
-  cudaMemcpyAsync(topk_idx, L->topk_idx, n * sizeof(int), cudaMemcpyDeviceToDevice, st);
-  cudaMemcpyAsync(topk_w, L->topk_w, n * sizeof(float), cudaMemcpyDeviceToDevice, st);
+  cudaMemcpyAsync(topk_idx, L->ws->topk_idx, n * sizeof(int), cudaMemcpyDeviceToDevice, st);
+  cudaMemcpyAsync(topk_w, L->ws->topk_w, n * sizeof(float), cudaMemcpyDeviceToDevice, st);
   return check_launch();
 }
 
@@ -474,9 +523,9 @@ foe_status foe_route_noalloc(int hidden, int n_clusters, int experts_per_cluster
 foe_status foe_get_aux(foe_layer* L, foe_aux* a) {
   if (!L || !a) return FOE_ERR_NULL;
   a->n_tokens = L->last_tokens;
-  a->r_full = L->r_full; a->u = L->u; a->logits = L->logits; a->topk_idx = L->topk_idx; a->topk_w = L->topk_w;
-  a->counts = L->pb.counts; a->offsets = L->pb.offsets; a->perm = L->pb.perm; a->inv = L->pb.inv;
-  a->qkv = L->qkv; a->attn_o = L->attn_o;
+  a->r_full = L->ws->r_full; a->u = L->ws->u; a->logits = L->ws->logits; a->topk_idx = L->ws->topk_idx; a->topk_w = L->ws->topk_w;
+  a->counts = L->ws->pb.counts; a->offsets = L->ws->pb.offsets; a->perm = L->ws->pb.perm; a->inv = L->ws->pb.inv;
+  a->qkv = L->ws->qkv; a->attn_o = L->ws->attn_o;
   return FOE_OK;
 }
 
@@ -484,9 +533,9 @@ foe_status foe_poll_status(foe_layer* L, int* device_status) {
   if (!L || !device_status) return FOE_ERR_NULL;
   if (cudaStreamSynchronize(L->last_stream) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
   int v = 0;
-  if (cudaMemcpy(&v, L->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FOE_ERR_CUDA;
+  if (cudaMemcpy(&v, L->ws->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FOE_ERR_CUDA;
   *device_status = v;
-  if (v != 0) cudaMemset(L->status, 0, sizeof(int));
+  if (v != 0) cudaMemset(L->ws->status, 0, sizeof(int));
   return FOE_OK;
 }
 

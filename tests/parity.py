@@ -103,7 +103,18 @@ def run_block_parity(shape, seed, q_lens: Sequence[int], ctx_lens: Sequence[int]
     aux = layer.aux()
     launches = layer.last_launch_count()
     layer.close()
+    res = compare_with_oracle(shape, W, x, q_lens, ctx_lens, cache, kv, out, aux, rows, stress=(wscale != 1.0))
+    res["launches"] = launches
+    if return_all:
+        res.update(out=out, aux=aux, kv=kv, W=W, x=x)
+    return res
 
+
+def compare_with_oracle(shape, W, x, q_lens, ctx_lens, cache, kv, out, aux, rows=None, stress=False) -> Dict:
+    """Stage-by-stage comparison of one finished GPU call (its output, intermediates `aux` and the cache `kv` it
+    wrote) with the oracle run on the same inputs.  `cache` is the logical cache from before the call."""
+    q_lens, ctx_lens = list(q_lens), list(ctx_lens)
+    S = sum(q_lens)
     cfg = adapter.cfg_from_shape(shape)
     Wn = adapter.weights_to_numpy(W)
     xn = adapter.to_np(x)
@@ -149,11 +160,8 @@ def run_block_parity(shape, seed, q_lens: Sequence[int], ctx_lens: Sequence[int]
 
     got = adapter.to_np(out)
     got = got[:, rsel] if shape.grouped_output else got[rsel]
-    if wscale == 1.0:
+    if not stress:
         mx, rel = assert_close(got, ref_g["out"], "block output")
     else:
         mx, rel = assert_close(got, ref_g["out"], "block output (scaled weights)", STAGE_MAX_TOL, STAGE_REL_TOL)
-    res = dict(max_abs=mx, rel_l1=rel, flips=int(flips.sum()), launches=launches, counts=maps["counts"])
-    if return_all:
-        res.update(out=out, aux=aux, ref=ref, kv=kv, W=W, x=x)
-    return res
+    return dict(max_abs=mx, rel_l1=rel, flips=int(flips.sum()), counts=maps["counts"], ref=ref)
