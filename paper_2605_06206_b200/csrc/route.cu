@@ -5,12 +5,12 @@
 //
 // Three kernels:
 //  1. ffn_norm:     one warp per token: inv_rms and the bf16 expert input u = r * inv_rms * gain.
-//  2. router_gemm:  SIMT fp32 GEMM, 64 tokens x 64 experts per CTA, 8 x 8 register tiles, k-major shared
+//  2. router_gemm:  SIMT fp32 GEMM, 64 tokens x 64 experts per CTA, 8 x 4 register tiles, k-major shared
 //                   tiles, register-staged double buffering; the normalisation is applied while the token
 //                   tile is loaded (u is never rounded to bf16 on this path).  For a handful of tokens the
 //                   reduction dimension is split over gridDim.z so that the grid still fills the GPU; the
 //                   partial scores are summed in a fixed order by kernel 3.
-//  3. topk_gates:   one warp per (token, cluster): bias, top-k by (score descending, expert id ascending),
+//  3. topk_gates:   8, 16 or 32 lanes per (token, cluster): bias, top-k by (score descending, expert id ascending),
 //                   softmax over the selected scores.
 #include <float.h>
 
@@ -66,10 +66,10 @@ __global__ void ffn_norm_kernel(const void* __restrict__ r_in, int r_is_bf16, co
 }
 
 // ------------------------------------------------------------------------------------------------ 2
-constexpr int kRgTM = 64, kRgTN = 64, kRgKC = 32, kRgThreads = 64;
+constexpr int kRgTM = 64, kRgTN = 64, kRgKC = 32, kRgThreads = 128;
 constexpr int kRgPA = kRgTM + 4, kRgPB = kRgTN + 4;      // padded pitches (floats), multiples of 4
 
-__global__ void __launch_bounds__(kRgThreads)
+__global__ void __launch_bounds__(kRgThreads, 4)
 router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __restrict__ inv_rms,
                    const bf16* __restrict__ gain, const float* __restrict__ wr, float* __restrict__ part,
                    int n_tokens, int d, int E, int k_per_split) {
@@ -78,17 +78,17 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
   const int tid = threadIdx.x;
   const int tok0 = blockIdx.x * kRgTM, exp0 = blockIdx.y * kRgTN;
   const int kbeg = blockIdx.z * k_per_split, kend = min(d, kbeg + k_per_split);
-  const int ty = tid >> 3, tx = tid & 7;                  // 8 x 8 threads, 8 tokens x 8 experts each
+  const int ty = tid >> 4, tx = tid & 15;                 // 8 x 16 threads, 8 tokens x 4 experts each
 
-  // loader roles: a tile is 64 rows x 8 float4; thread loads float4 (row = tid/8 + 8 j, k4 = tid%8), j < 8
+  // loader roles: a tile is 64 rows x 8 float4; thread loads float4 (row = tid/8 + 16 j, k4 = tid%8), j < 4
   const int l_k4 = tid & 7, l_r = tid >> 3;
-  float inv_t[8];
+  float inv_t[4];
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const int t = tok0 + l_r + 8 * j;
+  for (int j = 0; j < 4; ++j) {
+    const int t = tok0 + l_r + 16 * j;
     inv_t[j] = t < n_tokens ? inv_rms[t] : 0.f;
   }
-  float4 ra[8], rb[8];
+  float4 ra[4], rb[4];
 
   auto load_chunk = [&](int k0) {
     const int k = k0 + l_k4 * 4;
@@ -98,8 +98,8 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
       g4[0] = bf16_lo(gq.x); g4[1] = bf16_hi(gq.x); g4[2] = bf16_lo(gq.y); g4[3] = bf16_hi(gq.y);
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int t = tok0 + l_r + 8 * j;
+    for (int j = 0; j < 4; ++j) {
+      const int t = tok0 + l_r + 16 * j;
       float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
       if (t < n_tokens) {
         if (r_is_bf16) {
@@ -112,15 +112,15 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
       ra[j] = make_float4(v.x * inv_t[j] * g4[0], v.y * inv_t[j] * g4[1], v.z * inv_t[j] * g4[2], v.w * inv_t[j] * g4[3]);
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int e = min(exp0 + l_r + 8 * j, E - 1);
+    for (int j = 0; j < 4; ++j) {
+      const int e = min(exp0 + l_r + 16 * j, E - 1);
       rb[j] = __ldg(reinterpret_cast<const float4*>(wr + size_t(e) * d + k));
     }
   };
   auto store_chunk = [&](int buf) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int r = l_r + 8 * j;
+    for (int j = 0; j < 4; ++j) {
+      const int r = l_r + 16 * j;
       As[buf][l_k4 * 4 + 0][r] = ra[j].x; As[buf][l_k4 * 4 + 1][r] = ra[j].y;
       As[buf][l_k4 * 4 + 2][r] = ra[j].z; As[buf][l_k4 * 4 + 3][r] = ra[j].w;
       Bs[buf][l_k4 * 4 + 0][r] = rb[j].x; Bs[buf][l_k4 * 4 + 1][r] = rb[j].y;
@@ -128,11 +128,11 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
     }
   };
 
-  float acc[8][8];
+  float acc[8][4];
 #pragma unroll
   for (int a = 0; a < 8; ++a)
 #pragma unroll
-    for (int b = 0; b < 8; ++b) acc[a][b] = 0.f;
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
 
   load_chunk(kbeg);
   store_chunk(0);
@@ -145,14 +145,13 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
     for (int k = 0; k < kRgKC; ++k) {
       const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][k][ty * 8]);
       const float4 a1 = *reinterpret_cast<const float4*>(&As[buf][k][ty * 8 + 4]);
-      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 8]);
-      const float4 b1 = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 8 + 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 4]);
       const float a8[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-      const float b8[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+      const float b4[4] = {b0.x, b0.y, b0.z, b0.w};
 #pragma unroll
       for (int a = 0; a < 8; ++a)
 #pragma unroll
-        for (int b = 0; b < 8; ++b) acc[a][b] = fmaf(a8[a], b8[b], acc[a][b]);
+        for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(a8[a], b4[b], acc[a][b]);
     }
     if (more) store_chunk(buf ^ 1);
     __syncthreads();
@@ -163,10 +162,13 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
   for (int a = 0; a < 8; ++a) {
     const int t = tok0 + ty * 8 + a;
     if (t >= n_tokens) continue;
+    const int e = exp0 + tx * 4;
+    if (e + 3 < E && (E & 3) == 0) {
+      *reinterpret_cast<float4*>(dst + size_t(t) * E + e) = make_float4(acc[a][0], acc[a][1], acc[a][2], acc[a][3]);
+    } else {
 #pragma unroll
-    for (int b = 0; b < 8; ++b) {
-      const int e = exp0 + tx * 8 + b;
-      if (e < E) dst[size_t(t) * E + e] = acc[a][b];
+      for (int b = 0; b < 4; ++b)
+        if (e + b < E) dst[size_t(t) * E + e + b] = acc[a][b];
     }
   }
 }
@@ -175,54 +177,61 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
 __global__ void topk_gates_kernel(const float* __restrict__ part, int k_splits, const float* __restrict__ br,
                                   float* __restrict__ logits_out, int* __restrict__ idx_out, float* __restrict__ w_out,
                                   int n_tokens, int H, int Ec, int kc) {
-  const int task = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (task >= n_tokens * H) return;
-  const int i = task / H, h = task - i * H;
+  // a (token, cluster) task is handled by a group of W lanes (W = 8, 16 or 32), several tasks per warp
+  const int W = Ec <= 8 ? 8 : (Ec <= 16 ? 16 : 32);
+  const int per_warp = 32 / W;
+  const int lane = threadIdx.x & 31, li = lane & (W - 1);
+  const int warp_id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int task = warp_id * per_warp + lane / W;
+  const bool live = task < n_tokens * H;
+  const int i = live ? task / H : 0, h = live ? task - i * H : 0;
   const int E = H * Ec;
   float cand[4];
   bool taken[4];
 #pragma unroll
   for (int s = 0; s < 4; ++s) {
-    const int e = lane + 32 * s;
+    const int e = li + W * s;
     float v = -FLT_MAX;
-    if (e < Ec) {
+    if (live && e < Ec && (W == 32 || s == 0)) {
       const size_t o = size_t(i) * E + h * Ec + e;
       v = 0.f;
       for (int z = 0; z < k_splits; ++z) v += part[size_t(z) * n_tokens * E + o];
       if (br) v += __ldg(br + h * Ec + e);
       logits_out[o] = v;
+      taken[s] = false;
+    } else {
+      taken[s] = true;
     }
     cand[s] = v;
-    taken[s] = e >= Ec;
   }
-  float my_sel = -FLT_MAX;      // lane j keeps the j-th selected score
+  float my_sel = -FLT_MAX;      // lane j of the group keeps the j-th selected score
   int my_idx = 0;
   for (int j = 0; j < kc; ++j) {
     float bv = -FLT_MAX;
     int bi = 0x7fffffff;
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-      const int e = lane + 32 * s;
+      const int e = li + W * s;
       if (!taken[s] && (bi == 0x7fffffff || cand[s] > bv)) { bv = cand[s]; bi = e; }   // ascending e: first wins ties
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
+    for (int o = W >> 1; o > 0; o >>= 1) {
       const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
       const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
       if (oi != 0x7fffffff && (bi == 0x7fffffff || ov > bv || (ov == bv && oi < bi))) { bv = ov; bi = oi; }
     }
-    if ((bi & 31) == lane) {
+    if (bi != 0x7fffffff && (bi & (W - 1)) == li) {
 #pragma unroll
       for (int s = 0; s < 4; ++s)
-        if ((bi >> 5) == s) taken[s] = true;
+        if (bi / W == s) taken[s] = true;
     }
-    if (lane == j) { my_sel = bv; my_idx = bi; }
+    if (li == j) { my_sel = bv; my_idx = bi; }
   }
-  const float m = __shfl_sync(0xffffffffu, my_sel, 0);
-  const float ex = lane < kc ? expf(my_sel - m) : 0.f;
-  const float sum = warp_sum(ex);
-  if (lane < kc) {
-    const size_t o = (size_t(i) * H + h) * kc + lane;
+  const float m = __shfl_sync(0xffffffffu, my_sel, 0, W);
+  float ex = li < kc ? expf(my_sel - m) : 0.f;
+  float sum = ex;
+  for (int o = W >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if (live && li < kc) {
+    const size_t o = (size_t(i) * H + h) * kc + li;
     idx_out[o] = h * Ec + my_idx;
     w_out[o] = ex / sum;
   }
@@ -245,7 +254,9 @@ int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float*
   dim3 grid((n_tokens + kRgTM - 1) / kRgTM, (E + kRgTN - 1) / kRgTN, ks);
   router_gemm_kernel<<<grid, kRgThreads, 0, st>>>(r_in, r_is_bf16, inv_rms, gain, wr, part, n_tokens, d, E, d / ks);
   const int tasks = n_tokens * H;
-  topk_gates_kernel<<<(tasks * 32 + 255) / 256, 256, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc);
+  const int per_warp = Ec <= 8 ? 4 : (Ec <= 16 ? 2 : 1);
+  const int warps = (tasks + per_warp - 1) / per_warp;
+  topk_gates_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc);
   return 3;
 }
 
@@ -319,7 +330,9 @@ int launch_route_noalloc(const bf16* h, const bf16* gain, const float* wr, const
   dim3 grid((n_tokens + kRgTM - 1) / kRgTM, (E + kRgTN - 1) / kRgTN, ks);
   router_gemm_kernel<<<grid, kRgThreads, 0, st>>>(h, 1, inv, gain, wr, part, n_tokens, d, E, d / ks);
   const int tasks = n_tokens * H;
-  topk_gates_kernel<<<(tasks * 32 + 255) / 256, 256, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc);
+  const int per_warp = Ec <= 8 ? 4 : (Ec <= 16 ? 2 : 1);
+  const int warps = (tasks + per_warp - 1) / per_warp;
+  topk_gates_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc);
   return cudaGetLastError() == cudaSuccess ? 0 : -6;
 }
 
