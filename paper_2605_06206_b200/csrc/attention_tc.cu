@@ -70,8 +70,8 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   uint64_t* q_full = bars;                 // 1
   uint64_t* kv_full = bars + 1;            // kAtStages
   uint64_t* kv_empty = kv_full + kAtStages;
-  uint64_t* s_full = kv_empty + kAtStages; // 2
-  uint64_t* p_ready = s_full + 2;          // 2
+  uint64_t* s_full = kv_empty + kAtStages; // 2 tiles x 2 score buffers
+  uint64_t* p_ready = s_full + 4;          // 2
   uint64_t* o_full = p_ready + 2;          // 2
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_full + 2);
 
@@ -95,7 +95,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     mbar_init(q_full, 1);
     for (int s = 0; s < kAtStages; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(&s_full[t], 1); mbar_init(&p_ready[t], 4); mbar_init(&o_full[t], 1);
+      mbar_init(&s_full[2 * t], 1); mbar_init(&s_full[2 * t + 1], 1); mbar_init(&p_ready[t], 4); mbar_init(&o_full[t], 1);
     }
     mbar_fence_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -105,7 +105,8 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // tensor-memory columns: S of tile t at 64 t, per-step O of tile t at 128 + DH t
+  // tensor-memory columns: scores of tile t, step parity b at 128 t + 64 b (double-buffered so that the next
+  // step's Q K^T runs while this step's softmax is still reading); O of tile t at 256 + DH t
   const uint32_t q_u32 = smem_u32(smem + L::kQOff), kv_u32 = smem_u32(smem + L::kKVOff), p_u32 = smem_u32(smem + L::kPOff);
 
   if (warp == 0) {
@@ -144,16 +145,16 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         for (int ks = 0; ks < DH / 16; ++ks) {
           const uint32_t off_q = (ks >> 2) * (kAtRows * 128) + (ks & 3) * 32;
           const uint32_t off_k = (ks >> 2) * (kAtKeys * 128) + (ks & 3) * 32;
-          umma_bf16(tmem_base + t * 64, desc_kmajor(qb_ + off_q), desc_kmajor(kb_ + off_k), idesc_s, ks != 0);
+          umma_bf16(tmem_base + t * 128 + (j & 1) * 64, desc_kmajor(qb_ + off_q), desc_kmajor(kb_ + off_k), idesc_s, ks != 0);
         }
-        umma_commit(&s_full[t]);
+        umma_commit(&s_full[2 * t + (j & 1)]);
       };
       auto issue_o = [&](int t, int j) {                      // O_t = P_t V_j
         const int s = j % kAtStages;
         const uint32_t pb_ = p_u32 + (t * 2 + (j & 1)) * L::kPTile, vb_ = kv_u32 + s * 2 * L::kKVTile + L::kKVTile;
 #pragma unroll
         for (int kk = 0; kk < kAtKeys / 16; ++kk)
-          umma_bf16(tmem_base + 128 + t * DH, desc_kmajor(pb_ + kk * 32),
+          umma_bf16(tmem_base + 256 + t * DH, desc_kmajor(pb_ + kk * 32),
                     desc_mnmajor(vb_ + kk * (16 * 128), kAtKeys * 128, 1024), idesc_o, (j | kk) != 0);
         umma_commit(&o_full[t]);
       };
@@ -166,18 +167,15 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
       for (int j = 0; j < n_tiles && ok; ++j) {
         const uint32_t ph = j & 1;
-        bool next_ready = false;
-        for (int t = 0; t < n_tiles_q && ok; ++t) {
-          if (!mbar_wait(&p_ready[t], ph)) { ok = false; break; }       // P_t(j) in shared memory, S_t free again
+        // scores of the next step first: their buffer was released by p_ready(j-1), waited for one iteration ago
+        if (j + 1 < n_tiles) {
+          if (!mbar_wait(&kv_full[(j + 1) % kAtStages], ((j + 1) / kAtStages) & 1)) { ok = false; break; }
           tc_fence_after();
-          if (j + 1 < n_tiles) {
-            if (!next_ready) {
-              if (!mbar_wait(&kv_full[(j + 1) % kAtStages], ((j + 1) / kAtStages) & 1)) { ok = false; break; }
-              tc_fence_after();
-              next_ready = true;
-            }
-            issue_s(t, j + 1);
-          }
+          for (int t = 0; t < n_tiles_q; ++t) issue_s(t, j + 1);
+        }
+        for (int t = 0; t < n_tiles_q && ok; ++t) {
+          if (!mbar_wait(&p_ready[t], ph)) { ok = false; break; }       // P_t(j) is in shared memory
+          tc_fence_after();
           issue_o(t, j);
         }
         if (ok) umma_commit(&kv_empty[j % kAtStages]);                  // stage j reusable once those MMAs retire
@@ -191,8 +189,8 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const int quarter = warp & 3;
       const int row = quarter * 32 + lane;                   // row of the tile = TMEM lane
       const uint32_t lane_sel = static_cast<uint32_t>(quarter * 32) << 16;
-      const uint32_t s_addr = tmem_base + lane_sel + t * 64;
-      const uint32_t o_addr = tmem_base + lane_sel + 128 + t * DH;
+      const uint32_t s_base = tmem_base + lane_sel + t * 128;
+      const uint32_t o_addr = tmem_base + lane_sel + 256 + t * DH;
       const int qpos = ctx + q0 + row;
       const int first_mask_tile = (ctx + q0) / kAtKeys;
       uint8_t* p_rows = smem + L::kPOff + t * 2 * L::kPTile + row * 128;
@@ -200,23 +198,25 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       bool ok = true;
       for (int j = 0; j < n_tiles; ++j) {
         const uint32_t ph = j & 1;
-        if (!mbar_wait(&s_full[t], ph)) { ok = false; break; }
+        if (!mbar_wait(&s_full[2 * t + (j & 1)], (j >> 1) & 1)) { ok = false; break; }
         tc_fence_after();
+        const uint32_t s_addr = s_base + (j & 1) * 64;
         const bool masked = j >= first_mask_tile;
-        // pass 1: row maximum of the 64 scores
+        // the 64 scores of this row: two loads in flight, one wait
+        uint32_t r0[32], r1[32];
+        tmem_ld32(s_addr, r0);
+        tmem_ld32(s_addr + 32, r1);
+        tmem_ld_wait();
         float mx = -INFINITY;
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          uint32_t r[32];
-          tmem_ld32(s_addr + hf * 32, r);
-          tmem_ld_wait();
+        if (masked) {
 #pragma unroll
           for (int c = 0; c < 32; ++c) {
-            float v = __uint_as_float(r[c]);
-            if (masked && j * kAtKeys + hf * 32 + c > qpos) v = -INFINITY;
-            mx = fmaxf(mx, v);
+            if (j * kAtKeys + c > qpos) r0[c] = 0xff800000u;          // -inf: key after the query
+            if (j * kAtKeys + 32 + c > qpos) r1[c] = 0xff800000u;
           }
         }
+#pragma unroll
+        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, fmaxf(__uint_as_float(r0[c]), __uint_as_float(r1[c])));
         const float m_new = fmaxf(m_ref, mx * a.scale_log2);
         // move the reference maximum (and rescale O) only when it is off by more than 2^8; warp-uniform so that
         // the tensor-memory accesses stay aligned
@@ -241,23 +241,16 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           m_ref = m_new;
         }
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-        // pass 2: probabilities, written as the bf16 A operand of the PV product
+        // probabilities, written as the bf16 A operand of the PV product (exp2(-inf) = 0 handles the mask)
         uint8_t* p_row = p_rows + (j & 1) * L::kPTile;
         float rs = 0.f;
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
-          uint32_t r[32];
-          tmem_ld32(s_addr + hf * 32, r);
-          tmem_ld_wait();
           uint32_t pk[16];
 #pragma unroll
           for (int c = 0; c < 16; ++c) {
-            float v0 = __uint_as_float(r[2 * c]), v1 = __uint_as_float(r[2 * c + 1]);
-            float p0 = fast_exp2(fmaf(v0, a.scale_log2, -m_use)), p1 = fast_exp2(fmaf(v1, a.scale_log2, -m_use));
-            if (masked) {
-              if (j * kAtKeys + hf * 32 + 2 * c > qpos) p0 = 0.f;
-              if (j * kAtKeys + hf * 32 + 2 * c + 1 > qpos) p1 = 0.f;
-            }
+            const float v0 = __uint_as_float(hf ? r1[2 * c] : r0[2 * c]), v1 = __uint_as_float(hf ? r1[2 * c + 1] : r0[2 * c + 1]);
+            const float p0 = fast_exp2(fmaf(v0, a.scale_log2, -m_use)), p1 = fast_exp2(fmaf(v1, a.scale_log2, -m_use));
             rs += p0 + p1;
             pk[c] = pack_bf16(p0, p1);
           }
