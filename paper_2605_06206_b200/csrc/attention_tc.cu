@@ -215,8 +215,16 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             if (j * kAtKeys + 32 + c > qpos) r1[c] = 0xff800000u;
           }
         }
+        {                                                    // four independent chains, then a short tree
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, fmaxf(__uint_as_float(r0[c]), __uint_as_float(r1[c])));
+          for (int c = 0; c < 32; c += 4) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              m4[q] = fmaxf(m4[q], fmaxf(__uint_as_float(r0[c + q]), __uint_as_float(r1[c + q])));
+          }
+          mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        }
         const float m_new = fmaxf(m_ref, mx * a.scale_log2);
         // move the reference maximum (and rescale O) only when it is off by more than 2^8; warp-uniform so that
         // the tensor-memory accesses stay aligned
@@ -243,7 +251,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
         // probabilities, written as the bf16 A operand of the PV product (exp2(-inf) = 0 handles the mask)
         uint8_t* p_row = p_rows + (j & 1) * L::kPTile;
-        float rs = 0.f;
+        float rs4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
           uint32_t pk[16];
@@ -251,7 +259,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           for (int c = 0; c < 16; ++c) {
             const float v0 = __uint_as_float(hf ? r1[2 * c] : r0[2 * c]), v1 = __uint_as_float(hf ? r1[2 * c + 1] : r0[2 * c + 1]);
             const float p0 = fast_exp2(fmaf(v0, a.scale_log2, -m_use)), p1 = fast_exp2(fmaf(v1, a.scale_log2, -m_use));
-            rs += p0 + p1;
+            rs4[c & 3] += p0 + p1;
             pk[c] = pack_bf16(p0, p1);
           }
 #pragma unroll
@@ -259,7 +267,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             *reinterpret_cast<uint4*>(p_row + (((hf * 4 + q) ^ (row & 7)) << 4)) =
                 make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
         }
-        l_run += rs;
+        l_run += (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
         tc_fence_before();
         fence_async_smem();                                  // P visible to the tensor core's shared-memory reads
         __syncwarp();

@@ -43,7 +43,7 @@ __global__ void cu_q_kernel(const int* __restrict__ q_lens, int n_seqs, int* __r
   }
 }
 
-__global__ void token_map_kernel(const int* __restrict__ cu_q, int has_q_lens, const int* __restrict__ context_lens,
+__global__ void token_map_kernel(const int* __restrict__ cu_q, int* __restrict__ cu_q_out, int has_q_lens, const int* __restrict__ context_lens,
                                  const int* __restrict__ block_table, int n_seqs, int max_pages_per_seq,
                                  int num_pages, int page_size, int n_tokens, int max_context,
                                  int* __restrict__ tok_seq, int* __restrict__ tok_pos, int* __restrict__ tok_slot,
@@ -51,8 +51,11 @@ __global__ void token_map_kernel(const int* __restrict__ cu_q, int has_q_lens, c
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_tokens) return;
   int b;
-  if (!has_q_lens) b = i;
-  else {
+  if (!has_q_lens) {                         // one token per sequence: the prefix is the identity, written here
+    b = i;
+    cu_q_out[i] = i;
+    if (i == n_tokens - 1) cu_q_out[n_tokens] = n_tokens;
+  } else {
     int lo = 0, hi = n_seqs;                 // largest b with cu_q[b] <= i
     while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (cu_q[mid] <= i) lo = mid; else hi = mid; }
     b = lo;
@@ -71,14 +74,16 @@ __global__ void token_map_kernel(const int* __restrict__ cu_q, int has_q_lens, c
   tok_slot[i] = slot;
 }
 
-void launch_token_map(const int* q_lens, const int* context_lens, const int* block_table, int n_seqs,
+int launch_token_map(const int* q_lens, const int* context_lens, const int* block_table, int n_seqs,
                       int max_pages_per_seq, int num_pages, int page_size, int n_tokens, int max_context, int* cu_q,
                       int* tok_seq, int* tok_pos, int* tok_slot, int* status, cudaStream_t st) {
-  cu_q_kernel<<<1, 32, 0, st>>>(q_lens, n_seqs, cu_q);
-  if (n_tokens <= 0) return;
-  token_map_kernel<<<(n_tokens + 255) / 256, 256, 0, st>>>(cu_q, q_lens != nullptr, context_lens, block_table, n_seqs,
+  int launches = 0;
+  if (q_lens) { cu_q_kernel<<<1, 32, 0, st>>>(q_lens, n_seqs, cu_q); ++launches; }
+  if (n_tokens <= 0) return launches;
+  token_map_kernel<<<(n_tokens + 255) / 256, 256, 0, st>>>(cu_q, cu_q, q_lens != nullptr, context_lens, block_table, n_seqs,
                                                          max_pages_per_seq, num_pages, page_size, n_tokens,
                                                          max_context, tok_seq, tok_pos, tok_slot, status);
+  return launches + 1;
 }
 
 // ------------------------------------------------------------------ RoPE + KV page write

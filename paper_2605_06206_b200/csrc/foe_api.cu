@@ -142,8 +142,7 @@ void run_route_and_permute(foe_layer* L, const void* r, int r_is_bf16, int n, cu
   L->launches += launch_route(r, r_is_bf16, L->ffn_gain, L->router_w, L->router_b, L->ws->u, L->ws->inv_rms_f, L->ws->route_part,
                               L->ws->logits, L->ws->topk_idx, L->ws->topk_w, n, L->d, L->H, L->Ec, L->kc, L->cfg.rms_eps, L->n_sms, st);
   stage_mark(L, kStPermute, st);
-  launch_permute(L->ws->topk_idx, L->ws->pb, n, L->H * L->kc, L->E, 128, L->ws->status, st);
-  L->launches += 3;
+  L->launches += launch_permute(L->ws->topk_idx, L->ws->pb, n, L->H * L->kc, L->E, 128, L->ws->status, st);
 }
 
 foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* out, cudaStream_t st, bool decode) {
@@ -163,11 +162,13 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
 
   // ---- prep: token map and pre-attention RMS statistics
   stage_mark(L, kStPrep, st);
-  launch_token_map(decode ? nullptr : kv->q_lens, kv->context_lens, kv->block_table, kv->n_seqs, kv->max_pages_per_seq,
+  L->launches += launch_token_map(decode ? nullptr : kv->q_lens, kv->context_lens, kv->block_table, kv->n_seqs, kv->max_pages_per_seq,
                    kv->num_pages, 64, S, L->cfg.max_context, L->ws->cu_q, L->ws->tok_seq, L->ws->tok_pos, L->ws->tok_slot, L->ws->status, st);
   const int x_rows = L->first ? S : H * S;
-  launch_row_inv_rms(xb, L->ws->inv_rms, x_rows, d, L->cfg.rms_eps, st);
-  L->launches += 3;
+  if (!decode) {         // (the decode projection derives 1/rms from the rows it stages)
+    launch_row_inv_rms(xb, L->ws->inv_rms, x_rows, d, L->cfg.rms_eps, st);
+    L->launches += 1;
+  }
 
   // ---- per-cluster QKV projection (norm gain folded into the weights, 1/rms applied in the epilogue)
   stage_mark(L, kStQkv, st);
@@ -186,10 +187,10 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     memset(&sa, 0, sizeof(sa));
     sa.W = L->wqkv_t; sa.X = xb; sa.ldx = d; sa.n_groups = H; sa.rows_per_group = S; sa.x_group_stride = L->first ? 0 : S;
     sa.N = (L->g + 2 * L->c) * dh; sa.K = d; sa.epi = kEpiQKV; sa.out = L->ws->qkv; sa.ldo = L->qkv_cols;
-    sa.row_scale = L->ws->inv_rms; sa.scale_group_stride = L->first ? 0 : S;
+    sa.rms_eps = L->cfg.rms_eps;
     sa.q_cols = L->g * dh; sa.kv_cols = L->c * dh; sa.q_total = L->n_q * dh; sa.kv_total = L->n_kv * dh;
     sa.status = L->ws->status;
-    launch_smallm(L->tms_wqkv, sa, st);
+    launch_smallm(L->tms_wqkv, sa, L->n_sms, st);
   }
   L->launches += 1;
 
@@ -228,7 +229,7 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     sa.W = L->wo_t; sa.X = L->ws->attn_o; sa.ldx = L->n_q * dh; sa.n_groups = 1; sa.rows_per_group = S; sa.N = d;
     sa.K = L->n_q * dh; sa.epi = kEpiOProj; sa.out = L->ws->r_full; sa.ldo = d; sa.xsum = xb; sa.x_count = L->first ? 1 : H;
     sa.x_stride = size_t(S) * d; sa.out_scale = out_scale; sa.status = L->ws->status;
-    launch_smallm(L->tms_wo, sa, st);
+    launch_smallm(L->tms_wo, sa, L->n_sms, st);
   }
   L->launches += 1;
 
@@ -258,14 +259,14 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     s1.W = L->wgu_t; s1.X = L->ws->u; s1.ldx = d; s1.row_index = L->ws->pb.perm; s1.group_offsets = L->ws->pb.offsets;
     s1.n_groups = L->E; s1.N = 2 * L->I; s1.K = d; s1.epi = kEpiSwiGLU; s1.out = L->ws->hmid; s1.ldo = L->I;
     s1.status = L->ws->status;
-    launch_smallm(L->tms_wgu, s1, st);
+    launch_smallm(L->tms_wgu, s1, L->n_sms, st);
     stage_mark(L, kStGemm2, st);
     SmallMArgs s2;
     memset(&s2, 0, sizeof(s2));
     s2.W = L->wd_t; s2.X = L->ws->hmid; s2.ldx = L->I; s2.group_offsets = L->ws->pb.offsets; s2.n_groups = L->E; s2.N = d;
     s2.K = L->I; s2.epi = kEpiBf16; s2.out = L->ws->y; s2.ldo = d;
     s2.status = L->ws->status;
-    launch_smallm(L->tms_wd, s2, st);
+    launch_smallm(L->tms_wd, s2, L->n_sms, st);
     L->launches += 2;
   }
 

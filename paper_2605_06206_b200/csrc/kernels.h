@@ -16,7 +16,8 @@ typedef __nv_bfloat16 bf16;
 // inv_rms[r] = rsqrt(mean(x[r,:]^2) + eps) for n_rows rows of d bf16 values
 void launch_row_inv_rms(const bf16* x, float* inv_rms, int n_rows, int d, float eps, cudaStream_t st);
 // per-token position / sequence / cache slot from q_lens and context_lens (device arrays)
-void launch_token_map(const int* q_lens, const int* context_lens, const int* block_table, int n_seqs,
+// returns the number of kernels launched
+int launch_token_map(const int* q_lens, const int* context_lens, const int* block_table, int n_seqs,
                       int max_pages_per_seq, int num_pages, int page_size, int n_tokens, int max_context, int* cu_q,
                       int* tok_seq, int* tok_pos, int* tok_slot, int* status, cudaStream_t st);
 // RoPE on q (in place) and k, then K/V of the new tokens into their pages
@@ -55,8 +56,9 @@ struct PermuteBuffers {
   int* n_mtiles;      // scalar
 };
 constexpr int kPermuteBlockTokens = 256;
-void launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int sel_per_token, int E, int tile_rows,
-                    int* status, cudaStream_t st);
+// returns the number of kernels launched (1 for calls of at most 256 tokens, else 3)
+int launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int sel_per_token, int E, int tile_rows,
+                   int* status, cudaStream_t st);
 
 // ---- attention.cu
 struct AttnArgs {
@@ -100,12 +102,12 @@ struct SmallMArgs {
   int N, K;
   int epi;                  // GemmEpilogue
   void* out; int ldo;
-  const float* row_scale; int scale_group_stride;
+  float rms_eps;            // kEpiQKV: 1/rms of every activation row is computed from the staged rows themselves
   int q_cols, kv_cols, q_total, kv_total;
   const bf16* xsum; int x_count; size_t x_stride; float out_scale;
   int* status;
 };
 // tmW: tensor map of W as [n_groups*N][K] with 64-column boxes of 64 rows (32 rows for the SwiGLU packing)
-void launch_smallm(const CUtensorMap& tmW, const SmallMArgs& a, cudaStream_t st);
+void launch_smallm(const CUtensorMap& tmW, const SmallMArgs& a, int n_sms, cudaStream_t st);
 
 }  // namespace foe

@@ -35,6 +35,32 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
                : "memory");
 }
 
+struct SmTask {
+  int group, slab, row_begin, rows, out_row0;
+};
+
+// task t of the persistent loop -> (group, slab, rows).  A ragged group takes all its rows (in passes of 16);
+// a uniform group is cut into 16-row chunks so that the few slabs of a small projection still spread out.
+__device__ __forceinline__ SmTask sm_task(const SmallMArgs& a, int t, int slabs_per_group, int chunks) {
+  SmTask k;
+  const int sc = slabs_per_group * chunks;
+  k.group = t / sc;
+  const int r = t - k.group * sc;
+  k.slab = r / chunks;
+  const int chunk = r - k.slab * chunks;
+  if (a.group_offsets) {
+    k.row_begin = a.group_offsets[k.group];
+    k.rows = a.group_offsets[k.group + 1] - k.row_begin;
+    k.out_row0 = k.row_begin;
+  } else {
+    const int r0 = chunk * kSmRows;
+    k.row_begin = k.group * a.x_group_stride + r0;
+    k.rows = min(kSmRows, a.rows_per_group - r0);
+    k.out_row0 = r0;
+  }
+  return k;
+}
+
 template <int EPI>
 __global__ void __launch_bounds__(kSmThreads)
 smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
@@ -46,23 +72,9 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int slabs_per_group = a.N / kSmSlab;
-  const int group = blockIdx.x / slabs_per_group;
-  const int slab = blockIdx.x - group * slabs_per_group;
-
-  // rows of this CTA: a ragged group takes all its rows (in passes of 16); a uniform group is cut into
-  // 16-row chunks over blockIdx.y so that the few CTAs of a small projection still spread over the GPU
-  int row_begin, rows, out_row0;
-  if (a.group_offsets) {
-    row_begin = a.group_offsets[group];
-    rows = a.group_offsets[group + 1] - row_begin;
-    out_row0 = row_begin;
-  } else {
-    const int r0 = blockIdx.y * kSmRows;
-    row_begin = group * a.x_group_stride + r0;
-    rows = min(kSmRows, a.rows_per_group - r0);
-    out_row0 = r0;
-  }
-  if (rows <= 0) return;                                      // untouched group: its weights are never read
+  const int chunks = a.group_offsets ? 1 : (a.rows_per_group + kSmRows - 1) / kSmRows;
+  const int n_tasks = a.n_groups * slabs_per_group * chunks;
+  const int k_steps = a.K / kSmKStep;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSmStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kSmConsumers); }
@@ -70,59 +82,61 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
   }
   __syncthreads();
 
-  const int k_steps = a.K / kSmKStep;
-  const int passes = (rows + kSmRows - 1) / kSmRows;
-  const int total = passes * k_steps;
-
-  // first weight row of the slab inside the [n_groups * N][K] matrix.  SwiGLU slabs are 32 gate rows and
-  // their 32 up rows (128 rows further in the packed layout), everything else 64 consecutive rows.
-  int wrow0;
-  if (EPI == kEpiSwiGLU) {
-    const int i0 = slab * 32;
-    wrow0 = group * a.N + (i0 >> 7) * 256 + (i0 & 127);
-  } else {
-    wrow0 = group * a.N + slab * kSmSlab;
-  }
-
+  // The CTA is persistent: it walks tasks blockIdx.x, blockIdx.x + gridDim.x, ... and the stage ring keeps
+  // running across task boundaries, so the producer is already streaming the next slab while the consumers
+  // finish the current one.  Tasks of groups without rows are skipped by both roles: untouched experts are
+  // never read.
   if (warp == kSmConsumers) {
     // ---------------------------------------------------------------- producer warp
     // lane 0 arms the barrier and issues the weight boxes; lane r copies the 256-byte k-slice of activation
     // row r (gathered through row_index) next to them.
     bool ok = true;
-    const bf16* xsrc = nullptr;
-    int cur_pass = -1, rows_pass = 0;
-    for (int it = 0; it < total; ++it) {
-      const int s = it % kSmStages;
-      const uint32_t ph = (it / kSmStages) & 1;
-      const int pass = it / k_steps, ks = it - pass * k_steps;
-      if (pass != cur_pass) {
-        cur_pass = pass;
-        rows_pass = min(kSmRows, rows - pass * kSmRows);
+    int it = 0;
+    for (int t = blockIdx.x; t < n_tasks && ok; t += gridDim.x) {
+      const SmTask k = sm_task(a, t, slabs_per_group, chunks);
+      if (k.rows <= 0) continue;
+      // first weight row of the slab inside the [n_groups * N][K] matrix.  SwiGLU slabs are 32 gate rows and
+      // their 32 up rows (128 rows further in the packed layout), everything else 64 consecutive rows.
+      int wrow0;
+      if (EPI == kEpiSwiGLU) {
+        const int i0 = k.slab * 32;
+        wrow0 = k.group * a.N + (i0 >> 7) * 256 + (i0 & 127);
+      } else {
+        wrow0 = k.group * a.N + k.slab * kSmSlab;
+      }
+      const int passes = (k.rows + kSmRows - 1) / kSmRows;
+      for (int pass = 0; pass < passes && ok; ++pass) {
+        const int rows_pass = min(kSmRows, k.rows - pass * kSmRows);
+        const bf16* xsrc = nullptr;
         if (lane < rows_pass) {
-          int xrow = row_begin + pass * kSmRows + lane;
+          int xrow = k.row_begin + pass * kSmRows + lane;
           if (a.row_index) xrow = a.row_index[xrow];
           xsrc = a.X + size_t(xrow) * a.ldx;
         }
-      }
-      if (lane == 0) ok = mbar_wait(&empty[s], ph ^ 1);
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      uint8_t* dst = smem + s * kSmStageBytes;
-      if (lane == 0) {
-        mbar_expect_tx(&full[s], kSmWBytes + rows_pass * (kSmKStep * 2));
-        const int k0 = ks * kSmKStep;
+        for (int ks = 0; ks < k_steps; ++ks, ++it) {
+          const int s = it % kSmStages;
+          const uint32_t ph = (it / kSmStages) & 1;
+          if (lane == 0) ok = mbar_wait(&empty[s], ph ^ 1);
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (!ok) break;
+          uint8_t* dst = smem + s * kSmStageBytes;
+          if (lane == 0) {
+            mbar_expect_tx(&full[s], kSmWBytes + rows_pass * (kSmKStep * 2));
+            const int k0 = ks * kSmKStep;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          if (EPI == kEpiSwiGLU) {
-            tma_load_2d(dst + h * 8192, &tmW, &full[s], k0 + h * 64, wrow0);
-            tma_load_2d(dst + h * 8192 + 4096, &tmW, &full[s], k0 + h * 64, wrow0 + 128);
-          } else {
-            tma_load_2d(dst + h * 8192, &tmW, &full[s], k0 + h * 64, wrow0);
+            for (int h = 0; h < 2; ++h) {
+              if (EPI == kEpiSwiGLU) {
+                tma_load_2d(dst + h * 8192, &tmW, &full[s], k0 + h * 64, wrow0);
+                tma_load_2d(dst + h * 8192 + 4096, &tmW, &full[s], k0 + h * 64, wrow0 + 128);
+              } else {
+                tma_load_2d(dst + h * 8192, &tmW, &full[s], k0 + h * 64, wrow0);
+              }
+            }
           }
+          __syncwarp();
+          if (lane < rows_pass) bulk_load(dst + kSmWBytes + lane * kSmXPitch, xsrc + ks * kSmKStep, kSmKStep * 2, &full[s]);
         }
       }
-      __syncwarp();
-      if (lane < rows_pass) bulk_load(dst + kSmWBytes + lane * kSmXPitch, xsrc + ks * kSmKStep, kSmKStep * 2, &full[s]);
     }
     if (!ok && lane == 0) atomicExch(a.status, kStatusTimeout);
     return;
@@ -133,9 +147,6 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
   // shared-memory rows of the two weight rows this thread feeds (MMA rows g and g+8)
   const int sr_a = (EPI == kEpiSwiGLU) ? warp * 8 + g : warp * 16 + g;
   const int sr_b = (EPI == kEpiSwiGLU) ? 32 + warp * 8 + g : warp * 16 + g + 8;
-  // global output columns of those rows
-  const int n_a = (EPI == kEpiSwiGLU) ? slab * 32 + warp * 8 + g : slab * kSmSlab + warp * 16 + g;
-  const int n_b = (EPI == kEpiSwiGLU) ? n_a : n_a + 8;
   const uint32_t sw_a = uint32_t(sr_a * 128), sx_a = uint32_t(sr_a & 7);
   const uint32_t sw_b = uint32_t(sr_b * 128), sx_b = uint32_t(sr_b & 7);
   const uint32_t smem_base = smem_u32(smem);
@@ -148,11 +159,21 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
     return v;
   };
 
+  for (int t = blockIdx.x; t < n_tasks && ok; t += gridDim.x) {
+    const SmTask k = sm_task(a, t, slabs_per_group, chunks);
+    if (k.rows <= 0) continue;
+    const int group = k.group, rows = k.rows, out_row0 = k.out_row0;
+    // global output columns of this thread's two weight rows
+    const int n_a = (EPI == kEpiSwiGLU) ? k.slab * 32 + warp * 8 + g : k.slab * kSmSlab + warp * 16 + g;
+    const int n_b = (EPI == kEpiSwiGLU) ? n_a : n_a + 8;
+    const int passes = (rows + kSmRows - 1) / kSmRows;
+
   for (int pass = 0; pass < passes && ok; ++pass) {
     const int m0 = pass * kSmRows;
     float c[NT][4];
+    float ssq[NT];                        // sum of squares of activation row nt*8+g (QKV: fused RMS statistics)
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) { c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f; }
+    for (int nt = 0; nt < NT; ++nt) { c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f; ssq[nt] = 0.f; }
 
     for (int ks = 0; ks < k_steps; ++ks, ++it) {
       const int s = it % kSmStages;
@@ -171,6 +192,11 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
           if (m0 + nt * 8 < rows) {                          // warp-uniform
             const uint32_t xb = st_base + kSmWBytes + (nt * 8 + g) * kSmXPitch + h * 128 + t4 * 16;
             const uint4 x0 = lds128(xb), x1 = lds128(xb + 64);
+            if (EPI == kEpiQKV) {
+              const uint32_t xs[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+#pragma unroll
+              for (int q = 0; q < 8; ++q) { const float lo = bf16_lo(xs[q]), hi = bf16_hi(xs[q]); ssq[nt] += lo * lo + hi * hi; }
+            }
             { const uint32_t f[4] = {wa0.x, wb0.x, wa0.y, wb0.y}; mma_bf16_16816(c[nt], f, x0.x, x0.y); }
             { const uint32_t f[4] = {wa0.z, wb0.z, wa0.w, wb0.w}; mma_bf16_16816(c[nt], f, x0.z, x0.w); }
             { const uint32_t f[4] = {wa1.x, wb1.x, wa1.y, wb1.y}; mma_bf16_16816(c[nt], f, x1.x, x1.y); }
@@ -182,6 +208,17 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
       if (lane == 0) mbar_arrive(&empty[s]);
     }
     if (!ok) break;
+    if (EPI == kEpiQKV) {
+      // the four lanes of a quad saw disjoint quarters of row nt*8+g: finish the sum, turn it into 1/rms.
+      // (rows past the end hold stale shared memory; their value is never used)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        float v = ssq[nt];
+        v += __shfl_xor_sync(0xffffffffu, v, 1);
+        v += __shfl_xor_sync(0xffffffffu, v, 2);
+        ssq[nt] = rsqrtf(v / float(a.K) + a.rms_eps);
+      }
+    }
 
     // epilogue: c[nt][0..1] = (weight row A, tokens 2*t4, 2*t4+1), c[nt][2..3] = (weight row B, same tokens)
 #pragma unroll
@@ -199,7 +236,8 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
           o[n_a] = __float2bfloat16_rn(va);
           o[n_b] = __float2bfloat16_rn(vb);
         } else if (EPI == kEpiQKV) {
-          const float sc = a.row_scale[size_t(group) * a.scale_group_stride + out_row0 + r];
+          // 1/rms of token row nt*8 + 2*t4 + e sits in the quad whose g equals that row index
+          const float sc = __shfl_sync(0xffffffffu, ssq[nt], (t4 * 2 + e) * 4);
           bf16* o = static_cast<bf16*>(a.out) + size_t(out_row0 + r) * a.ldo;
 #pragma unroll
           for (int w = 0; w < 2; ++w) {
@@ -224,29 +262,31 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
       }
     }
   }
+  }
   if (!ok && lane == 0) atomicExch(a.status, kStatusTimeout);
 }
 
+
 template <int EPI>
-static void launch_one(const CUtensorMap& tmW, const SmallMArgs& a, cudaStream_t st) {
+static void launch_one(const CUtensorMap& tmW, const SmallMArgs& a, int n_sms, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(smallm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmSmemBytes));
     configured = true;
   }
-  const int blocks = a.n_groups * (a.N / kSmSlab);
-  if (blocks <= 0) return;
   const int chunks = a.group_offsets ? 1 : (a.rows_per_group + kSmRows - 1) / kSmRows;
-  if (chunks <= 0) return;
-  smallm_kernel<EPI><<<dim3(blocks, chunks), kSmThreads, kSmSmemBytes, st>>>(tmW, a);
+  const long long tasks = (long long)a.n_groups * (a.N / kSmSlab) * chunks;
+  if (tasks <= 0) return;
+  const int grid = int(tasks < 2LL * n_sms ? tasks : 2LL * n_sms);          // two resident CTAs per SM
+  smallm_kernel<EPI><<<grid, kSmThreads, kSmSmemBytes, st>>>(tmW, a);
 }
 
-void launch_smallm(const CUtensorMap& tmW, const SmallMArgs& a, cudaStream_t st) {
+void launch_smallm(const CUtensorMap& tmW, const SmallMArgs& a, int n_sms, cudaStream_t st) {
   switch (a.epi) {
-    case kEpiSwiGLU: launch_one<kEpiSwiGLU>(tmW, a, st); break;
-    case kEpiBf16: launch_one<kEpiBf16>(tmW, a, st); break;
-    case kEpiQKV: launch_one<kEpiQKV>(tmW, a, st); break;
-    default: launch_one<kEpiOProj>(tmW, a, st); break;
+    case kEpiSwiGLU: launch_one<kEpiSwiGLU>(tmW, a, n_sms, st); break;
+    case kEpiBf16: launch_one<kEpiBf16>(tmW, a, n_sms, st); break;
+    case kEpiQKV: launch_one<kEpiQKV>(tmW, a, n_sms, st); break;
+    default: launch_one<kEpiOProj>(tmW, a, n_sms, st); break;
   }
 }
 
