@@ -57,7 +57,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -194,31 +194,56 @@ def algorithmic_work(wl):
 
 
 def e2e_loop(wl, steps, warmup):
-    """Same call with HOST buffers: H2D of x from pinned memory, the block, D2H of the output."""
+    """Same call with HOST buffers: every step copies its input from pinned host memory to the device, runs the
+    block through the C ABI and copies the result back to pinned host memory.  The three legs run on three
+    streams with two sets of device buffers, so the copy of step i+1 and the read-back of step i-1 overlap the
+    compute of step i (the layer's workspace keeps the compute legs in order)."""
     layer, kv, S = wl["layer"], wl["kv"], wl["S"]
     x_host = wl["x"].cpu().pin_memory()
-    x_dev = torch.empty_like(wl["x"])
-    fn_dev, out_dev = step_fn(dict(wl, x=x_dev))
-    probe = fn_dev()
-    out_host = torch.empty(probe.shape, dtype=probe.dtype).pin_memory()
+    mq = max(wl["info"]["q_lens"])
+    probe = layer.prefill(wl["x"], kv, n_tokens=S, max_q_len=mq) if wl["kind"] == "prefill" else layer.decode(wl["x"], kv)
+    x_dev = [torch.empty_like(wl["x"]) for _ in range(2)]
+    out_dev = [torch.empty_like(probe) for _ in range(2)]
+    out_host = [torch.empty(probe.shape, dtype=probe.dtype).pin_memory() for _ in range(2)]
+    s_in, s_comp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_comp = [torch.cuda.Event() for _ in range(2)]
+    ev_out = [torch.cuda.Event() for _ in range(2)]
     torch.cuda.synchronize()
 
-    def one():
-        x_dev.copy_(x_host, non_blocking=True)
-        o = fn_dev()
-        out_host.copy_(o, non_blocking=True)
+    def one(i):
+        b = i & 1
+        with torch.cuda.stream(s_in):
+            s_in.wait_event(ev_comp[b])                     # the compute that last read x_dev[b] is done
+            x_dev[b].copy_(x_host, non_blocking=True)
+            ev_in[b].record(s_in)
+        with torch.cuda.stream(s_comp):
+            s_comp.wait_event(ev_in[b])
+            s_comp.wait_event(ev_out[b])                    # the read-back that last used out_dev[b] is done
+            if wl["kind"] == "prefill":
+                layer.prefill(x_dev[b], kv, n_tokens=S, max_q_len=mq, out=out_dev[b], stream=s_comp)
+            else:
+                layer.decode(x_dev[b], kv, out=out_dev[b], stream=s_comp)
+            ev_comp[b].record(s_comp)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_comp[b])
+            out_host[b].copy_(out_dev[b], non_blocking=True)
+            ev_out[b].record(s_out)
 
-    for _ in range(warmup):
-        one()
+    for i in range(warmup):
+        one(i)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        one()
-    e1.record()
+    e0.record(s_comp)
+    for i in range(steps):
+        one(i)
+    s_comp.wait_event(ev_out[(steps - 1) & 1])
+    if steps > 1:
+        s_comp.wait_event(ev_out[steps & 1])
+    e1.record(s_comp)
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
-    return ms, x_host.numel() * 2, out_host.numel() * 2
+    return ms, x_host.numel() * 2, out_host[0].numel() * 2
 
 
 # ----------------------------------------------------------------------------------------------
@@ -286,10 +311,12 @@ def measure(kind, args, dist_on, rank, world, peaks, with_cpu):
     sampler = ClockSampler(torch.cuda.current_device())
     sampler.start()
     ms_total = timed_loop(fn, args.steps, args.warmup, dist_on)
-    clocks = sampler.stop()
     ms = ms_total / args.steps
     launches = wl["layer"].last_launch_count()
+    # the per-stage pass runs the same steps back to back; the sampler stays on through it so that a short
+    # timed region still yields clock samples under the same load
     stages = stage_profile(wl, fn, max(3, min(args.steps, 20)))
+    clocks = sampler.stop()
     work = algorithmic_work(wl)
     S = wl["S"]
     res = dict(ms_per_step=ms, tokens_per_s=world * S / (ms * 1e-3), launches_per_step=launches, stages_ms=stages,
@@ -317,7 +344,7 @@ def measure(kind, args, dist_on, rank, world, peaks, with_cpu):
                                whole_step_gbs=work["total_bytes"] / (ms * 1e-3) / 1e9,
                                whole_step_frac=work["total_bytes"] / (ms * 1e-3) / 1e9 / peak)
     res["work"] = {k: v for k, v in work.items()}
-    e_ms, h2d, d2h = e2e_loop(wl, max(2, min(args.steps, 10)), 2)
+    e_ms, h2d, d2h = e2e_loop(wl, max(4, min(args.steps, 10)), 3)
     res["e2e"] = dict(value=world * S / (e_ms * 1e-3), unit="tokens/s", ms_per_step=e_ms, h2d_bytes_per_step=h2d,
                       d2h_bytes_per_step=d2h)
     wl["layer"].close()
@@ -333,7 +360,7 @@ def measure(kind, args, dist_on, rank, world, peaks, with_cpu):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", choices=["prefill", "decode"], default="prefill")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
