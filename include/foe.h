@@ -58,7 +58,7 @@ typedef enum { FOE_SYNC_MEAN = 0, FOE_SYNC_SUM = 1 } foe_sync;
 /* Layer description.  Validity: n_kv_heads % n_clusters == 0, n_q_heads % n_kv_heads == 0,
  * head_dim in {64, 128}, 1 <= top_k_per_cluster <= experts_per_cluster <= 128, top_k_per_cluster <= 32,
  * page_size == 64, hidden % 128 == 0, (n_q_heads * head_dim) % 128 == 0, ffn_inter % 128 == 0,
- * n_clusters * experts_per_cluster <= 1024, n_q_heads / n_kv_heads <= 16, max_* > 0.
+ * n_clusters <= 8, n_clusters * experts_per_cluster <= 1024, n_q_heads / n_kv_heads <= 16, max_* > 0.
  * position: FOE_FIRST/FOE_SINGLE take x as [S, hidden] (one shared attention, its residual used
  * in place of r_full); FOE_LAST/FOE_SINGLE write out as [S, hidden] (mean over clusters of x').
  * Otherwise x and out are [n_clusters, S, hidden]. */

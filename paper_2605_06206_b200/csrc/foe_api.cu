@@ -116,6 +116,7 @@ void ws_release(foe_workspace* W) {
 foe_status validate(const foe_config* c) {
   if (c->hidden <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->n_clusters <= 0) return FOE_ERR_CONFIG;
   if (c->n_kv_heads % c->n_clusters || c->n_q_heads % c->n_kv_heads) return FOE_ERR_CONFIG;
+  if (c->n_clusters > 8) return FOE_ERR_CONFIG;          // the sync epilogues add up to 8 residual streams
   if (c->head_dim != 64 && c->head_dim != 128) return FOE_ERR_CONFIG;
   if (c->n_q_heads / c->n_kv_heads > 16) return FOE_ERR_CONFIG;
   if (c->experts_per_cluster < 1 || c->experts_per_cluster > 128) return FOE_ERR_CONFIG;

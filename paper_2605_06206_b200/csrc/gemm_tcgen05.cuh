@@ -26,7 +26,6 @@ constexpr int kBBytes = kBN * kBK * 2;   // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kGemmThreads = 192;
 constexpr int kGatherThreads = 128;   // extra producer warps when the A rows are gathered
-constexpr int kGatherAhead = 2;       // cp.async groups a gather thread keeps in flight
 constexpr int kTmemCols = 512;
 constexpr int kStgPitch = 128 + 16;                 // staging row: 128 bytes of output + bank-spreading pad
 constexpr int kStgWarpBytes = 32 * kStgPitch;        // one epilogue warp stages its 32 rows
@@ -51,7 +50,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], GATHER ? 1 + kGatherThreads / 32 : 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], GATHER ? 1 + kGatherThreads : 1); mbar_init(&empty_bar[s], 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); }
     mbar_fence_init();
     tma_prefetch_desc(&tmA);
@@ -117,6 +116,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(&full_bar[stage], phase)) { ok = false; break; }
           tc_fence_after();
+          if constexpr (GATHER) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // cp.async-written A tile
           const uint32_t a_addr = smem_u32(smem + stage * kStageBytes);
           const uint32_t b_addr = a_addr + kABytes;
 #pragma unroll
@@ -135,25 +135,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // ------------------------------------------------------------ A-gather producers (4 warps, one tile row each)
     // Row r of the tile is row a_row_index[row0 + r] of a_gather: the dispatch permutation is applied while
     // the operand is staged, so the permuted activations are never written to memory.  Each thread copies one
-    // 16-byte chunk of eight rows per k-block with cp.async into the 128-byte-swizzled operand layout, keeps
-    // kGatherAhead groups in flight, and makes a finished group visible to the tensor core (async proxy
-    // fence) before its warp arrives on the stage's barrier.
+    // 16-byte chunk of eight rows per k-block with cp.async into the 128-byte-swizzled operand layout and lets
+    // the copies themselves arrive on the stage's barrier (cp.async.mbarrier.arrive.noinc); the MMA thread
+    // crosses to the async proxy with a fence before it issues the tensor-core reads.
     const int gt = threadIdx.x - kGemmThreads;            // 0..127
     const int gc = gt & 7, gr = gt >> 3;                  // 16-byte chunk of a row; rows gr + 16 j, j < 8:
                                                           // 8 lanes read one row's 128 bytes as a whole line
-    int stage = 0, arr_stage = 0;
+    int stage = 0;
     uint32_t phase = 0;
-    int issued = 0;
     bool ok = true;
-    auto retire = [&](int pending) {                       // arrive for the oldest un-signalled group
-      if (pending == 2) asm volatile("cp.async.wait_group 2;" ::: "memory");
-      else if (pending == 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
-      else asm volatile("cp.async.wait_group 0;" ::: "memory");
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&full_bar[arr_stage]);
-      if (++arr_stage == kStages) arr_stage = 0;
-    };
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int mt = tile / n_ntiles;
       const int group = args.mt_group[mt], row0 = args.mt_row0[mt], row_end = args.group_end[group];
@@ -172,18 +162,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + r * 128 + ((gc ^ (r & 7)) << 4)),
                        "l"(src[j] + size_t(kb) * 128) : "memory");
         }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        ++issued;
-        if (issued > kGatherAhead) retire(kGatherAhead);
+        // the barrier gets this thread's arrival when the copies above have landed; nothing blocks here, so a
+        // thread runs as far ahead as free stages allow
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&full_bar[stage])) : "memory");
         if (++stage == kStages) { stage = 0; phase ^= 1; }
       }
     }
-    if (ok) {
-      int left = issued < kGatherAhead ? issued : kGatherAhead;
-      while (left > 0) { retire(left - 1); --left; }
-    } else if (lane == 0) {
-      atomicExch(args.status, kStatusTimeout);
-    }
+    asm volatile("cp.async.wait_all;" ::: "memory");      // nothing of this thread may still be in flight at exit
+    if (!ok && lane == 0) atomicExch(args.status, kStatusTimeout);
   } else if (warp >= 2 && warp < 6) {
     // ------------------------------------------------------------ epilogue (4 warps = 128 TMEM lanes)
     const int quarter = warp & 3;                 // a warp may only touch TMEM lanes 32*(warp%4)..+31

@@ -26,8 +26,9 @@ constexpr int kSmRows = kSmNT * 8;              // activation rows per pass
 constexpr int kSmWBytes = kSmSlab * kSmKStep * 2;        // 16 KB of weights per stage
 constexpr int kSmXPitch = kSmKStep * 2 + 16;             // padded activation row (bank spread)
 constexpr int kSmStageBytes = ((kSmWBytes + kSmRows * kSmXPitch + 1023) / 1024) * 1024;
-constexpr int kSmStages = 5;
-constexpr size_t kSmSmemBytes = size_t(kSmStages) * kSmStageBytes + 1024 + 128;
+// ring depth: 5 stages of 21 KB, two CTAs per SM
+template <int EPI> __host__ __device__ constexpr int sm_stages() { return 5; }
+template <int EPI> constexpr size_t sm_smem_bytes() { return size_t(sm_stages<EPI>()) * kSmStageBytes + 1024 + 256 + 4 * kSmRows * 4; }
 
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -65,6 +66,7 @@ template <int EPI>
 __global__ void __launch_bounds__(kSmThreads)
 smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
   constexpr int NT = kSmNT;
+  constexpr int kSmStages = sm_stages<EPI>();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + kSmStages * kSmStageBytes);
@@ -192,10 +194,16 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
           if (m0 + nt * 8 < rows) {                          // warp-uniform
             const uint32_t xb = st_base + kSmWBytes + (nt * 8 + g) * kSmXPitch + h * 128 + t4 * 16;
             const uint4 x0 = lds128(xb), x1 = lds128(xb + 64);
-            if (EPI == kEpiQKV) {
+            if (EPI == kEpiQKV && (ks & 3) == warp) {        // each consumer warp covers a quarter of the k steps
               const uint32_t xs[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+              float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-              for (int q = 0; q < 8; ++q) { const float lo = bf16_lo(xs[q]), hi = bf16_hi(xs[q]); ssq[nt] += lo * lo + hi * hi; }
+              for (int q = 0; q < 8; q += 2) {
+                const float a0 = bf16_lo(xs[q]), a1 = bf16_hi(xs[q]), b0 = bf16_lo(xs[q + 1]), b1 = bf16_hi(xs[q + 1]);
+                s0 = fmaf(a0, a0, fmaf(a1, a1, s0));
+                s1 = fmaf(b0, b0, fmaf(b1, b1, s1));
+              }
+              ssq[nt] += s0 + s1;
             }
             { const uint32_t f[4] = {wa0.x, wb0.x, wa0.y, wb0.y}; mma_bf16_16816(c[nt], f, x0.x, x0.y); }
             { const uint32_t f[4] = {wa0.z, wb0.z, wa0.w, wb0.w}; mma_bf16_16816(c[nt], f, x0.z, x0.w); }
@@ -207,18 +215,28 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[s]);
     }
-    if (!ok) break;
-    if (EPI == kEpiQKV) {
-      // the four lanes of a quad saw disjoint quarters of row nt*8+g: finish the sum, turn it into 1/rms.
+    if (EPI == kEpiQKV) {   // (also reached after a timed-out wait, so that the warps never miss each other at bar.sync)
+      // the four lanes of a quad saw disjoint quarters of row nt*8+g and the four warps disjoint k steps: finish
+      // the sum (quad shuffle, then across the consumer warps through shared memory) and turn it into 1/rms.
       // (rows past the end hold stale shared memory; their value is never used)
+      float* red = reinterpret_cast<float*>(empty + kSmStages);          // [4 warps][NT * 8 rows]
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
         float v = ssq[nt];
         v += __shfl_xor_sync(0xffffffffu, v, 1);
         v += __shfl_xor_sync(0xffffffffu, v, 2);
+        if (t4 == 0) red[warp * (NT * 8) + nt * 8 + g] = v;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");                       // the four consumer warps only
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const int r = nt * 8 + g;
+        const float v = red[r] + red[NT * 8 + r] + red[2 * NT * 8 + r] + red[3 * NT * 8 + r];
         ssq[nt] = rsqrtf(v / float(a.K) + a.rms_eps);
       }
+      asm volatile("bar.sync 1, 128;" ::: "memory");                       // red is reused by the next pass
     }
+    if (!ok) break;
 
     // epilogue: c[nt][0..1] = (weight row A, tokens 2*t4, 2*t4+1), c[nt][2..3] = (weight row B, same tokens)
 #pragma unroll
@@ -250,11 +268,19 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
           }
         } else {  // kEpiOProj: r_full = scale * (C + sum_h x[h])
           float sa = va, sb = vb;
-          for (int h = 0; h < a.x_count; ++h) {
-            const bf16* xs = a.xsum + h * a.x_stride + size_t(out_row0 + r) * a.ldo;
-            sa += __bfloat162float(xs[n_a]);
-            sb += __bfloat162float(xs[n_b]);
+          bf16 xa[8], xb[8];
+#pragma unroll
+          for (int h = 0; h < 8; ++h) {                       // all loads first (up to 8 residual streams)
+            xa[h] = __float2bfloat16_rn(0.f);
+            xb[h] = xa[h];
+            if (h < a.x_count) {
+              const bf16* xs = a.xsum + h * a.x_stride + size_t(out_row0 + r) * a.ldo;
+              xa[h] = xs[n_a];
+              xb[h] = xs[n_b];
+            }
           }
+#pragma unroll
+          for (int h = 0; h < 8; ++h) { sa += __bfloat162float(xa[h]); sb += __bfloat162float(xb[h]); }
           float* o = static_cast<float*>(a.out) + size_t(out_row0 + r) * a.ldo;
           o[n_a] = sa * a.out_scale;
           o[n_b] = sb * a.out_scale;
@@ -271,14 +297,14 @@ template <int EPI>
 static void launch_one(const CUtensorMap& tmW, const SmallMArgs& a, int n_sms, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
-    cudaFuncSetAttribute(smallm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmSmemBytes));
+    cudaFuncSetAttribute(smallm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sm_smem_bytes<EPI>()));
     configured = true;
   }
   const int chunks = a.group_offsets ? 1 : (a.rows_per_group + kSmRows - 1) / kSmRows;
   const long long tasks = (long long)a.n_groups * (a.N / kSmSlab) * chunks;
   if (tasks <= 0) return;
   const int grid = int(tasks < 2LL * n_sms ? tasks : 2LL * n_sms);          // two resident CTAs per SM
-  smallm_kernel<EPI><<<grid, kSmThreads, kSmSmemBytes, st>>>(tmW, a);
+  smallm_kernel<EPI><<<grid, kSmThreads, sm_smem_bytes<EPI>(), st>>>(tmW, a);
 }
 
 void launch_smallm(const CUtensorMap& tmW, const SmallMArgs& a, int n_sms, cudaStream_t st) {
