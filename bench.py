@@ -28,7 +28,12 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2605_06206_b200 import synth  # noqa: E402
+from paper_2605_06206_b200 import replicas, synth  # noqa: E402
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernels, from the committed ncu captures
+# of these same workloads (profiles/): not re-measured by a plain bench run
+NCU_TRAFFIC = dict(expert_gemm1_prefill=965.5e6 + 252.9e6, attn_decode=1348.8e6 + 8.8e6)
 
 
 # ----------------------------------------------------------------------------------------------
@@ -123,12 +128,12 @@ def step_fn(wl):
 
 
 def timed_loop(fn, steps, warmup, dist_on):
-    import torch.distributed as dist
+    """W untimed steps, then exactly K steps between CUDA events, bracketed by a barrier and a device
+    synchronisation on both sides; returns this rank's milliseconds for the K steps."""
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
-    if dist_on:
-        dist.barrier()
+    replicas.barrier()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
@@ -137,11 +142,7 @@ def timed_loop(fn, steps, warmup, dist_on):
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
-    if dist_on:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.barrier()
-        ms = float(t.item())
+    replicas.barrier()
     return ms
 
 
@@ -310,8 +311,8 @@ def measure(kind, args, dist_on, rank, world, peaks, with_cpu):
         raise RuntimeError(f"device status {st} after the first {kind} step")
     sampler = ClockSampler(torch.cuda.current_device())
     sampler.start()
-    ms_total = timed_loop(fn, args.steps, args.warmup, dist_on)
-    ms = ms_total / args.steps
+    ms_local = timed_loop(fn, args.steps, args.warmup, dist_on)
+    tokens_per_s, ms = replicas.job_throughput(wl["S"], args.steps, ms_local, device="cuda")
     launches = wl["layer"].last_launch_count()
     # the per-stage pass runs the same steps back to back; the sampler stays on through it so that a short
     # timed region still yields clock samples under the same load
@@ -319,14 +320,15 @@ def measure(kind, args, dist_on, rank, world, peaks, with_cpu):
     clocks = sampler.stop()
     work = algorithmic_work(wl)
     S = wl["S"]
-    res = dict(ms_per_step=ms, tokens_per_s=world * S / (ms * 1e-3), launches_per_step=launches, stages_ms=stages,
+    res = dict(ms_per_step=ms, tokens_per_s=tokens_per_s, launches_per_step=launches, stages_ms=stages,
                clocks=clocks, tokens_per_step=S)
     if kind == "prefill":
         t = stages["expert_gemm1_swiglu"] * 1e-3
         ach = work["gemm1_flops"] / t / 1e12
         peak = peaks["bf16_tflops_sustained"]
         res["roofline"] = dict(bound="tensor", kernel="gemm_tcgen05_kernel<SwiGLU> (expert GEMM 1)", achieved=ach,
-                               peak=peak, unit="TFLOP/s", frac=ach / peak, traffic=None,
+                               peak=peak, unit="TFLOP/s", frac=ach / peak, traffic=NCU_TRAFFIC["expert_gemm1_prefill"],
+                               traffic_source="dram read+write bytes per launch, profiles/ncu_full_prefill_kernels_workload2.md",
                                peak_source=f"{peaks['source']} sustained bf16 (kernel timed inside the step)",
                                frac_of_nominal_2250=ach / 2250.0,
                                gemm2_tflops=work["gemm2_flops"] / (stages["expert_gemm2"] * 1e-3) / 1e12,
@@ -338,7 +340,9 @@ def measure(kind, args, dist_on, rank, world, peaks, with_cpu):
         g1 = work["gemm1_weight_bytes"] / (stages["expert_gemm1_swiglu"] * 1e-3) / 1e9
         g2 = work["gemm2_weight_bytes"] / (stages["expert_gemm2"] * 1e-3) / 1e9
         res["roofline"] = dict(bound="hbm", kernel="attn_decode_kernel (paged split-KV attention)", achieved=ach,
-                               peak=peak, unit="GB/s", frac=ach / peak, traffic=None,
+                               peak=peak, unit="GB/s", frac=ach / peak, traffic=NCU_TRAFFIC["attn_decode"],
+                               traffic_source="dram read+write bytes per launch, profiles/ncu_full_decode_kernels_workload3.md",
+                               algorithmic_bytes=work["kv_bytes"],
                                peak_source=f"{peaks['source']} copy bandwidth", frac_of_nominal_8000=ach / 8000.0,
                                gemm1_gbs=g1, gemm2_gbs=g2,
                                whole_step_gbs=work["total_bytes"] / (ms * 1e-3) / 1e9,
@@ -379,11 +383,7 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (the block has no CPU path)")
     torch.cuda.set_device(local)
-    dist_on = world > 1
-    if dist_on:
-        import torch.distributed as dist
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dist_on = replicas.init("nccl", torch.device("cuda", local))
     peaks = measured_peaks()
 
     main_kind = args.workload
@@ -412,9 +412,7 @@ def main():
                                gpu_launches=o["launches_per_step"] * args.steps,
                                cpu_baseline=o.get("cpu_baseline"))
         print(json.dumps(line))
-    if dist_on:
-        import torch.distributed as dist
-        dist.destroy_process_group()
+    replicas.shutdown()
 
 
 if __name__ == "__main__":

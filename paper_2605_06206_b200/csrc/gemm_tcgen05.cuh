@@ -144,15 +144,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
+    // The source rows of a tile come from two dependent loads (tile table, then dispatch map): they are fetched one
+    // tile ahead, so the producer never sits through that latency at a tile boundary.
+    auto tile_rows = [&](int tile, int (&rows)[8]) {
+      if (tile < total_tiles) {
+        const int mt = tile / n_ntiles;
+        const int group = args.mt_group[mt], row0 = args.mt_row0[mt], row_end = args.group_end[group];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) rows[j] = args.a_row_index[min(row0 + gr + 16 * j, row_end - 1)];
+      }
+    };
+    int next_rows[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    tile_rows(blockIdx.x, next_rows);
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const int mt = tile / n_ntiles;
-      const int group = args.mt_group[mt], row0 = args.mt_row0[mt], row_end = args.group_end[group];
       const uint8_t* src[8];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int src_row = args.a_row_index[min(row0 + gr + 16 * j, row_end - 1)];
-        src[j] = reinterpret_cast<const uint8_t*>(args.a_gather) + size_t(src_row) * args.K * 2 + gc * 16;
-      }
+      for (int j = 0; j < 8; ++j)
+        src[j] = reinterpret_cast<const uint8_t*>(args.a_gather) + size_t(next_rows[j]) * args.K * 2 + gc * 16;
+      tile_rows(tile + gridDim.x, next_rows);              // in flight while this tile's k-blocks are copied
       for (int kb = 0; kb < kblocks; ++kb) {
         if (!mbar_wait(&empty_bar[stage], phase ^ 1)) { ok = false; break; }
         const uint32_t dst = smem_u32(smem + stage * kStageBytes);
