@@ -115,7 +115,7 @@ typedef struct {
   const int* offsets;       /* [E+1] exclusive scan of counts */
   const int* perm;          /* [S*H*k_c] slot -> token */
   const int* inv;           /* [S][H][k_c] -> slot */
-  const void* qkv;          /* [S][(n_q+2*n_kv)*head_dim] bf16: q (after RoPE) | k | v (before RoPE) */
+  const void* q;            /* [S][n_q*head_dim] bf16 queries after RoPE (K and V of the call are in the cache pages) */
   const void* attn_o;       /* [S][n_q*head_dim] bf16 attention output before W_O */
 } foe_aux;
 

@@ -48,7 +48,7 @@ class FoeKvCache(ctypes.Structure):
 class FoeAux(ctypes.Structure):
     _fields_ = [("n_tokens", ctypes.c_int)] + [(n, ctypes.c_void_p) for n in
                                                ("r_full", "u", "logits", "topk_idx", "topk_w", "counts", "offsets",
-                                                "perm", "inv", "qkv", "attn_o")]
+                                                "perm", "inv", "q", "attn_o")]
 
 
 _lib = None
@@ -232,11 +232,10 @@ class FoeLayer:
         torch.cuda.synchronize()
         s = self.shape
         S, H, kc, E, d = a.n_tokens, s.n_clusters, s.top_k_per_cluster, s.n_experts, s.hidden
-        qkv_cols = (s.n_q_heads + 2 * s.n_kv_heads) * s.head_dim
         spec = dict(r_full=((S, d), torch.float32), u=((S, d), torch.bfloat16), logits=((S, E), torch.float32),
                     topk_idx=((S, H, kc), torch.int32), topk_w=((S, H, kc), torch.float32),
                     counts=((E,), torch.int32), offsets=((E + 1,), torch.int32), perm=((S * H * kc,), torch.int32),
-                    inv=((S, H, kc), torch.int32), qkv=((S, qkv_cols), torch.bfloat16),
+                    inv=((S, H, kc), torch.int32), q=((S, s.n_q_heads * s.head_dim), torch.bfloat16),
                     attn_o=((S, s.n_q_heads * s.head_dim), torch.bfloat16))
         return {k: _view(getattr(a, k), shp, dt).clone() for k, (shp, dt) in spec.items()}
 

@@ -60,7 +60,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   const int G = a.n_q / a.n_kv;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tok = a.cu_q[b];
-  const int ld_qkv = (a.n_q + 2 * a.n_kv) * DH;
+  const int ld_q = a.n_q * DH;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kDcStages; ++s) mbar_init(&full[s], 1);
@@ -69,7 +69,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   for (int q = threadIdx.x; q < 16 * (DH / 8); q += kDcThreads) {
     const int r = q / (DH / 8), ch = q - r * (DH / 8);
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (r < G) v = __ldg(reinterpret_cast<const uint4*>(a.qkv + size_t(tok) * ld_qkv + (kvh * G + r) * DH + ch * 8));
+    if (r < G) v = __ldg(reinterpret_cast<const uint4*>(a.q + size_t(tok) * ld_q + (kvh * G + r) * DH + ch * 8));
     *reinterpret_cast<uint4*>(q_s + tile_off<16>(r, ch * 8)) = v;
   }
   __syncthreads();

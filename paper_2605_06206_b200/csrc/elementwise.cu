@@ -86,62 +86,6 @@ int launch_token_map(const int* q_lens, const int* context_lens, const int* bloc
   return launches + 1;
 }
 
-// ------------------------------------------------------------------ RoPE + KV page write
-// One thread per (token, head, 8-wide chunk of the first half of the head): it owns elements
-// j..j+7 and j+dh/2..j+dh/2+7, i.e. eight rotation pairs.  q is rotated in place; k is rotated
-// into its page slot; v is copied into its page slot.
-__global__ void rope_kv_write_kernel(bf16* __restrict__ qkv, const float2* __restrict__ rope_tab,
-                                     const int* __restrict__ tok_pos, const int* __restrict__ tok_slot,
-                                     bf16* __restrict__ k_pages, bf16* __restrict__ v_pages, int n_tokens, int n_q,
-                                     int n_kv, int dh, int page_size) {
-  const int chunks = dh / 16;
-  const int heads = n_q + 2 * n_kv;
-  const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const long long total = (long long)n_tokens * heads * chunks;
-  if (gid >= total) return;
-  const int ch = int(gid % chunks);
-  const int head = int((gid / chunks) % heads);
-  const int tok = int(gid / (chunks * heads));
-  const int half = dh / 2;
-  bf16* src = qkv + size_t(tok) * heads * dh + size_t(head) * dh + ch * 8;
-  uint4 lo = *reinterpret_cast<const uint4*>(src);
-  uint4 hi = *reinterpret_cast<const uint4*>(src + half);
-  const int slot = tok_slot[tok];
-  if (head < n_q + n_kv) {
-    const float2* tab = rope_tab + size_t(tok_pos[tok]) * half + ch * 8;
-    uint32_t a[4] = {lo.x, lo.y, lo.z, lo.w}, b[4] = {hi.x, hi.y, hi.z, hi.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float2 cs0 = __ldg(tab + 2 * j), cs1 = __ldg(tab + 2 * j + 1);
-      const float a0 = bf16_lo(a[j]), a1 = bf16_hi(a[j]), b0 = bf16_lo(b[j]), b1 = bf16_hi(b[j]);
-      a[j] = pack_bf16(a0 * cs0.x - b0 * cs0.y, a1 * cs1.x - b1 * cs1.y);
-      b[j] = pack_bf16(b0 * cs0.x + a0 * cs0.y, b1 * cs1.x + a1 * cs1.y);
-    }
-    lo = make_uint4(a[0], a[1], a[2], a[3]);
-    hi = make_uint4(b[0], b[1], b[2], b[3]);
-  }
-  if (head < n_q) {
-    *reinterpret_cast<uint4*>(src) = lo;
-    *reinterpret_cast<uint4*>(src + half) = hi;
-    return;
-  }
-  if (slot < 0) return;
-  const int page = slot / page_size, off = slot - page * page_size;
-  const bool is_k = head < n_q + n_kv;
-  const int kvh = is_k ? head - n_q : head - n_q - n_kv;
-  bf16* dst = (is_k ? k_pages : v_pages) + ((size_t(page) * n_kv + kvh) * page_size + off) * dh + ch * 8;
-  *reinterpret_cast<uint4*>(dst) = lo;
-  *reinterpret_cast<uint4*>(dst + half) = hi;
-}
-
-void launch_rope_kv_write(bf16* qkv, const float2* rope_tab, const int* tok_pos, const int* tok_slot, bf16* k_pages,
-                          bf16* v_pages, int n_tokens, int n_q, int n_kv, int dh, int page_size, cudaStream_t st) {
-  const long long total = (long long)n_tokens * (n_q + 2 * n_kv) * (dh / 16);
-  if (total <= 0) return;
-  rope_kv_write_kernel<<<unsigned((total + 255) / 256), 256, 0, st>>>(qkv, rope_tab, tok_pos, tok_slot, k_pages,
-                                                                     v_pages, n_tokens, n_q, n_kv, dh, page_size);
-}
-
 // ------------------------------------------------------------------ combine (+ residual, + last-layer mean)
 // Block per token; each thread owns 8 consecutive columns.  x'[h,i] = r_full[i] + sum_j w[i,h,j] y[inv[i,h,j]].
 __global__ void combine_kernel(const float* __restrict__ r_full, const bf16* __restrict__ y, const float* __restrict__ w,
@@ -201,10 +145,12 @@ void launch_combine(const float* r_full, const bf16* y, const float* w, const in
 }
 
 // ------------------------------------------------------------------ create-time repacks
-// dst[b][n][k] = src[b][k][n] * gain[k]   (gain optional): makes the projection weights K-major.
+// dst[b][n'][k] = src[b][k][n] * gain[k]   (gain optional): makes the projection weights K-major.  With
+// interleave_dh > 0 the rows of every head of interleave_dh columns are stored as 0, dh/2, 1, dh/2+1, ... so that
+// the two members of a rotary pair are neighbours in the GEMM's accumulator.
 __global__ void transpose_batched_kernel(const bf16* __restrict__ src, size_t src_batch, int src_ld,
                                          bf16* __restrict__ dst, size_t dst_batch, int dst_ld, int K, int N,
-                                         const bf16* __restrict__ gain) {
+                                         const bf16* __restrict__ gain, int interleave_dh) {
   __shared__ float tile[32][33];
   const bf16* s = src + blockIdx.z * src_batch;
   bf16* d = dst + blockIdx.z * dst_batch;
@@ -221,15 +167,20 @@ __global__ void transpose_batched_kernel(const bf16* __restrict__ src, size_t sr
   __syncthreads();
   for (int r = threadIdx.y; r < 32; r += blockDim.y) {
     const int n = n0 + r, k = k0 + threadIdx.x;
-    if (k < K && n < N) d[size_t(n) * dst_ld + k] = __float2bfloat16_rn(tile[threadIdx.x][r]);
+    int nd = n;                                // destination row; heads may be stored with their halves interleaved
+    if (interleave_dh > 0) {
+      const int j = n % interleave_dh, half = interleave_dh >> 1;
+      nd = n - j + (j < half ? 2 * j : 2 * (j - half) + 1);
+    }
+    if (k < K && n < N) d[size_t(nd) * dst_ld + k] = __float2bfloat16_rn(tile[threadIdx.x][r]);
   }
 }
 
 void launch_transpose_batched(const bf16* src, size_t src_batch, int src_ld, bf16* dst, size_t dst_batch, int dst_ld,
-                              int K, int N, int batch, const bf16* gain, cudaStream_t st) {
+                              int K, int N, int batch, const bf16* gain, int interleave_dh, cudaStream_t st) {
   if (batch <= 0) return;
   dim3 grid((N + 31) / 32, (K + 31) / 32, batch), block(32, 8);
-  transpose_batched_kernel<<<grid, block, 0, st>>>(src, src_batch, src_ld, dst, dst_batch, dst_ld, K, N, gain);
+  transpose_batched_kernel<<<grid, block, 0, st>>>(src, src_batch, src_ld, dst, dst_batch, dst_ld, K, N, gain, interleave_dh);
 }
 
 // dst[e][b*256 + half*128 + j][k] = (half ? w_up : w_gate)[e][k][b*128 + j]: gate and up columns of one

@@ -44,8 +44,8 @@ bool make_map_2d(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-enum Stage { kStPrep = 0, kStQkv, kStRope, kStAttn, kStOproj, kStRoute, kStPermute, kStGemm1, kStGemm2, kStCombine, kNumStages };
-const char* kStageNames[kNumStages] = {"prep", "qkv_proj", "rope_kv_write", "attention", "o_proj_sync", "route",
+enum Stage { kStPrep = 0, kStQkv, kStAttn, kStOproj, kStRoute, kStPermute, kStGemm1, kStGemm2, kStCombine, kNumStages };
+const char* kStageNames[kNumStages] = {"prep", "qkv_rope_kv_write", "attention", "o_proj_sync", "route",
                                        "permute", "expert_gemm1_swiglu", "expert_gemm2", "combine"};
 
 }  // namespace
@@ -171,7 +171,8 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     L->launches += 1;
   }
 
-  // ---- per-cluster QKV projection (norm gain folded into the weights, 1/rms applied in the epilogue)
+  // ---- per-cluster QKV projection; its epilogue applies 1/rms (gain folded into the weights) and RoPE, writes q
+  //      and puts K / V of the new tokens straight into their cache pages
   stage_mark(L, kStQkv, st);
   if (!decode) {
     if (!make_map_2d(&tmX, x, x_rows, d, kBM)) return FOE_ERR_CUDA;
@@ -179,33 +180,32 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     memset(&ga, 0, sizeof(ga));
     ga.n_groups = H; ga.rows_per_group = S; ga.a_group_stride = L->first ? 0 : S;
     ga.N = (L->g + 2 * L->c) * dh; ga.K = d; ga.status = L->ws->status;
-    ga.out = L->ws->qkv; ga.ldo = L->qkv_cols;
+    ga.out = L->ws->qkv; ga.ldo = L->n_q * dh;
     ga.row_scale = L->ws->inv_rms; ga.scale_group_stride = L->first ? 0 : S;
-    ga.q_cols = L->g * dh; ga.kv_cols = L->c * dh; ga.q_total = L->n_q * dh; ga.kv_total = L->n_kv * dh;
+    ga.q_cols = L->g * dh; ga.kv_cols = L->c * dh; ga.dh = dh; ga.n_kv = L->n_kv;
+    ga.rope_tab = L->rope_tab; ga.tok_pos = L->ws->tok_pos; ga.tok_slot = L->ws->tok_slot;
+    ga.k_pages = static_cast<bf16*>(kv->k_pages); ga.v_pages = static_cast<bf16*>(kv->v_pages);
     launch_gemm(kEpiQKV, tmX, L->tm_wqkv, ga, L->n_sms, st);
   } else {
     SmallMArgs sa;
     memset(&sa, 0, sizeof(sa));
     sa.W = L->wqkv_t; sa.X = xb; sa.ldx = d; sa.n_groups = H; sa.rows_per_group = S; sa.x_group_stride = L->first ? 0 : S;
-    sa.N = (L->g + 2 * L->c) * dh; sa.K = d; sa.epi = kEpiQKV; sa.out = L->ws->qkv; sa.ldo = L->qkv_cols;
+    sa.N = (L->g + 2 * L->c) * dh; sa.K = d; sa.epi = kEpiQKV;
+    sa.out = L->ws->qkv; sa.ldo = L->n_q * dh;
     sa.rms_eps = L->cfg.rms_eps;
-    sa.q_cols = L->g * dh; sa.kv_cols = L->c * dh; sa.q_total = L->n_q * dh; sa.kv_total = L->n_kv * dh;
+    sa.q_cols = L->g * dh; sa.kv_cols = L->c * dh; sa.dh = dh; sa.n_kv = L->n_kv;
+    sa.rope_tab = L->rope_tab; sa.tok_pos = L->ws->tok_pos; sa.tok_slot = L->ws->tok_slot;
+    sa.k_pages = static_cast<bf16*>(kv->k_pages); sa.v_pages = static_cast<bf16*>(kv->v_pages);
     sa.status = L->ws->status;
     launch_smallm(L->tms_wqkv, sa, L->n_sms, st);
   }
-  L->launches += 1;
-
-  // ---- RoPE, K/V into the pages
-  stage_mark(L, kStRope, st);
-  launch_rope_kv_write(L->ws->qkv, L->rope_tab, L->ws->tok_pos, L->ws->tok_slot, static_cast<bf16*>(kv->k_pages),
-                       static_cast<bf16*>(kv->v_pages), S, L->n_q, L->n_kv, dh, 64, st);
   L->launches += 1;
 
   // ---- attention core over the paged cache
   stage_mark(L, kStAttn, st);
   AttnArgs aa;
   memset(&aa, 0, sizeof(aa));
-  aa.qkv = L->ws->qkv; aa.out = L->ws->attn_o; aa.cu_q = L->ws->cu_q; aa.context_lens = kv->context_lens;
+  aa.q = L->ws->qkv; aa.out = L->ws->attn_o; aa.cu_q = L->ws->cu_q; aa.context_lens = kv->context_lens;
   aa.q_lens = decode ? nullptr : kv->q_lens; aa.block_table = kv->block_table; aa.n_seqs = kv->n_seqs;
   aa.max_pages_per_seq = kv->max_pages_per_seq; aa.num_pages = kv->num_pages; aa.n_q = L->n_q; aa.n_kv = L->n_kv;
   aa.dh = dh; aa.max_q_len = decode ? 1 : kv->max_q_len; aa.scale_log2 = float(1.4426950408889634 / sqrt(double(dh)));
@@ -382,7 +382,7 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     ok = ok && walloc(W, &W->route_part, size_t(S) * E > (size_t(1) << 21) ? size_t(S) * E : (size_t(1) << 21));
     ok = ok && walloc(W, &W->topk_w, size_t(R));
     ok = ok && walloc(W, &W->topk_idx, size_t(R));
-    ok = ok && walloc(W, &W->qkv, size_t(S) * L->qkv_cols);
+    ok = ok && walloc(W, &W->qkv, size_t(S + 128) * L->n_q * dh);          // q after RoPE (k, v go to the pages)
     ok = ok && walloc(W, &W->attn_o, size_t(S + 128) * L->n_q * dh);
     ok = ok && walloc(W, &W->u, size_t(S) * d);
     ok = ok && walloc(W, &W->hmid, size_t(R + 128) * I);
@@ -409,7 +409,7 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     cudaMemsetAsync(W->hmid, 0, size_t(R + 128) * I * sizeof(bf16), st);
     ok = make_map_2d(&W->tm_attn_o, W->attn_o, uint64_t(S), uint64_t(L->n_q) * dh, kBM) &&
          make_map_2d(&W->tm_hmid, W->hmid, uint64_t(R), I, kBM) &&
-         make_map_2d(&W->tm_qkv, W->qkv, uint64_t(S), uint64_t(L->qkv_cols), 128);
+         make_map_2d(&W->tm_qkv, W->qkv, uint64_t(S), uint64_t(L->n_q) * dh, 128);
     if (!ok) { foe_layer_destroy(L); return FOE_ERR_CUDA; }
   }
 
@@ -417,17 +417,17 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
   const bf16* gain_a = static_cast<const bf16*>(w->attn_norm_g);
   const size_t qkv_batch = size_t(qkvN) * d;
   launch_transpose_batched(static_cast<const bf16*>(w->wq), size_t(d) * L->g * dh, L->g * dh, L->wqkv_t, qkv_batch, d, d,
-                           L->g * dh, H, gain_a, st);
+                           L->g * dh, H, gain_a, dh, st);
   launch_transpose_batched(static_cast<const bf16*>(w->wk), size_t(d) * L->c * dh, L->c * dh,
-                           L->wqkv_t + size_t(L->g) * dh * d, qkv_batch, d, d, L->c * dh, H, gain_a, st);
+                           L->wqkv_t + size_t(L->g) * dh * d, qkv_batch, d, d, L->c * dh, H, gain_a, dh, st);
   launch_transpose_batched(static_cast<const bf16*>(w->wv), size_t(d) * L->c * dh, L->c * dh,
-                           L->wqkv_t + size_t(L->g + L->c) * dh * d, qkv_batch, d, d, L->c * dh, H, gain_a, st);
-  launch_transpose_batched(static_cast<const bf16*>(w->wo), 0, d, L->wo_t, 0, L->n_q * dh, L->n_q * dh, d, 1, nullptr, st);
+                           L->wqkv_t + size_t(L->g + L->c) * dh * d, qkv_batch, d, d, L->c * dh, H, gain_a, dh, st);
+  launch_transpose_batched(static_cast<const bf16*>(w->wo), 0, d, L->wo_t, 0, L->n_q * dh, L->n_q * dh, d, 1, nullptr, 0, st);
   launch_pack_gate_up(static_cast<const bf16*>(w->w_gate), static_cast<const bf16*>(w->w_up), L->wgu_t, E, d, I, st);
   for (int e0 = 0; e0 < E; e0 += 32768) {
     const int nb = E - e0 < 32768 ? E - e0 : 32768;
     launch_transpose_batched(static_cast<const bf16*>(w->w_down) + size_t(e0) * I * d, size_t(I) * d, d,
-                             L->wd_t + size_t(e0) * d * I, size_t(d) * I, I, I, d, nb, nullptr, st);
+                             L->wd_t + size_t(e0) * d * I, size_t(d) * I, I, I, d, nb, nullptr, 0, st);
   }
   cudaMemcpyAsync(L->ffn_gain, w->ffn_norm_g, size_t(d) * sizeof(bf16), cudaMemcpyDeviceToDevice, st);
   cudaMemcpyAsync(L->router_w, w->router_w, size_t(E) * d * sizeof(float), cudaMemcpyDeviceToDevice, st);
@@ -527,7 +527,7 @@ foe_status foe_get_aux(foe_layer* L, foe_aux* a) {
   a->n_tokens = L->last_tokens;
   a->r_full = L->ws->r_full; a->u = L->ws->u; a->logits = L->ws->logits; a->topk_idx = L->ws->topk_idx; a->topk_w = L->ws->topk_w;
   a->counts = L->ws->pb.counts; a->offsets = L->ws->pb.offsets; a->perm = L->ws->pb.perm; a->inv = L->ws->pb.inv;
-  a->qkv = L->ws->qkv; a->attn_o = L->ws->attn_o;
+  a->q = L->ws->qkv; a->attn_o = L->ws->attn_o;
   return FOE_OK;
 }
 

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <vector_types.h>
 #include <stddef.h>
 
 namespace foe {
@@ -12,7 +13,7 @@ constexpr int kBN = 256;   // GEMM tile cols  (UMMA N)
 enum GemmEpilogue : int {
   kEpiBf16 = 0,     // C -> bf16 [row][ldo]
   kEpiSwiGLU = 1,   // columns [0,128) gate, [128,256) up of one 128-wide block: silu(gate)*up -> bf16
-  kEpiQKV = 2,      // row scale (1/rms) and scatter of the cluster's q|k|v columns into [S][(n_q+2n_kv)*dh]
+  kEpiQKV = 2,      // row scale (1/rms), RoPE, q -> [S][n_q*dh], k and v -> cache pages
   kEpiOProj = 3     // r_full = scale * (C + sum_h x[h]) -> fp32 [row][ldo]
 };
 
@@ -35,11 +36,19 @@ struct GemmArgs {
   // epilogue
   void* out;
   int ldo;                  // elements per output row
-  // kEpiQKV
+  // kEpiQKV: rows are tokens; the group's columns are its q heads, then its k heads, then its v heads, every head
+  // stored with its two halves interleaved (packed column 2i = natural i, 2i+1 = natural i + dh/2) so that a
+  // rotation pair sits in adjacent accumulator columns.  The epilogue applies 1/rms, rotates q and k (RoPE) in
+  // fp32 and writes q to out[token][n_q*dh] and k / v straight into their cache pages.
   const float* row_scale;   // [n_groups * scale_group_stride]
   int scale_group_stride;
   int q_cols, kv_cols;      // g*dh and c*dh of one cluster
-  int q_total, kv_total;    // n_q*dh and n_kv*dh
+  int dh, n_kv;
+  const float2* rope_tab;   // [max_context][dh/2] (cos, sin)
+  const int* tok_pos;       // [tokens] position of the token in its sequence
+  const int* tok_slot;      // [tokens] page * 64 + offset of the token in the cache, -1 = none
+  __nv_bfloat16* k_pages;   // [num_pages][n_kv][64][dh]
+  __nv_bfloat16* v_pages;
   // kEpiOProj
   const __nv_bfloat16* xsum; // [x_count][x_stride] residual streams added to C
   int x_count;

@@ -240,6 +240,38 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         } else if constexpr (EPI == kEpiOProj) {
           tmem_ld32(taddr + ps * 32, w);
           tmem_ld_wait();
+        } else if constexpr (EPI == kEpiQKV) {
+          // 64 packed columns = 32 rotation pairs (natural columns i0+m and i0+m+dh/2 of one head).  The first
+          // 64 bytes of the staged row are the first-half columns, the second 64 bytes their partners.
+          const bool rotate = n < args.q_cols + args.kv_cols;          // q and k heads; v is only de-interleaved
+          const int i0 = (n % args.dh) >> 1;
+          // the 32 (cos, sin) pairs of this row's position are fetched before the accumulator is read, so their
+          // latency overlaps the tensor-memory load
+          const float4* tab = reinterpret_cast<const float4*>(
+              args.rope_tab + size_t(row_ok ? args.tok_pos[row_local] : 0) * (args.dh >> 1) + i0);
+          float4 cs4[16];
+#pragma unroll
+          for (int m = 0; m < 16; ++m) cs4[m] = rotate ? __ldg(tab + m) : make_float4(1.f, 0.f, 1.f, 0.f);
+          uint32_t r[32];
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            tmem_ld32(taddr + ps * 64 + hf * 32, r);
+            tmem_ld_wait();
+            float lo[16], hi[16];
+#pragma unroll
+            for (int m = 0; m < 16; ++m) {
+              const float a = __uint_as_float(r[2 * m]) * scale, b = __uint_as_float(r[2 * m + 1]) * scale;
+              const float4 c4 = cs4[hf * 8 + (m >> 1)];
+              const float cx = (m & 1) ? c4.z : c4.x, cy = (m & 1) ? c4.w : c4.y;
+              lo[m] = a * cx - b * cy;
+              hi[m] = b * cx + a * cy;
+            }
+#pragma unroll
+            for (int m = 0; m < 8; ++m) {
+              w[hf * 8 + m] = pack_bf16(lo[2 * m], lo[2 * m + 1]);
+              w[16 + hf * 8 + m] = pack_bf16(hi[2 * m], hi[2 * m + 1]);
+            }
+          }
         } else {
           uint32_t r[32];
 #pragma unroll
@@ -248,7 +280,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             tmem_ld_wait();
 #pragma unroll
             for (int c = 0; c < 16; ++c)
-              w[hf * 16 + c] = pack_bf16(__uint_as_float(r[2 * c]) * scale, __uint_as_float(r[2 * c + 1]) * scale);
+              w[hf * 16 + c] = pack_bf16(__uint_as_float(r[2 * c]), __uint_as_float(r[2 * c + 1]));
           }
         }
         if (ps == kTilePasses - 1 || (EPI != kEpiSwiGLU && n + kPassCols >= args.N)) {
@@ -304,14 +336,27 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const int grow = row0 + quarter * 32 + rr;
             if (grow >= row_end) continue;
             const uint4 v = *reinterpret_cast<const uint4*>(stg + rr * kStgPitch + wr_chunk * 16);
-            int col = n, orow = grow;
             if constexpr (EPI == kEpiQKV) {
-              orow = grow - group_row0;
-              if (n < args.q_cols) col = group * args.q_cols + n;
-              else if (n < args.q_cols + args.kv_cols) col = args.q_total + group * args.kv_cols + (n - args.q_cols);
-              else col = args.q_total + args.kv_total + group * args.kv_cols + (n - args.q_cols - args.kv_cols);
+              const int tok = grow - group_row0;
+              // natural column inside the head of this lane's 8 values: chunks 0-3 first half, 4-7 second half
+              const int hcol = ((n % args.dh) >> 1) + (wr_chunk & 3) * 8 + (wr_chunk >> 2) * (args.dh >> 1);
+              if (n < args.q_cols) {
+                const int head = group * (args.q_cols / args.dh) + n / args.dh;
+                *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + size_t(tok) * args.ldo + head * args.dh + hcol) = v;
+              } else {
+                const bool is_k = n < args.q_cols + args.kv_cols;
+                const int nn = n - args.q_cols - (is_k ? 0 : args.kv_cols);
+                const int kvh = group * (args.kv_cols / args.dh) + nn / args.dh;
+                const int slot = args.tok_slot[tok];
+                if (slot >= 0) {
+                  const int page = slot >> 6, off = slot & 63;
+                  __nv_bfloat16* base = is_k ? args.k_pages : args.v_pages;
+                  *reinterpret_cast<uint4*>(base + ((size_t(page) * args.n_kv + kvh) * 64 + off) * args.dh + hcol) = v;
+                }
+              }
+            } else {
+              *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + size_t(grow) * args.ldo + n + wr_chunk * 8) = v;
             }
-            *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + size_t(orow) * args.ldo + col + wr_chunk * 8) = v;
           }
         }
       }

@@ -20,15 +20,12 @@ void launch_row_inv_rms(const bf16* x, float* inv_rms, int n_rows, int d, float 
 int launch_token_map(const int* q_lens, const int* context_lens, const int* block_table, int n_seqs,
                       int max_pages_per_seq, int num_pages, int page_size, int n_tokens, int max_context, int* cu_q,
                       int* tok_seq, int* tok_pos, int* tok_slot, int* status, cudaStream_t st);
-// RoPE on q (in place) and k, then K/V of the new tokens into their pages
-void launch_rope_kv_write(bf16* qkv, const float2* rope_tab, const int* tok_pos, const int* tok_slot, bf16* k_pages,
-                          bf16* v_pages, int n_tokens, int n_q, int n_kv, int dh, int page_size, cudaStream_t st);
 // combine: out = r_full + sum_j w * y[inv]  (per cluster), optional mean over clusters
 void launch_combine(const float* r_full, const bf16* y, const float* w, const int* inv, bf16* out, int n_tokens,
                     int d, int H, int kc, int last_mean, cudaStream_t st);
 // weight repacks (create time)
 void launch_transpose_batched(const bf16* src, size_t src_batch, int src_ld, bf16* dst, size_t dst_batch, int dst_ld,
-                              int K, int N, int batch, const bf16* gain, cudaStream_t st);
+                              int K, int N, int batch, const bf16* gain, int interleave_dh, cudaStream_t st);
 void launch_pack_gate_up(const bf16* wg, const bf16* wu, bf16* dst, int E, int d, int I, cudaStream_t st);
 
 // ---- route.cu
@@ -62,7 +59,7 @@ int launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int s
 
 // ---- attention.cu
 struct AttnArgs {
-  const bf16* qkv;          // [S][(n_q+2n_kv)*dh]; q after RoPE
+  const bf16* q;            // [S][n_q*dh] queries after RoPE
   bf16* out;                // [S][n_q*dh]
   const int* cu_q;          // [n_seqs+1]
   const int* context_lens;  // [n_seqs]
@@ -103,7 +100,8 @@ struct SmallMArgs {
   int epi;                  // GemmEpilogue
   void* out; int ldo;
   float rms_eps;            // kEpiQKV: 1/rms of every activation row is computed from the staged rows themselves
-  int q_cols, kv_cols, q_total, kv_total;
+  int q_cols, kv_cols, dh, n_kv;   // kEpiQKV: see GemmArgs (interleaved heads, RoPE, q -> out, k / v -> pages)
+  const float2* rope_tab; const int* tok_pos; const int* tok_slot; bf16* k_pages; bf16* v_pages;
   const bf16* xsum; int x_count; size_t x_stride; float out_scale;
   int* status;
 };

@@ -147,8 +147,9 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
   // ------------------------------------------------------------------ consumers
   const int g = lane >> 2, t4 = lane & 3;
   // shared-memory rows of the two weight rows this thread feeds (MMA rows g and g+8)
-  const int sr_a = (EPI == kEpiSwiGLU) ? warp * 8 + g : warp * 16 + g;
-  const int sr_b = (EPI == kEpiSwiGLU) ? 32 + warp * 8 + g : warp * 16 + g + 8;
+  // (QKV: heads are stored with their halves interleaved, so rows 2g and 2g+1 are the two members of a rotary pair)
+  const int sr_a = (EPI == kEpiSwiGLU) ? warp * 8 + g : (EPI == kEpiQKV ? warp * 16 + 2 * g : warp * 16 + g);
+  const int sr_b = (EPI == kEpiSwiGLU) ? 32 + warp * 8 + g : (EPI == kEpiQKV ? warp * 16 + 2 * g + 1 : warp * 16 + g + 8);
   const uint32_t sw_a = uint32_t(sr_a * 128), sx_a = uint32_t(sr_a & 7);
   const uint32_t sw_b = uint32_t(sr_b * 128), sx_b = uint32_t(sr_b & 7);
   const uint32_t smem_base = smem_u32(smem);
@@ -166,8 +167,9 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
     if (k.rows <= 0) continue;
     const int group = k.group, rows = k.rows, out_row0 = k.out_row0;
     // global output columns of this thread's two weight rows
-    const int n_a = (EPI == kEpiSwiGLU) ? k.slab * 32 + warp * 8 + g : k.slab * kSmSlab + warp * 16 + g;
-    const int n_b = (EPI == kEpiSwiGLU) ? n_a : n_a + 8;
+    const int n_a = (EPI == kEpiSwiGLU) ? k.slab * 32 + warp * 8 + g
+                                        : (EPI == kEpiQKV ? k.slab * kSmSlab + warp * 16 + 2 * g : k.slab * kSmSlab + warp * 16 + g);
+    const int n_b = (EPI == kEpiSwiGLU) ? n_a : (EPI == kEpiQKV ? n_a + 1 : n_a + 8);
     const int passes = (rows + kSmRows - 1) / kSmRows;
 
   for (int pass = 0; pass < passes && ok; ++pass) {
@@ -256,15 +258,31 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
         } else if (EPI == kEpiQKV) {
           // 1/rms of token row nt*8 + 2*t4 + e sits in the quad whose g equals that row index
           const float sc = __shfl_sync(0xffffffffu, ssq[nt], (t4 * 2 + e) * 4);
-          bf16* o = static_cast<bf16*>(a.out) + size_t(out_row0 + r) * a.ldo;
-#pragma unroll
-          for (int w = 0; w < 2; ++w) {
-            const int n = w ? n_b : n_a;
-            int col;
-            if (n < a.q_cols) col = group * a.q_cols + n;
-            else if (n < a.q_cols + a.kv_cols) col = a.q_total + group * a.kv_cols + (n - a.q_cols);
-            else col = a.q_total + a.kv_total + group * a.kv_cols + (n - a.q_cols - a.kv_cols);
-            o[col] = __float2bfloat16_rn((w ? vb : va) * sc);
+          const int tok = out_row0 + r;
+          // packed columns n_a = 2i and n_a + 1 of a head are its natural columns i and i + dh/2: one rotary pair
+          const int i = (n_a % a.dh) >> 1, half = a.dh >> 1;
+          float lo = va * sc, hi = vb * sc;
+          const bool is_q = n_a < a.q_cols, is_k = !is_q && n_a < a.q_cols + a.kv_cols;
+          if (is_q || is_k) {
+            const float2 cs = __ldg(a.rope_tab + size_t(a.tok_pos[tok]) * half + i);
+            const float x0 = lo, x1 = hi;
+            lo = x0 * cs.x - x1 * cs.y;
+            hi = x1 * cs.x + x0 * cs.y;
+          }
+          if (is_q) {
+            const int head = group * (a.q_cols / a.dh) + n_a / a.dh;
+            bf16* o = static_cast<bf16*>(a.out) + size_t(tok) * a.ldo + head * a.dh;
+            o[i] = __float2bfloat16_rn(lo);
+            o[i + half] = __float2bfloat16_rn(hi);
+          } else {
+            const int nn = n_a - a.q_cols - (is_k ? 0 : a.kv_cols);
+            const int kvh = group * (a.kv_cols / a.dh) + nn / a.dh;
+            const int slot = a.tok_slot[tok];
+            if (slot >= 0) {
+              bf16* o = (is_k ? a.k_pages : a.v_pages) + ((size_t(slot >> 6) * a.n_kv + kvh) * 64 + (slot & 63)) * a.dh;
+              o[i] = __float2bfloat16_rn(lo);
+              o[i + half] = __float2bfloat16_rn(hi);
+            }
           }
         } else {  // kEpiOProj: r_full = scale * (C + sum_h x[h])
           float sa = va, sb = vb;

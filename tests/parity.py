@@ -125,8 +125,8 @@ def compare_with_oracle(shape, W, x, q_lens, ctx_lens, cache, kv, out, aux, rows
 
     # tier (i): everything up to the sync
     nq, nkv, dh = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
-    qkv = adapter.to_np(aux["qkv"])
-    assert_close(qkv[rsel, :nq * dh].reshape(len(rsel), nq, dh), ref["q"], "q after RoPE", STAGE_MAX_TOL, STAGE_REL_TOL)
+    q_gpu = adapter.to_np(aux["q"])
+    assert_close(q_gpu[rsel].reshape(len(rsel), nq, dh), ref["q"], "q after RoPE", STAGE_MAX_TOL, STAGE_REL_TOL)
     full = [c + q for c, q in zip(ctx_lens, q_lens)]
     newc = adapter.logical_cache(kv.k_pages, kv.v_pages, kv.block_table, full, 64)
     k_new = np.concatenate([newc[b][0][ctx_lens[b]:] for b in range(len(q_lens))])

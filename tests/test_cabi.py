@@ -60,7 +60,7 @@ def test_null_and_config_errors_need_no_device(lib):
     assert lib.foe_layer_destroy(None) == 0
     assert lib.foe_prefill(None, None, None, None, None) == -1
     assert lib.foe_last_launch_count(None) == 0
-    assert lib.foe_num_stages() == 10 and lib.foe_stage_name(7).decode() == "expert_gemm1_swiglu"
+    assert lib.foe_num_stages() == 9 and lib.foe_stage_name(6).decode() == "expert_gemm1_swiglu"
 
 
 def test_product_path_fails_loudly_without_a_gpu():
