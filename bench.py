@@ -361,6 +361,31 @@ def measure(kind, args, dist_on, rank, world, peaks, with_cpu):
     return res
 
 
+def run_sweep(args):
+    """Latency of one block at the paper's 7B layer shape for the token-batch sizes of its forward-latency table
+    (1 ... 24,576 tokens, as sequences of at most 2,048 tokens), on one GPU.  Context for that table's shape only:
+    the paper's numbers are whole 16-layer models on 8 H100s."""
+    from paper_2605_06206_b200 import binding
+    shape = synth.LayerShape(2048, 16, 8, 8, 128, 8, 1, 1024, rope_theta=5.0e5)
+    W = synth.make_weights(shape, 7, "cuda")
+    sizes = [1, 64, 128, 256, 512, 1024, 2048, 4096, 8192, 12288, 16384, 24576]
+    layer = binding.FoeLayer(shape, W, max_tokens=max(sizes), max_seqs=16, max_context=2048)
+    rows = []
+    for S in sizes:
+        q_lens = [2048] * (S // 2048) + ([S % 2048] if S % 2048 else [])
+        x = synth.make_x(shape, 7, S, "cuda")
+        kv = synth.make_paged_cache(shape, 7, [0] * len(q_lens), q_lens, "cuda", fill_random=False)
+        out = torch.empty_like(x)
+        fn = lambda: layer.prefill(x, kv, n_tokens=S, max_q_len=max(q_lens), out=out)
+        ms = timed_loop(fn, args.steps, args.warmup, False) / args.steps
+        rows.append(dict(tokens=S, ms_per_block=ms, tokens_per_s=S / (ms * 1e-3)))
+    layer.close()
+    print(json.dumps(dict(metric="foe_block_latency_sweep", unit="ms", data="synthetic", dtype="bf16",
+                          config=dict(workload="paper 7B layer shape (hidden 2048, 16q/8kv, 8 groups x 8 experts top-1, "
+                                               "inter 1024), prefill of S tokens in sequences of <= 2048"),
+                          steps=args.steps, warmup=args.warmup, sweep=rows)))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -370,6 +395,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-secondary", action="store_true", help="skip the other workload's measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle (profiler runs)")
+    ap.add_argument("--sweep", action="store_true", help="token-batch latency sweep at the paper's 7B layer shape")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
@@ -383,6 +409,9 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (the block has no CPU path)")
     torch.cuda.set_device(local)
+    if args.sweep:
+        run_sweep(args)
+        return
     dist_on = replicas.init("nccl", torch.device("cuda", local))
     peaks = measured_peaks()
 

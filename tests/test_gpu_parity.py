@@ -253,3 +253,16 @@ def test_workload4_skewed_routing_sampled():
     c = r["counts"].reshape(shape.n_clusters, shape.experts_per_cluster)
     print("workload 4:", {k: r[k] for k in ("max_abs", "rel_l1", "flips")}, "max/mean rows", c.max() / c.mean())
     assert (c == 0).sum() >= 2 * shape.n_clusters and c.max() > 3 * c.mean()       # empty and overfull experts
+
+
+# ------------------------------------------------------------------------------------------ the paper's own model shape
+def test_paper_7b_layer_shape_prefill_and_decode():
+    """The "Full" model of the paper's training-configuration table: hidden 2048, 16 query / 8 KV heads of 128,
+    64 experts, top-8, 8 groups (so 8 experts and top-1 per group), expert FFN multiplier 1/2 (inter 1024),
+    RoPE base 500,000."""
+    shape = synth.LayerShape(2048, 16, 8, 8, 128, 8, 1, 1024, rope_theta=5.0e5)
+    rows = _sample_rows([1024, 3000], 10, 7)
+    r = run_block_parity(shape, 70, [1024, 3000], [0, 0], rows=rows)
+    print("paper 7B layer, prefill:", {k: r[k] for k in ("max_abs", "rel_l1", "flips")})
+    r = run_block_parity(shape, 71, [1] * 12, [17, 900, 2048, 5000, 63, 64, 4095, 4096, 30000, 1, 777, 12000], decode=True)
+    print("paper 7B layer, decode:", {k: r[k] for k in ("max_abs", "rel_l1", "flips")})
