@@ -229,10 +229,15 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         // move the reference maximum (and rescale O) only when it is off by more than 2^8; warp-uniform so that
         // the tensor-memory accesses stay aligned
         const bool move = __any_sync(0xffffffffu, m_new > m_ref + 8.0f);
+        // A parity wait only tells phases apart if the waiter is at most one phase behind the barrier, so every step
+        // observes the completion of the previous step's P V product exactly once: here when O has to be rescaled,
+        // otherwise at the end of the step, when it has long landed.
+        bool o_seen = (j == 0);
         if (move) {
           const float alpha = (m_ref == -INFINITY) ? 0.f : fast_exp2(m_ref - m_new);
           if (j > 0) {
             if (!mbar_wait(&o_full[t], ph ^ 1)) { ok = false; break; }      // every P V product so far has landed
+            o_seen = true;
             tc_fence_after();
 #pragma unroll
             for (int ch = 0; ch < DH / 32; ++ch) {
@@ -272,6 +277,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         fence_async_smem();                                  // P visible to the tensor core's shared-memory reads
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_ready[t]);
+        if (!o_seen && !mbar_wait(&o_full[t], ph ^ 1)) { ok = false; break; }
       }
       if (ok && n_tiles > 0) ok = mbar_wait(&o_full[t], (n_tiles - 1) & 1);
       tc_fence_after();

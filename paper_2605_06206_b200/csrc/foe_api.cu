@@ -75,6 +75,7 @@ struct foe_layer {
   int max_splits, pages_per_split;
   // tensor maps of the weights
   CUtensorMap tm_wqkv, tm_wo, tm_wgu, tm_wd;
+  CUtensorMap tmp_wd;                              // 128-row boxes: each CTA of a pair loads half of a B tile
   CUtensorMap tms_wqkv, tms_wo, tms_wgu, tms_wd;   // same weights, boxes sized for the decode kernels
   // call state
   cudaStream_t last_stream;
@@ -143,7 +144,7 @@ void run_route_and_permute(foe_layer* L, const void* r, int r_is_bf16, int n, cu
   L->launches += launch_route(r, r_is_bf16, L->ffn_gain, L->router_w, L->router_b, L->ws->u, L->ws->inv_rms_f, L->ws->route_part,
                               L->ws->logits, L->ws->topk_idx, L->ws->topk_w, n, L->d, L->H, L->Ec, L->kc, L->cfg.rms_eps, L->n_sms, st);
   stage_mark(L, kStPermute, st);
-  L->launches += launch_permute(L->ws->topk_idx, L->ws->pb, n, L->H * L->kc, L->E, 128, L->ws->status, st);
+  L->launches += launch_permute(L->ws->topk_idx, L->ws->pb, n, L->H * L->kc, L->E, L->ws->status, st);
 }
 
 foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* out, cudaStream_t st, bool decode) {
@@ -251,7 +252,8 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     GemmArgs g2 = g1;
     g2.a_gather = nullptr; g2.a_row_index = nullptr;
     g2.N = d; g2.K = L->I; g2.out = L->ws->y; g2.ldo = d;
-    launch_gemm(kEpiBf16, L->ws->tm_hmid, L->tm_wd, g2, L->n_sms, st);
+    g2.mt_group = L->ws->pb.mt2_group; g2.mt_row0 = L->ws->pb.mt2_row0; g2.n_mtiles = L->ws->pb.n_mtiles2;   // 256-row tiles
+    launch_gemm_pair(L->ws->tm_hmid, L->tmp_wd, g2, L->n_sms, st);
     L->launches += 2;
   } else {
     stage_mark(L, kStGemm1, st);
@@ -403,6 +405,9 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     ok = ok && walloc(W, &W->pb.mt_group, size_t(R / 128 + E + 1));
     ok = ok && walloc(W, &W->pb.mt_row0, size_t(R / 128 + E + 1));
     ok = ok && walloc(W, &W->pb.n_mtiles, size_t(1));
+    ok = ok && walloc(W, &W->pb.mt2_group, size_t(R / 256 + E + 1));
+    ok = ok && walloc(W, &W->pb.mt2_row0, size_t(R / 256 + E + 1));
+    ok = ok && walloc(W, &W->pb.n_mtiles2, size_t(1));
     if (!ok) { foe_layer_destroy(L); return FOE_ERR_OOM; }
     cudaMemsetAsync(W->status, 0, sizeof(int), st);
     cudaMemsetAsync(W->attn_o, 0, size_t(S + 128) * L->n_q * dh * sizeof(bf16), st);
@@ -454,6 +459,7 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
        make_map_2d(&L->tm_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, kBN) &&
        make_map_2d(&L->tm_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, kBN) &&
        make_map_2d(&L->tm_wd, L->wd_t, uint64_t(E) * d, I, kBN) &&
+       make_map_2d(&L->tmp_wd, L->wd_t, uint64_t(E) * d, I, 128) &&
        make_map_2d(&L->tms_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, 64) &&
        make_map_2d(&L->tms_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, 64) &&
        make_map_2d(&L->tms_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, 32) &&

@@ -9,7 +9,7 @@
 // The activation rows themselves are not moved here: expert GEMM 1 gathers them through perm while it stages
 // its A operand.  Three launches: (1) every block of 256 tokens builds a token-bitmap per expert in shared memory,
 // from which each selection reads its rank inside the block; (2) one block scans block counts and
-// expert totals and writes the m-tile table the grouped GEMM walks; (3) every selection computes its
+// expert totals and writes the m-tile tables the grouped GEMMs walk; (3) every selection computes its
 // slot.
 #include "common.cuh"
 #include "kernels.h"
@@ -54,13 +54,22 @@ permute_count_kernel(const int* __restrict__ idx, int* __restrict__ rank, int* _
   }
 }
 
-// Single block.  blk_counts[b][e] becomes the exclusive prefix over b; counts/offsets and the m-tile table
-// (group and first row of every tile_rows-row tile of every non-empty expert) are written.
+// Tile tables the grouped GEMMs walk: expert and first row of every 128-row tile and of every 256-row tile of
+// every non-empty expert.  Expert e owns tiles1 / tiles2 entries from tile0_1 / tile0_2 on; the last expert also
+// writes the table lengths (sum1, sum2).
+__device__ __forceinline__ void write_tile_tables(const PermuteBuffers& pb, int e, int E, int row0, int tiles1,
+                                                  int tile0_1, int tiles2, int tile0_2, int sum1, int sum2) {
+  if (e == E - 1) { *pb.n_mtiles = sum1; *pb.n_mtiles2 = sum2; }
+  for (int j = 0; j < tiles1; ++j) { pb.mt_group[tile0_1 + j] = e; pb.mt_row0[tile0_1 + j] = row0 + j * 128; }
+  for (int j = 0; j < tiles2; ++j) { pb.mt2_group[tile0_2 + j] = e; pb.mt2_row0[tile0_2 + j] = row0 + j * 256; }
+}
+
+// Single block.  blk_counts[b][e] becomes the exclusive prefix over b; counts/offsets and the tile tables are written.
 __global__ void __launch_bounds__(1024)
-permute_scan_kernel(int* __restrict__ blk_counts, int n_blocks, int E, int tile_rows, int* __restrict__ counts,
-                    int* __restrict__ offsets, int* __restrict__ mt_group, int* __restrict__ mt_row0,
-                    int* __restrict__ n_mtiles) {
-  __shared__ int s_a[1024], s_b[1024];
+permute_scan_kernel(int* __restrict__ blk_counts, int n_blocks, int E, const PermuteBuffers pb) {
+  __shared__ int s_a[1024], s_b[1024], s_c[1024];
+  int* counts = pb.counts;
+  int* offsets = pb.offsets;
   const int e = threadIdx.x;
   int total = 0;
   if (e < E) {
@@ -71,24 +80,27 @@ permute_scan_kernel(int* __restrict__ blk_counts, int n_blocks, int E, int tile_
     }
     counts[e] = total;
   }
-  const int tiles = (total + tile_rows - 1) / tile_rows;
-  // two inclusive Hillis-Steele scans over the expert id (rows and tiles)
+  const int tiles1 = (total + 127) / 128, tiles2 = (total + 255) / 256;
+  // three inclusive Hillis-Steele scans over the expert id (rows, 128-row tiles, 256-row tiles)
   s_a[e] = total;
-  s_b[e] = tiles;
+  s_b[e] = tiles1;
+  s_c[e] = tiles2;
   __syncthreads();
   for (int o = 1; o < 1024; o <<= 1) {
     const int va = e >= o ? s_a[e - o] : 0;
     const int vb = e >= o ? s_b[e - o] : 0;
+    const int vc = e >= o ? s_c[e - o] : 0;
     __syncthreads();
     s_a[e] += va;
     s_b[e] += vb;
+    s_c[e] += vc;
     __syncthreads();
   }
   if (e < E) {
-    const int row0 = s_a[e] - total, tile0 = s_b[e] - tiles;
+    const int row0 = s_a[e] - total;
     offsets[e] = row0;
-    if (e == E - 1) { offsets[E] = s_a[e]; *n_mtiles = s_b[e]; }
-    for (int j = 0; j < tiles; ++j) { mt_group[tile0 + j] = e; mt_row0[tile0 + j] = row0 + j * tile_rows; }
+    if (e == E - 1) offsets[E] = s_a[e];
+    write_tile_tables(pb, e, E, row0, tiles1, s_b[e] - tiles1, tiles2, s_c[e] - tiles2, s_b[e], s_c[e]);
   }
 }
 
@@ -108,11 +120,14 @@ __global__ void permute_scatter_kernel(const int* __restrict__ idx, const int* _
 // All three steps in one block, for calls of at most 256 tokens (a decode step): bitmap, scan over the
 // experts, slots.  Same results as the three-kernel path, two launches fewer.
 __global__ void __launch_bounds__(1024)
-permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, int tile_rows, int* __restrict__ counts,
-                     int* __restrict__ offsets, int* __restrict__ mt_group, int* __restrict__ mt_row0,
-                     int* __restrict__ n_mtiles, int* __restrict__ perm, int* __restrict__ inv, int* __restrict__ status) {
+permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, const PermuteBuffers pb,
+                     int* __restrict__ status) {
   extern __shared__ uint32_t bm[];            // [E][8]
-  __shared__ int s_a[1024], s_b[1024], s_off[1024];
+  __shared__ int s_a[1024], s_b[1024], s_c[1024], s_off[1024];
+  int* counts = pb.counts;
+  int* offsets = pb.offsets;
+  int* perm = pb.perm;
+  int* inv = pb.inv;
   const int t = threadIdx.x;
   for (int q = t; q < E * 8; q += 1024) bm[q] = 0u;
   __syncthreads();
@@ -130,24 +145,27 @@ permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, 
     for (int k = 0; k < 8; ++k) total += __popc(bm[t * 8 + k]);
     counts[t] = total;
   }
-  const int tiles = (total + tile_rows - 1) / tile_rows;
+  const int tiles1 = (total + 127) / 128, tiles2 = (total + 255) / 256;
   s_a[t] = total;
-  s_b[t] = tiles;
+  s_b[t] = tiles1;
+  s_c[t] = tiles2;
   __syncthreads();
   for (int o = 1; o < 1024; o <<= 1) {
     const int va = t >= o ? s_a[t - o] : 0;
     const int vb = t >= o ? s_b[t - o] : 0;
+    const int vc = t >= o ? s_c[t - o] : 0;
     __syncthreads();
     s_a[t] += va;
     s_b[t] += vb;
+    s_c[t] += vc;
     __syncthreads();
   }
   if (t < E) {
-    const int row0 = s_a[t] - total, tile0 = s_b[t] - tiles;
+    const int row0 = s_a[t] - total;
     offsets[t] = row0;
     s_off[t] = row0;
-    if (t == E - 1) { offsets[E] = s_a[t]; *n_mtiles = s_b[t]; }
-    for (int j = 0; j < tiles; ++j) { mt_group[tile0 + j] = t; mt_row0[tile0 + j] = row0 + j * tile_rows; }
+    if (t == E - 1) offsets[E] = s_a[t];
+    write_tile_tables(pb, t, E, row0, tiles1, s_b[t] - tiles1, tiles2, s_c[t] - tiles2, s_b[t], s_c[t]);
   }
   __syncthreads();
   for (int q = t; q < n_tokens * sel; q += 1024) {
@@ -164,18 +182,16 @@ permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, 
   }
 }
 
-int launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int sel, int E, int tile_rows, int* status,
+int launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int sel, int E, int* status,
                    cudaStream_t st) {
   if (n_tokens <= 0) return 0;
   if (n_tokens <= kPB) {
-    permute_small_kernel<<<1, 1024, size_t(E) * 32, st>>>(idx, n_tokens, sel, E, tile_rows, pb.counts, pb.offsets,
-                                                         pb.mt_group, pb.mt_row0, pb.n_mtiles, pb.perm, pb.inv, status);
+    permute_small_kernel<<<1, 1024, size_t(E) * 32, st>>>(idx, n_tokens, sel, E, pb, status);
     return 1;
   }
   const int n_blocks = (n_tokens + kPB - 1) / kPB;
   permute_count_kernel<<<n_blocks, kPB, size_t(E) * 32, st>>>(idx, pb.rank, pb.blk_counts, n_tokens, sel, E, status);
-  permute_scan_kernel<<<1, 1024, 0, st>>>(pb.blk_counts, n_blocks, E, tile_rows, pb.counts, pb.offsets, pb.mt_group,
-                                          pb.mt_row0, pb.n_mtiles);
+  permute_scan_kernel<<<1, 1024, 0, st>>>(pb.blk_counts, n_blocks, E, pb);
   const int total = n_tokens * sel;
   permute_scatter_kernel<<<(total + 255) / 256, 256, 0, st>>>(idx, pb.rank, pb.blk_counts, pb.offsets, pb.perm, pb.inv,
                                                             n_tokens, sel, E);

@@ -249,7 +249,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
         if (r >= rows) continue;
         const float va = c[nt][e], vb = c[nt][2 + e];
         if (EPI == kEpiSwiGLU) {
-          const float h = va / (1.0f + __expf(-va)) * vb;
+          const float h = __fdividef(va, 1.0f + __expf(-va)) * vb;
           static_cast<bf16*>(a.out)[size_t(out_row0 + r) * a.ldo + n_a] = __float2bfloat16_rn(h);
         } else if (EPI == kEpiBf16) {
           bf16* o = static_cast<bf16*>(a.out) + size_t(out_row0 + r) * a.ldo;

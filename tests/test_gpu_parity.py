@@ -187,6 +187,31 @@ def test_same_inputs_give_bit_identical_outputs():
     assert torch.equal(outs[0], outs[1])
 
 
+@pytest.mark.parametrize("dh,q_lens,ctx", [(128, [130, 300, 63, 65], [0, 0, 0, 0]), (64, [700, 333, 129], [64, 0, 130])])
+def test_repeated_prefill_is_bit_stable_under_timing_noise(dh, q_lens, ctx):
+    """The same call repeated many times, with the L2 flushed at irregular intervals, must give the same bits every
+    time: a warp that runs a pipeline phase ahead of its neighbours may not change what it reads."""
+    shape = synth.LayerShape(512, 8, 2, 2, 128, 4, 2, 256) if dh == 128 else synth.LayerShape(256, 8, 4, 4, 64, 8, 2, 128)
+    W = scaled_weights(shape, 14, "cuda", 4.0)
+    S = sum(q_lens)
+    x = synth.make_x(shape, 14, S, "cuda")
+    layer = binding.FoeLayer(shape, W, max_tokens=S, max_seqs=len(q_lens), max_context=max(c + q for c, q in zip(ctx, q_lens)))
+    first = None
+    for it in range(120):
+        kv = synth.make_paged_cache(shape, 14, ctx, q_lens, "cuda")
+        if it % 3 == 1:
+            torch.empty(192 << 20, dtype=torch.uint8, device="cuda").fill_(1)
+        out = layer.prefill(x, kv)
+        assert layer.poll_status() == 0
+        cur = (out.clone(), layer.aux()["attn_o"].clone(), kv.k_pages.clone(), kv.v_pages.clone())
+        if first is None:
+            first = cur
+        else:
+            for a, b, name in zip(first, cur, ("out", "attn_o", "k_pages", "v_pages")):
+                assert torch.equal(a, b), f"repeat {it}: {name} changed"
+    layer.close()
+
+
 # ------------------------------------------------------------------------------------------ error paths (host side)
 def test_host_side_argument_errors():
     shape = shape_small()
