@@ -8,7 +8,14 @@
 namespace foe {
 
 constexpr int kBM = 128;   // GEMM tile rows  (UMMA M)
-constexpr int kBN = 256;   // GEMM tile cols  (UMMA N)
+constexpr int kBN = 256;   // widest GEMM tile (UMMA N); the launcher narrows it in steps of 64 so that N splits evenly
+
+// Tile width for N columns per group: as few tiles as 256 allows, all of the same width (384 columns are two tiles
+// of 192, not one of 256 and a half-empty one).
+__host__ __device__ constexpr int gemm_tile_cols(int N) {
+  const int tiles = (N + kBN - 1) / kBN;
+  return tiles <= 0 ? kBN : ((((N + tiles - 1) / tiles) + 63) / 64) * 64;
+}
 
 enum GemmEpilogue : int {
   kEpiBf16 = 0,     // C -> bf16 [row][ldo]
@@ -29,6 +36,7 @@ struct GemmArgs {
   const int* n_mtiles;      // device scalar
   int N;                    // columns per group (rows of B per group)
   int K;
+  int bn;                   // tile width, set by the launcher (gemm_tile_cols(N); 256 for kEpiSwiGLU)
   int* status;              // device status word
   // gathered A operand (expert GEMM 1): A row r of a tile is a_gather[a_row_index[r]][:]; nullptr = A through tmA
   const __nv_bfloat16* a_gather;

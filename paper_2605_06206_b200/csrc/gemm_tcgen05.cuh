@@ -2,10 +2,11 @@
 //
 //   C_g[m, n] = sum_k A[row_g(m), k] * B_g[n, k]          fp32 accumulation in tensor memory
 //
-// One persistent CTA per SM walks a static round-robin list of 128 x 256 output tiles.  Warp 0 is
-// the TMA producer, warp 1 issues the MMAs and owns the TMEM allocation, warps 2..5 drain the
-// accumulator (tcgen05.ld) and apply the epilogue.  Two accumulator stages (2 x 256 TMEM columns)
-// let the epilogue of one tile overlap the MMAs of the next.  Groups are either uniform (every
+// One persistent CTA per SM walks a static round-robin list of 128 x bn output tiles (bn <= 256).  Warp 0 is
+// the TMA producer, warp 1 issues the MMAs and owns the TMEM allocation, warps 2..9 drain the
+// accumulator (tcgen05.ld) and apply the epilogue: two warps per 32-lane quarter of tensor memory, which take
+// alternate column passes, so that twice as many global loads and stores of the epilogue are in flight.  Two
+// accumulator stages (2 x 256 TMEM columns) let the epilogue of one tile overlap the MMAs of the next.  Groups are either uniform (every
 // group has the same row count: the per-cluster QKV projection, the output projection) or ragged
 // (the experts: an m-tile table built on the device by the permute step, so no host sync).
 //
@@ -24,23 +25,28 @@ constexpr int kStages = 4;
 constexpr int kABytes = kBM * kBK * 2;   // 16 KB
 constexpr int kBBytes = kBN * kBK * 2;   // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kGemmThreads = 192;
+constexpr int kEpiWarps = 8;          // two per tensor-memory lane quarter
+constexpr int kGemmThreads = 64 + kEpiWarps * 32;
 constexpr int kGatherThreads = 128;   // extra producer warps when the A rows are gathered
 constexpr int kTmemCols = 512;
-constexpr int kStgPitch = 128 + 16;                 // staging row: 128 bytes of output + bank-spreading pad
+constexpr int kStgPitch = 128;                       // staging row: 128 bytes of output, 16-byte chunks XOR-swizzled by row
 constexpr int kStgWarpBytes = 32 * kStgPitch;        // one epilogue warp stages its 32 rows
-constexpr size_t kGemmSmemBytes = size_t(kStages) * kStageBytes + 4 * kStgWarpBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr size_t kGemmSmemBytes = size_t(kStages) * kStageBytes + kEpiWarps * kStgWarpBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+// byte offset of 16-byte chunk c of staging row r (conflict-free for row-per-lane writes and 8-lanes-per-row reads)
+__device__ __forceinline__ int stg_off(int r, int c) { return r * kStgPitch + ((c ^ (r & 7)) << 4); }
 
 // z * sigmoid(z) with the fast exponential and the fast (two-ulp) division: two special-function operations per value
 __device__ __forceinline__ float silu_f(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
 
-// Epilogue of one 128 x 256 accumulator tile, run by the four epilogue warps (warp `quarter` owns TMEM lanes
-// 32*quarter ..).  `row0` is the first A row of the CTA's 128 rows, `release` is called once, right after the
-// last tensor-memory read, and hands the accumulator stage back to the MMA issuer.
+// Epilogue of one 128 x tile_cols accumulator tile, run by the eight epilogue warps: the two warps of `quarter` own
+// TMEM lanes 32*quarter .. and take the column passes of their `half` (passes half, half + 2, ...).  `row0` is the
+// first A row of the CTA's 128 rows; `release` is called once per warp, right after its last tensor-memory read,
+// and hands the accumulator stage back to the MMA issuer.
 template <int EPI, class ReleaseFn>
 __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_t taddr, uint8_t* stg, int lane, int quarter,
-                                                   int row0, int row_end, int group, int group_row0, int n0,
-                                                   ReleaseFn release) {
+                                                   int half, int row0, int row_end, int group, int group_row0, int n0,
+                                                   int tile_cols, ReleaseFn release) {
   const int row = row0 + quarter * 32 + lane;      // A row of this thread's accumulator lane
   const bool row_ok = row < row_end;
         // Every pass turns 128 bytes of output per row into registers (thread = accumulator row), parks them
@@ -51,13 +57,13 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
         if constexpr (EPI == kEpiQKV) {
           if (row_ok) scale = args.row_scale[size_t(group) * args.scale_group_stride + row_local];
         }
-        constexpr int kPassCols = (EPI == kEpiOProj) ? 32 : 64;          // output columns per pass
-        constexpr int kTilePasses = (EPI == kEpiSwiGLU) ? 2 : kBN / kPassCols;
+        constexpr int kPassCols = (EPI == kEpiOProj) ? 32 : 64;          // accumulator columns per pass (SwiGLU: 64 + 64)
+        const int n_pass = (EPI == kEpiSwiGLU) ? 2 : (tile_cols + kPassCols - 1) / kPassCols;
         const int wr_row = lane >> 3, wr_chunk = lane & 7;                // write-out role: row (+4j), 16-byte chunk
+        if (half >= n_pass) { release(); return; }                        // nothing for this warp in a one-pass tile
   #pragma unroll 1
-        for (int ps = 0; ps < kTilePasses; ++ps) {
+        for (int ps = half; ps < n_pass; ps += 2) {
           const int n = (EPI == kEpiSwiGLU) ? (n0 >> 1) + ps * 64 : n0 + ps * kPassCols;   // output column in the group
-          if (EPI != kEpiSwiGLU && n >= args.N) break;                    // warp-uniform
           uint32_t w[32];                                                // 128 bytes of this row's output
           __syncwarp();
           if constexpr (EPI == kEpiSwiGLU) {
@@ -120,10 +126,10 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
                 w[hf * 16 + c] = pack_bf16(__uint_as_float(r[2 * c]), __uint_as_float(r[2 * c + 1]));
             }
           }
-          if (ps == kTilePasses - 1 || (EPI != kEpiSwiGLU && n + kPassCols >= args.N)) release();   // last TMEM read of the tile
+          if (ps + 2 >= n_pass) release();                               // this warp's last TMEM read of the tile
   #pragma unroll
           for (int c = 0; c < 8; ++c)
-            *reinterpret_cast<uint4*>(stg + lane * kStgPitch + c * 16) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+            *reinterpret_cast<uint4*>(stg + stg_off(lane, c)) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
           __syncwarp();
           if constexpr (EPI == kEpiOProj) {
             // r_full = scale * (C + sum_h x[h]): the residual streams are read here.  This GEMM moves almost as many
@@ -147,8 +153,8 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
               const int rr = or_row + 8 * j;
               const int grow = row0 + quarter * 32 + rr;
               if (grow >= row_end) continue;
-              const float4 c0 = *reinterpret_cast<const float4*>(stg + rr * kStgPitch + or_cg * 32);
-              const float4 c1 = *reinterpret_cast<const float4*>(stg + rr * kStgPitch + or_cg * 32 + 16);
+              const float4 c0 = *reinterpret_cast<const float4*>(stg + stg_off(rr, 2 * or_cg));
+              const float4 c1 = *reinterpret_cast<const float4*>(stg + stg_off(rr, 2 * or_cg + 1));
               float a8[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
   #pragma unroll
               for (int h = 0; h < 8; ++h) {
@@ -167,7 +173,7 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
               const int rr = wr_row + 4 * j;                              // row inside the warp's 32
               const int grow = row0 + quarter * 32 + rr;
               if (grow >= row_end) continue;
-              const uint4 v = *reinterpret_cast<const uint4*>(stg + rr * kStgPitch + wr_chunk * 16);
+              const uint4 v = *reinterpret_cast<const uint4*>(stg + stg_off(rr, wr_chunk));
               if constexpr (EPI == kEpiQKV) {
                 const int tok = grow - group_row0;
                 // natural column inside the head of this lane's 8 values: chunks 0-3 first half, 4-7 second half
@@ -201,7 +207,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stg_all = smem + kStages * kStageBytes;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(stg_all + 4 * kStgWarpBytes);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(stg_all + kEpiWarps * kStgWarpBytes);
   uint64_t* empty_bar = full_bar + kStages;
   uint64_t* acc_full = empty_bar + kStages;
   uint64_t* acc_empty = acc_full + 2;
@@ -212,7 +218,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], GATHER ? 1 + kGatherThreads : 1); mbar_init(&empty_bar[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], kEpiWarps); }
     mbar_fence_init();
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
@@ -229,7 +235,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const bool ragged = args.n_mtiles != nullptr;
   const int tiles_per_group = (args.rows_per_group + kBM - 1) / kBM;
   const int n_mtiles = ragged ? *args.n_mtiles : args.n_groups * tiles_per_group;
-  const int n_ntiles = (args.N + kBN - 1) / kBN;
+  const int bn = args.bn;                                   // tile width = rows of the B map's box
+  const int n_ntiles = (args.N + bn - 1) / bn;
   const int total_tiles = n_mtiles * n_ntiles;
   const int kblocks = (args.K + kBK - 1) / kBK;
 
@@ -244,14 +251,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int group, row0;
         if (ragged) { group = args.mt_group[mt]; row0 = args.mt_row0[mt]; }
         else { group = mt / tiles_per_group; row0 = group * args.a_group_stride + (mt - group * tiles_per_group) * kBM; }
-        const int brow0 = group * args.N + nt * kBN;
+        const int brow0 = group * args.N + nt * bn;
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1)) { ok = false; break; }
           uint8_t* sa = smem + stage * kStageBytes;
           if constexpr (GATHER) {
-            mbar_expect_tx(&full_bar[stage], kBBytes);       // the A half arrives through the gather warps
+            mbar_expect_tx(&full_bar[stage], bn * (kBK * 2));            // the A half arrives through the gather warps
           } else {
-            mbar_expect_tx(&full_bar[stage], kStageBytes);
+            mbar_expect_tx(&full_bar[stage], kABytes + bn * (kBK * 2));
             tma_load_2d(sa, &tmA, &full_bar[stage], kb * kBK, row0);
           }
           tma_load_2d(sa + kABytes, &tmB, &full_bar[stage], kb * kBK, brow0);
@@ -263,7 +270,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (one thread)
     if (elect_one()) {
-      constexpr uint32_t idesc = umma_idesc_bf16(kBM, kBN);
+      const uint32_t idesc = umma_idesc_bf16(kBM, bn);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
@@ -292,7 +299,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
       if (!ok) atomicExch(args.status, kStatusTimeout);
     }
-  } else if (GATHER && warp >= 6) {
+  } else if (GATHER && warp >= 2 + kEpiWarps) {
     // ------------------------------------------------------------ A-gather producers (4 warps, one tile row each)
     // Row r of the tile is row a_row_index[row0 + r] of a_gather: the dispatch permutation is applied while
     // the operand is staged, so the permuted activations are never written to memory.  Each thread copies one
@@ -340,10 +347,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     asm volatile("cp.async.wait_all;" ::: "memory");      // nothing of this thread may still be in flight at exit
     if (!ok && lane == 0) atomicExch(args.status, kStatusTimeout);
-  } else if (warp >= 2 && warp < 6) {
-    // ------------------------------------------------------------ epilogue (4 warps = 128 TMEM lanes)
+  } else if (warp >= 2 && warp < 2 + kEpiWarps) {
+    // ------------------------------------------------------------ epilogue (2 x 4 warps over the 128 TMEM lanes)
     const int quarter = warp & 3;                 // a warp may only touch TMEM lanes 32*(warp%4)..+31
-    uint8_t* stg = stg_all + quarter * kStgWarpBytes;
+    const int half = (warp - 2) >> 2;             // which of the quarter's two warps
+    uint8_t* stg = stg_all + (warp - 2) * kStgWarpBytes;
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
@@ -357,15 +365,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         row0 = group_row0 + (mt - group * tiles_per_group) * kBM;
         row_end = group_row0 + args.rows_per_group;
       }
-      const int n0 = nt * kBN;                     // column inside the group
+      const int n0 = nt * bn;                      // column inside the group
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
       if (!mbar_wait(&acc_full[acc], acc_phase)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kBN;
 
-      gemm_epilogue_tile<EPI>(args, taddr, stg, lane, quarter, row0, row_end, group, group_row0, n0, [&]() {
-        // last read of this accumulator stage: hand it back to the MMA warp before the stores
+      gemm_epilogue_tile<EPI>(args, taddr, stg, lane, quarter, half, row0, row_end, group, group_row0, n0,
+                              min(bn, args.N - n0), [&]() {
+        // this warp's last read of the accumulator stage: hand it back to the MMA warp before the stores
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty[acc]);

@@ -8,7 +8,7 @@
 //   full[s]      used in the leader: 1 arrival (leader's expect_tx) + the bytes of BOTH CTAs' TMA loads
 //   empty[s]     used in each CTA: 1 arrival from the leader's multicast tcgen05.commit
 //   acc_full[a]  used in each CTA: 1 arrival from the leader's multicast tcgen05.commit
-//   acc_empty[a] used in the leader: 8 arrivals (4 epilogue warps of each CTA; the peer's arrive remotely)
+//   acc_empty[a] used in the leader: 16 arrivals (8 epilogue warps of each CTA; the peer's arrive remotely)
 #pragma once
 
 #include "gemm_tcgen05.cuh"
@@ -18,7 +18,7 @@ namespace foe {
 constexpr int kPairStages = 6;
 constexpr int kPairBBytes = (kBN / 2) * kBK * 2;                       // this CTA's half of the B tile: 16 KB
 constexpr int kPairStageBytes = kABytes + kPairBBytes;                 // 32 KB
-constexpr size_t kPairSmemBytes = size_t(kPairStages) * kPairStageBytes + 4 * kStgWarpBytes + 1024 + 256;
+constexpr size_t kPairSmemBytes = size_t(kPairStages) * kPairStageBytes + kEpiWarps * kStgWarpBytes + 1024 + 256;
 constexpr int kPairTileRows = 2 * kBM;                                 // 256 rows per pair tile
 
 template <int EPI>
@@ -28,7 +28,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stg_all = smem + kPairStages * kPairStageBytes;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(stg_all + 4 * kStgWarpBytes);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(stg_all + kEpiWarps * kStgWarpBytes);
   uint64_t* empty_bar = full_bar + kPairStages;
   uint64_t* acc_full = empty_bar + kPairStages;
   uint64_t* acc_empty = acc_full + 2;
@@ -45,7 +45,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
-    for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 8); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 2 * kEpiWarps); }
     mbar_fence_init();
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
@@ -65,7 +65,8 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
   const bool ragged = args.n_mtiles != nullptr;
   const int tiles_per_group = (args.rows_per_group + kPairTileRows - 1) / kPairTileRows;
   const int n_mtiles = ragged ? *args.n_mtiles : args.n_groups * tiles_per_group;
-  const int n_ntiles = (args.N + kBN - 1) / kBN;
+  const int bn = args.bn;                                // tile width; each CTA stages bn / 2 rows of B (= the B map's box)
+  const int n_ntiles = (args.N + bn - 1) / bn;
   const int total_tiles = n_mtiles * n_ntiles;
   const int kblocks = (args.K + kBK - 1) / kBK;
 
@@ -92,11 +93,11 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
       for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
         int group, row0, row_end, group_row0, nt;
         tile_coords(tile, group, row0, row_end, group_row0, nt);
-        const int brow0 = group * args.N + nt * kBN + int(rank) * (kBN / 2);     // this CTA's half of the B rows
+        const int brow0 = group * args.N + nt * bn + int(rank) * (bn / 2);       // this CTA's half of the B rows
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1)) { ok = false; break; }
           uint8_t* sa = smem + stage * kPairStageBytes;
-          if (leader) mbar_expect_tx(&full_bar[stage], 2 * kPairStageBytes);
+          if (leader) mbar_expect_tx(&full_bar[stage], 2 * (kABytes + (bn / 2) * (kBK * 2)));
           tma_load_2d_pair(sa, &tmA, &full_bar[stage], kb * kBK, row0);
           tma_load_2d_pair(sa + kABytes, &tmB, &full_bar[stage], kb * kBK, brow0);
           if (++stage == kPairStages) { stage = 0; phase ^= 1; }
@@ -107,7 +108,7 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (one thread of the leader CTA)
     if (leader && elect_one()) {
-      constexpr uint32_t idesc = umma_idesc_bf16(kPairTileRows, kBN);
+      const uint32_t idesc = umma_idesc_bf16(kPairTileRows, bn);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
@@ -135,23 +136,25 @@ gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
       }
       if (!ok) atomicExch(args.status, kStatusTimeout);
     }
-  } else if (warp >= 2 && warp < 6) {
-    // ------------------------------------------------------------ epilogue (4 warps per CTA, own 128 rows)
+  } else if (warp >= 2 && warp < 2 + kEpiWarps) {
+    // ------------------------------------------------------------ epilogue (8 warps per CTA, own 128 rows)
     const int quarter = warp & 3;
-    uint8_t* stg = stg_all + quarter * kStgWarpBytes;
+    const int half = (warp - 2) >> 2;
+    uint8_t* stg = stg_all + (warp - 2) * kStgWarpBytes;
     const uint32_t leader_acc_empty0 = mapa_u32(smem_u32(&acc_empty[0]), 0);
     int it = 0;
     bool ok = true;
     for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++it) {
       int group, row0, row_end, group_row0, nt;
       tile_coords(tile, group, row0, row_end, group_row0, nt);
-      const int n0 = nt * kBN;
+      const int n0 = nt * bn;
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
       if (!mbar_wait(&acc_full[acc], acc_phase)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kBN;
-      gemm_epilogue_tile<EPI>(args, taddr, stg, lane, quarter, row0, row_end, group, group_row0, n0, [&]() {
+      gemm_epilogue_tile<EPI>(args, taddr, stg, lane, quarter, half, row0, row_end, group, group_row0, n0,
+                              min(bn, args.N - n0), [&]() {
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(leader_acc_empty0 + acc * 8);

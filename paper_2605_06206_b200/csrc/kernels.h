@@ -87,7 +87,7 @@ void launch_attn_decode(const CUtensorMap& tmK, const CUtensorMap& tmV, const At
 // ---- gemm_tcgen05.cu
 void launch_gemm(int epi, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args, int n_sms,
                  cudaStream_t st);
-void launch_gemm_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args, int n_sms,
+void launch_gemm_pair(int epi, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args, int n_sms,
                       cudaStream_t st);
 cudaError_t gemm_configure();   // opt in to the dynamic shared memory the kernels need
 
