@@ -74,8 +74,7 @@ struct foe_layer {
   foe_workspace* ws;
   int max_splits, pages_per_split;
   // tensor maps of the weights
-  CUtensorMap tm_wo, tm_wgu;
-  CUtensorMap tmp_wqkv, tmp_wd;                    // half-tile boxes: each CTA of a pair loads half of a B tile
+  CUtensorMap tm_wqkv, tm_wo, tm_wgu, tm_wd;       // weights; box = the rows of B one CTA of a pair stages per k-block
   CUtensorMap tms_wqkv, tms_wo, tms_wgu, tms_wd;   // same weights, boxes sized for the decode kernels
   // call state
   cudaStream_t last_stream;
@@ -186,7 +185,7 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     ga.q_cols = L->g * dh; ga.kv_cols = L->c * dh; ga.dh = dh; ga.n_kv = L->n_kv;
     ga.rope_tab = L->rope_tab; ga.tok_pos = L->ws->tok_pos; ga.tok_slot = L->ws->tok_slot;
     ga.k_pages = static_cast<bf16*>(kv->k_pages); ga.v_pages = static_cast<bf16*>(kv->v_pages);
-    launch_gemm_pair(kEpiQKV, tmX, L->tmp_wqkv, ga, L->n_sms, st);
+    launch_gemm(kEpiQKV, tmX, L->tm_wqkv, ga, L->n_sms, st);
   } else {
     SmallMArgs sa;
     memset(&sa, 0, sizeof(sa));
@@ -252,8 +251,7 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     GemmArgs g2 = g1;
     g2.a_gather = nullptr; g2.a_row_index = nullptr;
     g2.N = d; g2.K = L->I; g2.out = L->ws->y; g2.ldo = d;
-    g2.mt_group = L->ws->pb.mt2_group; g2.mt_row0 = L->ws->pb.mt2_row0; g2.n_mtiles = L->ws->pb.n_mtiles2;   // 256-row tiles
-    launch_gemm_pair(kEpiBf16, L->ws->tm_hmid, L->tmp_wd, g2, L->n_sms, st);
+    launch_gemm(kEpiBf16, L->ws->tm_hmid, L->tm_wd, g2, L->n_sms, st);
     L->launches += 2;
   } else {
     stage_mark(L, kStGemm1, st);
@@ -402,12 +400,9 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     ok = ok && walloc(W, &W->pb.inv, size_t(R));
     ok = ok && walloc(W, &W->pb.rank, size_t(R));
     ok = ok && walloc(W, &W->pb.blk_counts, size_t(n_blocks) * E);
-    ok = ok && walloc(W, &W->pb.mt_group, size_t(R / 128 + E + 1));
-    ok = ok && walloc(W, &W->pb.mt_row0, size_t(R / 128 + E + 1));
+    ok = ok && walloc(W, &W->pb.mt_group, size_t(R / 256 + E + 1));
+    ok = ok && walloc(W, &W->pb.mt_row0, size_t(R / 256 + E + 1));
     ok = ok && walloc(W, &W->pb.n_mtiles, size_t(1));
-    ok = ok && walloc(W, &W->pb.mt2_group, size_t(R / 256 + E + 1));
-    ok = ok && walloc(W, &W->pb.mt2_row0, size_t(R / 256 + E + 1));
-    ok = ok && walloc(W, &W->pb.n_mtiles2, size_t(1));
     if (!ok) { foe_layer_destroy(L); return FOE_ERR_OOM; }
     cudaMemsetAsync(W->status, 0, sizeof(int), st);
     cudaMemsetAsync(W->attn_o, 0, size_t(S + 128) * L->n_q * dh * sizeof(bf16), st);
@@ -455,11 +450,10 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     foe_layer_destroy(L);
     return FOE_ERR_CUDA;
   }
-  // box rows of a B map = the tile width its GEMM runs with (half of it for the CTA-pair kernel)
-  ok = make_map_2d(&L->tm_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, gemm_tile_cols(d)) &&
-       make_map_2d(&L->tm_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, kBN) &&
-       make_map_2d(&L->tmp_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, gemm_tile_cols(qkvN) / 2) &&
-       make_map_2d(&L->tmp_wd, L->wd_t, uint64_t(E) * d, I, gemm_tile_cols(d) / 2) &&
+  ok = make_map_2d(&L->tm_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, gemm_tile_rows_b(kEpiQKV, qkvN)) &&
+       make_map_2d(&L->tm_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, gemm_tile_rows_b(kEpiOProj, d)) &&
+       make_map_2d(&L->tm_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, gemm_tile_rows_b(kEpiSwiGLU, 2 * I)) &&
+       make_map_2d(&L->tm_wd, L->wd_t, uint64_t(E) * d, I, gemm_tile_rows_b(kEpiBf16, d)) &&
        make_map_2d(&L->tms_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, 64) &&
        make_map_2d(&L->tms_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, 64) &&
        make_map_2d(&L->tms_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, 32) &&

@@ -7,7 +7,7 @@
 
 namespace foe {
 
-constexpr int kBM = 128;   // GEMM tile rows  (UMMA M)
+constexpr int kBM = 128;   // GEMM tile rows per CTA (UMMA M of a CTA pair = 256)
 constexpr int kBN = 256;   // widest GEMM tile (UMMA N); the launcher narrows it in steps of 64 so that N splits evenly
 
 // Tile width for N columns per group: as few tiles as 256 allows, all of the same width (384 columns are two tiles
@@ -24,6 +24,10 @@ enum GemmEpilogue : int {
   kEpiOProj = 3     // r_full = scale * (C + sum_h x[h]) -> fp32 [row][ldo]
 };
 
+// Rows of B one CTA of a pair stages per k-block = box rows of the B tensor map: half a tile.  The SwiGLU epilogue
+// needs the full 256-wide tile (128 gate columns, 128 up columns).
+__host__ __device__ constexpr int gemm_tile_rows_b(int epi, int N) { return (epi == kEpiSwiGLU ? kBN : gemm_tile_cols(N)) / 2; }
+
 struct GemmArgs {
   // uniform groups
   int n_groups;
@@ -36,7 +40,7 @@ struct GemmArgs {
   const int* n_mtiles;      // device scalar
   int N;                    // columns per group (rows of B per group)
   int K;
-  int bn;                   // tile width, set by the launcher (gemm_tile_cols(N); 256 for kEpiSwiGLU)
+  int bn;                   // tile width, set by the launcher (2 * gemm_tile_rows_b)
   int* status;              // device status word
   // gathered A operand (expert GEMM 1): A row r of a tile is a_gather[a_row_index[r]][:]; nullptr = A through tmA
   const __nv_bfloat16* a_gather;

@@ -2,13 +2,27 @@
 //
 //   C_g[m, n] = sum_k A[row_g(m), k] * B_g[n, k]          fp32 accumulation in tensor memory
 //
-// One persistent CTA per SM walks a static round-robin list of 128 x bn output tiles (bn <= 256).  Warp 0 is
-// the TMA producer, warp 1 issues the MMAs and owns the TMEM allocation, warps 2..9 drain the
-// accumulator (tcgen05.ld) and apply the epilogue: two warps per 32-lane quarter of tensor memory, which take
-// alternate column passes, so that twice as many global loads and stores of the epilogue are in flight.  Two
-// accumulator stages (2 x 256 TMEM columns) let the epilogue of one tile overlap the MMAs of the next.  Groups are either uniform (every
-// group has the same row count: the per-cluster QKV projection, the output projection) or ragged
-// (the experts: an m-tile table built on the device by the permute step, so no host sync).
+// A cluster of two CTAs (two SMs) computes one 256 x bn output tile (bn <= 256) with tcgen05.mma.cta_group::2 and
+// walks a static round-robin list of tiles.  Each CTA stages only its own 128 A rows and its own half of the B rows,
+// so the shared-memory traffic per SM and k-block (TMA writes + tensor-core reads) is a third lower than with one
+// CTA per tile -- and that traffic, not the MMA rate, is what bounds a one-CTA 128 x 256 tile -- and six stages fit
+// where four did.  The leader CTA (cluster rank 0) issues the MMAs for both; accumulators live in each CTA's own
+// tensor memory (its 128 rows x 256 columns, two stages, so the epilogue of one tile overlaps the MMAs of the next)
+// and each CTA's epilogue warps drain their half.
+//
+// Warp roles per CTA: warp 0 TMA producer, warp 1 MMA issuer (leader) / gather relay (peer), warps 2..9 epilogue (two
+// warps per 32-lane quarter of tensor memory, alternate column passes), warps 10..13 A-gather producers (GATHER only).
+// Groups are either uniform (every group has the same row count: the per-cluster QKV projection, the output
+// projection) or ragged (the experts: an m-tile table built on the device by the permute step, so no host sync).
+//
+// Barrier protocol (every barrier exists in both CTAs at the same shared-memory offset):
+//   full[s]      used in the leader: 1 arrival (leader's expect_tx) + the bytes of BOTH CTAs' TMA loads; with a
+//                gathered A also one arrival per gather thread of the leader (carried by its cp.async copies) and
+//                one from the peer's relay thread
+//   a_full[s]    gathered A only, used in the peer: one arrival per gather thread of the peer
+//   empty[s]     used in each CTA: 1 arrival from the leader's multicast tcgen05.commit
+//   acc_full[a]  used in each CTA: 1 arrival from the leader's multicast tcgen05.commit
+//   acc_empty[a] used in the leader: 16 arrivals (8 epilogue warps of each CTA; the peer's arrive remotely)
 //
 // Used for steps of the paper's Table 2: Attn_h's projections ("Attn. residual" row), the sync
 // ("Cross-group avg." row, fused into the output-projection epilogue) and FFN_e ("MoE update" row).
@@ -21,10 +35,11 @@ namespace foe {
 
 constexpr int kBK = 64;              // k-block: 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;
-constexpr int kStages = 4;
-constexpr int kABytes = kBM * kBK * 2;   // 16 KB
-constexpr int kBBytes = kBN * kBK * 2;   // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kStages = 6;
+constexpr int kABytes = kBM * kBK * 2;                 // this CTA's 128 A rows of a k-block: 16 KB
+constexpr int kBHalfBytes = (kBN / 2) * kBK * 2;       // this CTA's half of the widest B tile: 16 KB
+constexpr int kStageBytes = kABytes + kBHalfBytes;     // 32 KB
+constexpr int kPairTileRows = 2 * kBM;                 // 256 rows per tile
 constexpr int kEpiWarps = 8;          // two per tensor-memory lane quarter
 constexpr int kGemmThreads = 64 + kEpiWarps * 32;
 constexpr int kGatherThreads = 128;   // extra producer warps when the A rows are gathered
@@ -201,9 +216,9 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
 }
 
 template <int EPI, bool GATHER>
-__global__ void __launch_bounds__(kGemmThreads + (GATHER ? kGatherThreads : 0), 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads + (GATHER ? kGatherThreads : 0), 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const GemmArgs args) {
+                         const GemmArgs args) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stg_all = smem + kStages * kStageBytes;
@@ -211,71 +226,90 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   uint64_t* empty_bar = full_bar + kStages;
   uint64_t* acc_full = empty_bar + kStages;
   uint64_t* acc_empty = acc_full + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* a_full = acc_empty + 2;                      // gathered A only (peer CTA)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(a_full + kStages);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();               // 0 = leader
+  const bool leader = rank == 0;
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], GATHER ? 1 + kGatherThreads : 1); mbar_init(&empty_bar[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], kEpiWarps); }
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&full_bar[s], GATHER ? 1 + kGatherThreads + 1 : 1);
+      mbar_init(&empty_bar[s], 1);
+      mbar_init(&a_full[s], kGatherThreads);
+    }
+    for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 2 * kEpiWarps); }
     mbar_fence_init();
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
   }
+  __syncthreads();
+  cluster_sync_all();                                    // both CTAs' barriers exist before anything remote touches them
   if (warp == 1) {
-    tmem_alloc(tmem_slot, kTmemCols);
-    tmem_relinquish();
+    tmem_alloc_pair(tmem_slot, kTmemCols);
+    tmem_relinquish_pair();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // tiles: groups are cut into 256-row pair tiles (the device-built table for the ragged experts uses the same size)
   const bool ragged = args.n_mtiles != nullptr;
-  const int tiles_per_group = (args.rows_per_group + kBM - 1) / kBM;
+  const int tiles_per_group = (args.rows_per_group + kPairTileRows - 1) / kPairTileRows;
   const int n_mtiles = ragged ? *args.n_mtiles : args.n_groups * tiles_per_group;
-  const int bn = args.bn;                                   // tile width = rows of the B map's box
+  const int bn = args.bn;                                // tile width; each CTA stages bn / 2 rows of B (= the B map's box)
   const int n_ntiles = (args.N + bn - 1) / bn;
   const int total_tiles = n_mtiles * n_ntiles;
   const int kblocks = (args.K + kBK - 1) / kBK;
 
+  auto tile_coords = [&](int tile, int& group, int& row0, int& row_end, int& group_row0, int& nt) {
+    const int mt = tile / n_ntiles;
+    nt = tile - mt * n_ntiles;
+    if (ragged) {
+      group = args.mt_group[mt]; row0 = args.mt_row0[mt]; row_end = args.group_end[group]; group_row0 = 0;
+    } else {
+      group = mt / tiles_per_group;
+      group_row0 = group * args.a_group_stride;
+      row0 = group_row0 + (mt - group * tiles_per_group) * kPairTileRows;
+      row_end = group_row0 + args.rows_per_group;
+    }
+    row0 += int(rank) * kBM;                             // this CTA's 128 rows of the pair tile
+  };
+
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer (one thread)
+    // ------------------------------------------------------------ TMA producer (one thread per CTA)
     if (elect_one()) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int mt = tile / n_ntiles, nt = tile - mt * n_ntiles;
-        int group, row0;
-        if (ragged) { group = args.mt_group[mt]; row0 = args.mt_row0[mt]; }
-        else { group = mt / tiles_per_group; row0 = group * args.a_group_stride + (mt - group * tiles_per_group) * kBM; }
-        const int brow0 = group * args.N + nt * bn;
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
+        int group, row0, row_end, group_row0, nt;
+        tile_coords(tile, group, row0, row_end, group_row0, nt);
+        const int brow0 = group * args.N + nt * bn + int(rank) * (bn / 2);       // this CTA's half of the B rows
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1)) { ok = false; break; }
           uint8_t* sa = smem + stage * kStageBytes;
-          if constexpr (GATHER) {
-            mbar_expect_tx(&full_bar[stage], bn * (kBK * 2));            // the A half arrives through the gather warps
-          } else {
-            mbar_expect_tx(&full_bar[stage], kABytes + bn * (kBK * 2));
-            tma_load_2d(sa, &tmA, &full_bar[stage], kb * kBK, row0);
-          }
-          tma_load_2d(sa + kABytes, &tmB, &full_bar[stage], kb * kBK, brow0);
+          if (leader) mbar_expect_tx(&full_bar[stage], 2 * ((GATHER ? 0 : kABytes) + (bn / 2) * (kBK * 2)));
+          if constexpr (!GATHER) tma_load_2d_pair(sa, &tmA, &full_bar[stage], kb * kBK, row0);
+          tma_load_2d_pair(sa + kABytes, &tmB, &full_bar[stage], kb * kBK, brow0);
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
       }
       if (!ok) atomicExch(args.status, kStatusTimeout);
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer (one thread)
-    if (elect_one()) {
-      const uint32_t idesc = umma_idesc_bf16(kBM, bn);
+    // ------------------------------------------------------------ MMA issuer (one thread of the leader CTA)
+    if (leader && elect_one()) {
+      const uint32_t idesc = umma_idesc_bf16(kPairTileRows, bn);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++it) {
         const int acc = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1;
         if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1)) { ok = false; break; }
@@ -284,54 +318,74 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(&full_bar[stage], phase)) { ok = false; break; }
           tc_fence_after();
-          if constexpr (GATHER) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // cp.async-written A tile
+          if constexpr (GATHER) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the leader's cp.async-written rows
           const uint32_t a_addr = smem_u32(smem + stage * kStageBytes);
           const uint32_t b_addr = a_addr + kABytes;
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
-            umma_bf16(d_tmem, umma_desc_sw128(a_addr + k * kUmmaK * 2), umma_desc_sw128(b_addr + k * kUmmaK * 2),
-                      idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_bf16_pair(d_tmem, umma_desc_sw128(a_addr + k * kUmmaK * 2), umma_desc_sw128(b_addr + k * kUmmaK * 2),
+                           idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          umma_commit(&empty_bar[stage]);
+          umma_commit_pair(&empty_bar[stage], 3);          // both CTAs may refill this stage
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
-        if (ok) umma_commit(&acc_full[acc]);
+        if (ok) umma_commit_pair(&acc_full[acc], 3);       // both CTAs' epilogues may drain their halves
+      }
+      if (!ok) atomicExch(args.status, kStatusTimeout);
+    } else if (GATHER && !leader && elect_one()) {
+      // relay (the peer's otherwise idle warp 1): the peer's gathered A rows of a stage have landed -> make them
+      // visible to the tensor core's reads and tell the leader's MMA thread.  The arrival is relaxed: a releasing
+      // remote arrival costs about a microsecond each, more than two k-blocks, and orders nothing that matters
+      // here: the rows are in shared memory once the copies have arrived on a_full, the proxy fence below comes
+      // before the arrival in program order, and the reader is the tensor core, which starts after the leader has
+      // seen this arrival.
+      const uint32_t leader_full0 = mapa_u32(smem_u32(&full_bar[0]), 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(&a_full[stage], phase)) { ok = false; break; }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          mbar_arrive_cluster_relaxed(leader_full0 + stage * 8);
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
       }
       if (!ok) atomicExch(args.status, kStatusTimeout);
     }
   } else if (GATHER && warp >= 2 + kEpiWarps) {
-    // ------------------------------------------------------------ A-gather producers (4 warps, one tile row each)
-    // Row r of the tile is row a_row_index[row0 + r] of a_gather: the dispatch permutation is applied while
-    // the operand is staged, so the permuted activations are never written to memory.  Each thread copies one
-    // 16-byte chunk of eight rows per k-block with cp.async into the 128-byte-swizzled operand layout and lets
-    // the copies themselves arrive on the stage's barrier (cp.async.mbarrier.arrive.noinc); the MMA thread
-    // crosses to the async proxy with a fence before it issues the tensor-core reads.
-    const int gt = threadIdx.x - kGemmThreads;            // 0..127
-    const int gc = gt & 7, gr = gt >> 3;                  // 16-byte chunk of a row; rows gr + 16 j, j < 8:
-                                                          // 8 lanes read one row's 128 bytes as a whole line
+    // ------------------------------------------------------------ A-gather producers (4 warps in each CTA, own 128 rows)
+    // Row r of the tile is row a_row_index[row0 + r] of a_gather.  Each thread copies one 16-byte chunk of eight
+    // rows per k-block with cp.async into the swizzled operand layout; the copies themselves arrive on a barrier of
+    // their own CTA (cp.async.mbarrier.arrive.noinc): the leader's on full[s], the peer's on a_full[s].  One lane
+    // per warp polls the stage's empty barrier: it receives its arrivals from the other SM, and a crowd of
+    // pollers slows those down.
+    const int gt = threadIdx.x - kGemmThreads;
+    const int gc = gt & 7, gr = gt >> 3;
+    uint64_t* my_full = leader ? full_bar : a_full;
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
-    // The source rows of a tile come from two dependent loads (tile table, then dispatch map): they are fetched one
-    // tile ahead, so the producer never sits through that latency at a tile boundary.
     auto tile_rows = [&](int tile, int (&rows)[8]) {
       if (tile < total_tiles) {
-        const int mt = tile / n_ntiles;
-        const int group = args.mt_group[mt], row0 = args.mt_row0[mt], row_end = args.group_end[group];
+        int group, row0, row_end, group_row0, nt;
+        tile_coords(tile, group, row0, row_end, group_row0, nt);
 #pragma unroll
         for (int j = 0; j < 8; ++j) rows[j] = args.a_row_index[min(row0 + gr + 16 * j, row_end - 1)];
       }
     };
     int next_rows[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    tile_rows(blockIdx.x, next_rows);
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+    tile_rows(pair, next_rows);
+    for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
       const uint8_t* src[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j)
         src[j] = reinterpret_cast<const uint8_t*>(args.a_gather) + size_t(next_rows[j]) * args.K * 2 + gc * 16;
-      tile_rows(tile + gridDim.x, next_rows);              // in flight while this tile's k-blocks are copied
+      tile_rows(tile + n_pairs, next_rows);
       for (int kb = 0; kb < kblocks; ++kb) {
-        if (!mbar_wait(&empty_bar[stage], phase ^ 1)) { ok = false; break; }
+        if (lane == 0) ok = mbar_wait(&empty_bar[stage], phase ^ 1);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
         const uint32_t dst = smem_u32(smem + stage * kStageBytes);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -339,56 +393,46 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + r * 128 + ((gc ^ (r & 7)) << 4)),
                        "l"(src[j] + size_t(kb) * 128) : "memory");
         }
-        // the barrier gets this thread's arrival when the copies above have landed; nothing blocks here, so a
-        // thread runs as far ahead as free stages allow
-        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&full_bar[stage])) : "memory");
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&my_full[stage])) : "memory");
         if (++stage == kStages) { stage = 0; phase ^= 1; }
       }
     }
-    asm volatile("cp.async.wait_all;" ::: "memory");      // nothing of this thread may still be in flight at exit
+    asm volatile("cp.async.wait_all;" ::: "memory");
     if (!ok && lane == 0) atomicExch(args.status, kStatusTimeout);
   } else if (warp >= 2 && warp < 2 + kEpiWarps) {
-    // ------------------------------------------------------------ epilogue (2 x 4 warps over the 128 TMEM lanes)
-    const int quarter = warp & 3;                 // a warp may only touch TMEM lanes 32*(warp%4)..+31
-    const int half = (warp - 2) >> 2;             // which of the quarter's two warps
+    // ------------------------------------------------------------ epilogue (8 warps per CTA, own 128 rows)
+    const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;
     uint8_t* stg = stg_all + (warp - 2) * kStgWarpBytes;
+    const uint32_t leader_acc_empty0 = mapa_u32(smem_u32(&acc_empty[0]), 0);
     int it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-      const int mt = tile / n_ntiles, nt = tile - mt * n_ntiles;
-      int group, row0, row_end, group_row0;
-      if (ragged) {
-        group = args.mt_group[mt]; row0 = args.mt_row0[mt]; row_end = args.group_end[group]; group_row0 = 0;
-      } else {
-        group = mt / tiles_per_group;
-        group_row0 = group * args.a_group_stride;
-        row0 = group_row0 + (mt - group * tiles_per_group) * kBM;
-        row_end = group_row0 + args.rows_per_group;
-      }
-      const int n0 = nt * bn;                      // column inside the group
+    for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++it) {
+      int group, row0, row_end, group_row0, nt;
+      tile_coords(tile, group, row0, row_end, group_row0, nt);
+      const int n0 = nt * bn;
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
       if (!mbar_wait(&acc_full[acc], acc_phase)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kBN;
-
       gemm_epilogue_tile<EPI>(args, taddr, stg, lane, quarter, half, row0, row_end, group, group_row0, n0,
                               min(bn, args.N - n0), [&]() {
-        // this warp's last read of the accumulator stage: hand it back to the MMA warp before the stores
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&acc_empty[acc]);
+        if (lane == 0) mbar_arrive_cluster_relaxed(leader_acc_empty0 + acc * 8);   // tensor memory is not ordered by a release anyway
       });
     }
     if (!ok && lane == 0) atomicExch(args.status, kStatusTimeout);
   }
 
-  // ---------------------------------------------------------------- teardown
+  // ---------------------------------------------------------------- teardown (both CTAs, together)
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
+    tmem_dealloc_pair(tmem_base, kTmemCols);
   }
 }
 

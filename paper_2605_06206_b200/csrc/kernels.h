@@ -48,12 +48,9 @@ struct PermuteBuffers {
   int* inv;           // [S*H*kc]
   int* rank;          // [S*H*kc] rank of the selection inside its token block
   int* blk_counts;    // [n_blocks][E]
-  int* mt_group;      // [R/128 + E] tiles of 128 rows: expert and first row of each
-  int* mt_row0;
+  int* mt_group;      // [R/256 + E] tiles of 256 rows (one per CTA pair of the grouped GEMM): expert of each
+  int* mt_row0;       //             and its first row
   int* n_mtiles;      // scalar
-  int* mt2_group;     // [R/256 + E] the same for tiles of 256 rows (CTA-pair GEMM)
-  int* mt2_row0;
-  int* n_mtiles2;     // scalar
 };
 constexpr int kPermuteBlockTokens = 256;
 // returns the number of kernels launched (1 for calls of at most 256 tokens, else 3)
@@ -87,8 +84,6 @@ void launch_attn_decode(const CUtensorMap& tmK, const CUtensorMap& tmV, const At
 // ---- gemm_tcgen05.cu
 void launch_gemm(int epi, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args, int n_sms,
                  cudaStream_t st);
-void launch_gemm_pair(int epi, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args, int n_sms,
-                      cudaStream_t st);
 cudaError_t gemm_configure();   // opt in to the dynamic shared memory the kernels need
 
 // ---- smallm.cu  (weight-streaming GEMMs for a handful of rows per group)

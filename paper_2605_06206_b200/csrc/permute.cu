@@ -9,7 +9,7 @@
 // The activation rows themselves are not moved here: expert GEMM 1 gathers them through perm while it stages
 // its A operand.  Three launches: (1) every block of 256 tokens builds a token-bitmap per expert in shared memory,
 // from which each selection reads its rank inside the block; (2) one block scans block counts and
-// expert totals and writes the m-tile tables the grouped GEMMs walk; (3) every selection computes its
+// expert totals and writes the m-tile table the grouped GEMMs walk; (3) every selection computes its
 // slot.
 #include "common.cuh"
 #include "kernels.h"
@@ -54,20 +54,19 @@ permute_count_kernel(const int* __restrict__ idx, int* __restrict__ rank, int* _
   }
 }
 
-// Tile tables the grouped GEMMs walk: expert and first row of every 128-row tile and of every 256-row tile of
-// every non-empty expert.  Expert e owns tiles1 / tiles2 entries from tile0_1 / tile0_2 on; the last expert also
-// writes the table lengths (sum1, sum2).
-__device__ __forceinline__ void write_tile_tables(const PermuteBuffers& pb, int e, int E, int row0, int tiles1,
-                                                  int tile0_1, int tiles2, int tile0_2, int sum1, int sum2) {
-  if (e == E - 1) { *pb.n_mtiles = sum1; *pb.n_mtiles2 = sum2; }
-  for (int j = 0; j < tiles1; ++j) { pb.mt_group[tile0_1 + j] = e; pb.mt_row0[tile0_1 + j] = row0 + j * 128; }
-  for (int j = 0; j < tiles2; ++j) { pb.mt2_group[tile0_2 + j] = e; pb.mt2_row0[tile0_2 + j] = row0 + j * 256; }
+// Tile table the grouped GEMMs walk: expert and first row of every 256-row tile of every non-empty expert.  Expert e
+// owns `tiles` entries from tile0 on; the last expert also writes the table length.
+constexpr int kTileRows = 256;
+__device__ __forceinline__ void write_tile_table(const PermuteBuffers& pb, int e, int E, int row0, int tiles, int tile0,
+                                                 int n_tiles_all) {
+  if (e == E - 1) *pb.n_mtiles = n_tiles_all;
+  for (int j = 0; j < tiles; ++j) { pb.mt_group[tile0 + j] = e; pb.mt_row0[tile0 + j] = row0 + j * kTileRows; }
 }
 
-// Single block.  blk_counts[b][e] becomes the exclusive prefix over b; counts/offsets and the tile tables are written.
+// Single block.  blk_counts[b][e] becomes the exclusive prefix over b; counts/offsets and the tile table are written.
 __global__ void __launch_bounds__(1024)
 permute_scan_kernel(int* __restrict__ blk_counts, int n_blocks, int E, const PermuteBuffers pb) {
-  __shared__ int s_a[1024], s_b[1024], s_c[1024];
+  __shared__ int s_a[1024], s_b[1024];
   int* counts = pb.counts;
   int* offsets = pb.offsets;
   const int e = threadIdx.x;
@@ -80,27 +79,24 @@ permute_scan_kernel(int* __restrict__ blk_counts, int n_blocks, int E, const Per
     }
     counts[e] = total;
   }
-  const int tiles1 = (total + 127) / 128, tiles2 = (total + 255) / 256;
-  // three inclusive Hillis-Steele scans over the expert id (rows, 128-row tiles, 256-row tiles)
+  const int tiles = (total + kTileRows - 1) / kTileRows;
+  // two inclusive Hillis-Steele scans over the expert id (rows and tiles)
   s_a[e] = total;
-  s_b[e] = tiles1;
-  s_c[e] = tiles2;
+  s_b[e] = tiles;
   __syncthreads();
   for (int o = 1; o < 1024; o <<= 1) {
     const int va = e >= o ? s_a[e - o] : 0;
     const int vb = e >= o ? s_b[e - o] : 0;
-    const int vc = e >= o ? s_c[e - o] : 0;
     __syncthreads();
     s_a[e] += va;
     s_b[e] += vb;
-    s_c[e] += vc;
     __syncthreads();
   }
   if (e < E) {
     const int row0 = s_a[e] - total;
     offsets[e] = row0;
     if (e == E - 1) offsets[E] = s_a[e];
-    write_tile_tables(pb, e, E, row0, tiles1, s_b[e] - tiles1, tiles2, s_c[e] - tiles2, s_b[e], s_c[e]);
+    write_tile_table(pb, e, E, row0, tiles, s_b[e] - tiles, s_b[e]);
   }
 }
 
@@ -123,7 +119,7 @@ __global__ void __launch_bounds__(1024)
 permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, const PermuteBuffers pb,
                      int* __restrict__ status) {
   extern __shared__ uint32_t bm[];            // [E][8]
-  __shared__ int s_a[1024], s_b[1024], s_c[1024], s_off[1024];
+  __shared__ int s_a[1024], s_b[1024], s_off[1024];
   int* counts = pb.counts;
   int* offsets = pb.offsets;
   int* perm = pb.perm;
@@ -145,19 +141,16 @@ permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, 
     for (int k = 0; k < 8; ++k) total += __popc(bm[t * 8 + k]);
     counts[t] = total;
   }
-  const int tiles1 = (total + 127) / 128, tiles2 = (total + 255) / 256;
+  const int tiles = (total + kTileRows - 1) / kTileRows;
   s_a[t] = total;
-  s_b[t] = tiles1;
-  s_c[t] = tiles2;
+  s_b[t] = tiles;
   __syncthreads();
   for (int o = 1; o < 1024; o <<= 1) {
     const int va = t >= o ? s_a[t - o] : 0;
     const int vb = t >= o ? s_b[t - o] : 0;
-    const int vc = t >= o ? s_c[t - o] : 0;
     __syncthreads();
     s_a[t] += va;
     s_b[t] += vb;
-    s_c[t] += vc;
     __syncthreads();
   }
   if (t < E) {
@@ -165,7 +158,7 @@ permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, 
     offsets[t] = row0;
     s_off[t] = row0;
     if (t == E - 1) offsets[E] = s_a[t];
-    write_tile_tables(pb, t, E, row0, tiles1, s_b[t] - tiles1, tiles2, s_c[t] - tiles2, s_b[t], s_c[t]);
+    write_tile_table(pb, t, E, row0, tiles, s_b[t] - tiles, s_b[t]);
   }
   __syncthreads();
   for (int q = t; q < n_tokens * sel; q += 1024) {
