@@ -70,6 +70,8 @@ struct foe_layer {
   // repacked weights
   bf16 *wqkv_t, *wo_t, *wgu_t, *wd_t, *ffn_gain;
   float *router_w, *router_b;
+  bf16* router_split;    // [3][E padded to 64][d]: bf16 terms of router weights x FFN-norm gain
+  CUtensorMap tm_router;
   float2* rope_tab;
   foe_workspace* ws;
   int max_splits, pages_per_split;
@@ -140,8 +142,8 @@ foe_status check_launch() { return cudaGetLastError() == cudaSuccess ? FOE_OK : 
 
 // routing + dispatch maps for n tokens whose synced residual is r (fp32 internal or bf16 from the caller)
 void run_route_and_permute(foe_layer* L, const void* r, int r_is_bf16, int n, cudaStream_t st) {
-  L->launches += launch_route(r, r_is_bf16, L->ffn_gain, L->router_w, L->router_b, L->ws->u, L->ws->inv_rms_f, L->ws->route_part,
-                              L->ws->logits, L->ws->topk_idx, L->ws->topk_w, n, L->d, L->H, L->Ec, L->kc, L->cfg.rms_eps, L->n_sms, st);
+  L->launches += launch_route(r, r_is_bf16, L->ffn_gain, L->router_w, &L->tm_router, L->router_b, L->ws->u, L->ws->inv_rms_f, L->ws->route_part,
+                              L->ws->logits, L->ws->topk_idx, L->ws->topk_w, n, L->d, L->H, L->Ec, L->kc, L->cfg.rms_eps, L->n_sms, L->ws->status, st);
   stage_mark(L, kStPermute, st);
   L->launches += launch_permute(L->ws->topk_idx, L->ws->pb, n, L->H * L->kc, L->E, L->ws->status, st);
 }
@@ -364,6 +366,7 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
   ok = ok && dalloc(L, &L->ffn_gain, size_t(d));
   ok = ok && dalloc(L, &L->router_w, size_t(E) * d);
   ok = ok && dalloc(L, &L->router_b, size_t(E));
+  ok = ok && dalloc(L, &L->router_split, size_t(3) * router_padded_experts(E) * d);
   ok = ok && dalloc(L, &L->rope_tab, size_t(cfg->max_context) * (dh / 2));
   if (!ok) { foe_layer_destroy(L); return FOE_ERR_OOM; }
   cudaStream_t st = 0;
@@ -431,6 +434,7 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
   }
   cudaMemcpyAsync(L->ffn_gain, w->ffn_norm_g, size_t(d) * sizeof(bf16), cudaMemcpyDeviceToDevice, st);
   cudaMemcpyAsync(L->router_w, w->router_w, size_t(E) * d * sizeof(float), cudaMemcpyDeviceToDevice, st);
+  launch_split_router_weights(L->router_w, L->ffn_gain, L->router_split, E, d, st);
   if (w->router_b) cudaMemcpyAsync(L->router_b, w->router_b, size_t(E) * sizeof(float), cudaMemcpyDeviceToDevice, st);
   else cudaMemsetAsync(L->router_b, 0, size_t(E) * sizeof(float), st);
   // rotary table in double precision on the host: (cos, sin)(p * theta^(-2j/dh))
@@ -450,7 +454,8 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     foe_layer_destroy(L);
     return FOE_ERR_CUDA;
   }
-  ok = make_map_2d(&L->tm_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, gemm_tile_rows_b(kEpiQKV, qkvN)) &&
+  ok = make_map_2d(&L->tm_router, L->router_split, uint64_t(3) * router_padded_experts(E), d, kRouterChunk) &&
+       make_map_2d(&L->tm_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, gemm_tile_rows_b(kEpiQKV, qkvN)) &&
        make_map_2d(&L->tm_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, gemm_tile_rows_b(kEpiOProj, d)) &&
        make_map_2d(&L->tm_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, gemm_tile_rows_b(kEpiSwiGLU, 2 * I)) &&
        make_map_2d(&L->tm_wd, L->wd_t, uint64_t(E) * d, I, gemm_tile_rows_b(kEpiBf16, d)) &&

@@ -32,9 +32,18 @@ void launch_pack_gate_up(const bf16* wg, const bf16* wu, bf16* dst, int E, int d
 // FFN norm + fp32 router + per-cluster top-k + gates.  r_in is fp32 or bf16 [S][d].
 // Returns the number of kernels launched.  inv_rms: [S] scratch; part: scratch for the split-K partial scores
 // (at least max(S*E, 2^21) floats).
-int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const float* br, bf16* u_out,
-                 float* inv_rms, float* part, float* logits, int* idx, float* w, int n_tokens, int d, int H, int Ec,
-                 int kc, float eps, int n_sms, cudaStream_t st);
+// tm_wr_split: map of the split router weights (launch_split_router_weights; box 64 x 64), or null: plain-ALU scores
+// at every size.
+constexpr int kRouterTcMinTokens = 2048;
+constexpr int kRouterChunk = 64;              // experts per CTA of the tensor-core score kernel
+inline int router_padded_experts(int E) { return (E + kRouterChunk - 1) / kRouterChunk * kRouterChunk; }
+int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const CUtensorMap* tm_wr_split,
+                 const float* br, bf16* u_out, float* inv_rms, float* part, float* logits, int* idx, float* w,
+                 int n_tokens, int d, int H, int Ec, int kc, float eps, int n_sms, int* status, cudaStream_t st);
+// planes: [3][router_padded_experts(E)][d] bf16 terms of gain * W
+void launch_split_router_weights(const float* wr, const bf16* gain, bf16* planes, int E, int d, cudaStream_t st);
+void launch_router_tc(const CUtensorMap& tmW, const float* r, const float* inv_rms, float* part, int n_tokens, int d,
+                      int E, int* status, cudaStream_t st);
 
 // routing on the library's built-in scratch area (no allocation); 0, -3 (too large) or -6 (CUDA error)
 int launch_route_noalloc(const bf16* h, const bf16* gain, const float* wr, const float* br, int* idx, float* w,

@@ -3,7 +3,7 @@
 // scores.  Everything on this path is fp32 on the plain ALUs: the decision it takes (which experts)
 // is an integer result that must agree with a float32 reference, so no reduced-precision tensor path.
 //
-// Three kernels:
+// Three kernels (for calls of kRouterTcMinTokens tokens or more, the tensor-core kernel of router_tc.cu replaces 2):
 //  1. ffn_norm:     one warp per token: inv_rms and the bf16 expert input u = r * inv_rms * gain.
 //  2. router_gemm:  SIMT fp32 GEMM, 64 tokens x 64 experts per CTA, 8 x 4 register tiles, k-major shared
 //                   tiles, register-staged double buffering; the normalisation is applied while the token
@@ -244,15 +244,20 @@ int route_k_splits(int n_tokens, int d, int E, int n_sms) {
   return ks;
 }
 
-int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const float* br, bf16* u_out,
-                 float* inv_rms, float* part, float* logits, int* idx, float* w, int n_tokens, int d, int H, int Ec,
-                 int kc, float eps, int n_sms, cudaStream_t st) {
+int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const CUtensorMap* tm_wr_split,
+                 const float* br, bf16* u_out, float* inv_rms, float* part, float* logits, int* idx, float* w,
+                 int n_tokens, int d, int H, int Ec, int kc, float eps, int n_sms, int* status, cudaStream_t st) {
   if (n_tokens <= 0) return 0;
   const int E = H * Ec;
   ffn_norm_kernel<<<(n_tokens * 32 + 255) / 256, 256, 0, st>>>(r_in, r_is_bf16, gain, u_out, inv_rms, n_tokens, d, eps);
-  const int ks = route_k_splits(n_tokens, d, E, n_sms);
-  dim3 grid((n_tokens + kRgTM - 1) / kRgTM, (E + kRgTN - 1) / kRgTN, ks);
-  router_gemm_kernel<<<grid, kRgThreads, 0, st>>>(r_in, r_is_bf16, inv_rms, gain, wr, part, n_tokens, d, E, d / ks);
+  int ks = 1;
+  if (tm_wr_split && !r_is_bf16 && n_tokens >= kRouterTcMinTokens) {
+    launch_router_tc(*tm_wr_split, static_cast<const float*>(r_in), inv_rms, part, n_tokens, d, E, status, st);
+  } else {
+    ks = route_k_splits(n_tokens, d, E, n_sms);
+    dim3 grid((n_tokens + kRgTM - 1) / kRgTM, (E + kRgTN - 1) / kRgTN, ks);
+    router_gemm_kernel<<<grid, kRgThreads, 0, st>>>(r_in, r_is_bf16, inv_rms, gain, wr, part, n_tokens, d, E, d / ks);
+  }
   const int tasks = n_tokens * H;
   const int per_warp = Ec <= 8 ? 4 : (Ec <= 16 ? 2 : 1);
   const int warps = (tasks + per_warp - 1) / per_warp;
