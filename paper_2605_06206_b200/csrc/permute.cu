@@ -72,10 +72,15 @@ permute_scan_kernel(int* __restrict__ blk_counts, int n_blocks, int E, const Per
   const int e = threadIdx.x;
   int total = 0;
   if (e < E) {
-    for (int b = 0; b < n_blocks; ++b) {
-      const int c = blk_counts[size_t(b) * E + e];
-      blk_counts[size_t(b) * E + e] = total;
-      total += c;
+    for (int b0 = 0; b0 < n_blocks; b0 += 16) {          // 16 independent loads in flight, then their prefix
+      int c[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) c[j] = b0 + j < n_blocks ? blk_counts[size_t(b0 + j) * E + e] : 0;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        if (b0 + j < n_blocks) blk_counts[size_t(b0 + j) * E + e] = total;
+        total += c[j];
+      }
     }
     counts[e] = total;
   }

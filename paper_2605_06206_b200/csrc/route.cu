@@ -237,6 +237,65 @@ __global__ void topk_gates_kernel(const float* __restrict__ part, int k_splits, 
   }
 }
 
+// The same selection with one thread per (token, cluster) and the cluster's scores in registers: for the common
+// cluster sizes (a power of two up to 32) there is nothing to exchange between lanes.  Ties and order exactly as in
+// topk_gates_kernel: score descending, expert id ascending.
+template <int EC>
+__global__ void topk_gates_thread_kernel(const float* __restrict__ part, int k_splits, const float* __restrict__ br,
+                                         float* __restrict__ logits_out, int* __restrict__ idx_out,
+                                         float* __restrict__ w_out, int n_tokens, int H, int kc) {
+  const int task = blockIdx.x * blockDim.x + threadIdx.x;
+  if (task >= n_tokens * H) return;
+  const int i = task / H, h = task - i * H;
+  const size_t o = size_t(i) * H * EC + size_t(h) * EC;
+  const size_t split_stride = size_t(n_tokens) * H * EC;
+  float v[EC];
+#pragma unroll
+  for (int e = 0; e < EC; e += 4) {
+    float4 a = *reinterpret_cast<const float4*>(part + o + e);
+    for (int z = 1; z < k_splits; ++z) {
+      const float4 b = *reinterpret_cast<const float4*>(part + z * split_stride + o + e);
+      a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+    }
+    if (br) { a.x += __ldg(br + h * EC + e); a.y += __ldg(br + h * EC + e + 1); a.z += __ldg(br + h * EC + e + 2); a.w += __ldg(br + h * EC + e + 3); }
+    v[e] = a.x; v[e + 1] = a.y; v[e + 2] = a.z; v[e + 3] = a.w;
+    *reinterpret_cast<float4*>(logits_out + o + e) = a;
+  }
+  uint32_t taken = 0u;
+  float m = 0.f, sum = 0.f;
+  const size_t oo = size_t(task) * kc;
+  for (int j = 0; j < kc; ++j) {
+    float bv = -FLT_MAX;
+    int bi = -1;
+#pragma unroll
+    for (int e = 0; e < EC; ++e)
+      if (!((taken >> e) & 1u) && (bi < 0 || v[e] > bv)) { bv = v[e]; bi = e; }      // ascending e: first wins ties
+    taken |= 1u << bi;
+    if (j == 0) m = bv;
+    const float ex = expf(bv - m);
+    sum += ex;
+    idx_out[oo + j] = h * EC + bi;
+    w_out[oo + j] = ex;                 // normalised below
+  }
+  for (int j = 0; j < kc; ++j) w_out[oo + j] = w_out[oo + j] / sum;
+}
+
+static void launch_topk_gates(const float* part, int ks, const float* br, float* logits, int* idx, float* w,
+                              int n_tokens, int H, int Ec, int kc, cudaStream_t st) {
+  const int tasks = n_tokens * H;
+  const int tb = (tasks + 127) / 128;
+  switch (Ec) {
+    case 4: topk_gates_thread_kernel<4><<<tb, 128, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, kc); return;
+    case 8: topk_gates_thread_kernel<8><<<tb, 128, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, kc); return;
+    case 16: topk_gates_thread_kernel<16><<<tb, 128, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, kc); return;
+    case 32: topk_gates_thread_kernel<32><<<tb, 128, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, kc); return;
+    default: break;
+  }
+  const int per_warp = Ec <= 8 ? 4 : (Ec <= 16 ? 2 : 1);
+  const int warps = (tasks + per_warp - 1) / per_warp;
+  topk_gates_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc);
+}
+
 int route_k_splits(int n_tokens, int d, int E, int n_sms) {
   const int ctas = ((n_tokens + kRgTM - 1) / kRgTM) * ((E + kRgTN - 1) / kRgTN);
   int ks = 1;
@@ -258,10 +317,7 @@ int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float*
     dim3 grid((n_tokens + kRgTM - 1) / kRgTM, (E + kRgTN - 1) / kRgTN, ks);
     router_gemm_kernel<<<grid, kRgThreads, 0, st>>>(r_in, r_is_bf16, inv_rms, gain, wr, part, n_tokens, d, E, d / ks);
   }
-  const int tasks = n_tokens * H;
-  const int per_warp = Ec <= 8 ? 4 : (Ec <= 16 ? 2 : 1);
-  const int warps = (tasks + per_warp - 1) / per_warp;
-  topk_gates_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc);
+  launch_topk_gates(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc, st);
   return 3;
 }
 
@@ -334,10 +390,7 @@ int launch_route_noalloc(const bf16* h, const bf16* gain, const float* wr, const
   while (ks > 1 && size_t(ks) * n_tokens * E > kNaMaxPartial) ks >>= 1;
   dim3 grid((n_tokens + kRgTM - 1) / kRgTM, (E + kRgTN - 1) / kRgTN, ks);
   router_gemm_kernel<<<grid, kRgThreads, 0, st>>>(h, 1, inv, gain, wr, part, n_tokens, d, E, d / ks);
-  const int tasks = n_tokens * H;
-  const int per_warp = Ec <= 8 ? 4 : (Ec <= 16 ? 2 : 1);
-  const int warps = (tasks + per_warp - 1) / per_warp;
-  topk_gates_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc);
+  launch_topk_gates(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc, st);
   return cudaGetLastError() == cudaSuccess ? 0 : -6;
 }
 
