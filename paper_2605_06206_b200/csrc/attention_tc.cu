@@ -256,16 +256,21 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
         // probabilities, written as the bf16 A operand of the PV product (exp2(-inf) = 0 handles the mask)
         uint8_t* p_row = p_rows + (j & 1) * L::kPTile;
+        // Written in stages over 32 values: all scalings, then all exponentials back to back, then sums and packing.
         float rs4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
+          uint32_t (&rr)[32] = hf ? r1 : r0;
+          float e[32];
+#pragma unroll
+          for (int c = 0; c < 32; ++c) e[c] = fmaf(__uint_as_float(rr[c]), a.scale_log2, -m_use);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(e[c]) : "f"(e[c]));
           uint32_t pk[16];
 #pragma unroll
           for (int c = 0; c < 16; ++c) {
-            const float v0 = __uint_as_float(hf ? r1[2 * c] : r0[2 * c]), v1 = __uint_as_float(hf ? r1[2 * c + 1] : r0[2 * c + 1]);
-            const float p0 = fast_exp2(fmaf(v0, a.scale_log2, -m_use)), p1 = fast_exp2(fmaf(v1, a.scale_log2, -m_use));
-            rs4[c & 3] += p0 + p1;
-            pk[c] = pack_bf16(p0, p1);
+            rs4[c & 3] += e[2 * c] + e[2 * c + 1];
+            pk[c] = pack_bf16(e[2 * c], e[2 * c + 1]);
           }
 #pragma unroll
           for (int q = 0; q < 4; ++q)
@@ -273,11 +278,13 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
         }
         l_run += (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
+        // (before this warp's arrival below: P V of step j cannot have been issued yet, so the barrier is at most one
+        // phase ahead of what is waited for)
+        if (!o_seen && !mbar_wait(&o_full[t], ph ^ 1)) { ok = false; break; }
         tc_fence_before();
         fence_async_smem();                                  // P visible to the tensor core's shared-memory reads
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_ready[t]);
-        if (!o_seen && !mbar_wait(&o_full[t], ph ^ 1)) { ok = false; break; }
       }
       if (ok && n_tiles > 0) ok = mbar_wait(&o_full[t], (n_tiles - 1) & 1);
       tc_fence_after();
