@@ -196,16 +196,17 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       uint8_t* p_rows = smem + L::kPOff + t * 2 * L::kPTile + row * 128;
       float m_ref = -INFINITY, l_run = 0.f;                  // m_ref: the (possibly stale) maximum the exponentials use
       bool ok = true;
+      uint32_t r0[32], r1[32];                               // the 64 scores of this row
+      bool preloaded = false;                                // the loads of step j were issued at the end of step j-1
       for (int j = 0; j < n_tiles; ++j) {
         const uint32_t ph = j & 1;
-        if (!mbar_wait(&s_full[2 * t + (j & 1)], (j >> 1) & 1)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t s_addr = s_base + (j & 1) * 64;
         const bool masked = j >= first_mask_tile;
-        // the 64 scores of this row: two loads in flight, one wait
-        uint32_t r0[32], r1[32];
-        tmem_ld32(s_addr, r0);
-        tmem_ld32(s_addr + 32, r1);
+        if (!preloaded) {
+          if (!mbar_wait(&s_full[2 * t + (j & 1)], (j >> 1) & 1)) { ok = false; break; }
+          tc_fence_after();
+          tmem_ld32(s_base + (j & 1) * 64, r0);              // two loads in flight, one wait
+          tmem_ld32(s_base + (j & 1) * 64 + 32, r1);
+        }
         tmem_ld_wait();
         float mx = -INFINITY;
         if (masked) {
@@ -221,7 +222,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           for (int c = 0; c < 32; c += 4) {
 #pragma unroll
             for (int q = 0; q < 4; ++q)
-              m4[q] = fmaxf(m4[q], fmaxf(__uint_as_float(r0[c + q]), __uint_as_float(r1[c + q])));
+              m4[q] = fmax3(m4[q], __uint_as_float(r0[c + q]), __uint_as_float(r1[c + q]));
           }
           mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         }
@@ -278,6 +279,20 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
                 make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
         }
         l_run += (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
+        // The scores are used up: if the next step's are already there (they usually are, the issuer runs a step
+        // ahead), start loading them now, so that the load's latency passes behind the stores and arrivals below.
+        preloaded = false;
+        if (j + 1 < n_tiles) {
+          const int jn = j + 1;
+          bool ready = false;
+          if (lane == 0) ready = mbar_test(&s_full[2 * t + (jn & 1)], (jn >> 1) & 1);
+          preloaded = __shfl_sync(0xffffffffu, ready, 0);
+          if (preloaded) {
+            tc_fence_after();
+            tmem_ld32(s_base + (jn & 1) * 64, r0);
+            tmem_ld32(s_base + (jn & 1) * 64 + 32, r1);
+          }
+        }
         // (before this warp's arrival below: P V of step j cannot have been issued yet, so the barrier is at most one
         // phase ahead of what is waited for)
         if (!o_seen && !mbar_wait(&o_full[t], ph ^ 1)) { ok = false; break; }
