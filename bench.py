@@ -33,7 +33,7 @@ from paper_2605_06206_b200 import replicas, synth  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernels, from the committed ncu captures
 # of these same workloads (profiles/): not re-measured by a plain bench run
-NCU_TRAFFIC = dict(expert_gemm1_prefill=965.5e6 + 252.9e6, attn_decode=1348.8e6 + 8.8e6)
+NCU_TRAFFIC = dict(expert_gemm1_prefill=973.0e6 + 255.7e6, attn_decode=1348.7e6 + 9.0e6)
 
 
 # ----------------------------------------------------------------------------------------------
@@ -326,7 +326,7 @@ def measure(kind, args, dist_on, rank, world, peaks, with_cpu):
         t = stages["expert_gemm1_swiglu"] * 1e-3
         ach = work["gemm1_flops"] / t / 1e12
         peak = peaks["bf16_tflops_sustained"]
-        res["roofline"] = dict(bound="tensor", kernel="gemm_tcgen05_kernel<SwiGLU> (expert GEMM 1)", achieved=ach,
+        res["roofline"] = dict(bound="tensor", kernel="gemm_tcgen05_kernel<SwiGLU, gather> (expert GEMM 1, CTA pairs)", achieved=ach,
                                peak=peak, unit="TFLOP/s", frac=ach / peak, traffic=NCU_TRAFFIC["expert_gemm1_prefill"],
                                traffic_source="dram read+write bytes per launch, profiles/ncu_full_prefill_kernels_workload2.md",
                                peak_source=f"{peaks['source']} sustained bf16 (kernel timed inside the step)",
