@@ -12,7 +12,7 @@ constexpr int kBN = 256;   // widest GEMM tile (UMMA N); the launcher narrows it
 
 // Tile width for N columns per group: as few tiles as 256 allows, all of the same width (384 columns are two tiles
 // of 192, not one of 256 and a half-empty one).
-__host__ __device__ constexpr int gemm_tile_cols(int N) {
+constexpr int gemm_tile_cols(int N) {
   const int tiles = (N + kBN - 1) / kBN;
   return tiles <= 0 ? kBN : ((((N + tiles - 1) / tiles) + 63) / 64) * 64;
 }
@@ -26,7 +26,7 @@ enum GemmEpilogue : int {
 
 // Rows of B one CTA of a pair stages per k-block = box rows of the B tensor map: half a tile.  The SwiGLU epilogue
 // needs the full 256-wide tile (128 gate columns, 128 up columns).
-__host__ __device__ constexpr int gemm_tile_rows_b(int epi, int N) { return (epi == kEpiSwiGLU ? kBN : gemm_tile_cols(N)) / 2; }
+constexpr int gemm_tile_rows_b(int epi, int N) { return (epi == kEpiSwiGLU ? kBN : gemm_tile_cols(N)) / 2; }
 
 struct GemmArgs {
   // uniform groups

@@ -98,6 +98,13 @@ def test_chunked_prefill_over_cached_context():
     run_block_parity(shape, 15, [40, 17, 130], [100, 64, 1], wscale=4.0)
 
 
+def test_mixed_batch_of_prefill_chunks_and_decode_tokens():
+    """One prefill call carrying fresh prompts, a chunk of a longer prompt and single decode tokens of running
+    sequences (q_len 1 over a long cached context): the serving batch shape of Section 4's engine."""
+    shape = shape_small()
+    run_block_parity(shape, 18, [1, 200, 1, 64, 1], [300, 0, 1000, 64, 63], wscale=4.0)
+
+
 def test_empty_and_single_token_calls():
     shape = shape_small()
     W = synth.make_weights(shape, 16, "cuda")
