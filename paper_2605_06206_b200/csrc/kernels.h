@@ -42,8 +42,8 @@ int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float*
                  int n_tokens, int d, int H, int Ec, int kc, float eps, int n_sms, int* status, cudaStream_t st);
 // planes: [3][router_padded_experts(E)][d] bf16 terms of gain * W
 void launch_split_router_weights(const float* wr, const bf16* gain, bf16* planes, int E, int d, cudaStream_t st);
-void launch_router_tc(const CUtensorMap& tmW, const float* r, const float* inv_rms, float* part, int n_tokens, int d,
-                      int E, int* status, cudaStream_t st);
+void launch_router_tc(const CUtensorMap& tmW, const void* r, int r_is_bf16, const float* inv_rms, float* part,
+                      int n_tokens, int d, int E, int* status, cudaStream_t st);
 
 // routing on the library's built-in scratch area (no allocation); 0, -3 (too large) or -6 (CUDA error)
 int launch_route_noalloc(const bf16* h, const bf16* gain, const float* wr, const float* br, int* idx, float* w,

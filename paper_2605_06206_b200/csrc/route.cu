@@ -310,8 +310,8 @@ int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float*
   const int E = H * Ec;
   ffn_norm_kernel<<<(n_tokens * 32 + 255) / 256, 256, 0, st>>>(r_in, r_is_bf16, gain, u_out, inv_rms, n_tokens, d, eps);
   int ks = 1;
-  if (tm_wr_split && !r_is_bf16 && n_tokens >= kRouterTcMinTokens) {
-    launch_router_tc(*tm_wr_split, static_cast<const float*>(r_in), inv_rms, part, n_tokens, d, E, status, st);
+  if (tm_wr_split && n_tokens >= kRouterTcMinTokens) {
+    launch_router_tc(*tm_wr_split, r_in, r_is_bf16, inv_rms, part, n_tokens, d, E, status, st);
   } else {
     ks = route_k_splits(n_tokens, d, E, n_sms);
     dim3 grid((n_tokens + kRgTM - 1) / kRgTM, (E + kRgTN - 1) / kRgTN, ks);

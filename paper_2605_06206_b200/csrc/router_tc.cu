@@ -61,7 +61,7 @@ __global__ void split_router_weights_kernel(const float* __restrict__ wr, const 
 }
 
 __global__ void __launch_bounds__(kRtThreads, 1)
-router_tc_kernel(const __grid_constant__ CUtensorMap tmW, const float* __restrict__ r_in,
+router_tc_kernel(const __grid_constant__ CUtensorMap tmW, const void* __restrict__ r_in, int r_is_bf16,
                  const float* __restrict__ inv_rms, float* __restrict__ part, int n_tokens, int d, int E, int E_pad,
                  int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
@@ -132,21 +132,29 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmW, const float* __restric
     const int cw = warp - 6;
     const int sub = lane >> 4, c4 = lane & 15;             // row inside the pair; float4 column (4 k values)
     const int chunk16 = c4 >> 1, half8 = (c4 & 1) * 8;      // 16-byte chunk of the bf16 row and offset inside it
-    const float* src[8];
+    size_t src[8];                                          // element offset of this lane's four values in k-block 0
     int trow[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       trow[i] = cw * 16 + 2 * i + sub;                      // row of the tile
-      src[i] = r_in + size_t(min(row0 + trow[i], n_tokens - 1)) * d + c4 * 4;   // rows past the end repeat the last one
+      src[i] = size_t(min(row0 + trow[i], n_tokens - 1)) * d + c4 * 4;          // rows past the end repeat the last one
     }
+    // the residual comes as fp32 (inside a block) or as bf16 (routing call on a caller's tensor)
+    auto load4 = [&](size_t off) {
+      if (r_is_bf16) {
+        const uint2 q = __ldg(reinterpret_cast<const uint2*>(static_cast<const bf16*>(r_in) + off));
+        return make_float4(bf16_lo(q.x), bf16_hi(q.x), bf16_lo(q.y), bf16_hi(q.y));
+      }
+      return __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(r_in) + off));
+    };
     bool ok = true;
     float4 cur[8], nxt[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) cur[i] = __ldg(reinterpret_cast<const float4*>(src[i]));
+    for (int i = 0; i < 8; ++i) cur[i] = load4(src[i]);
     for (int kb = 0; kb < kblocks; ++kb) {
       if (kb + 1 < kblocks) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) nxt[i] = __ldg(reinterpret_cast<const float4*>(src[i] + (kb + 1) * kRtBK));
+        for (int i = 0; i < 8; ++i) nxt[i] = load4(src[i] + size_t(kb + 1) * kRtBK);
       }
       const int s = kb % kRtStages;
       if (lane == 0) ok = mbar_wait(&empty_bar[s], ((kb / kRtStages) & 1) ^ 1);
@@ -224,8 +232,8 @@ void launch_split_router_weights(const float* wr, const bf16* gain, bf16* planes
   split_router_weights_kernel<<<unsigned((total + 255) / 256), 256, 0, st>>>(wr, gain, planes, E, E_pad, d);
 }
 
-void launch_router_tc(const CUtensorMap& tmW, const float* r, const float* inv_rms, float* part, int n_tokens, int d,
-                      int E, int* status, cudaStream_t st) {
+void launch_router_tc(const CUtensorMap& tmW, const void* r, int r_is_bf16, const float* inv_rms, float* part,
+                      int n_tokens, int d, int E, int* status, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(router_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kRtSmemBytes));
@@ -233,7 +241,7 @@ void launch_router_tc(const CUtensorMap& tmW, const float* r, const float* inv_r
   }
   const int E_pad = router_padded_experts(E);
   dim3 grid((n_tokens + kRtRows - 1) / kRtRows, E_pad / kRtChunk);
-  router_tc_kernel<<<grid, kRtThreads, kRtSmemBytes, st>>>(tmW, r, inv_rms, part, n_tokens, d, E, E_pad, status);
+  router_tc_kernel<<<grid, kRtThreads, kRtSmemBytes, st>>>(tmW, r, r_is_bf16, inv_rms, part, n_tokens, d, E, E_pad, status);
 }
 
 }  // namespace foe
