@@ -248,7 +248,7 @@ def e2e_loop(wl, steps, warmup):
 
 
 # ----------------------------------------------------------------------------------------------
-def oracle_sample(kind: str, n_tokens: int, seed: int = 0):
+def oracle_sample(kind: str, n_tokens: int, seed: int = 0, n_seqs: int = 1):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload.  Returns (seconds, tokens,
     threads, description)."""
     import numpy as np
@@ -259,11 +259,11 @@ def oracle_sample(kind: str, n_tokens: int, seed: int = 0):
     cfg = adapter.cfg_from_shape(shape)
     threads = os.cpu_count() or 1
     if kind == "prefill":
-        x = adapter.to_np(synth.make_x(shape, info["seed"] + seed, n_tokens))
+        x = adapter.to_np(synth.make_x(shape, info["seed"] + seed, n_tokens * n_seqs))
         t0 = time.perf_counter()
-        orc.foe_block(cfg, W, x, [n_tokens])
+        orc.foe_block(cfg, W, x, [n_tokens] * n_seqs)
         dt = time.perf_counter() - t0
-        return dt, n_tokens, threads, f"one sequence of {n_tokens} tokens, full block, workload-2 layer"
+        return dt, n_tokens * n_seqs, threads, f"{n_seqs} sequence(s) of {n_tokens} tokens, full block, workload-2 layer"
     n_seqs = n_tokens
     ctx = info["context_lens"][:n_seqs]
     kv = synth.make_paged_cache(shape, info["seed"], ctx, [1] * n_seqs)
@@ -355,7 +355,7 @@ def measure(kind, args, dist_on, rank, world, peaks, with_cpu):
     del wl
     torch.cuda.empty_cache()
     if with_cpu:
-        dt, ntk, thr, desc = oracle_sample(kind, 1024 if kind == "prefill" else 16)
+        dt, ntk, thr, desc = oracle_sample(kind, 4096 if kind == "prefill" else 64, n_seqs=2)   # about 10 s of host work
         res["cpu_baseline"] = dict(value=ntk / dt, unit="tokens/s", cores=thr, kind="oracle", sample=desc,
                                    seconds=dt)
     return res
