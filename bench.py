@@ -386,6 +386,35 @@ def run_sweep(args):
                           steps=args.steps, warmup=args.warmup, sweep=rows)))
 
 
+def run_serve(args):
+    """Request-level run: Poisson arrivals of long-prompt requests served with continuous batching (chunked prefill
+    mixed with decode tokens) by a 4-layer stack of the workload-2 layer; TTFT / TBT / end-to-end latency as mean,
+    p50, p99 (the format of the paper's latency tables; its numbers are whole models on 8 GPUs, context only)."""
+    from paper_2605_06206_b200 import serving as sv
+    shape, _ = synth.workload(2)
+    n_layers, max_batch_tokens, max_seqs, chunk, max_context = 4, 8192, 64, 2048, 16384 + 256
+    n_req, rate = args.requests, args.rate
+    reqs = sv.synthetic_trace(n_req, rate=rate, seed=11)
+    num_pages = 4096                                        # 262,144 tokens of KV per layer
+    runner = sv.FoeStackRunner(shape, n_layers, seed=2, num_pages=num_pages, max_batch_tokens=max_batch_tokens,
+                               max_seqs=max_seqs, max_context=max_context)
+    warm = sv.synthetic_trace(3, rate=1e6, seed=12, prompt_range=(512, 4096), output_range=(2, 4))
+    sv.Engine(sv.Scheduler(sv.PagePool(num_pages), max_batch_tokens, max_seqs, chunk), runner.forward).run(warm)
+    eng = sv.Engine(sv.Scheduler(sv.PagePool(num_pages), max_batch_tokens, max_seqs, chunk), runner.forward)
+    done = eng.run(reqs)
+    runner.close()
+    rep = sv.latency_report(done)
+    toks = sum(r.prompt_len + r.output_len - 1 for r in done)
+    print(json.dumps(dict(metric="foe_stack_request_latency", unit="ms", data="synthetic", dtype="bf16",
+                          config=dict(workload=f"{n_layers}-layer stack of the workload-2 layer; {n_req} requests, Poisson "
+                                               f"{rate} req/s, prompts log-uniform 1024..16384, outputs 32..256; continuous "
+                                               f"batching, <= {max_batch_tokens} tokens and {max_seqs} sequences per iteration, "
+                                               f"prompt chunks of {chunk}"),
+                          requests=len(done), iterations=eng.iterations, busy_seconds=eng.clock,
+                          tokens_per_s=toks / eng.clock, mean_batch_tokens=sum(eng.batch_tokens) / max(1, len(eng.batch_tokens)),
+                          **rep)))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -396,6 +425,9 @@ def main():
     ap.add_argument("--no-secondary", action="store_true", help="skip the other workload's measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle (profiler runs)")
     ap.add_argument("--sweep", action="store_true", help="token-batch latency sweep at the paper's 7B layer shape")
+    ap.add_argument("--serve", action="store_true", help="request-level latency run (continuous batching on a 4-layer stack)")
+    ap.add_argument("--requests", type=int, default=48)
+    ap.add_argument("--rate", type=float, default=20.0, help="--serve: Poisson arrival rate, requests per second")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
@@ -411,6 +443,9 @@ def main():
     torch.cuda.set_device(local)
     if args.sweep:
         run_sweep(args)
+        return
+    if args.serve:
+        run_serve(args)
         return
     dist_on = replicas.init("nccl", torch.device("cuda", local))
     peaks = measured_peaks()
