@@ -64,155 +64,155 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
                                                    int tile_cols, ReleaseFn release) {
   const int row = row0 + quarter * 32 + lane;      // A row of this thread's accumulator lane
   const bool row_ok = row < row_end;
-        // Every pass turns 128 bytes of output per row into registers (thread = accumulator row), parks them
-        // in the warp's staging tile and writes them out again with 8 lanes per row, so that global stores
-        // are whole 128-byte lines instead of 32 scattered 16-byte pieces.
-        const int row_local = row - group_row0;
-        float scale = 1.0f;
+  // Every pass turns 128 bytes of output per row into registers (thread = accumulator row), parks them
+  // in the warp's staging tile and writes them out again with 8 lanes per row, so that global stores
+  // are whole 128-byte lines instead of 32 scattered 16-byte pieces.
+  const int row_local = row - group_row0;
+  float scale = 1.0f;
+  if constexpr (EPI == kEpiQKV) {
+    if (row_ok) scale = args.row_scale[size_t(group) * args.scale_group_stride + row_local];
+  }
+  constexpr int kPassCols = (EPI == kEpiOProj) ? 32 : 64;          // accumulator columns per pass (SwiGLU: 64 + 64)
+  const int n_pass = (EPI == kEpiSwiGLU) ? 2 : (tile_cols + kPassCols - 1) / kPassCols;
+  const int wr_row = lane >> 3, wr_chunk = lane & 7;                // write-out role: row (+4j), 16-byte chunk
+  if (half >= n_pass) { release(); return; }                        // nothing for this warp in a one-pass tile
+#pragma unroll 1
+  for (int ps = half; ps < n_pass; ps += 2) {
+    const int n = (EPI == kEpiSwiGLU) ? (n0 >> 1) + ps * 64 : n0 + ps * kPassCols;   // output column in the group
+    uint32_t w[32];                                                // 128 bytes of this row's output
+    __syncwarp();
+    if constexpr (EPI == kEpiSwiGLU) {
+      uint32_t gt[32], up[32];
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        tmem_ld32(taddr + ps * 64 + hf * 32, gt);
+        tmem_ld32(taddr + 128 + ps * 64 + hf * 32, up);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          const float h0 = silu_f(__uint_as_float(gt[2 * c])) * __uint_as_float(up[2 * c]);
+          const float h1 = silu_f(__uint_as_float(gt[2 * c + 1])) * __uint_as_float(up[2 * c + 1]);
+          w[hf * 16 + c] = pack_bf16(h0, h1);
+        }
+      }
+    } else if constexpr (EPI == kEpiOProj) {
+      tmem_ld32(taddr + ps * 32, w);
+      tmem_ld_wait();
+    } else if constexpr (EPI == kEpiQKV) {
+      // 64 packed columns = 32 rotation pairs (natural columns i0+m and i0+m+dh/2 of one head).  The first
+      // 64 bytes of the staged row are the first-half columns, the second 64 bytes their partners.
+      const bool rotate = n < args.q_cols + args.kv_cols;          // q and k heads; v is only de-interleaved
+      const int i0 = (n % args.dh) >> 1;
+      // the 32 (cos, sin) pairs of this row's position are fetched before the accumulator is read, so their
+      // latency overlaps the tensor-memory load
+      const float4* tab = reinterpret_cast<const float4*>(
+          args.rope_tab + size_t(row_ok ? args.tok_pos[row_local] : 0) * (args.dh >> 1) + i0);
+      float4 cs4[16];
+#pragma unroll
+      for (int m = 0; m < 16; ++m) cs4[m] = rotate ? __ldg(tab + m) : make_float4(1.f, 0.f, 1.f, 0.f);
+      uint32_t r[32];
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        tmem_ld32(taddr + ps * 64 + hf * 32, r);
+        tmem_ld_wait();
+        float lo[16], hi[16];
+#pragma unroll
+        for (int m = 0; m < 16; ++m) {
+          const float a = __uint_as_float(r[2 * m]) * scale, b = __uint_as_float(r[2 * m + 1]) * scale;
+          const float4 c4 = cs4[hf * 8 + (m >> 1)];
+          const float cx = (m & 1) ? c4.z : c4.x, cy = (m & 1) ? c4.w : c4.y;
+          lo[m] = a * cx - b * cy;
+          hi[m] = b * cx + a * cy;
+        }
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          w[hf * 8 + m] = pack_bf16(lo[2 * m], lo[2 * m + 1]);
+          w[16 + hf * 8 + m] = pack_bf16(hi[2 * m], hi[2 * m + 1]);
+        }
+      }
+    } else {
+      uint32_t r[32];
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        tmem_ld32(taddr + ps * 64 + hf * 32, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 16; ++c)
+          w[hf * 16 + c] = pack_bf16(__uint_as_float(r[2 * c]), __uint_as_float(r[2 * c + 1]));
+      }
+    }
+    if (ps + 2 >= n_pass) release();                               // this warp's last TMEM read of the tile
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+      *reinterpret_cast<uint4*>(stg + stg_off(lane, c)) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+    __syncwarp();
+    if constexpr (EPI == kEpiOProj) {
+      // r_full = scale * (C + sum_h x[h]): the residual streams are read here.  This GEMM moves almost as many
+      // bytes as it has flops to hide them, so the epilogue has to keep ~256 bytes per thread in flight:
+      // 4 lanes x 16 bytes per row and stream, and all loads of the pass are issued before the first use.
+      const int or_row = lane >> 2, or_cg = lane & 3;           // row (+8j) and group of 8 columns
+      uint4 xq[4][8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int grow = row0 + quarter * 32 + or_row + 8 * j;
+        const size_t off = size_t(grow) * args.ldo + n + or_cg * 8;
+#pragma unroll
+        for (int h = 0; h < 8; ++h) {
+          xq[j][h] = make_uint4(0u, 0u, 0u, 0u);
+          if (h < args.x_count && grow < row_end)
+            xq[j][h] = __ldg(reinterpret_cast<const uint4*>(args.xsum + h * args.x_stride + off));
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int rr = or_row + 8 * j;
+        const int grow = row0 + quarter * 32 + rr;
+        if (grow >= row_end) continue;
+        const float4 c0 = *reinterpret_cast<const float4*>(stg + stg_off(rr, 2 * or_cg));
+        const float4 c1 = *reinterpret_cast<const float4*>(stg + stg_off(rr, 2 * or_cg + 1));
+        float a8[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+#pragma unroll
+        for (int h = 0; h < 8; ++h) {
+          const uint32_t w4[4] = {xq[j][h].x, xq[j][h].y, xq[j][h].z, xq[j][h].w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) { a8[2 * q] += bf16_lo(w4[q]); a8[2 * q + 1] += bf16_hi(w4[q]); }
+        }
+        float* dst = static_cast<float*>(args.out) + size_t(grow) * args.ldo + n + or_cg * 8;
+        const float sc = args.out_scale;
+        *reinterpret_cast<float4*>(dst) = make_float4(a8[0] * sc, a8[1] * sc, a8[2] * sc, a8[3] * sc);
+        *reinterpret_cast<float4*>(dst + 4) = make_float4(a8[4] * sc, a8[5] * sc, a8[6] * sc, a8[7] * sc);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int rr = wr_row + 4 * j;                              // row inside the warp's 32
+        const int grow = row0 + quarter * 32 + rr;
+        if (grow >= row_end) continue;
+        const uint4 v = *reinterpret_cast<const uint4*>(stg + stg_off(rr, wr_chunk));
         if constexpr (EPI == kEpiQKV) {
-          if (row_ok) scale = args.row_scale[size_t(group) * args.scale_group_stride + row_local];
-        }
-        constexpr int kPassCols = (EPI == kEpiOProj) ? 32 : 64;          // accumulator columns per pass (SwiGLU: 64 + 64)
-        const int n_pass = (EPI == kEpiSwiGLU) ? 2 : (tile_cols + kPassCols - 1) / kPassCols;
-        const int wr_row = lane >> 3, wr_chunk = lane & 7;                // write-out role: row (+4j), 16-byte chunk
-        if (half >= n_pass) { release(); return; }                        // nothing for this warp in a one-pass tile
-  #pragma unroll 1
-        for (int ps = half; ps < n_pass; ps += 2) {
-          const int n = (EPI == kEpiSwiGLU) ? (n0 >> 1) + ps * 64 : n0 + ps * kPassCols;   // output column in the group
-          uint32_t w[32];                                                // 128 bytes of this row's output
-          __syncwarp();
-          if constexpr (EPI == kEpiSwiGLU) {
-            uint32_t gt[32], up[32];
-  #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-              tmem_ld32(taddr + ps * 64 + hf * 32, gt);
-              tmem_ld32(taddr + 128 + ps * 64 + hf * 32, up);
-              tmem_ld_wait();
-  #pragma unroll
-              for (int c = 0; c < 16; ++c) {
-                const float h0 = silu_f(__uint_as_float(gt[2 * c])) * __uint_as_float(up[2 * c]);
-                const float h1 = silu_f(__uint_as_float(gt[2 * c + 1])) * __uint_as_float(up[2 * c + 1]);
-                w[hf * 16 + c] = pack_bf16(h0, h1);
-              }
-            }
-          } else if constexpr (EPI == kEpiOProj) {
-            tmem_ld32(taddr + ps * 32, w);
-            tmem_ld_wait();
-          } else if constexpr (EPI == kEpiQKV) {
-            // 64 packed columns = 32 rotation pairs (natural columns i0+m and i0+m+dh/2 of one head).  The first
-            // 64 bytes of the staged row are the first-half columns, the second 64 bytes their partners.
-            const bool rotate = n < args.q_cols + args.kv_cols;          // q and k heads; v is only de-interleaved
-            const int i0 = (n % args.dh) >> 1;
-            // the 32 (cos, sin) pairs of this row's position are fetched before the accumulator is read, so their
-            // latency overlaps the tensor-memory load
-            const float4* tab = reinterpret_cast<const float4*>(
-                args.rope_tab + size_t(row_ok ? args.tok_pos[row_local] : 0) * (args.dh >> 1) + i0);
-            float4 cs4[16];
-  #pragma unroll
-            for (int m = 0; m < 16; ++m) cs4[m] = rotate ? __ldg(tab + m) : make_float4(1.f, 0.f, 1.f, 0.f);
-            uint32_t r[32];
-  #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-              tmem_ld32(taddr + ps * 64 + hf * 32, r);
-              tmem_ld_wait();
-              float lo[16], hi[16];
-  #pragma unroll
-              for (int m = 0; m < 16; ++m) {
-                const float a = __uint_as_float(r[2 * m]) * scale, b = __uint_as_float(r[2 * m + 1]) * scale;
-                const float4 c4 = cs4[hf * 8 + (m >> 1)];
-                const float cx = (m & 1) ? c4.z : c4.x, cy = (m & 1) ? c4.w : c4.y;
-                lo[m] = a * cx - b * cy;
-                hi[m] = b * cx + a * cy;
-              }
-  #pragma unroll
-              for (int m = 0; m < 8; ++m) {
-                w[hf * 8 + m] = pack_bf16(lo[2 * m], lo[2 * m + 1]);
-                w[16 + hf * 8 + m] = pack_bf16(hi[2 * m], hi[2 * m + 1]);
-              }
-            }
+          const int tok = grow - group_row0;
+          // natural column inside the head of this lane's 8 values: chunks 0-3 first half, 4-7 second half
+          const int hcol = ((n % args.dh) >> 1) + (wr_chunk & 3) * 8 + (wr_chunk >> 2) * (args.dh >> 1);
+          if (n < args.q_cols) {
+            const int head = group * (args.q_cols / args.dh) + n / args.dh;
+            *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + size_t(tok) * args.ldo + head * args.dh + hcol) = v;
           } else {
-            uint32_t r[32];
-  #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-              tmem_ld32(taddr + ps * 64 + hf * 32, r);
-              tmem_ld_wait();
-  #pragma unroll
-              for (int c = 0; c < 16; ++c)
-                w[hf * 16 + c] = pack_bf16(__uint_as_float(r[2 * c]), __uint_as_float(r[2 * c + 1]));
+            const bool is_k = n < args.q_cols + args.kv_cols;
+            const int nn = n - args.q_cols - (is_k ? 0 : args.kv_cols);
+            const int kvh = group * (args.kv_cols / args.dh) + nn / args.dh;
+            const int slot = args.tok_slot[tok];
+            if (slot >= 0) {
+              const int page = slot >> 6, off = slot & 63;
+              __nv_bfloat16* base = is_k ? args.k_pages : args.v_pages;
+              *reinterpret_cast<uint4*>(base + ((size_t(page) * args.n_kv + kvh) * 64 + off) * args.dh + hcol) = v;
             }
           }
-          if (ps + 2 >= n_pass) release();                               // this warp's last TMEM read of the tile
-  #pragma unroll
-          for (int c = 0; c < 8; ++c)
-            *reinterpret_cast<uint4*>(stg + stg_off(lane, c)) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
-          __syncwarp();
-          if constexpr (EPI == kEpiOProj) {
-            // r_full = scale * (C + sum_h x[h]): the residual streams are read here.  This GEMM moves almost as many
-            // bytes as it has flops to hide them, so the epilogue has to keep ~256 bytes per thread in flight:
-            // 4 lanes x 16 bytes per row and stream, and all loads of the pass are issued before the first use.
-            const int or_row = lane >> 2, or_cg = lane & 3;           // row (+8j) and group of 8 columns
-            uint4 xq[4][8];
-  #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const int grow = row0 + quarter * 32 + or_row + 8 * j;
-              const size_t off = size_t(grow) * args.ldo + n + or_cg * 8;
-  #pragma unroll
-              for (int h = 0; h < 8; ++h) {
-                xq[j][h] = make_uint4(0u, 0u, 0u, 0u);
-                if (h < args.x_count && grow < row_end)
-                  xq[j][h] = __ldg(reinterpret_cast<const uint4*>(args.xsum + h * args.x_stride + off));
-              }
-            }
-  #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const int rr = or_row + 8 * j;
-              const int grow = row0 + quarter * 32 + rr;
-              if (grow >= row_end) continue;
-              const float4 c0 = *reinterpret_cast<const float4*>(stg + stg_off(rr, 2 * or_cg));
-              const float4 c1 = *reinterpret_cast<const float4*>(stg + stg_off(rr, 2 * or_cg + 1));
-              float a8[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-  #pragma unroll
-              for (int h = 0; h < 8; ++h) {
-                const uint32_t w4[4] = {xq[j][h].x, xq[j][h].y, xq[j][h].z, xq[j][h].w};
-  #pragma unroll
-                for (int q = 0; q < 4; ++q) { a8[2 * q] += bf16_lo(w4[q]); a8[2 * q + 1] += bf16_hi(w4[q]); }
-              }
-              float* dst = static_cast<float*>(args.out) + size_t(grow) * args.ldo + n + or_cg * 8;
-              const float sc = args.out_scale;
-              *reinterpret_cast<float4*>(dst) = make_float4(a8[0] * sc, a8[1] * sc, a8[2] * sc, a8[3] * sc);
-              *reinterpret_cast<float4*>(dst + 4) = make_float4(a8[4] * sc, a8[5] * sc, a8[6] * sc, a8[7] * sc);
-            }
-          } else {
-  #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const int rr = wr_row + 4 * j;                              // row inside the warp's 32
-              const int grow = row0 + quarter * 32 + rr;
-              if (grow >= row_end) continue;
-              const uint4 v = *reinterpret_cast<const uint4*>(stg + stg_off(rr, wr_chunk));
-              if constexpr (EPI == kEpiQKV) {
-                const int tok = grow - group_row0;
-                // natural column inside the head of this lane's 8 values: chunks 0-3 first half, 4-7 second half
-                const int hcol = ((n % args.dh) >> 1) + (wr_chunk & 3) * 8 + (wr_chunk >> 2) * (args.dh >> 1);
-                if (n < args.q_cols) {
-                  const int head = group * (args.q_cols / args.dh) + n / args.dh;
-                  *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + size_t(tok) * args.ldo + head * args.dh + hcol) = v;
-                } else {
-                  const bool is_k = n < args.q_cols + args.kv_cols;
-                  const int nn = n - args.q_cols - (is_k ? 0 : args.kv_cols);
-                  const int kvh = group * (args.kv_cols / args.dh) + nn / args.dh;
-                  const int slot = args.tok_slot[tok];
-                  if (slot >= 0) {
-                    const int page = slot >> 6, off = slot & 63;
-                    __nv_bfloat16* base = is_k ? args.k_pages : args.v_pages;
-                    *reinterpret_cast<uint4*>(base + ((size_t(page) * args.n_kv + kvh) * 64 + off) * args.dh + hcol) = v;
-                  }
-                }
-              } else {
-                *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + size_t(grow) * args.ldo + n + wr_chunk * 8) = v;
-              }
-            }
-          }
+        } else {
+          *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + size_t(grow) * args.ldo + n + wr_chunk * 8) = v;
         }
+      }
+    }
+  }
 }
 
 template <int EPI, bool GATHER>
