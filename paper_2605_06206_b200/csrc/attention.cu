@@ -200,39 +200,44 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     a.part_o[pidx * DH + c] = acc;
     if (c == 0) { a.part_ml[pidx * 2] = m; a.part_ml[pidx * 2 + 1] = l; }
   }
-}
 
-// one warp per (sequence, query head): combine the splits that exist for that sequence
-template <int DH>
-__global__ void attn_decode_merge_kernel(const AttnArgs a) {
-  const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (wid >= a.n_seqs * a.n_q) return;
-  const int b = wid / a.n_q, head = wid - b * a.n_q;
-  const int n_pages = (a.context_lens[b] + 1 + 63) >> 6;
+  // The CTA that finishes last among the splits of this (sequence, KV head) combines them (always in split order, so
+  // the result does not depend on which one that is) and re-arms the counter for the next call: no merge launch.
   const int n_splits = min(a.max_splits, (n_pages + a.pages_per_split - 1) / a.pages_per_split);
-  const size_t base = (size_t(b) * a.n_q + head) * a.max_splits;
-  float m = -INFINITY;
-  for (int s = 0; s < n_splits; ++s) m = fmaxf(m, a.part_ml[(base + s) * 2]);
-  float acc[DH / 32];
+  int* ticket_s = reinterpret_cast<int*>(ml + 64);
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) *ticket_s = atomicAdd(&a.split_done[b * a.n_kv + kvh], 1);
+  __syncthreads();
+  if (*ticket_s != n_splits - 1) return;
+  if (threadIdx.x == 0) a.split_done[b * a.n_kv + kvh] = 0;
+  __threadfence();
+  for (int r = warp; r < G; r += kDcThreads / 32) {                 // one warp per query head of the group
+    const int head = kvh * G + r;
+    const size_t base = (size_t(b) * a.n_q + head) * a.max_splits;
+    float m = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) m = fmaxf(m, __ldcg(a.part_ml + (base + s) * 2));
+    float acc[DH / 32];
 #pragma unroll
-  for (int q = 0; q < DH / 32; ++q) acc[q] = 0.f;
-  float l = 0.f;
-  for (int s = 0; s < n_splits; ++s) {
-    const float f = fast_exp2(a.part_ml[(base + s) * 2] - m);
-    l += f * a.part_ml[(base + s) * 2 + 1];
+    for (int q = 0; q < DH / 32; ++q) acc[q] = 0.f;
+    float l = 0.f;
+    for (int s = 0; s < n_splits; ++s) {
+      const float f = fast_exp2(__ldcg(a.part_ml + (base + s) * 2) - m);
+      l += f * __ldcg(a.part_ml + (base + s) * 2 + 1);
 #pragma unroll
-    for (int q = 0; q < DH / 32; ++q) acc[q] += f * a.part_o[(base + s) * DH + q * 32 + lane];
+      for (int q = 0; q < DH / 32; ++q) acc[q] += f * __ldcg(a.part_o + (base + s) * DH + q * 32 + lane);
+    }
+    const float inv = 1.f / l;
+    bf16* dst = a.out + size_t(tok) * (a.n_q * DH) + head * DH;
+#pragma unroll
+    for (int q = 0; q < DH / 32; ++q) dst[q * 32 + lane] = __float2bfloat16_rn(acc[q] * inv);
   }
-  const float inv = 1.f / l;
-  bf16* dst = a.out + size_t(a.cu_q[b]) * (a.n_q * DH) + head * DH;
-#pragma unroll
-  for (int q = 0; q < DH / 32; ++q) dst[q * 32 + lane] = __float2bfloat16_rn(acc[q] * inv);
 }
 
 template <int DH>
 static void launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st) {
   constexpr size_t smem = kDcStages * 2 * 64 * DH * 2 + 16 * DH * 2 + 1024 + 64;
-  static_assert(kDcStages * 2 * 64 * DH * 2 >= (4 * 16 * DH + 128) * 4, "merge buffer must fit in the stages");
+  static_assert(kDcStages * 2 * 64 * DH * 2 >= (4 * 16 * DH + 128 + 4) * 4, "merge buffer must fit in the stages");
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(attn_decode_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
@@ -240,8 +245,6 @@ static void launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, cons
   }
   dim3 grid(a.max_splits, a.n_kv, a.n_seqs);
   attn_decode_kernel<DH><<<grid, kDcThreads, smem, st>>>(tmK, tmV, a);
-  const int warps = a.n_seqs * a.n_q;
-  attn_decode_merge_kernel<DH><<<(warps * 32 + 127) / 128, 128, 0, st>>>(a);
 }
 
 void launch_attn_decode(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st) {

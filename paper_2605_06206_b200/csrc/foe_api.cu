@@ -57,7 +57,7 @@ struct foe_workspace {
   std::vector<void*> allocs;
   float *inv_rms, *inv_rms_f, *route_part, *r_full, *logits, *topk_w, *part_o, *part_ml;
   bf16 *qkv, *attn_o, *u, *hmid, *y;
-  int *topk_idx, *cu_q, *tok_seq, *tok_pos, *tok_slot, *status;
+  int *topk_idx, *cu_q, *tok_seq, *tok_pos, *tok_slot, *status, *split_done;
   PermuteBuffers pb;
   CUtensorMap tm_attn_o, tm_hmid, tm_qkv;       // maps of workspace buffers (A operands, attention Q)
 };
@@ -212,8 +212,8 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
   aa.max_pages_per_seq = kv->max_pages_per_seq; aa.num_pages = kv->num_pages; aa.n_q = L->n_q; aa.n_kv = L->n_kv;
   aa.dh = dh; aa.max_q_len = decode ? 1 : kv->max_q_len; aa.scale_log2 = float(1.4426950408889634 / sqrt(double(dh)));
   aa.status = L->ws->status; aa.part_o = L->ws->part_o; aa.part_ml = L->ws->part_ml; aa.max_splits = L->max_splits;
-  aa.pages_per_split = L->pages_per_split;
-  if (decode) { launch_attn_decode(tmK, tmV, aa, st); L->launches += 2; }
+  aa.pages_per_split = L->pages_per_split; aa.split_done = L->ws->split_done;
+  if (decode) { launch_attn_decode(tmK, tmV, aa, st); L->launches += 1; }
   else { launch_attn_prefill_tc(L->ws->tm_qkv, tmK, tmV, aa, st); L->launches += 1; }
 
   // ---- output projection; the cross-cluster sync is its K-reduction plus the sum of x[h] in the epilogue
@@ -397,6 +397,7 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     ok = ok && walloc(W, &W->status, size_t(1));
     ok = ok && walloc(W, &W->part_o, size_t(cfg->max_seqs) * L->n_q * L->max_splits * dh);
     ok = ok && walloc(W, &W->part_ml, size_t(cfg->max_seqs) * L->n_q * L->max_splits * 2);
+    ok = ok && walloc(W, &W->split_done, size_t(cfg->max_seqs) * L->n_kv);
     ok = ok && walloc(W, &W->pb.counts, size_t(E));
     ok = ok && walloc(W, &W->pb.offsets, size_t(E) + 1);
     ok = ok && walloc(W, &W->pb.perm, size_t(R));
@@ -408,6 +409,7 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     ok = ok && walloc(W, &W->pb.n_mtiles, size_t(1));
     if (!ok) { foe_layer_destroy(L); return FOE_ERR_OOM; }
     cudaMemsetAsync(W->status, 0, sizeof(int), st);
+    cudaMemsetAsync(W->split_done, 0, size_t(cfg->max_seqs) * L->n_kv * sizeof(int), st);
     cudaMemsetAsync(W->attn_o, 0, size_t(S + 128) * L->n_q * dh * sizeof(bf16), st);
     cudaMemsetAsync(W->hmid, 0, size_t(R + 128) * I * sizeof(bf16), st);
     ok = make_map_2d(&W->tm_attn_o, W->attn_o, uint64_t(S), uint64_t(L->n_q) * dh, kBM) &&

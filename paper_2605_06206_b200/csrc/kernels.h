@@ -82,6 +82,7 @@ struct AttnArgs {
   // decode only
   float* part_o;            // [n_seqs][n_q][max_splits][dh]
   float* part_ml;           // [n_seqs][n_q][max_splits][2]
+  int* split_done;          // [n_seqs][n_kv] splits finished so far (zero between calls)
   int max_splits;
   int pages_per_split;
 };
