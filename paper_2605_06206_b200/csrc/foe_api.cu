@@ -142,6 +142,13 @@ foe_status check_launch() { return cudaGetLastError() == cudaSuccess ? FOE_OK : 
 
 // routing + dispatch maps for n tokens whose synced residual is r (fp32 internal or bf16 from the caller)
 void run_route_and_permute(foe_layer* L, const void* r, int r_is_bf16, int n, cudaStream_t st) {
+  if (n <= kRouteSmallMaxTokens) {          // a decode step: two launches for norm, scores, top-k, gates and maps
+    L->launches += launch_route_small(r, r_is_bf16, L->ffn_gain, L->router_w, L->router_b, L->ws->u, L->ws->route_part,
+                                      L->ws->logits, L->ws->topk_idx, L->ws->topk_w, L->ws->pb, n, L->d, L->H, L->Ec,
+                                      L->kc, L->cfg.rms_eps, L->ws->status, st);
+    stage_mark(L, kStPermute, st);
+    return;
+  }
   L->launches += launch_route(r, r_is_bf16, L->ffn_gain, L->router_w, &L->tm_router, L->router_b, L->ws->u, L->ws->inv_rms_f, L->ws->route_part,
                               L->ws->logits, L->ws->topk_idx, L->ws->topk_w, n, L->d, L->H, L->Ec, L->kc, L->cfg.rms_eps, L->n_sms, L->ws->status, st);
   stage_mark(L, kStPermute, st);

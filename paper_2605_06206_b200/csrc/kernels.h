@@ -45,6 +45,16 @@ void launch_split_router_weights(const float* wr, const bf16* gain, bf16* planes
 void launch_router_tc(const CUtensorMap& tmW, const void* r, int r_is_bf16, const float* inv_rms, float* part,
                       int n_tokens, int d, int E, int* status, cudaStream_t st);
 
+// Calls of at most kRouteSmallMaxTokens tokens: FFN norm + scores in one launch, top-k + gates + dispatch maps in a
+// second one (launch_route followed by launch_permute give the same results in up to six).
+constexpr int kRouteSmallMaxTokens = 256;
+struct PermuteBuffers;
+int launch_route_small(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const float* br, bf16* u_out,
+                       float* scores, float* logits, int* idx, float* w, const PermuteBuffers& pb, int n_tokens, int d,
+                       int H, int Ec, int kc, float eps, int* status, cudaStream_t st);
+int launch_topk_permute_small(const float* scores, int k_splits, const float* bias, float* logits, int* idx, float* w,
+                              const PermuteBuffers& pb, int n_tokens, int H, int Ec, int kc, int* status, cudaStream_t st);
+
 // routing on the library's built-in scratch area (no allocation); 0, -3 (too large) or -6 (CUDA error)
 int launch_route_noalloc(const bf16* h, const bf16* gain, const float* wr, const float* br, int* idx, float* w,
                          int n_tokens, int d, int H, int Ec, int kc, float eps, cudaStream_t st);

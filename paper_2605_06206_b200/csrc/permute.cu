@@ -120,9 +120,22 @@ __global__ void permute_scatter_kernel(const int* __restrict__ idx, const int* _
 
 // All three steps in one block, for calls of at most 256 tokens (a decode step): bitmap, scan over the
 // experts, slots.  Same results as the three-kernel path, two launches fewer.
+// With `scores` given, the block first takes the routing decision itself (so that a decode step needs one launch for
+// top-k, gates and maps): one thread per (token, cluster) adds the bias, writes the scores, selects the k_c largest of
+// the cluster's E_c (larger score first, equal scores: lower expert id first) and their softmax gates.
+struct TopkSmall {
+  const float* scores;    // [k_splits][n_tokens][E] partial router scores, or nullptr: idx is an input
+  int k_splits;
+  const float* bias;      // [E] or nullptr
+  float* logits_out;      // [n_tokens][E]
+  int* idx_out;           // [n_tokens][H][kc]
+  float* w_out;
+  int H, Ec, kc;
+};
+
 __global__ void __launch_bounds__(1024)
 permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, const PermuteBuffers pb,
-                     int* __restrict__ status) {
+                     int* __restrict__ status, const TopkSmall tk) {
   extern __shared__ uint32_t bm[];            // [E][8]
   __shared__ int s_a[1024], s_b[1024], s_off[1024];
   int* counts = pb.counts;
@@ -130,6 +143,42 @@ permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, 
   int* perm = pb.perm;
   int* inv = pb.inv;
   const int t = threadIdx.x;
+  if (tk.scores) {
+    const int H = tk.H, Ec = tk.Ec, kc = tk.kc;
+    // scores = partial sums in fixed order + bias, all threads; then one thread per (token, cluster)
+    for (int q = t; q < n_tokens * E; q += 1024) {
+      float v = 0.f;
+      for (int z = 0; z < tk.k_splits; ++z) v += tk.scores[size_t(z) * n_tokens * E + q];
+      tk.logits_out[q] = v + (tk.bias ? tk.bias[q % E] : 0.f);
+    }
+    __threadfence_block();
+    __syncthreads();
+    for (int task = t; task < n_tokens * H; task += 1024) {
+      const int i = task / H, h = task - i * H;
+      const size_t o = size_t(i) * E + size_t(h) * Ec;
+      uint32_t taken[4] = {0u, 0u, 0u, 0u};                 // E_c <= 128
+      float m = 0.f, sum = 0.f;
+      const size_t oo = size_t(task) * kc;
+      for (int j = 0; j < kc; ++j) {
+        float bv = 0.f;
+        int bi = -1;
+        for (int e = 0; e < Ec; ++e) {
+          if ((taken[e >> 5] >> (e & 31)) & 1u) continue;
+          const float v = tk.logits_out[o + e];
+          if (bi < 0 || v > bv) { bv = v; bi = e; }         // ascending e: first wins ties
+        }
+        taken[bi >> 5] |= 1u << (bi & 31);
+        if (j == 0) m = bv;
+        const float ex = expf(bv - m);
+        sum += ex;
+        tk.idx_out[oo + j] = h * Ec + bi;
+        tk.w_out[oo + j] = ex;
+      }
+      for (int j = 0; j < kc; ++j) tk.w_out[oo + j] = tk.w_out[oo + j] / sum;
+    }
+    __threadfence_block();
+    __syncthreads();                            // idx (== tk.idx_out) is read below by other threads of this block
+  }
   for (int q = t; q < E * 8; q += 1024) bm[q] = 0u;
   __syncthreads();
   if (t < n_tokens) {
@@ -184,7 +233,9 @@ int launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int s
                    cudaStream_t st) {
   if (n_tokens <= 0) return 0;
   if (n_tokens <= kPB) {
-    permute_small_kernel<<<1, 1024, size_t(E) * 32, st>>>(idx, n_tokens, sel, E, pb, status);
+    TopkSmall none;
+    none.scores = nullptr;
+    permute_small_kernel<<<1, 1024, size_t(E) * 32, st>>>(idx, n_tokens, sel, E, pb, status, none);
     return 1;
   }
   const int n_blocks = (n_tokens + kPB - 1) / kPB;
@@ -194,6 +245,17 @@ int launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int s
   permute_scatter_kernel<<<(total + 255) / 256, 256, 0, st>>>(idx, pb.rank, pb.blk_counts, pb.offsets, pb.perm, pb.inv,
                                                             n_tokens, sel, E);
   return 3;
+}
+
+// top-k + gates + dispatch maps of a call of at most 256 tokens in one launch (scores: [k_splits][n_tokens][E])
+int launch_topk_permute_small(const float* scores, int k_splits, const float* bias, float* logits, int* idx, float* w,
+                              const PermuteBuffers& pb, int n_tokens, int H, int Ec, int kc, int* status, cudaStream_t st) {
+  if (n_tokens <= 0) return 0;
+  TopkSmall tk;
+  tk.scores = scores; tk.k_splits = k_splits; tk.bias = bias; tk.logits_out = logits; tk.idx_out = idx; tk.w_out = w; tk.H = H; tk.Ec = Ec; tk.kc = kc;
+  const int E = H * Ec;
+  permute_small_kernel<<<1, 1024, size_t(E) * 32, st>>>(idx, n_tokens, H * kc, E, pb, status, tk);
+  return 1;
 }
 
 }  // namespace foe

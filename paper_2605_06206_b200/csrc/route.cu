@@ -237,6 +237,84 @@ __global__ void topk_gates_kernel(const float* __restrict__ part, int k_splits, 
   }
 }
 
+// ------------------------------------------------------------------------------------------------ 1+2, small calls
+// FFN norm and router scores of a call of at most 256 tokens (a decode step) in one launch: a CTA owns 4 tokens and
+// 64 experts.  It first reduces its tokens' rows to 1/rms, then walks K in tiles of 64: the normalised activations
+// (fp32, never rounded on this path) and a 64 x 64 tile of router weights go through shared memory, every thread
+// accumulates one (token, expert) score in four interleaved fp32 chains.  K is also split over gridDim.z (partial
+// scores, summed in a fixed order by the top-k kernel).  The CTAs of the first expert chunk also write the bf16
+// expert input u for their slice of K.
+constexpr int kRsTok = 4, kRsExp = 64, kRsK = 64, kRsThreads = kRsTok * kRsExp;
+
+__global__ void __launch_bounds__(kRsThreads)
+route_scores_small_kernel(const void* __restrict__ r_in, int r_is_bf16, const bf16* __restrict__ gain,
+                          const float* __restrict__ wr, bf16* __restrict__ u_out, float* __restrict__ scores,
+                          int n_tokens, int d, int E, float eps, int k_per_split) {
+  __shared__ float w_s[kRsK][kRsExp + 1];
+  __shared__ float u_s[kRsTok][kRsK];
+  __shared__ float red[kRsTok][2];
+  const int tid = threadIdx.x, el = tid & 63, tq = tid >> 6;
+  const int tok = min(blockIdx.x * kRsTok + tq, n_tokens - 1);          // rows past the end repeat the last one
+  const int e0 = blockIdx.y * kRsExp;
+  auto load_r = [&](int k) -> float {
+    return r_is_bf16 ? __bfloat162float(static_cast<const bf16*>(r_in)[size_t(tok) * d + k])
+                     : static_cast<const float*>(r_in)[size_t(tok) * d + k];
+  };
+  // 1/rms of this thread's token: 64 threads per token
+  float ss = 0.f;
+  for (int k = el; k < d; k += 64) { const float v = load_r(k); ss += v * v; }
+  ss = warp_sum(ss);
+  if ((tid & 31) == 0) red[tq][(tid >> 5) & 1] = ss;
+  __syncthreads();
+  const float inv = rsqrtf((red[tq][0] + red[tq][1]) / float(d) + eps);
+
+  // loader roles for the weight tile: float4 (row = i >> 4, column group = i & 15), i = tid + 256 j
+  float4 wq[4];
+  float uq;
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = tid + kRsThreads * j;
+      const int e = min(e0 + (i >> 4), E - 1);
+      wq[j] = __ldg(reinterpret_cast<const float4*>(wr + size_t(e) * d + k0 + (i & 15) * 4));
+    }
+    uq = load_r(k0 + el) * inv * __bfloat162float(gain[k0 + el]);
+  };
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  const int kbeg = blockIdx.z * k_per_split, kend = min(d, kbeg + k_per_split);   // this CTA's slice of K
+  fetch(kbeg);
+  for (int k0 = kbeg; k0 < kend; k0 += kRsK) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = tid + kRsThreads * j, row = i >> 4, c = (i & 15) * 4;
+      w_s[c][row] = wq[j].x; w_s[c + 1][row] = wq[j].y; w_s[c + 2][row] = wq[j].z; w_s[c + 3][row] = wq[j].w;
+    }
+    u_s[tq][el] = uq;
+    if (blockIdx.y == 0 && blockIdx.x * kRsTok + tq < n_tokens) u_out[size_t(tok) * d + k0 + el] = __float2bfloat16_rn(uq);
+    __syncthreads();
+    if (k0 + kRsK < kend) fetch(k0 + kRsK);            // in flight during the products below
+#pragma unroll
+    for (int k = 0; k < kRsK; ++k) acc[k & 3] = fmaf(u_s[tq][k], w_s[k][el], acc[k & 3]);
+    __syncthreads();
+  }
+  if (blockIdx.x * kRsTok + tq < n_tokens && e0 + el < E)
+    scores[(size_t(blockIdx.z) * n_tokens + tok) * E + e0 + el] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+}
+
+int launch_route_small(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const float* br, bf16* u_out,
+                       float* scores, float* logits, int* idx, float* w, const PermuteBuffers& pb, int n_tokens, int d,
+                       int H, int Ec, int kc, float eps, int* status, cudaStream_t st) {
+  if (n_tokens <= 0) return 0;
+  const int E = H * Ec;
+  // K is cut into slices so that a few dozen tokens still spread over the GPU; the partial scores are summed in a
+  // fixed order by the second kernel
+  int ks = 1;
+  while (ks < 16 && (d / (ks * 2)) % kRsK == 0 && d / (ks * 2) >= 2 * kRsK) ks *= 2;
+  dim3 grid((n_tokens + kRsTok - 1) / kRsTok, (E + kRsExp - 1) / kRsExp, ks);
+  route_scores_small_kernel<<<grid, kRsThreads, 0, st>>>(r_in, r_is_bf16, gain, wr, u_out, scores, n_tokens, d, E, eps, d / ks);
+  return 1 + launch_topk_permute_small(scores, ks, br, logits, idx, w, pb, n_tokens, H, Ec, kc, status, st);
+}
+
 // The same selection with one thread per (token, cluster) and the cluster's scores in registers: for the common
 // cluster sizes (a power of two up to 32) there is nothing to exchange between lanes.  Ties and order exactly as in
 // topk_gates_kernel: score descending, expert id ascending.
