@@ -56,7 +56,7 @@ typedef enum { FOE_MIDDLE = 0, FOE_FIRST = 1, FOE_LAST = 2, FOE_SINGLE = 3 } foe
 typedef enum { FOE_SYNC_MEAN = 0, FOE_SYNC_SUM = 1 } foe_sync;
 
 /* Layer description.  Validity: n_kv_heads % n_clusters == 0, n_q_heads % n_kv_heads == 0,
- * head_dim in {64, 128}, 1 <= top_k_per_cluster <= experts_per_cluster <= 128, top_k_per_cluster <= 32,
+ * head_dim in {64, 96, 128}, 1 <= top_k_per_cluster <= experts_per_cluster <= 128, top_k_per_cluster <= 32,
  * page_size == 64, hidden % 128 == 0, (n_q_heads * head_dim) % 128 == 0, ffn_inter % 128 == 0,
  * n_clusters <= 8, n_clusters * experts_per_cluster <= 1024, n_q_heads / n_kv_heads <= 16, max_* > 0.
  * position: FOE_FIRST/FOE_SINGLE take x as [S, hidden] (one shared attention, its residual used
@@ -115,7 +115,8 @@ typedef struct {
   const int* offsets;       /* [E+1] exclusive scan of counts */
   const int* perm;          /* [S*H*k_c] slot -> token */
   const int* inv;           /* [S][H][k_c] -> slot */
-  const void* q;            /* [S][n_q*head_dim] bf16 queries after RoPE (K and V of the call are in the cache pages) */
+  const void* q;            /* [S][n_q][head_dim, padded to 128 when it is 96] bf16 queries after RoPE (K and V of the
+                               call are in the cache pages) */
   const void* attn_o;       /* [S][n_q*head_dim] bf16 attention output before W_O */
 } foe_aux;
 

@@ -235,9 +235,12 @@ class FoeLayer:
         spec = dict(r_full=((S, d), torch.float32), u=((S, d), torch.bfloat16), logits=((S, E), torch.float32),
                     topk_idx=((S, H, kc), torch.int32), topk_w=((S, H, kc), torch.float32),
                     counts=((E,), torch.int32), offsets=((E + 1,), torch.int32), perm=((S * H * kc,), torch.int32),
-                    inv=((S, H, kc), torch.int32), q=((S, s.n_q_heads * s.head_dim), torch.bfloat16),
+                    inv=((S, H, kc), torch.int32), q=((S, s.n_q_heads, 128 if s.head_dim == 96 else s.head_dim), torch.bfloat16),
                     attn_o=((S, s.n_q_heads * s.head_dim), torch.bfloat16))
-        return {k: _view(getattr(a, k), shp, dt).clone() for k, (shp, dt) in spec.items()}
+        out = {k: _view(getattr(a, k), shp, dt).clone() for k, (shp, dt) in spec.items()}
+        # q is kept with its heads padded to the attention kernels' tile width (head_dim 96 -> 128)
+        out["q"] = out["q"][:, :, :s.head_dim].reshape(S, s.n_q_heads * s.head_dim).contiguous()
+        return out
 
     def poll_status(self) -> int:
         v = ctypes.c_int(0)

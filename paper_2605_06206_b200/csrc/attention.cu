@@ -228,9 +228,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
       for (int q = 0; q < DH / 32; ++q) acc[q] += f * __ldcg(a.part_o + (base + s) * DH + q * 32 + lane);
     }
     const float inv = 1.f / l;
-    bf16* dst = a.out + size_t(tok) * (a.n_q * DH) + head * DH;
+    bf16* dst = a.out + size_t(tok) * (a.n_q * a.dh) + head * a.dh;       // (a 96-wide head is computed zero-padded to 128)
 #pragma unroll
-    for (int q = 0; q < DH / 32; ++q) dst[q * 32 + lane] = __float2bfloat16_rn(acc[q] * inv);
+    for (int q = 0; q < DH / 32; ++q)
+      if (q * 32 + lane < a.dh) dst[q * 32 + lane] = __float2bfloat16_rn(acc[q] * inv);
   }
 }
 
@@ -249,7 +250,7 @@ static void launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, cons
 
 void launch_attn_decode(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st) {
   if (a.n_seqs <= 0) return;
-  if (a.dh == 128) launch_decode_t<128>(tmK, tmV, a, st);
+  if (a.dh > 64) launch_decode_t<128>(tmK, tmV, a, st);
   else launch_decode_t<64>(tmK, tmV, a, st);
 }
 

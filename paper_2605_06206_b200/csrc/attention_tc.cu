@@ -330,8 +330,8 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         for (int r0 = 0; r0 < 32; r0 += RPI) {
           const int rr = r0 + lane / CH, c = lane % CH;
           const int grow = quarter * 32 + rr;
-          if (grow < rows_here)
-            *reinterpret_cast<uint4*>(a.out + size_t(tok0 + grow) * (a.n_q * DH) + (head0 + t) * DH + c * 8) =
+          if (grow < rows_here && c * 8 < a.dh)            // (a 96-wide head is computed zero-padded to 128)
+            *reinterpret_cast<uint4*>(a.out + size_t(tok0 + grow) * (a.n_q * a.dh) + (head0 + t) * a.dh + c * 8) =
                 *reinterpret_cast<const uint4*>(stg + rr * (DH * 2) + ((c ^ (rr & 7)) << 4));
         }
       }
@@ -364,7 +364,7 @@ static void launch_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUte
 void launch_attn_prefill_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
                             cudaStream_t st) {
   if (a.n_seqs <= 0 || a.max_q_len <= 0) return;
-  if (a.dh == 128) launch_tc<128>(tmQ, tmK, tmV, a, st);
+  if (a.dh > 64) launch_tc<128>(tmQ, tmK, tmV, a, st);
   else launch_tc<64>(tmQ, tmK, tmV, a, st);
 }
 

@@ -65,6 +65,7 @@ struct foe_workspace {
 struct foe_layer {
   foe_config cfg;
   int H, g, c, dh, d, I, E, Ec, kc, n_q, n_kv, qkv_cols, S_max, R_max, n_sms;
+  int dhp;               // head width the attention kernels work with: head_dim, or 128 for head_dim 96 (zero-padded)
   bool first, last;
   std::vector<void*> allocs;
   // repacked weights
@@ -119,7 +120,7 @@ foe_status validate(const foe_config* c) {
   if (c->hidden <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->n_clusters <= 0) return FOE_ERR_CONFIG;
   if (c->n_kv_heads % c->n_clusters || c->n_q_heads % c->n_kv_heads) return FOE_ERR_CONFIG;
   if (c->n_clusters > 8) return FOE_ERR_CONFIG;          // the sync epilogues add up to 8 residual streams
-  if (c->head_dim != 64 && c->head_dim != 128) return FOE_ERR_CONFIG;
+  if (c->head_dim != 64 && c->head_dim != 96 && c->head_dim != 128) return FOE_ERR_CONFIG;
   if (c->n_q_heads / c->n_kv_heads > 16) return FOE_ERR_CONFIG;
   if (c->experts_per_cluster < 1 || c->experts_per_cluster > 128) return FOE_ERR_CONFIG;
   if (c->top_k_per_cluster < 1 || c->top_k_per_cluster > c->experts_per_cluster || c->top_k_per_cluster > 32)
@@ -189,7 +190,7 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     memset(&ga, 0, sizeof(ga));
     ga.n_groups = H; ga.rows_per_group = S; ga.a_group_stride = L->first ? 0 : S;
     ga.N = (L->g + 2 * L->c) * dh; ga.K = d; ga.status = L->ws->status;
-    ga.out = L->ws->qkv; ga.ldo = L->n_q * dh;
+    ga.out = L->ws->qkv; ga.ldo = L->n_q * L->dhp; ga.q_head_stride = L->dhp;
     ga.row_scale = L->ws->inv_rms; ga.scale_group_stride = L->first ? 0 : S;
     ga.q_cols = L->g * dh; ga.kv_cols = L->c * dh; ga.dh = dh; ga.n_kv = L->n_kv;
     ga.rope_tab = L->rope_tab; ga.tok_pos = L->ws->tok_pos; ga.tok_slot = L->ws->tok_slot;
@@ -200,7 +201,7 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
     memset(&sa, 0, sizeof(sa));
     sa.W = L->wqkv_t; sa.X = xb; sa.ldx = d; sa.n_groups = H; sa.rows_per_group = S; sa.x_group_stride = L->first ? 0 : S;
     sa.N = (L->g + 2 * L->c) * dh; sa.K = d; sa.epi = kEpiQKV;
-    sa.out = L->ws->qkv; sa.ldo = L->n_q * dh;
+    sa.out = L->ws->qkv; sa.ldo = L->n_q * L->dhp; sa.q_head_stride = L->dhp;
     sa.rms_eps = L->cfg.rms_eps;
     sa.q_cols = L->g * dh; sa.kv_cols = L->c * dh; sa.dh = dh; sa.n_kv = L->n_kv;
     sa.rope_tab = L->rope_tab; sa.tok_pos = L->ws->tok_pos; sa.tok_slot = L->ws->tok_slot;
@@ -349,7 +350,7 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
   foe_layer* L = new (std::nothrow) foe_layer();
   if (!L) return FOE_ERR_OOM;
   L->cfg = *cfg;
-  L->H = cfg->n_clusters; L->n_q = cfg->n_q_heads; L->n_kv = cfg->n_kv_heads; L->dh = cfg->head_dim;
+  L->H = cfg->n_clusters; L->n_q = cfg->n_q_heads; L->n_kv = cfg->n_kv_heads; L->dh = cfg->head_dim; L->dhp = cfg->head_dim == 96 ? 128 : cfg->head_dim;
   L->g = L->n_q / L->H; L->c = L->n_kv / L->H; L->d = cfg->hidden; L->I = cfg->ffn_inter;
   L->Ec = cfg->experts_per_cluster; L->E = L->H * L->Ec; L->kc = cfg->top_k_per_cluster;
   L->qkv_cols = (L->n_q + 2 * L->n_kv) * L->dh;
@@ -392,7 +393,7 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     ok = ok && walloc(W, &W->route_part, size_t(S) * E > (size_t(1) << 21) ? size_t(S) * E : (size_t(1) << 21));
     ok = ok && walloc(W, &W->topk_w, size_t(R));
     ok = ok && walloc(W, &W->topk_idx, size_t(R));
-    ok = ok && walloc(W, &W->qkv, size_t(S + 128) * L->n_q * dh);          // q after RoPE (k, v go to the pages)
+    ok = ok && walloc(W, &W->qkv, size_t(S + 128) * L->n_q * L->dhp);      // q after RoPE (k, v go to the pages)
     ok = ok && walloc(W, &W->attn_o, size_t(S + 128) * L->n_q * dh);
     ok = ok && walloc(W, &W->u, size_t(S) * d);
     ok = ok && walloc(W, &W->hmid, size_t(R + 128) * I);
@@ -402,7 +403,7 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     ok = ok && walloc(W, &W->tok_pos, size_t(S));
     ok = ok && walloc(W, &W->tok_slot, size_t(S));
     ok = ok && walloc(W, &W->status, size_t(1));
-    ok = ok && walloc(W, &W->part_o, size_t(cfg->max_seqs) * L->n_q * L->max_splits * dh);
+    ok = ok && walloc(W, &W->part_o, size_t(cfg->max_seqs) * L->n_q * L->max_splits * L->dhp);
     ok = ok && walloc(W, &W->part_ml, size_t(cfg->max_seqs) * L->n_q * L->max_splits * 2);
     ok = ok && walloc(W, &W->split_done, size_t(cfg->max_seqs) * L->n_kv);
     ok = ok && walloc(W, &W->pb.counts, size_t(E));
@@ -418,10 +419,11 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     cudaMemsetAsync(W->status, 0, sizeof(int), st);
     cudaMemsetAsync(W->split_done, 0, size_t(cfg->max_seqs) * L->n_kv * sizeof(int), st);
     cudaMemsetAsync(W->attn_o, 0, size_t(S + 128) * L->n_q * dh * sizeof(bf16), st);
+    cudaMemsetAsync(W->qkv, 0, size_t(S + 128) * L->n_q * L->dhp * sizeof(bf16), st);   // padding columns stay zero
     cudaMemsetAsync(W->hmid, 0, size_t(R + 128) * I * sizeof(bf16), st);
     ok = make_map_2d(&W->tm_attn_o, W->attn_o, uint64_t(S), uint64_t(L->n_q) * dh, kBM) &&
          make_map_2d(&W->tm_hmid, W->hmid, uint64_t(R), I, kBM) &&
-         make_map_2d(&W->tm_qkv, W->qkv, uint64_t(S), uint64_t(L->n_q) * dh, 128);
+         make_map_2d(&W->tm_qkv, W->qkv, uint64_t(S), uint64_t(L->n_q) * L->dhp, 128);
     if (!ok) { foe_layer_destroy(L); return FOE_ERR_CUDA; }
   }
 

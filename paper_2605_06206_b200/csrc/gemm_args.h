@@ -56,6 +56,8 @@ struct GemmArgs {
   int scale_group_stride;
   int q_cols, kv_cols;      // g*dh and c*dh of one cluster
   int dh, n_kv;
+  int q_head_stride;        // elements between the heads of a q row in out (head_dim, or 128 for head_dim 96: the
+                            // attention kernels read q with zero padding up to their tile width)
   const float2* rope_tab;   // [max_context][dh/2] (cos, sin)
   const int* tok_pos;       // [tokens] position of the token in its sequence
   const int* tok_slot;      // [tokens] page * 64 + offset of the token in the cache, -1 = none

@@ -73,12 +73,15 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
     if (row_ok) scale = args.row_scale[size_t(group) * args.scale_group_stride + row_local];
   }
   constexpr int kPassCols = (EPI == kEpiOProj) ? 32 : 64;          // accumulator columns per pass (SwiGLU: 64 + 64)
-  const int n_pass = (EPI == kEpiSwiGLU) ? 2 : (tile_cols + kPassCols - 1) / kPassCols;
+  // a head of 96 columns is not a whole number of 64-column passes: its QKV epilogue takes 32 columns at a time
+  const bool narrow = (EPI == kEpiQKV) && (args.dh & 63) != 0;
+  const int pass_cols = narrow ? 32 : kPassCols;
+  const int n_pass = (EPI == kEpiSwiGLU) ? 2 : (tile_cols + pass_cols - 1) / pass_cols;
   const int wr_row = lane >> 3, wr_chunk = lane & 7;                // write-out role: row (+4j), 16-byte chunk
   if (half >= n_pass) { release(); return; }                        // nothing for this warp in a one-pass tile
 #pragma unroll 1
   for (int ps = half; ps < n_pass; ps += 2) {
-    const int n = (EPI == kEpiSwiGLU) ? (n0 >> 1) + ps * 64 : n0 + ps * kPassCols;   // output column in the group
+    const int n = (EPI == kEpiSwiGLU) ? (n0 >> 1) + ps * 64 : n0 + ps * pass_cols;   // output column in the group
     uint32_t w[32];                                                // 128 bytes of this row's output
     __syncwarp();
     if constexpr (EPI == kEpiSwiGLU) {
@@ -109,8 +112,30 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
           args.rope_tab + size_t(row_ok ? args.tok_pos[row_local] : 0) * (args.dh >> 1) + i0);
       float4 cs4[16];
 #pragma unroll
-      for (int m = 0; m < 16; ++m) cs4[m] = rotate ? __ldg(tab + m) : make_float4(1.f, 0.f, 1.f, 0.f);
+      for (int m = 0; m < 16; ++m) cs4[m] = (rotate && (m < 8 || !narrow)) ? __ldg(tab + m) : make_float4(1.f, 0.f, 1.f, 0.f);
       uint32_t r[32];
+      if (narrow) {
+        // 32 packed columns = 16 pairs: the first 32 bytes of the staged row are the first-half columns, the next 32
+        // bytes their partners; the rest of the row is unused
+        tmem_ld32(taddr + ps * 32, r);
+        tmem_ld_wait();
+        float lo[16], hi[16];
+#pragma unroll
+        for (int m = 0; m < 16; ++m) {
+          const float a = __uint_as_float(r[2 * m]) * scale, b = __uint_as_float(r[2 * m + 1]) * scale;
+          const float4 c4 = cs4[m >> 1];
+          const float cx = (m & 1) ? c4.z : c4.x, cy = (m & 1) ? c4.w : c4.y;
+          lo[m] = a * cx - b * cy;
+          hi[m] = b * cx + a * cy;
+        }
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          w[m] = pack_bf16(lo[2 * m], lo[2 * m + 1]);
+          w[8 + m] = pack_bf16(hi[2 * m], hi[2 * m + 1]);
+          w[16 + m] = 0u;
+          w[24 + m] = 0u;
+        }
+      } else
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
         tmem_ld32(taddr + ps * 64 + hf * 32, r);
@@ -192,10 +217,13 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
         if constexpr (EPI == kEpiQKV) {
           const int tok = grow - group_row0;
           // natural column inside the head of this lane's 8 values: chunks 0-3 first half, 4-7 second half
-          const int hcol = ((n % args.dh) >> 1) + (wr_chunk & 3) * 8 + (wr_chunk >> 2) * (args.dh >> 1);
+          // (32-column passes: chunks 0-1 first half, 2-3 second half, 4-7 nothing)
+          if (narrow && wr_chunk >= 4) continue;
+          const int hcol = narrow ? ((n % args.dh) >> 1) + (wr_chunk & 1) * 8 + (wr_chunk >> 1) * (args.dh >> 1)
+                                  : ((n % args.dh) >> 1) + (wr_chunk & 3) * 8 + (wr_chunk >> 2) * (args.dh >> 1);
           if (n < args.q_cols) {
             const int head = group * (args.q_cols / args.dh) + n / args.dh;
-            *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + size_t(tok) * args.ldo + head * args.dh + hcol) = v;
+            *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + size_t(tok) * args.ldo + head * args.q_head_stride + hcol) = v;
           } else {
             const bool is_k = n < args.q_cols + args.kv_cols;
             const int nn = n - args.q_cols - (is_k ? 0 : args.kv_cols);

@@ -85,7 +85,8 @@ struct AttnArgs {
   const int* q_lens;        // [n_seqs] or nullptr (1 each)
   const int* block_table;   // [n_seqs][max_pages_per_seq]
   int n_seqs, max_pages_per_seq, num_pages;
-  int n_q, n_kv, dh;
+  int n_q, n_kv, dh;        // dh: the real head_dim (64, 96 or 128); kernels are instantiated for 64 and 128 and read
+                            // a 96-wide head zero-padded: q with a head stride of 128, K/V through the tensor maps
   int max_q_len;
   float scale_log2;         // log2(e) / sqrt(dh)
   int* status;
@@ -121,6 +122,7 @@ struct SmallMArgs {
   void* out; int ldo;
   float rms_eps;            // kEpiQKV: 1/rms of every activation row is computed from the staged rows themselves
   int q_cols, kv_cols, dh, n_kv;   // kEpiQKV: see GemmArgs (interleaved heads, RoPE, q -> out, k / v -> pages)
+  int q_head_stride;
   const float2* rope_tab; const int* tok_pos; const int* tok_slot; bf16* k_pages; bf16* v_pages;
   const bf16* xsum; int x_count; size_t x_stride; float out_scale;
   int* status;

@@ -73,7 +73,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
   uint64_t* empty = full + kSmStages;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int slabs_per_group = a.N / kSmSlab;
+  const int slabs_per_group = (a.N + kSmSlab - 1) / kSmSlab;    // the last slab of a group may be partly past its rows
   const int chunks = a.group_offsets ? 1 : (a.rows_per_group + kSmRows - 1) / kSmRows;
   const int n_tasks = a.n_groups * slabs_per_group * chunks;
   const int k_steps = a.K / kSmKStep;
@@ -248,6 +248,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
         const int r = m0 + nt * 8 + t4 * 2 + e;              // logical row inside the group
         if (r >= rows) continue;
         const float va = c[nt][e], vb = c[nt][2 + e];
+        if (EPI != kEpiSwiGLU && n_a >= a.N) continue;       // (both columns of a thread lie on the same side of the end)
         if (EPI == kEpiSwiGLU) {
           const float h = __fdividef(va, 1.0f + __expf(-va)) * vb;
           static_cast<bf16*>(a.out)[size_t(out_row0 + r) * a.ldo + n_a] = __float2bfloat16_rn(h);
@@ -271,7 +272,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
           }
           if (is_q) {
             const int head = group * (a.q_cols / a.dh) + n_a / a.dh;
-            bf16* o = static_cast<bf16*>(a.out) + size_t(tok) * a.ldo + head * a.dh;
+            bf16* o = static_cast<bf16*>(a.out) + size_t(tok) * a.ldo + head * a.q_head_stride;
             o[i] = __float2bfloat16_rn(lo);
             o[i + half] = __float2bfloat16_rn(hi);
           } else {
@@ -319,7 +320,7 @@ static void launch_one(const CUtensorMap& tmW, const SmallMArgs& a, int n_sms, c
     configured = true;
   }
   const int chunks = a.group_offsets ? 1 : (a.rows_per_group + kSmRows - 1) / kSmRows;
-  const long long tasks = (long long)a.n_groups * (a.N / kSmSlab) * chunks;
+  const long long tasks = (long long)a.n_groups * ((a.N + kSmSlab - 1) / kSmSlab) * chunks;
   if (tasks <= 0) return;
   const int grid = int(tasks < 2LL * n_sms ? tasks : 2LL * n_sms);          // two resident CTAs per SM
   smallm_kernel<EPI><<<grid, kSmThreads, sm_smem_bytes<EPI>(), st>>>(tmW, a);

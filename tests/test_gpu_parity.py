@@ -94,6 +94,28 @@ def test_head_dim_128_and_ragged_tiles():
     run_block_parity(shape, 14, [130, 300, 63, 65], [0, 0, 0, 0], wscale=4.0)       # several 128-row tiles + tails
 
 
+def test_head_dim_96_prefill_and_decode():
+    """head_dim 96 (the paper's 1B model): the attention kernels work on heads zero-padded to 128, the projection
+    epilogues on 32-column passes."""
+    shape = synth.LayerShape(256, 4, 2, 2, 96, 4, 2, 128)
+    run_block_parity(shape, 31, [130, 70, 1, 200], [0, 64, 300, 0], wscale=4.0)
+    run_block_parity(shape, 32, [1] * 5, [0, 63, 64, 200, 1500], decode=True, wscale=4.0)
+    for position in ("first", "last"):
+        sh = synth.LayerShape(256, 4, 2, 2, 96, 4, 2, 128, position=position)
+        run_block_parity(sh, 33, [90, 41], [0, 10], wscale=4.0)
+
+
+def test_paper_1b_layer_shape_prefill_and_decode():
+    """Layer shape of the paper's 1B model (Table 8): hidden 768, 8 query / 8 KV heads of 96, 8 groups x 8 experts
+    top-1, intermediate 384, rope theta 5e5.  One query and one KV head per group: 288 projection columns per group,
+    not a multiple of the 64-row slabs and 64-column passes used elsewhere."""
+    shape = synth.LayerShape(768, 8, 8, 8, 96, 8, 1, 384, rope_theta=5.0e5)
+    r = run_block_parity(shape, 34, [700, 333, 129], [0, 0, 64])
+    print("1B shape prefill:", {k: r[k] for k in ("max_abs", "rel_l1", "flips")})
+    r = run_block_parity(shape, 35, [1] * 6, [0, 100, 1000, 2047, 2048, 3000], decode=True)
+    print("1B shape decode:", {k: r[k] for k in ("max_abs", "rel_l1", "flips")})
+
+
 def test_chunked_prefill_over_cached_context():
     shape = shape_small()
     run_block_parity(shape, 15, [40, 17, 130], [100, 64, 1], wscale=4.0)
