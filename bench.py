@@ -362,11 +362,16 @@ def measure(kind, args, dist_on, rank, world, peaks, with_cpu):
 
 
 def run_sweep(args):
-    """Latency of one block at the paper's 7B layer shape for the token-batch sizes of its forward-latency table
+    """Latency of one block at the paper's 7B (or 1B) layer shape for the token-batch sizes of its forward-latency table
     (1 ... 24,576 tokens, as sequences of at most 2,048 tokens), on one GPU.  Context for that table's shape only:
     the paper's numbers are whole 16-layer models on 8 H100s."""
     from paper_2605_06206_b200 import binding
-    shape = synth.LayerShape(2048, 16, 8, 8, 128, 8, 1, 1024, rope_theta=5.0e5)
+    if args.sweep_shape == "1b":
+        shape = synth.LayerShape(768, 8, 8, 8, 96, 8, 1, 384, rope_theta=5.0e5)
+        desc = "paper 1B layer shape (hidden 768, 8q/8kv heads of 96, 8 groups x 8 experts top-1, inter 384)"
+    else:
+        shape = synth.LayerShape(2048, 16, 8, 8, 128, 8, 1, 1024, rope_theta=5.0e5)
+        desc = "paper 7B layer shape (hidden 2048, 16q/8kv, 8 groups x 8 experts top-1, inter 1024)"
     W = synth.make_weights(shape, 7, "cuda")
     sizes = [1, 64, 128, 256, 512, 1024, 2048, 4096, 8192, 12288, 16384, 24576]
     layer = binding.FoeLayer(shape, W, max_tokens=max(sizes), max_seqs=16, max_context=2048)
@@ -381,8 +386,7 @@ def run_sweep(args):
         rows.append(dict(tokens=S, ms_per_block=ms, tokens_per_s=S / (ms * 1e-3)))
     layer.close()
     print(json.dumps(dict(metric="foe_block_latency_sweep", unit="ms", data="synthetic", dtype="bf16",
-                          config=dict(workload="paper 7B layer shape (hidden 2048, 16q/8kv, 8 groups x 8 experts top-1, "
-                                               "inter 1024), prefill of S tokens in sequences of <= 2048"),
+                          config=dict(workload=desc + ", prefill of S tokens in sequences of <= 2048"),
                           steps=args.steps, warmup=args.warmup, sweep=rows)))
 
 
@@ -425,6 +429,7 @@ def main():
     ap.add_argument("--no-secondary", action="store_true", help="skip the other workload's measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle (profiler runs)")
     ap.add_argument("--sweep", action="store_true", help="token-batch latency sweep at the paper's 7B layer shape")
+    ap.add_argument("--sweep-shape", choices=["7b", "1b"], default="7b")
     ap.add_argument("--serve", action="store_true", help="request-level latency run (continuous batching on a 4-layer stack)")
     ap.add_argument("--requests", type=int, default=48)
     ap.add_argument("--rate", type=float, default=20.0, help="--serve: Poisson arrival rate, requests per second")
