@@ -212,7 +212,7 @@ class Engine:
 class FoeStackRunner:
     """forward() for Engine on a stack of FoE layers (first, middle..., last) with per-layer page pools.
 
-    One mixed batch = one foe_prefill per layer: sequences in scheduler order, their new tokens concatenated; the
+    One batch = one foe_prefill per layer (foe_decode when every sequence contributes a single token): sequences in scheduler order, their new tokens concatenated; the
     block table row of a sequence lists the pages reserved for the request."""
 
     def __init__(self, base_shape, n_layers: int, seed: int, num_pages: int, max_batch_tokens: int, max_seqs: int,
@@ -263,7 +263,8 @@ class FoeStackRunner:
         h = x
         for l, layer in enumerate(self.layers):
             kv = synth.PagedKV(self.k[l], self.v[l], bt, ctx, ql)
-            h = layer.prefill(h, kv, n_tokens=S, max_q_len=mq)
+            # an iteration of decode tokens only takes the decode entry point (split-KV attention, weight streaming)
+            h = layer.decode(h, kv) if mq == 1 else layer.prefill(h, kv, n_tokens=S, max_q_len=mq)
         e1.record()
         torch.cuda.synchronize()
         status = self.layers[0].poll_status()
