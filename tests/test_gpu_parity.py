@@ -53,6 +53,27 @@ def test_route_bit_exact(wl, n_tok, zipf):
         assert live.max() > 4 * max(1, live.min())                                          # skewed load
 
 
+def test_route_bit_exact_tensor_core_scores_odd_k_blocks():
+    """The tensor-core score kernel spreads the k-blocks over eight accumulators; hidden 768 gives 12 k-blocks (an
+    uneven spread), 8 experts per cluster the narrowest register top-k."""
+    shape = synth.LayerShape(768, 8, 8, 8, 96, 8, 1, 384)
+    W = synth.make_weights(shape, 41, "cuda")
+    n_tok = 2304
+    h = synth.normal_bf16(41, 77, (n_tok, shape.hidden), 1.5, 0.0, "cuda")
+    layer = binding.FoeLayer(shape, W, max_tokens=n_tok, max_seqs=1, max_context=64)
+    idx, w = layer.route(h)
+    assert layer.poll_status() == 0
+    aux = layer.aux()
+    layer.close()
+    cfg = adapter.cfg_from_shape(shape)
+    Wn = {k: adapter.to_np(W[k]) for k in ("ffn_norm_g", "router_w", "router_b")}
+    rt = orc.route(cfg, Wn, adapter.to_np(h))
+    exempt = check_routing(shape, idx.cpu().numpy(), w.cpu().numpy().astype(np.float64), rt["logits"], rt["idx"], rt["w"])
+    assert exempt <= n_tok // 200
+    assert np.abs(adapter.to_np(aux["logits"]) - rt["logits"]).max() <= 2e-5 * max(1.0, np.abs(rt["logits"]).max())
+    check_maps(shape, aux, idx.cpu().numpy())
+
+
 def test_route_is_deterministic():
     shape, info = synth.workload(1)
     W = synth.make_weights(shape, 0, "cuda")
