@@ -419,6 +419,55 @@ def run_serve(args):
                           **rep)))
 
 
+def run_stack(args):
+    """The 16-layer stack (first, 14 middle, last layer; hidden 4096, 32q/8kv heads, 8 clusters x 16 experts top-2,
+    inter 1408; 72 GB of weights): prefill of 2 x 16,384 tokens, then 128 decode steps on the caches it wrote, once as
+    FoE and once as the equal-size one-cluster MoE (128 experts, top-16) on the same kernels."""
+    import dataclasses
+    from paper_2605_06206_b200.stack import FoeStack
+    shape, info = synth.workload(5)
+    q_lens, L, steps = info["q_lens"], info["layers"], info.get("decode_steps", 128)
+    rows = []
+    for H in (shape.n_clusters, 1):
+        sh = shape if H != 1 else dataclasses.replace(shape, n_clusters=1, experts_per_cluster=128, top_k_per_cluster=16)
+        st = FoeStack(sh, L, info["seed"], q_lens, steps)
+        S = sum(q_lens)
+        x0 = synth.make_x(st.shapes[0], info["seed"], S, "cuda")
+        st.forward(x0, [0] * len(q_lens), decode=False)                      # warm-up (also writes the caches)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 3
+        e0.record()
+        for _ in range(reps):
+            st.forward(x0, [0] * len(q_lens), decode=False)
+        e1.record()
+        torch.cuda.synchronize()
+        prefill_ms = e0.elapsed_time(e1) / reps
+        xs = [synth.make_x(st.shapes[0], info["seed"], len(q_lens), "cuda", tid=synth.TID["x_step"] + s) for s in range(steps)]
+        ctx = list(q_lens)
+        for s in range(3):                                                   # warm-up steps (not counted)
+            st.forward(xs[s], ctx, decode=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for s in range(steps):
+            st.forward(xs[s], ctx, decode=True)
+            ctx = [c + 1 for c in ctx]
+        e1.record()
+        torch.cuda.synchronize()
+        decode_ms = e0.elapsed_time(e1) / steps
+        assert st.status() == 0
+        rows.append(dict(n_clusters=H, prefill_ms=prefill_ms, prefill_tokens_per_s=S / (prefill_ms * 1e-3),
+                         decode_ms_per_step=decode_ms, decode_tokens_per_s=len(q_lens) / (decode_ms * 1e-3)))
+        st.close()
+        del st, x0, xs
+        torch.cuda.empty_cache()
+    print(json.dumps(dict(metric="foe_stack_tokens_per_s", unit="tokens/s", data="synthetic", dtype="bf16",
+                          config=dict(workload="workload 5: 16-layer stack, hidden 4096, 32q/8kv heads, 8 clusters x 16 experts "
+                                               "top-2 (and 1 cluster x 128 experts top-16), inter 1408; prefill 2 x 16384 tokens, "
+                                               "then 128 decode steps (host tensor set-up of every step included)"),
+                          stacks=rows)))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -430,6 +479,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle (profiler runs)")
     ap.add_argument("--sweep", action="store_true", help="token-batch latency sweep at the paper's 7B layer shape")
     ap.add_argument("--sweep-shape", choices=["7b", "1b"], default="7b")
+    ap.add_argument("--stack", action="store_true", help="16-layer stack (workload 5): FoE and the one-cluster MoE twin")
     ap.add_argument("--serve", action="store_true", help="request-level latency run (continuous batching on a 4-layer stack)")
     ap.add_argument("--requests", type=int, default=48)
     ap.add_argument("--rate", type=float, default=20.0, help="--serve: Poisson arrival rate, requests per second")
@@ -451,6 +501,9 @@ def main():
         return
     if args.serve:
         run_serve(args)
+        return
+    if args.stack:
+        run_stack(args)
         return
     dist_on = replicas.init("nccl", torch.device("cuda", local))
     peaks = measured_peaks()
