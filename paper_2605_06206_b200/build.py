@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfoe.so")
-SOURCES = ["foe_api.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "smallm.cu", "route.cu", "router_tc.cu", "permute.cu", "elementwise.cu"]
+SOURCES = ["foe_api.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "smallm.cu", "route.cu", "router_tc.cu", "permute.cu", "elementwise.cu", "shard.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
          "-cudart", "static"]
 
@@ -17,7 +17,7 @@ def _stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(HERE, "..", "include", "foe.h"),
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(HERE, "..", "include", "foe.h"), os.path.join(HERE, "..", "include", "foe_shard.h"),
                                                                  os.path.abspath(__file__)]
     return any(os.path.getmtime(p) > t for p in deps)
 

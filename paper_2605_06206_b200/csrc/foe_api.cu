@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "../../include/foe.h"
+#include "../../include/foe_shard.h"
 #include "kernels.h"
 
 using namespace foe;
@@ -82,12 +83,38 @@ struct foe_layer {
   // call state
   cudaStream_t last_stream;
   int last_tokens, launches;
+  bool last_decode;
+  int shard_stage;       // 0: no sharded call in flight; 1: foe_shard_attend done, foe_shard_ffn owed
   int profiling;
   cudaEvent_t ev[kNumStages + 1];
   bool ev_valid;
 };
 
+// One rank's end of the exchange of a cluster-per-GPU group.
+struct foe_shard {
+  foe_shard_config cfg;
+  int span;                         // columns each rank owns
+  size_t S_cap;
+  uint8_t* buf[8];                  // every rank's exchange buffer as seen from here
+  ShardPeerTable table;
+  unsigned int epoch;               // exchanges started
+  unsigned int slot_expect, gather_expect;   // running totals the counters must reach for the current exchange
+  int S;                            // tokens of the current exchange
+  int stage;                        // 0 idle, 1 pushed, 2 reduced
+  int* status;
+  unsigned long long limit_ns;
+  cudaStream_t last_stream;
+};
+
 namespace {
+
+constexpr size_t kShardHeaderBytes = 1024;       // slot counters at 0, gather counters at 128
+
+bool shard_config_ok(const foe_shard_config* c) {
+  return c && c->n_ranks >= 1 && c->n_ranks <= 8 && c->rank >= 0 && c->rank < c->n_ranks && c->hidden > 0 &&
+         c->hidden % (32 * c->n_ranks) == 0 && c->max_tokens > 0 && c->wait_limit_ms >= 0;
+}
+size_t shard_slots_bytes(const foe_shard_config* c) { return size_t(2) * c->max_tokens * c->hidden * sizeof(bf16); }
 
 template <typename T>
 bool dalloc(foe_layer* L, T** p, size_t count) {
@@ -156,11 +183,15 @@ void run_route_and_permute(foe_layer* L, const void* r, int r_is_bf16, int n, cu
   L->launches += launch_permute(L->ws->topk_idx, L->ws->pb, n, L->H * L->kc, L->E, L->ws->status, st);
 }
 
-foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* out, cudaStream_t st, bool decode) {
+// Attention half of the block: token map, QKV projection, attention core, output projection.  With `sh` the
+// O-projection's result is this rank's partial of the synced residual and goes to the column owners' receive
+// slots; otherwise it is r_full itself, in the workspace.
+foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaStream_t st, bool decode, foe_shard* sh) {
   const int S = decode ? kv->n_seqs : kv->n_tokens;
   L->last_stream = st;
   L->launches = 0;
   L->last_tokens = S;
+  L->last_decode = decode;
   L->ev_valid = false;
   if (S == 0) return FOE_OK;
   const int H = L->H, d = L->d, dh = L->dh;
@@ -226,28 +257,54 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
 
   // ---- output projection; the cross-cluster sync is its K-reduction plus the sum of x[h] in the epilogue
   stage_mark(L, kStOproj, st);
-  const float out_scale = (L->first || L->cfg.sync == FOE_SYNC_SUM) ? 1.0f : 1.0f / float(H);
+  // one device: r_full = (sum_h (x[h] + Attn_h W_O[h])) / H, with the sum over h inside the GEMM's K loop.
+  // one rank of a group: the partial (x[h] + Attn_h W_O[h]) / H; a first layer's shared x comes from rank 0 alone.
+  float out_scale = (L->first || L->cfg.sync == FOE_SYNC_SUM) ? 1.0f : 1.0f / float(H);
+  int x_count = L->first ? 1 : H;
+  if (sh) {
+    out_scale = (L->first || L->cfg.sync == FOE_SYNC_SUM) ? 1.0f : 1.0f / float(sh->cfg.n_ranks);
+    x_count = (L->first && sh->cfg.rank != 0) ? 0 : 1;
+  }
+  const long long slot_off = sh ? (long long)((size_t(sh->epoch & 1) * sh->cfg.n_ranks + sh->cfg.rank) * sh->S_cap * sh->span) : 0;
   if (!decode) {
     GemmArgs ga;
     memset(&ga, 0, sizeof(ga));
     ga.n_groups = 1; ga.rows_per_group = S; ga.a_group_stride = 0; ga.N = d; ga.K = L->n_q * dh; ga.status = L->ws->status;
-    ga.out = L->ws->r_full; ga.ldo = d; ga.xsum = xb; ga.x_count = L->first ? 1 : H; ga.x_stride = size_t(S) * d;
+    ga.out = L->ws->r_full; ga.ldo = d; ga.xsum = xb; ga.x_count = x_count; ga.x_stride = size_t(S) * d;
     ga.out_scale = out_scale;
+    if (sh) {     // the epilogue stores each tile straight into the owners' slots
+      for (int o = 0; o < sh->cfg.n_ranks; ++o) { ga.push_base[o] = sh->table.slots[o]; ga.push_cnt[o] = sh->table.slot_cnt[o]; }
+      ga.push_span = sh->span;
+      ga.push_slot_off = slot_off;
+    }
     launch_gemm(kEpiOProj, L->ws->tm_attn_o, L->tm_wo, ga, L->n_sms, st);
   } else {
     SmallMArgs sa;
     memset(&sa, 0, sizeof(sa));
     sa.W = L->wo_t; sa.X = L->ws->attn_o; sa.ldx = L->n_q * dh; sa.n_groups = 1; sa.rows_per_group = S; sa.N = d;
-    sa.K = L->n_q * dh; sa.epi = kEpiOProj; sa.out = L->ws->r_full; sa.ldo = d; sa.xsum = xb; sa.x_count = L->first ? 1 : H;
+    sa.K = L->n_q * dh; sa.epi = kEpiOProj; sa.out = L->ws->r_full; sa.ldo = d; sa.xsum = xb; sa.x_count = x_count;
     sa.x_stride = size_t(S) * d; sa.out_scale = out_scale; sa.status = L->ws->status;
     launch_smallm(L->tms_wo, sa, L->n_sms, st);
+    if (sh) {     // a decode step's partial is a few hundred KB: one more launch pushes it
+      launch_shard_push(L->ws->r_full, 1, 1.0f, S, d, sh->cfg.n_ranks, sh->table, slot_off, st);
+      L->launches += 1;
+    }
   }
   L->launches += 1;
+  return check_launch();
+}
+
+// FFN half of the block on the synced residual in the workspace: routing, dispatch maps, experts, combine.
+foe_status run_ffn(foe_layer* L, void* out, cudaStream_t st) {
+  const int S = L->last_tokens, H = L->H, d = L->d;
+  const bool decode = L->last_decode;
+  if (S == 0) return FOE_OK;
 
   // ---- router, top-k, gates, dispatch maps
   stage_mark(L, kStRoute, st);
   run_route_and_permute(L, L->ws->r_full, 0, S, st);
   const int R = S * H * L->kc;
+  (void)R;
 
   if (!decode) {
     stage_mark(L, kStGemm1, st);
@@ -287,6 +344,27 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
   L->launches += 1;
   if (L->profiling) { cudaEventRecord(L->ev[kNumStages], st); L->ev_valid = true; }
   return check_launch();
+}
+
+foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* out, cudaStream_t st, bool decode) {
+  L->shard_stage = 0;
+  const foe_status a = run_attend(L, x, kv, st, decode, nullptr);
+  if (a != FOE_OK) return a;
+  return run_ffn(L, out, st);
+}
+
+// argument checks shared by foe_prefill / foe_decode and foe_shard_attend (x and out are checked by the callers)
+foe_status check_call(const foe_layer* L, const foe_kv_cache* kv, bool decode) {
+  if (!kv->k_pages || !kv->v_pages || !kv->block_table || !kv->context_lens) return FOE_ERR_NULL;
+  if (decode) {
+    if (kv->n_seqs > L->cfg.max_seqs || kv->max_pages_per_seq <= 0 || kv->num_pages <= 0) return FOE_ERR_SHAPE;
+    return FOE_OK;
+  }
+  if (!kv->q_lens) return FOE_ERR_NULL;
+  if (kv->n_tokens > L->cfg.max_tokens || kv->n_seqs > L->cfg.max_seqs || kv->n_seqs == 0) return FOE_ERR_SHAPE;
+  if (kv->max_q_len <= 0 || kv->max_q_len > kv->n_tokens || kv->max_pages_per_seq <= 0 || kv->num_pages <= 0)
+    return FOE_ERR_SHAPE;
+  return FOE_OK;
 }
 
 }  // namespace
@@ -485,10 +563,8 @@ foe_status foe_prefill(foe_layer* L, const void* x, const foe_kv_cache* kv, void
   if (kv->n_tokens < 0 || kv->n_seqs < 0) return FOE_ERR_SHAPE;
   if (kv->n_tokens == 0) { L->launches = 0; L->last_tokens = 0; return FOE_OK; }
   if (!x || !out) return FOE_ERR_NULL;
-  if (!kv->k_pages || !kv->v_pages || !kv->block_table || !kv->context_lens || !kv->q_lens) return FOE_ERR_NULL;
-  if (kv->n_tokens > L->cfg.max_tokens || kv->n_seqs > L->cfg.max_seqs || kv->n_seqs == 0) return FOE_ERR_SHAPE;
-  if (kv->max_q_len <= 0 || kv->max_q_len > kv->n_tokens || kv->max_pages_per_seq <= 0 || kv->num_pages <= 0)
-    return FOE_ERR_SHAPE;
+  const foe_status c = check_call(L, kv, false);
+  if (c != FOE_OK) return c;
   if (x == out) return FOE_ERR_UNSUPPORTED;
   return run_block(L, x, kv, out, static_cast<cudaStream_t>(stream), false);
 }
@@ -498,8 +574,8 @@ foe_status foe_decode(foe_layer* L, const void* x, const foe_kv_cache* kv, void*
   if (kv->n_seqs < 0) return FOE_ERR_SHAPE;
   if (kv->n_seqs == 0) { L->launches = 0; L->last_tokens = 0; return FOE_OK; }
   if (!x || !out) return FOE_ERR_NULL;
-  if (!kv->k_pages || !kv->v_pages || !kv->block_table || !kv->context_lens) return FOE_ERR_NULL;
-  if (kv->n_seqs > L->cfg.max_seqs || kv->max_pages_per_seq <= 0 || kv->num_pages <= 0) return FOE_ERR_SHAPE;
+  const foe_status c = check_call(L, kv, true);
+  if (c != FOE_OK) return c;
   if (x == out) return FOE_ERR_UNSUPPORTED;
   return run_block(L, x, kv, out, static_cast<cudaStream_t>(stream), true);
 }
@@ -575,6 +651,193 @@ foe_status foe_get_stage_ms(foe_layer* L, float* ms, int n) {
   if (cudaEventSynchronize(L->ev[kNumStages]) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
   for (int i = 0; i < kNumStages; ++i)
     if (cudaEventElapsedTime(&ms[i], L->ev[i], L->ev[i + 1]) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  return FOE_OK;
+}
+
+// ------------------------------------------------------------------ cluster-per-GPU group (include/foe_shard.h)
+
+size_t foe_shard_buffer_bytes(const foe_shard_config* c) {
+  if (!shard_config_ok(c)) return 0;
+  return kShardHeaderBytes + 2 * shard_slots_bytes(c);       // slots and gather buffer have the same size
+}
+
+foe_status foe_shard_buffer_alloc(const foe_shard_config* c, void** buffer) {
+  if (!c || !buffer) return FOE_ERR_NULL;
+  *buffer = nullptr;
+  const size_t bytes = foe_shard_buffer_bytes(c);
+  if (bytes == 0) return FOE_ERR_CONFIG;
+  void* p = nullptr;
+  if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_OOM; }
+  if (cudaMemset(p, 0, bytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+    cudaGetLastError();
+    cudaFree(p);
+    return FOE_ERR_CUDA;
+  }
+  *buffer = p;
+  return FOE_OK;
+}
+
+foe_status foe_shard_buffer_free(void* buffer) {
+  if (buffer && cudaFree(buffer) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  return FOE_OK;
+}
+
+foe_status foe_shard_buffer_export(void* buffer, unsigned char handle[64]) {
+  if (!buffer || !handle) return FOE_ERR_NULL;
+  static_assert(sizeof(cudaIpcMemHandle_t) == 64, "IPC handle size");
+  cudaIpcMemHandle_t h;
+  if (cudaIpcGetMemHandle(&h, buffer) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  memcpy(handle, &h, sizeof(h));
+  return FOE_OK;
+}
+
+foe_status foe_shard_buffer_import(const unsigned char handle[64], void** buffer) {
+  if (!handle || !buffer) return FOE_ERR_NULL;
+  *buffer = nullptr;
+  cudaIpcMemHandle_t h;
+  memcpy(&h, handle, sizeof(h));
+  void* p = nullptr;
+  if (cudaIpcOpenMemHandle(&p, h, cudaIpcMemLazyEnablePeerAccess) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  *buffer = p;
+  return FOE_OK;
+}
+
+foe_status foe_shard_buffer_close(void* imported) {
+  if (imported && cudaIpcCloseMemHandle(imported) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  return FOE_OK;
+}
+
+foe_status foe_shard_create(const foe_shard_config* c, void* const* buffers, foe_shard** out) {
+  if (!c || !buffers || !out) return FOE_ERR_NULL;
+  *out = nullptr;
+  if (!shard_config_ok(c)) return FOE_ERR_CONFIG;
+  for (int r = 0; r < c->n_ranks; ++r)
+    if (!buffers[r]) return FOE_ERR_NULL;
+  foe_shard* sh = new (std::nothrow) foe_shard();
+  if (!sh) return FOE_ERR_OOM;
+  sh->cfg = *c;
+  sh->span = c->hidden / c->n_ranks;
+  sh->S_cap = size_t(c->max_tokens);
+  sh->limit_ns = (unsigned long long)(c->wait_limit_ms > 0 ? c->wait_limit_ms : 2000) * 1000000ull;
+  for (int r = 0; r < c->n_ranks; ++r) {
+    uint8_t* b = static_cast<uint8_t*>(buffers[r]);
+    sh->buf[r] = b;
+    sh->table.slots[r] = reinterpret_cast<bf16*>(b + kShardHeaderBytes);
+    sh->table.gather[r] = reinterpret_cast<bf16*>(b + kShardHeaderBytes + shard_slots_bytes(c));
+    sh->table.slot_cnt[r] = reinterpret_cast<unsigned int*>(b) + c->rank;        // rank r's counter of MY pushes
+    sh->table.gather_cnt[r] = reinterpret_cast<unsigned int*>(b + 128);          // rank r's counters, one per owner
+  }
+  if (cudaMalloc(reinterpret_cast<void**>(&sh->status), sizeof(int)) != cudaSuccess) { cudaGetLastError(); delete sh; return FOE_ERR_OOM; }
+  cudaMemset(sh->status, 0, sizeof(int));
+  *out = sh;
+  return FOE_OK;
+}
+
+foe_status foe_shard_destroy(foe_shard* sh) {
+  if (!sh) return FOE_OK;
+  cudaFree(sh->status);
+  delete sh;
+  return FOE_OK;
+}
+
+// starts exchange number epoch + 1 for S tokens: buffer half and the totals its counters will have to reach
+static foe_status shard_begin(foe_shard* sh, int S, cudaStream_t st) {
+  if (sh->stage != 0) return FOE_ERR_UNSUPPORTED;
+  if (S < 0 || S > sh->cfg.max_tokens) return FOE_ERR_SHAPE;
+  sh->epoch += 1;
+  sh->S = S;
+  sh->slot_expect += unsigned(S) * unsigned(sh->span);
+  sh->gather_expect += unsigned(S) * unsigned(sh->span);
+  sh->stage = 1;
+  sh->last_stream = st;
+  return FOE_OK;
+}
+
+foe_status foe_shard_attend(foe_layer* L, foe_shard* sh, const void* x, const foe_kv_cache* kv, int decode, void* stream) {
+  if (!L || !sh || !kv) return FOE_ERR_NULL;
+  if (L->H != 1 || L->d != sh->cfg.hidden) return FOE_ERR_CONFIG;
+  if (kv->n_tokens < 0 || kv->n_seqs < 0) return FOE_ERR_SHAPE;
+  const int S = decode ? kv->n_seqs : kv->n_tokens;
+  if (S > 0) {
+    if (!x) return FOE_ERR_NULL;
+    const foe_status c = check_call(L, kv, decode != 0);
+    if (c != FOE_OK) return c;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const foe_status b = shard_begin(sh, S, st);
+  if (b != FOE_OK) return b;
+  L->shard_stage = 1;
+  if (S == 0) { L->launches = 0; L->last_tokens = 0; return FOE_OK; }
+  return run_attend(L, x, kv, st, decode != 0, sh);
+}
+
+foe_status foe_shard_push(foe_shard* sh, const void* src, int n_tokens, float scale, void* stream) {
+  if (!sh) return FOE_ERR_NULL;
+  if (n_tokens > 0 && !src) return FOE_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const foe_status b = shard_begin(sh, n_tokens, st);
+  if (b != FOE_OK) return b;
+  if (n_tokens == 0) return FOE_OK;
+  const long long slot_off = (long long)((size_t(sh->epoch & 1) * sh->cfg.n_ranks + sh->cfg.rank) * sh->S_cap * sh->span);
+  launch_shard_push(src, 0, scale, n_tokens, sh->cfg.hidden, sh->cfg.n_ranks, sh->table, slot_off, st);
+  return check_launch();
+}
+
+foe_status foe_shard_reduce(foe_shard* sh, void* stream) {
+  if (!sh) return FOE_ERR_NULL;
+  if (sh->stage != 1) return FOE_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  sh->stage = 2;
+  sh->last_stream = st;
+  if (sh->S == 0) return FOE_OK;
+  const int H = sh->cfg.n_ranks, me = sh->cfg.rank;
+  const size_t half = size_t(sh->epoch & 1);
+  const bf16* my_slots = sh->table.slots[me] + half * H * sh->S_cap * sh->span;
+  const unsigned int* my_cnt = reinterpret_cast<const unsigned int*>(sh->buf[me]);
+  launch_shard_reduce(my_slots, my_cnt, sh->slot_expect, sh->S, sh->S_cap, sh->cfg.hidden, H, me, sh->table,
+                      (long long)(half * sh->S_cap * sh->cfg.hidden), sh->limit_ns, sh->status, st);
+  return check_launch();
+}
+
+static foe_status shard_finish(foe_shard* sh, float* dst_f32, bf16* dst_bf16, cudaStream_t st) {
+  if (sh->stage != 2) return FOE_ERR_UNSUPPORTED;
+  sh->stage = 0;
+  sh->last_stream = st;
+  if (sh->S == 0) return FOE_OK;
+  const int me = sh->cfg.rank;
+  const bf16* my_gather = sh->table.gather[me] + size_t(sh->epoch & 1) * sh->S_cap * sh->cfg.hidden;
+  launch_shard_gather(my_gather, sh->table.gather_cnt[me], sh->gather_expect, sh->S, sh->cfg.hidden, sh->cfg.n_ranks,
+                      dst_f32, dst_bf16, sh->limit_ns, sh->status, st);
+  return check_launch();
+}
+
+foe_status foe_shard_ffn(foe_layer* L, foe_shard* sh, void* out, void* stream) {
+  if (!L || !sh) return FOE_ERR_NULL;
+  if (L->shard_stage != 1 || L->last_tokens != sh->S) return FOE_ERR_UNSUPPORTED;
+  if (sh->S > 0 && !out) return FOE_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const foe_status f = shard_finish(sh, L->ws->r_full, nullptr, st);      // r_full of the whole group, as fp32
+  if (f != FOE_OK) return f;
+  L->shard_stage = 0;
+  L->last_stream = st;
+  if (sh->S == 0) return FOE_OK;
+  L->launches += 1;
+  return run_ffn(L, out, st);
+}
+
+foe_status foe_shard_gather(foe_shard* sh, void* dst, void* stream) {
+  if (!sh) return FOE_ERR_NULL;
+  if (sh->S > 0 && !dst) return FOE_ERR_NULL;
+  return shard_finish(sh, nullptr, static_cast<bf16*>(dst), static_cast<cudaStream_t>(stream));
+}
+
+foe_status foe_shard_poll_status(foe_shard* sh, int* device_status) {
+  if (!sh || !device_status) return FOE_ERR_NULL;
+  if (cudaStreamSynchronize(sh->last_stream) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  int v = 0;
+  if (cudaMemcpy(&v, sh->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FOE_ERR_CUDA;
+  *device_status = v;
+  if (v != 0) cudaMemset(sh->status, 0, sizeof(int));
   return FOE_OK;
 }
 

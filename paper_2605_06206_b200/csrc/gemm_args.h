@@ -68,6 +68,15 @@ struct GemmArgs {
   int x_count;
   size_t x_stride;
   float out_scale;
+  // kEpiOProj on one rank of a cluster-per-GPU group (push_span != 0): the scaled tile is not written to `out` but
+  // pushed as bf16 to the rank that owns its columns -- columns [o * push_span, (o + 1) * push_span) belong to rank
+  // o -- at push_base[o] + push_slot_off + row * push_span + (column - o * push_span); push_cnt[o] then grows by
+  // the number of elements written (after a system-scope fence), which is what the owner's reduction waits for.
+  // The pointers are this rank's mappings of the owners' buffers (peer memory, or plain local memory).
+  __nv_bfloat16* push_base[8];
+  unsigned int* push_cnt[8];
+  int push_span;
+  long long push_slot_off;
 };
 
 }  // namespace foe

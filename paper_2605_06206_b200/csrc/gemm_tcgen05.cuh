@@ -79,6 +79,17 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
   const int n_pass = (EPI == kEpiSwiGLU) ? 2 : (tile_cols + pass_cols - 1) / pass_cols;
   const int wr_row = lane >> 3, wr_chunk = lane & 7;                // write-out role: row (+4j), 16-byte chunk
   if (half >= n_pass) { release(); return; }                        // nothing for this warp in a one-pass tile
+  // pushed O-proj tiles: elements this warp has written to the current owner since its last counter update
+  int push_owner = -1;
+  unsigned int push_n = 0;
+  auto push_flush = [&]() {
+    if (push_n) {
+      __threadfence_system();                                       // every lane: its stores before the count
+      __syncwarp();
+      if (lane == 0) atomicAdd_system(args.push_cnt[push_owner], push_n);
+      push_n = 0;
+    }
+  };
 #pragma unroll 1
   for (int ps = half; ps < n_pass; ps += 2) {
     const int n = (EPI == kEpiSwiGLU) ? (n0 >> 1) + ps * 64 : n0 + ps * pass_cols;   // output column in the group
@@ -202,10 +213,25 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
 #pragma unroll
           for (int q = 0; q < 4; ++q) { a8[2 * q] += bf16_lo(w4[q]); a8[2 * q + 1] += bf16_hi(w4[q]); }
         }
-        float* dst = static_cast<float*>(args.out) + size_t(grow) * args.ldo + n + or_cg * 8;
         const float sc = args.out_scale;
-        *reinterpret_cast<float4*>(dst) = make_float4(a8[0] * sc, a8[1] * sc, a8[2] * sc, a8[3] * sc);
-        *reinterpret_cast<float4*>(dst + 4) = make_float4(a8[4] * sc, a8[5] * sc, a8[6] * sc, a8[7] * sc);
+        if (args.push_span) {
+          // the 32 columns of a pass lie inside one owner's span (a multiple of 32)
+          const int owner = n / args.push_span;
+          __nv_bfloat16* dst = args.push_base[owner] + args.push_slot_off + size_t(grow) * args.push_span +
+                               (n - owner * args.push_span) + or_cg * 8;
+          *reinterpret_cast<uint4*>(dst) = make_uint4(pack_bf16(a8[0] * sc, a8[1] * sc), pack_bf16(a8[2] * sc, a8[3] * sc),
+                                                      pack_bf16(a8[4] * sc, a8[5] * sc), pack_bf16(a8[6] * sc, a8[7] * sc));
+        } else {
+          float* dst = static_cast<float*>(args.out) + size_t(grow) * args.ldo + n + or_cg * 8;
+          *reinterpret_cast<float4*>(dst) = make_float4(a8[0] * sc, a8[1] * sc, a8[2] * sc, a8[3] * sc);
+          *reinterpret_cast<float4*>(dst + 4) = make_float4(a8[4] * sc, a8[5] * sc, a8[6] * sc, a8[7] * sc);
+        }
+      }
+      if (args.push_span) {
+        const int owner = n / args.push_span;
+        if (owner != push_owner) { push_flush(); push_owner = owner; }
+        const int rows_here = min(32, max(0, row_end - (row0 + quarter * 32)));
+        push_n += unsigned(rows_here) * 32u;
       }
     } else {
 #pragma unroll
@@ -241,6 +267,7 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
       }
     }
   }
+  if constexpr (EPI == kEpiOProj) push_flush();
 }
 
 template <int EPI, bool GATHER>

@@ -130,4 +130,29 @@ struct SmallMArgs {
 // tmW: tensor map of W as [n_groups*N][K] with 64-column boxes of 64 rows (32 rows for the SwiGLU packing)
 void launch_smallm(const CUtensorMap& tmW, const SmallMArgs& a, int n_sms, cudaStream_t st);
 
+// ---- shard.cu  (sync of a cluster-per-GPU group over peer memory)
+// This rank's mappings of every rank's exchange buffer: receive slots ([2][H][S_cap][d/H] bf16), gather buffer
+// ([2][S_cap][d] bf16), arrival counters of the slots ([H], one per source) and of the gather buffer ([H], one per owner).
+struct ShardPeerTable {
+  bf16* slots[8];
+  bf16* gather[8];
+  unsigned int* slot_cnt[8];      // slot_cnt[o]: the counter on rank o that counts THIS rank's pushes
+  unsigned int* gather_cnt[8];    // gather_cnt[p]: rank p's array of H counters (indexed by owner)
+};
+// src ([S][d] bf16 or fp32) * scale -> bf16 into this rank's slot on every owner; slot_off = element offset of that
+// slot ((parity * H + rank) * S_cap * (d/H)).  Adds S * d/H to every slot_cnt[o].
+void launch_shard_push(const void* src, int src_is_f32, float scale, int S, int d, int H, const ShardPeerTable& t,
+                       long long slot_off, cudaStream_t st);
+// waits until my_slot_cnt[0..H) reached `expect`, sums the H slots (my_slots = this parity's [H][S_cap][d/H]) and
+// writes the bf16 result to gather[p] + gather_off + row * d + rank * d/H of every rank p; adds S * d/H to
+// gather_cnt[p][rank].
+void launch_shard_reduce(const bf16* my_slots, const unsigned int* my_slot_cnt, unsigned int expect, int S, size_t S_cap,
+                         int d, int H, int rank, const ShardPeerTable& t, long long gather_off,
+                         unsigned long long limit_ns, int* status, cudaStream_t st);
+// waits until my_gather_cnt[0..H) reached `expect` and copies the [S][d] gathered tensor (my_gather = this parity's
+// half) to dst_f32 and / or dst_bf16 (either may be null)
+void launch_shard_gather(const bf16* my_gather, const unsigned int* my_gather_cnt, unsigned int expect, int S, int d,
+                         int H, float* dst_f32, bf16* dst_bf16, unsigned long long limit_ns, int* status,
+                         cudaStream_t st);
+
 }  // namespace foe

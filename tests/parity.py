@@ -110,9 +110,12 @@ def run_block_parity(shape, seed, q_lens: Sequence[int], ctx_lens: Sequence[int]
     return res
 
 
-def compare_with_oracle(shape, W, x, q_lens, ctx_lens, cache, kv, out, aux, rows=None, stress=False) -> Dict:
+def compare_with_oracle(shape, W, x, q_lens, ctx_lens, cache, kv, out, aux, rows=None, stress=False,
+                        cluster_maps=None) -> Dict:
     """Stage-by-stage comparison of one finished GPU call (its output, intermediates `aux` and the cache `kv` it
-    wrote) with the oracle run on the same inputs.  `cache` is the logical cache from before the call."""
+    wrote) with the oracle run on the same inputs.  `cache` is the logical cache from before the call.
+    `cluster_maps`: for a block that ran as one handle per cluster, the H per-cluster dispatch maps (each over the
+    cluster's own E_c experts, ids local to the cluster) instead of one map over all experts in `aux`."""
     q_lens, ctx_lens = list(q_lens), list(ctx_lens)
     S = sum(q_lens)
     cfg = adapter.cfg_from_shape(shape)
@@ -151,12 +154,23 @@ def compare_with_oracle(shape, W, x, q_lens, ctx_lens, cache, kv, out, aux, rows
     assert not unexplained.any(), f"{int(unexplained.sum())} routing flips with margin above the noise bound"
     assert_close(u_gpu, ref["u"], "FFN-normed u", STAGE_MAX_TOL, STAGE_REL_TOL)
 
-    maps = check_maps(shape, aux, idx_gpu)
     H, kc = shape.n_clusters, shape.top_k_per_cluster
-    assert int(maps["counts"].sum()) == S * H * kc
     Ec = shape.experts_per_cluster
-    for h in range(H):                                                             # every cluster gets S*k_c rows
-        assert int(maps["counts"][h * Ec:(h + 1) * Ec].sum()) == S * kc
+    if cluster_maps is None:
+        maps = check_maps(shape, aux, idx_gpu)
+        assert int(maps["counts"].sum()) == S * H * kc
+        for h in range(H):                                                         # every cluster gets S*k_c rows
+            assert int(maps["counts"][h * Ec:(h + 1) * Ec].sum()) == S * kc
+        counts = maps["counts"]
+    else:
+        per = []
+        for h in range(H):
+            mp = orc.permute(idx_gpu[:, h:h + 1] - h * Ec, Ec)
+            for k in ("counts", "offsets", "perm", "inv"):
+                assert np.array_equal(cluster_maps[h][k].cpu().numpy(), mp[k]), f"cluster {h}: dispatch map {k} differs"
+            assert int(mp["counts"].sum()) == S * kc
+            per.append(mp["counts"])
+        counts = np.concatenate(per)
 
     got = adapter.to_np(out)
     got = got[:, rsel] if shape.grouped_output else got[rsel]
@@ -164,4 +178,4 @@ def compare_with_oracle(shape, W, x, q_lens, ctx_lens, cache, kv, out, aux, rows
         mx, rel = assert_close(got, ref_g["out"], "block output")
     else:
         mx, rel = assert_close(got, ref_g["out"], "block output (scaled weights)", STAGE_MAX_TOL, STAGE_REL_TOL)
-    return dict(max_abs=mx, rel_l1=rel, flips=int(flips.sum()), counts=maps["counts"], ref=ref)
+    return dict(max_abs=mx, rel_l1=rel, flips=int(flips.sum()), counts=counts, ref=ref)
