@@ -468,6 +468,79 @@ def run_stack(args):
                           stacks=rows)))
 
 
+def run_shard(args):
+    """One cluster per rank, all ranks on this one device: what each rank's own kernels cost.  Ranks on one device run
+    one after the other, so a rank's time is the sum of its three phases (attention + push, owner-side reduce +
+    all-gather, wait + routing + experts + combine), taken with CUDA events around each; the exchange moves through
+    local memory here, so the NVLink time is NOT in these numbers -- its bytes are reported beside them."""
+    from paper_2605_06206_b200 import shard
+    rows = []
+    for kind in ("prefill", "decode"):
+        n = 2 if kind == "prefill" else 3
+        shape, info = synth.workload(n)
+        H, d = shape.n_clusters, shape.hidden
+        seed, q_lens, ctx = info["seed"], info["q_lens"], info["context_lens"]
+        S = sum(q_lens)
+        decode = kind == "decode"
+        W = synth.make_weights(shape, seed, "cuda")
+        x = synth.make_x(shape, seed, S, "cuda")
+        kv = synth.make_paged_cache(shape, seed, ctx, q_lens, "cuda")
+        kvs = [shard.split_cache(shape, kv, h) for h in range(H)]
+        max_ctx = max(c + q for c, q in zip(ctx, q_lens))
+        one = build_workload(kind, "cuda")
+        fn, _ = step_fn(one)
+        one_ms = timed_loop(fn, args.steps, args.warmup, False) / args.steps
+        one["layer"].close()
+        del one, kv
+        group = shard.LocalGroup(shape, max_tokens=S)
+        layers = group.make_layer(shape, W, S, len(q_lens), max_ctx)
+        del W
+        torch.cuda.empty_cache()
+        outs = [torch.empty(S, d, dtype=torch.bfloat16, device="cuda") for _ in range(H)]
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(H)]
+        acc = [[0.0, 0.0, 0.0] for _ in range(H)]
+        for it in range(args.warmup + args.steps):
+            torch.cuda._sleep(20_000_000)      # ~10 ms of device spin: the host queues the whole step behind it, so the
+                                               # events see kernel time, not launch gaps
+            for h, l in enumerate(layers):
+                ev[h][0].record(); l.attend(x[h], kvs[h], decode); ev[h][1].record()
+            for h, l in enumerate(layers):
+                ev[h][2].record(); l.reduce(); ev[h][3].record()
+            for h, l in enumerate(layers):
+                ev[h][4].record(); l.ffn(out=outs[h]); ev[h][5].record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                for h in range(H):
+                    for p in range(3):
+                        acc[h][p] += ev[h][2 * p].elapsed_time(ev[h][2 * p + 1])
+        assert group.poll_status() == 0 and all(l.layer.poll_status() == 0 for l in layers)
+        per = [[v / args.steps for v in a] for a in acc]
+        rank_ms = [sum(a) for a in per]
+        # per rank and layer: reduce-scatter sends (H-1)/H of its [S][d] bf16 partial, all-gather sends its d/H columns
+        # to H-1 peers: 2 * S * d * 2 * (H-1)/H bytes out (and as many in).  Conventional expert parallelism over the
+        # same H GPUs moves every token to its k experts and back: 2 * S * k * d * 2 * (H-1)/H bytes (Section 3.2).
+        k = H * shape.top_k_per_cluster
+        sync_bytes = 2 * S * d * 2 * (H - 1) / H
+        ep_bytes = 2 * S * k * d * 2 * (H - 1) / H
+        rows.append(dict(workload=f"workload {n} ({kind})", n_ranks=H, tokens=S, one_device_ms=one_ms,
+                         rank_ms_max=max(rank_ms), rank_ms_mean=sum(rank_ms) / H,
+                         phases_ms_mean=dict(attend_push=sum(a[0] for a in per) / H, reduce_allgather=sum(a[1] for a in per) / H,
+                                             wait_route_experts_combine=sum(a[2] for a in per) / H),
+                         launches_per_rank=layers[0].layer.last_launch_count() + 1,
+                         sync_bytes_out_per_rank=sync_bytes, sync_ms_at_770_GBs=sync_bytes / 770e9 * 1e3,
+                         expert_parallel_alltoall_bytes_out_per_rank=ep_bytes, bytes_ratio=ep_bytes / sync_bytes))
+        for l in layers:
+            l.close()
+        group.close()
+        del layers, group, kvs, outs
+        torch.cuda.empty_cache()
+    print(json.dumps(dict(metric="foe_rank_ms_per_layer", unit="ms", data="synthetic", dtype="bf16",
+                          config=dict(workload="one cluster per rank, all ranks emulated on one device; exchange through local "
+                                               "memory (NVLink time not included: see sync_ms_at_770_GBs)",
+                                      steps=args.steps, warmup=args.warmup),
+                          groups=rows)))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -480,6 +553,7 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="token-batch latency sweep at the paper's 7B layer shape")
     ap.add_argument("--sweep-shape", choices=["7b", "1b"], default="7b")
     ap.add_argument("--stack", action="store_true", help="16-layer stack (workload 5): FoE and the one-cluster MoE twin")
+    ap.add_argument("--shard", action="store_true", help="one cluster per rank, all ranks emulated on this device: per-rank kernel time")
     ap.add_argument("--serve", action="store_true", help="request-level latency run (continuous batching on a 4-layer stack)")
     ap.add_argument("--requests", type=int, default=48)
     ap.add_argument("--rate", type=float, default=20.0, help="--serve: Poisson arrival rate, requests per second")
@@ -504,6 +578,9 @@ def main():
         return
     if args.stack:
         run_stack(args)
+        return
+    if args.shard:
+        run_shard(args)
         return
     dist_on = replicas.init("nccl", torch.device("cuda", local))
     peaks = measured_peaks()

@@ -161,3 +161,60 @@ def test_a_wait_that_nothing_satisfies_runs_out_and_is_reported():
     group.close()
     y = torch.ones(4, device="cuda") * 2
     assert float(y.sum()) == 8.0
+
+
+def test_group_stack_prefill_then_decode_on_per_cluster_caches():
+    """Three layers (first, middle, last), a prefill and two decode steps: every layer runs once on one device and once
+    as a group of ranks with per-cluster caches, both fed the one-device path's input to that layer.  The decode steps
+    read what the group's own prefill wrote into the per-cluster pages."""
+    base, L, q_lens, steps = shape_small(), 3, [70, 130], 2
+    H, Ec, S, n_seqs = base.n_clusters, base.experts_per_cluster, sum(q_lens), len(q_lens)
+    max_ctx = max(q_lens) + steps
+    group = shard.LocalGroup(base, max_tokens=S)
+    ones, groups, kv_one, kv_grp = [], [], [], []
+    total = [q + steps for q in q_lens]
+    for l in range(L):
+        sh = dataclasses.replace(base, position=("first", "middle", "last")[l])
+        W = scaled_weights(sh, 21, "cuda", layer=l + 1)
+        ones.append(binding.FoeLayer(sh, W, S, n_seqs, max_ctx))
+        groups.append(group.make_layer(sh, W, S, n_seqs, max_ctx))
+        kv = synth.make_paged_cache(base, 21, [0] * n_seqs, total, "cuda", fill_random=False)
+        kv_one.append(kv)
+        kv_grp.append([shard.split_cache(base, kv, h) for h in range(H)])
+
+    def run_all(x, ctx, decode):
+        ctx_t = torch.tensor(ctx, dtype=torch.int32, device="cuda")
+        q_t = torch.tensor([1] * n_seqs if decode else q_lens, dtype=torch.int32, device="cuda")
+        h_in = x
+        for l in range(L):
+            for kv in [kv_one[l]] + kv_grp[l]:
+                kv.context_lens, kv.q_lens = ctx_t, q_t
+            ref = ones[l].decode(h_in, kv_one[l]) if decode else ones[l].prefill(h_in, kv_one[l])
+            got = group.forward(groups[l], h_in, kv_grp[l], decode)
+            idx_one = ones[l].aux()["topk_idx"]
+            idx_grp = torch.cat([r.layer.aux()["topk_idx"] + h * Ec for h, r in enumerate(groups[l])], 1)
+            same = (torch.sort(idx_one, -1).values == torch.sort(idx_grp, -1).values).all(-1).all(-1)
+            assert same.float().mean() > 0.7
+            grouped = ones[l].shape.grouped_output
+            a = got[:, same] if grouped else got[same]
+            b = ref[:, same] if grouped else ref[same]
+            assert_close(a.float().cpu().numpy(), b.float().cpu().numpy(), f"layer {l} ({'decode' if decode else 'prefill'})", 2e-2, 4e-3)
+            h_in = ref
+        return h_in
+
+    run_all(synth.make_x(dataclasses.replace(base, position="first"), 21, S, "cuda"), [0] * n_seqs, False)
+    for s in range(steps):
+        run_all(synth.make_x(dataclasses.replace(base, position="first"), 21, n_seqs, "cuda", tid=synth.TID["x_step"] + s),
+                [q + s for q in q_lens], True)
+    # the per-cluster pages hold what the one-device cache holds for the cluster's KV heads
+    c = base.kv_per_cluster
+    for l in range(L):
+        for h in range(H):
+            ref_k = kv_one[l].k_pages[:, h * c:(h + 1) * c].float()
+            assert_close(kv_grp[l][h].k_pages.float().cpu().numpy(), ref_k.cpu().numpy(), f"K pages, layer {l}, cluster {h}", 3e-2, 1.5e-2)
+    assert group.poll_status() == 0
+    for l in range(L):
+        ones[l].close()
+        for r in groups[l]:
+            r.close()
+    group.close()
