@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfoe.so")
-SOURCES = ["foe_api.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "smallm.cu", "route.cu", "router_tc.cu", "permute.cu", "elementwise.cu", "shard.cu"]
+SOURCES = ["foe_api.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "smallm.cu", "route.cu", "router_tc.cu", "permute.cu", "elementwise.cu", "shard.cu", "decode_proj.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
          "-cudart", "static"]
 

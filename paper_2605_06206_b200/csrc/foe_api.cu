@@ -61,6 +61,7 @@ struct foe_workspace {
   int *topk_idx, *cu_q, *tok_seq, *tok_pos, *tok_slot, *status, *split_done;
   PermuteBuffers pb;
   CUtensorMap tm_attn_o, tm_hmid, tm_qkv;       // maps of workspace buffers (A operands, attention Q)
+  CUtensorMap tm_attn_o64;                       // attention output with 64-row boxes (decode O-projection)
 };
 
 struct foe_layer {
@@ -80,6 +81,8 @@ struct foe_layer {
   // tensor maps of the weights
   CUtensorMap tm_wqkv, tm_wo, tm_wgu, tm_wd;       // weights; box = the rows of B one CTA of a pair stages per k-block
   CUtensorMap tms_wqkv, tms_wo, tms_wgu, tms_wd;   // same weights, boxes sized for the decode kernels
+  CUtensorMap tmt_wqkv, tmt_wo;                    // 128-row boxes: slabs of the tensor-core decode projections
+  bool dp_qkv, dp_oproj;                           // shapes those kernels take (else the weight-streaming kernels)
   // call state
   cudaStream_t last_stream;
   int last_tokens, launches;
@@ -227,6 +230,17 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
     ga.rope_tab = L->rope_tab; ga.tok_pos = L->ws->tok_pos; ga.tok_slot = L->ws->tok_slot;
     ga.k_pages = static_cast<bf16*>(kv->k_pages); ga.v_pages = static_cast<bf16*>(kv->v_pages);
     launch_gemm(kEpiQKV, tmX, L->tm_wqkv, ga, L->n_sms, st);
+  } else if (L->dp_qkv) {
+    if (!make_map_2d(&tmX, x, x_rows, d, 64)) return FOE_ERR_CUDA;
+    DecodeProjArgs pa;
+    memset(&pa, 0, sizeof(pa));
+    pa.n_groups = H; pa.rows_per_group = S; pa.x_group_stride = L->first ? 0 : S; pa.N = (L->g + 2 * L->c) * dh; pa.K = d;
+    pa.epi = kEpiQKV; pa.status = L->ws->status;
+    pa.out = L->ws->qkv; pa.ldo = L->n_q * L->dhp; pa.q_head_stride = L->dhp; pa.rms_eps = L->cfg.rms_eps;
+    pa.q_cols = L->g * dh; pa.kv_cols = L->c * dh; pa.dh = dh; pa.n_kv = L->n_kv;
+    pa.rope_tab = L->rope_tab; pa.tok_pos = L->ws->tok_pos; pa.tok_slot = L->ws->tok_slot;
+    pa.k_pages = static_cast<bf16*>(kv->k_pages); pa.v_pages = static_cast<bf16*>(kv->v_pages);
+    launch_decode_proj(L->tmt_wqkv, tmX, pa, L->n_sms, st);
   } else {
     SmallMArgs sa;
     memset(&sa, 0, sizeof(sa));
@@ -278,6 +292,17 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
       ga.push_slot_off = slot_off;
     }
     launch_gemm(kEpiOProj, L->ws->tm_attn_o, L->tm_wo, ga, L->n_sms, st);
+  } else if (L->dp_oproj) {
+    DecodeProjArgs pa;
+    memset(&pa, 0, sizeof(pa));
+    pa.n_groups = 1; pa.rows_per_group = S; pa.x_group_stride = 0; pa.N = d; pa.K = L->n_q * dh; pa.epi = kEpiOProj;
+    pa.status = L->ws->status;
+    pa.out = L->ws->r_full; pa.ldo = d; pa.xsum = xb; pa.x_count = x_count; pa.x_stride = size_t(S) * d; pa.out_scale = out_scale;
+    launch_decode_proj(L->tmt_wo, L->ws->tm_attn_o64, pa, L->n_sms, st);
+    if (sh) {
+      launch_shard_push(L->ws->r_full, 1, 1.0f, S, d, sh->cfg.n_ranks, sh->table, slot_off, st);
+      L->launches += 1;
+    }
   } else {
     SmallMArgs sa;
     memset(&sa, 0, sizeof(sa));
@@ -501,7 +526,8 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     cudaMemsetAsync(W->hmid, 0, size_t(R + 128) * I * sizeof(bf16), st);
     ok = make_map_2d(&W->tm_attn_o, W->attn_o, uint64_t(S), uint64_t(L->n_q) * dh, kBM) &&
          make_map_2d(&W->tm_hmid, W->hmid, uint64_t(R), I, kBM) &&
-         make_map_2d(&W->tm_qkv, W->qkv, uint64_t(S), uint64_t(L->n_q) * L->dhp, 128);
+         make_map_2d(&W->tm_qkv, W->qkv, uint64_t(S), uint64_t(L->n_q) * L->dhp, 128) &&
+         make_map_2d(&W->tm_attn_o64, W->attn_o, uint64_t(S), uint64_t(L->n_q) * dh, 64);
     if (!ok) { foe_layer_destroy(L); return FOE_ERR_CUDA; }
   }
 
@@ -551,7 +577,11 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
        make_map_2d(&L->tms_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, 64) &&
        make_map_2d(&L->tms_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, 64) &&
        make_map_2d(&L->tms_wgu, L->wgu_t, uint64_t(E) * 2 * I, d, 32) &&
-       make_map_2d(&L->tms_wd, L->wd_t, uint64_t(E) * d, I, 64);
+       make_map_2d(&L->tms_wd, L->wd_t, uint64_t(E) * d, I, 64) &&
+       make_map_2d(&L->tmt_wqkv, L->wqkv_t, uint64_t(H) * qkvN, d, 128) &&
+       make_map_2d(&L->tmt_wo, L->wo_t, uint64_t(d), uint64_t(L->n_q) * dh, 128);
+  L->dp_qkv = decode_proj_supported(kEpiQKV, qkvN, d, dh);
+  L->dp_oproj = decode_proj_supported(kEpiOProj, d, L->n_q * dh, dh);
   if (!ok) { foe_layer_destroy(L); return FOE_ERR_CUDA; }
   for (int i = 0; i <= kNumStages; ++i) cudaEventCreate(&L->ev[i]);
   *out = L;

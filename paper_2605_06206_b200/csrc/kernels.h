@@ -130,6 +130,27 @@ struct SmallMArgs {
 // tmW: tensor map of W as [n_groups*N][K] with 64-column boxes of 64 rows (32 rows for the SwiGLU packing)
 void launch_smallm(const CUtensorMap& tmW, const SmallMArgs& a, int n_sms, cudaStream_t st);
 
+// ---- decode_proj.cu  (dense projections of a decode step on tcgen05, weights as the MMA's M operand)
+struct DecodeProjArgs {
+  int n_groups;
+  int rows_per_group;       // tokens S (the same tokens for every group)
+  int x_group_stride;       // activation row of (group g, token t) = g * x_group_stride + t
+  int N, K;                 // weight rows per group (a multiple of 128), reduction length (a multiple of 64)
+  int k_splits;             // set by the launcher: CTAs per cluster (1, 2, 4 or 8), each with its share of K
+  int epi;                  // kEpiQKV or kEpiOProj
+  int* status;
+  void* out; int ldo;
+  // kEpiQKV (see GemmArgs; 1/rms is computed from the staged activation rows)
+  float rms_eps;
+  int q_cols, kv_cols, dh, n_kv, q_head_stride;
+  const float2* rope_tab; const int* tok_pos; const int* tok_slot; bf16* k_pages; bf16* v_pages;
+  // kEpiOProj
+  const bf16* xsum; int x_count; size_t x_stride; float out_scale;
+};
+bool decode_proj_supported(int epi, int N, int K, int dh);
+// tmW: the weights [n_groups * N][K] with 64-column boxes of 128 rows; tmX: the activations with 64 x 64 boxes
+void launch_decode_proj(const CUtensorMap& tmW, const CUtensorMap& tmX, DecodeProjArgs a, int n_sms, cudaStream_t st);
+
 // ---- shard.cu  (sync of a cluster-per-GPU group over peer memory)
 // This rank's mappings of every rank's exchange buffer: receive slots ([2][H][S_cap][d/H] bf16), gather buffer
 // ([2][S_cap][d] bf16), arrival counters of the slots ([H], one per source) and of the gather buffer ([H], one per owner).
