@@ -70,6 +70,8 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       : "memory");
 }
 
+}  // namespace
+
 template <int EPI>
 __global__ void __launch_bounds__(kDpThreads, 1)
 decode_proj_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
@@ -293,6 +295,8 @@ decode_proj_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     tmem_dealloc(tmem_base, 64);
   }
 }
+
+namespace {
 
 template <int EPI>
 void launch_one(const CUtensorMap& tmW, const CUtensorMap& tmX, DecodeProjArgs a, int tiles, cudaStream_t st) {

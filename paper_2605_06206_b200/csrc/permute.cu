@@ -89,7 +89,7 @@ permute_scan_kernel(int* __restrict__ blk_counts, int n_blocks, int E, const Per
   s_a[e] = total;
   s_b[e] = tiles;
   __syncthreads();
-  for (int o = 1; o < 1024; o <<= 1) {
+  for (int o = 1; o < E; o <<= 1) {                 // (entries from E on are zero)
     const int va = e >= o ? s_a[e - o] : 0;
     const int vb = e >= o ? s_b[e - o] : 0;
     __syncthreads();
@@ -146,9 +146,18 @@ permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, 
   if (tk.scores) {
     const int H = tk.H, Ec = tk.Ec, kc = tk.kc;
     // scores = partial sums in fixed order + bias, all threads; then one thread per (token, cluster)
+    // (sixteen loads in flight per element: the partials sit in L2, and one round trip per split would cost more
+    // than everything else in this kernel)
     for (int q = t; q < n_tokens * E; q += 1024) {
       float v = 0.f;
-      for (int z = 0; z < tk.k_splits; ++z) v += tk.scores[size_t(z) * n_tokens * E + q];
+      for (int z0 = 0; z0 < tk.k_splits; z0 += 16) {
+        float p[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u)
+          p[u] = (z0 + u < tk.k_splits) ? __ldcg(tk.scores + size_t(z0 + u) * n_tokens * E + q) : 0.f;
+#pragma unroll
+        for (int u = 0; u < 16; ++u) v += p[u];             // split order; the zeros of absent splits change nothing
+      }
       tk.logits_out[q] = v + (tk.bias ? tk.bias[q % E] : 0.f);
     }
     __threadfence_block();
@@ -199,7 +208,7 @@ permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, 
   s_a[t] = total;
   s_b[t] = tiles;
   __syncthreads();
-  for (int o = 1; o < 1024; o <<= 1) {
+  for (int o = 1; o < E; o <<= 1) {                 // (entries from E on are zero)
     const int va = t >= o ? s_a[t - o] : 0;
     const int vb = t >= o ? s_b[t - o] : 0;
     __syncthreads();
