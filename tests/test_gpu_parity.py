@@ -179,6 +179,17 @@ def test_decode_head_dim_128_many_splits():
     run_block_parity(shape, 22, [1] * 4, [10, 1030, 2100, 5000], decode=True, wscale=4.0)
 
 
+@pytest.mark.parametrize("dh,position,n_seqs", [(64, "middle", 130), (128, "middle", 200), (64, "first", 65), (128, "last", 256)])
+def test_decode_more_sequences_than_one_token_tile(dh, position, n_seqs):
+    # the decode projections take 64 tokens per CTA: several token tiles, the last one ragged (or exactly full)
+    if dh == 64:
+        shape = shape_small(position=position)
+    else:
+        shape = synth.LayerShape(512, 8, 2, 2, 128, 4, 2, 256, position=position)
+    ctx = [(37 * i) % 300 for i in range(n_seqs)]
+    run_block_parity(shape, 29, [1] * n_seqs, ctx, decode=True, wscale=4.0)
+
+
 @pytest.mark.parametrize("position", ["first", "last"])
 def test_decode_boundary_layers(position):
     shape = shape_small(position=position)
