@@ -27,6 +27,61 @@ __global__ void row_inv_rms_kernel(const bf16* __restrict__ x, float* __restrict
   if (lane == 0) inv_rms[warp] = rsqrtf(ss / float(d) + eps);
 }
 
+// The same statistics for the H residual streams x[h] of a middle or last layer, plus their sum: one warp per token
+// reads its H rows once, writes inv_rms[h * S + s] and xsum[s][:] = sum_h x[h][s][:] (fp32, h ascending).  The output
+// projection then adds ONE fp32 tensor in its epilogue instead of reading the H streams again.
+template <int H>
+__global__ void row_inv_rms_xsum_kernel(const bf16* __restrict__ x, float* __restrict__ inv_rms, float* __restrict__ xsum,
+                                        int S, int d, float eps) {
+  const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (s >= S) return;
+  float ss[H];
+#pragma unroll
+  for (int h = 0; h < H; ++h) ss[h] = 0.f;
+  for (int c = lane; c < d / 8; c += 32) {
+    uint4 q[H];
+#pragma unroll
+    for (int h = 0; h < H; ++h) q[h] = __ldg(reinterpret_cast<const uint4*>(x + (size_t(h) * S + s) * d) + c);
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int h = 0; h < H; ++h) {
+      const uint32_t w[4] = {q[h].x, q[h].y, q[h].z, q[h].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float a = bf16_lo(w[j]), b = bf16_hi(w[j]);
+        ss[h] += a * a + b * b;
+        acc[2 * j] += a;
+        acc[2 * j + 1] += b;
+      }
+    }
+    float4* o = reinterpret_cast<float4*>(xsum + size_t(s) * d + c * 8);
+    o[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    o[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+  }
+#pragma unroll
+  for (int h = 0; h < H; ++h) {
+    const float t = warp_sum(ss[h]);
+    if (lane == 0) inv_rms[size_t(h) * S + s] = rsqrtf(t / float(d) + eps);
+  }
+}
+
+bool launch_row_inv_rms_xsum(const bf16* x, float* inv_rms, float* xsum, int S, int d, int H, float eps, cudaStream_t st) {
+  if (S <= 0) return true;
+  const int threads = 256;
+  const int blocks = (S * 32 + threads - 1) / threads;
+  switch (H) {
+    case 2: row_inv_rms_xsum_kernel<2><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
+    case 3: row_inv_rms_xsum_kernel<3><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
+    case 4: row_inv_rms_xsum_kernel<4><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
+    case 5: row_inv_rms_xsum_kernel<5><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
+    case 6: row_inv_rms_xsum_kernel<6><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
+    case 7: row_inv_rms_xsum_kernel<7><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
+    case 8: row_inv_rms_xsum_kernel<8><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
+    default: return false;
+  }
+}
+
 void launch_row_inv_rms(const bf16* x, float* inv_rms, int n_rows, int d, float eps, cudaStream_t st) {
   if (n_rows <= 0) return;
   const int threads = 256;

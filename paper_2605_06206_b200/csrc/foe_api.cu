@@ -210,8 +210,11 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
   L->launches += launch_token_map(decode ? nullptr : kv->q_lens, kv->context_lens, kv->block_table, kv->n_seqs, kv->max_pages_per_seq,
                    kv->num_pages, 64, S, L->cfg.max_context, L->ws->cu_q, L->ws->tok_seq, L->ws->tok_pos, L->ws->tok_slot, L->ws->status, st);
   const int x_rows = L->first ? S : H * S;
+  bool x_summed = false;   // r_full holds sum_h x[h] (fp32) for the output projection to add
   if (!decode) {         // (the decode projection derives 1/rms from the rows it stages)
-    launch_row_inv_rms(xb, L->ws->inv_rms, x_rows, d, L->cfg.rms_eps, st);
+    if (!L->first && H > 1 && !sh)
+      x_summed = launch_row_inv_rms_xsum(xb, L->ws->inv_rms, L->ws->r_full, S, d, H, L->cfg.rms_eps, st);
+    if (!x_summed) launch_row_inv_rms(xb, L->ws->inv_rms, x_rows, d, L->cfg.rms_eps, st);
     L->launches += 1;
   }
 
@@ -286,6 +289,7 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
     ga.n_groups = 1; ga.rows_per_group = S; ga.a_group_stride = 0; ga.N = d; ga.K = L->n_q * dh; ga.status = L->ws->status;
     ga.out = L->ws->r_full; ga.ldo = d; ga.xsum = xb; ga.x_count = x_count; ga.x_stride = size_t(S) * d;
     ga.out_scale = out_scale;
+    if (x_summed) { ga.x_count = 0; ga.x_in_out = 1; }
     if (sh) {     // the epilogue stores each tile straight into the owners' slots
       for (int o = 0; o < sh->cfg.n_ranks; ++o) { ga.push_base[o] = sh->table.slots[o]; ga.push_cnt[o] = sh->table.slot_cnt[o]; }
       ga.push_span = sh->span;

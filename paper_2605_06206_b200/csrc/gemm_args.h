@@ -21,7 +21,7 @@ enum GemmEpilogue : int {
   kEpiBf16 = 0,     // C -> bf16 [row][ldo]
   kEpiSwiGLU = 1,   // columns [0,128) gate, [128,256) up of one 128-wide block: silu(gate)*up -> bf16
   kEpiQKV = 2,      // row scale (1/rms), RoPE, q -> [S][n_q*dh], k and v -> cache pages
-  kEpiOProj = 3     // r_full = scale * (C + sum_h x[h]) -> fp32 [row][ldo]
+  kEpiOProj = 3     // r_full = scale * (C + sum_h x[h]) -> fp32 [row][ldo]; the sum either read as bf16 streams or found in r_full
 };
 
 // Rows of B one CTA of a pair stages per k-block = box rows of the B tensor map: half a tile.  The SwiGLU epilogue
@@ -64,10 +64,11 @@ struct GemmArgs {
   __nv_bfloat16* k_pages;   // [num_pages][n_kv][64][dh]
   __nv_bfloat16* v_pages;
   // kEpiOProj
-  const __nv_bfloat16* xsum; // [x_count][x_stride] residual streams added to C
+  const __nv_bfloat16* xsum; // one bf16 residual stream [rows][ldo] added to C when x_count == 1 (x_count is 0 or 1)
   int x_count;
   size_t x_stride;
   float out_scale;
+  int x_in_out;              // `out` already holds the fp32 sum of the residual streams: out = scale * (C + out)
   // kEpiOProj on one rank of a cluster-per-GPU group (push_span != 0): the scaled tile is not written to `out` but
   // pushed as bf16 to the rank that owns its columns -- columns [o * push_span, (o + 1) * push_span) belong to rank
   // o -- at push_base[o] + push_slot_off + row * push_span + (column - o * push_span); push_cnt[o] then grows by

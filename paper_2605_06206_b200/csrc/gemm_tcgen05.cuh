@@ -183,20 +183,25 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
       *reinterpret_cast<uint4*>(stg + stg_off(lane, c)) = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
     __syncwarp();
     if constexpr (EPI == kEpiOProj) {
-      // r_full = scale * (C + sum_h x[h]): the residual streams are read here.  This GEMM moves almost as many
-      // bytes as it has flops to hide them, so the epilogue has to keep ~256 bytes per thread in flight:
-      // 4 lanes x 16 bytes per row and stream, and all loads of the pass are issued before the first use.
+      // r_full = scale * (C + sum_h x[h]); all loads of the pass are issued before the first use.
       const int or_row = lane >> 2, or_cg = lane & 3;           // row (+8j) and group of 8 columns
-      uint4 xq[4][8];
+      // what is added to C: the fp32 sum of the residual streams already sitting in `out` (two float4 per row), or
+      // one bf16 stream (a first layer's shared x, a rank's own x[h]), or nothing
+      float4 xf[4][2];
+      uint4 xq[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int grow = row0 + quarter * 32 + or_row + 8 * j;
         const size_t off = size_t(grow) * args.ldo + n + or_cg * 8;
-#pragma unroll
-        for (int h = 0; h < 8; ++h) {
-          xq[j][h] = make_uint4(0u, 0u, 0u, 0u);
-          if (h < args.x_count && grow < row_end)
-            xq[j][h] = __ldg(reinterpret_cast<const uint4*>(args.xsum + h * args.x_stride + off));
+        xf[j][0] = xf[j][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        xq[j] = make_uint4(0u, 0u, 0u, 0u);
+        if (grow < row_end) {
+          if (args.x_in_out) {
+            xf[j][0] = *reinterpret_cast<const float4*>(static_cast<const float*>(args.out) + off);
+            xf[j][1] = *reinterpret_cast<const float4*>(static_cast<const float*>(args.out) + off + 4);
+          } else if (args.x_count > 0) {
+            xq[j] = __ldg(reinterpret_cast<const uint4*>(args.xsum + off));
+          }
         }
       }
 #pragma unroll
@@ -206,10 +211,10 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
         if (grow >= row_end) continue;
         const float4 c0 = *reinterpret_cast<const float4*>(stg + stg_off(rr, 2 * or_cg));
         const float4 c1 = *reinterpret_cast<const float4*>(stg + stg_off(rr, 2 * or_cg + 1));
-        float a8[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-#pragma unroll
-        for (int h = 0; h < 8; ++h) {
-          const uint32_t w4[4] = {xq[j][h].x, xq[j][h].y, xq[j][h].z, xq[j][h].w};
+        float a8[8] = {c0.x + xf[j][0].x, c0.y + xf[j][0].y, c0.z + xf[j][0].z, c0.w + xf[j][0].w,
+                       c1.x + xf[j][1].x, c1.y + xf[j][1].y, c1.z + xf[j][1].z, c1.w + xf[j][1].w};
+        {
+          const uint32_t w4[4] = {xq[j].x, xq[j].y, xq[j].z, xq[j].w};
 #pragma unroll
           for (int q = 0; q < 4; ++q) { a8[2 * q] += bf16_lo(w4[q]); a8[2 * q + 1] += bf16_hi(w4[q]); }
         }

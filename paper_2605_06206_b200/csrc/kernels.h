@@ -15,6 +15,8 @@ typedef __nv_bfloat16 bf16;
 // ---- elementwise.cu
 // inv_rms[r] = rsqrt(mean(x[r,:]^2) + eps) for n_rows rows of d bf16 values
 void launch_row_inv_rms(const bf16* x, float* inv_rms, int n_rows, int d, float eps, cudaStream_t st);
+// the same for x = [H][S][d], plus xsum[s][:] = sum_h x[h][s][:] in fp32; false (nothing launched) unless 2 <= H <= 8
+bool launch_row_inv_rms_xsum(const bf16* x, float* inv_rms, float* xsum, int S, int d, int H, float eps, cudaStream_t st);
 // per-token position / sequence / cache slot from q_lens and context_lens (device arrays)
 // returns the number of kernels launched
 int launch_token_map(const int* q_lens, const int* context_lens, const int* block_table, int n_seqs,
