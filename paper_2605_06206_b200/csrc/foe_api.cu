@@ -111,6 +111,7 @@ struct foe_shard {
 
 namespace {
 
+constexpr int kFewTokens = 256;                  // calls up to this size take the decode-step kernels where they fit
 constexpr size_t kShardHeaderBytes = 1024;       // slot counters at 0, gather counters at 128
 
 bool shard_config_ok(const foe_shard_config* c) {
@@ -210,18 +211,25 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
   L->launches += launch_token_map(decode ? nullptr : kv->q_lens, kv->context_lens, kv->block_table, kv->n_seqs, kv->max_pages_per_seq,
                    kv->num_pages, 64, S, L->cfg.max_context, L->ws->cu_q, L->ws->tok_seq, L->ws->tok_pos, L->ws->tok_slot, L->ws->status, st);
   const int x_rows = L->first ? S : H * S;
+  // Kernel family of the two projections: a call of a few hundred tokens (any decode step, a short prompt chunk, a
+  // small mixed batch) is a weight-streaming problem and takes the decode kernels, whatever entry point it came by.
+  const bool few = decode || S <= kFewTokens;
+  const bool qkv_dp = few && L->dp_qkv, qkv_gemm = !qkv_dp && !decode;
+  const bool oproj_dp = few && L->dp_oproj, oproj_gemm = !oproj_dp && !decode;
   bool x_summed = false;   // r_full holds sum_h x[h] (fp32) for the output projection to add
-  if (!decode) {         // (the decode projection derives 1/rms from the rows it stages)
-    if (!L->first && H > 1 && !sh)
-      x_summed = launch_row_inv_rms_xsum(xb, L->ws->inv_rms, L->ws->r_full, S, d, H, L->cfg.rms_eps, st);
-    if (!x_summed) launch_row_inv_rms(xb, L->ws->inv_rms, x_rows, d, L->cfg.rms_eps, st);
+  if (oproj_gemm && !L->first && H > 1 && !sh) {
+    x_summed = launch_row_inv_rms_xsum(xb, L->ws->inv_rms, L->ws->r_full, S, d, H, L->cfg.rms_eps, st);
+    if (x_summed) L->launches += 1;
+  }
+  if (qkv_gemm && !x_summed) {   // (the decode projections derive 1/rms from the rows they stage)
+    launch_row_inv_rms(xb, L->ws->inv_rms, x_rows, d, L->cfg.rms_eps, st);
     L->launches += 1;
   }
 
   // ---- per-cluster QKV projection; its epilogue applies 1/rms (gain folded into the weights) and RoPE, writes q
   //      and puts K / V of the new tokens straight into their cache pages
   stage_mark(L, kStQkv, st);
-  if (!decode) {
+  if (qkv_gemm) {
     if (!make_map_2d(&tmX, x, x_rows, d, kBM)) return FOE_ERR_CUDA;
     GemmArgs ga;
     memset(&ga, 0, sizeof(ga));
@@ -233,7 +241,7 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
     ga.rope_tab = L->rope_tab; ga.tok_pos = L->ws->tok_pos; ga.tok_slot = L->ws->tok_slot;
     ga.k_pages = static_cast<bf16*>(kv->k_pages); ga.v_pages = static_cast<bf16*>(kv->v_pages);
     launch_gemm(kEpiQKV, tmX, L->tm_wqkv, ga, L->n_sms, st);
-  } else if (L->dp_qkv) {
+  } else if (qkv_dp) {
     if (!make_map_2d(&tmX, x, x_rows, d, 64)) return FOE_ERR_CUDA;
     DecodeProjArgs pa;
     memset(&pa, 0, sizeof(pa));
@@ -283,7 +291,7 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
     x_count = (L->first && sh->cfg.rank != 0) ? 0 : 1;
   }
   const long long slot_off = sh ? (long long)((size_t(sh->epoch & 1) * sh->cfg.n_ranks + sh->cfg.rank) * sh->S_cap * sh->span) : 0;
-  if (!decode) {
+  if (oproj_gemm) {
     GemmArgs ga;
     memset(&ga, 0, sizeof(ga));
     ga.n_groups = 1; ga.rows_per_group = S; ga.a_group_stride = 0; ga.N = d; ga.K = L->n_q * dh; ga.status = L->ws->status;
@@ -296,7 +304,7 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
       ga.push_slot_off = slot_off;
     }
     launch_gemm(kEpiOProj, L->ws->tm_attn_o, L->tm_wo, ga, L->n_sms, st);
-  } else if (L->dp_oproj) {
+  } else if (oproj_dp) {
     DecodeProjArgs pa;
     memset(&pa, 0, sizeof(pa));
     pa.n_groups = 1; pa.rows_per_group = S; pa.x_group_stride = 0; pa.N = d; pa.K = L->n_q * dh; pa.epi = kEpiOProj;
@@ -333,9 +341,11 @@ foe_status run_ffn(foe_layer* L, void* out, cudaStream_t st) {
   stage_mark(L, kStRoute, st);
   run_route_and_permute(L, L->ws->r_full, 0, S, st);
   const int R = S * H * L->kc;
-  (void)R;
+  // experts: the weight-streaming kernels take 16 rows of an expert per pass over its weights; up to 8 rows per
+  // expert on average (few experts need a second pass) they beat the tiled GEMMs, at 16 they no longer do
+  const bool stream_experts = decode || (S <= kFewTokens && R <= 8 * L->E);
 
-  if (!decode) {
+  if (!stream_experts) {
     stage_mark(L, kStGemm1, st);
     GemmArgs g1;
     memset(&g1, 0, sizeof(g1));
