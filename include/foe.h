@@ -141,6 +141,8 @@ foe_status foe_layer_destroy(foe_layer* layer);
 /* Table 2 (all four rows) for S = kv->n_tokens new tokens of kv->n_seqs sequences: attention over the
  * paged cache plus the new tokens (causal), sync, routing, experts, combine.  x: [H][S][hidden] bf16
  * ([S][hidden] on a first layer); out likewise ([S][hidden] on a last layer); out must not alias x.
+ * Calls of a few hundred tokens (short prompt chunks, small mixed batches) are run with the weight-streaming kernels
+ * of the decode step where those fit; results do not depend on the entry point beyond rounding.
  * Errors: FOE_ERR_NULL, FOE_ERR_SHAPE (S > max_tokens, n_seqs > max_seqs, S == 0 is FOE_OK, no work). */
 foe_status foe_prefill(foe_layer* layer, const void* x, const foe_kv_cache* kv, void* out, void* stream);
 
