@@ -168,6 +168,15 @@ def test_skewed_router_bias_small():
     assert (r["counts"] == 0).sum() >= 12                                         # dead experts stay empty
 
 
+def test_small_prefill_with_skewed_routing_streams_experts_in_several_passes():
+    # 120 tokens, 16 experts per cluster, top-1: few enough rows per expert on average for the weight-streaming
+    # expert kernels, but the skewed bias sends dozens of rows to single experts (several 16-row passes) and none to others
+    shape = shape_small(experts_per_cluster=16, top_k_per_cluster=1)
+    bias = synth.zipf_router_bias(shape, 19, 1.5, 1.2, dead_per_cluster=4)
+    r = run_block_parity(shape, 19, [70, 50], [0, 33], wscale=4.0, router_bias=bias)
+    assert r["counts"].max() > 16 and (r["counts"] == 0).sum() >= 16
+
+
 # ------------------------------------------------------------------------------------------ decode
 def test_decode_small_elementwise():
     shape = shape_small()
