@@ -133,6 +133,39 @@ struct TopkSmall {
   int H, Ec, kc;
 };
 
+// Top-k and gates of one (token, cluster) with the cluster's E_c scores in registers (E_c a power of two up to 32):
+// all loads at once, then k_c selection passes without touching memory.  Order and ties as in the generic loop of
+// the kernel below: score descending, expert id ascending.
+template <int EC>
+__device__ __forceinline__ void topk_small_regs(const TopkSmall& tk, int task) {
+  const int H = tk.H, kc = tk.kc;
+  const int i = task / H, h = task - i * H;
+  const float* src = tk.logits_out + (size_t(i) * H + h) * EC;
+  float v[EC];
+#pragma unroll
+  for (int e = 0; e < EC; e += 4) {
+    const float4 a = *reinterpret_cast<const float4*>(src + e);
+    v[e] = a.x; v[e + 1] = a.y; v[e + 2] = a.z; v[e + 3] = a.w;
+  }
+  uint32_t taken = 0u;
+  float m = 0.f, sum = 0.f;
+  const size_t oo = size_t(task) * kc;
+  for (int j = 0; j < kc; ++j) {
+    float bv = 0.f;
+    int bi = -1;
+#pragma unroll
+    for (int e = 0; e < EC; ++e)
+      if (!((taken >> e) & 1u) && (bi < 0 || v[e] > bv)) { bv = v[e]; bi = e; }
+    taken |= 1u << bi;
+    if (j == 0) m = bv;
+    const float x = expf(bv - m);
+    sum += x;
+    tk.idx_out[oo + j] = h * EC + bi;
+    tk.w_out[oo + j] = x;
+  }
+  for (int j = 0; j < kc; ++j) tk.w_out[oo + j] = tk.w_out[oo + j] / sum;
+}
+
 __global__ void __launch_bounds__(1024)
 permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, const PermuteBuffers pb,
                      int* __restrict__ status, const TopkSmall tk) {
@@ -162,7 +195,18 @@ permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, 
     }
     __threadfence_block();
     __syncthreads();
-    for (int task = t; task < n_tokens * H; task += 1024) {
+    const bool in_regs = Ec == 4 || Ec == 8 || Ec == 16 || Ec == 32;
+    if (in_regs) {
+      for (int task = t; task < n_tokens * H; task += 1024) {
+        switch (Ec) {
+          case 4: topk_small_regs<4>(tk, task); break;
+          case 8: topk_small_regs<8>(tk, task); break;
+          case 16: topk_small_regs<16>(tk, task); break;
+          default: topk_small_regs<32>(tk, task); break;
+        }
+      }
+    }
+    for (int task = in_regs ? n_tokens * H : t; task < n_tokens * H; task += 1024) {
       const int i = task / H, h = task - i * H;
       const size_t o = size_t(i) * E + size_t(h) * Ec;
       uint32_t taken[4] = {0u, 0u, 0u, 0u};                 // E_c <= 128
