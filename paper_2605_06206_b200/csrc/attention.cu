@@ -41,6 +41,8 @@ constexpr int kDcStages = 3;
 template <int DH>
 __global__ void __launch_bounds__(kDcThreads, 2)
 attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
+  pdl_launch_dependents();
+  pdl_wait();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int kTileBytes = 64 * DH * 2;
@@ -245,7 +247,7 @@ static void launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, cons
     configured = true;
   }
   dim3 grid(a.max_splits, a.n_kv, a.n_seqs);
-  attn_decode_kernel<DH><<<grid, kDcThreads, smem, st>>>(tmK, tmV, a);
+  launch_pdl(attn_decode_kernel<DH>, grid, dim3(kDcThreads), smem, st, tmK, tmV, a);
 }
 
 void launch_attn_decode(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st) {

@@ -62,6 +62,8 @@ template <int DH>
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
+  pdl_launch_dependents();
+  pdl_wait();
   using L = AtSmem<DH>;
   constexpr int HN = DH / 64;
   extern __shared__ uint8_t smem_raw[];
@@ -358,7 +360,7 @@ static void launch_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUte
   const int G = a.n_q / a.n_kv;
   const int heads_per_cta = (G % 2 == 0) ? 2 : 1;
   dim3 grid((a.max_q_len + kAtRows - 1) / kAtRows, a.n_q / heads_per_cta, a.n_seqs);
-  attn_prefill_tc_kernel<DH><<<grid, kAtThreads, AtSmem<DH>::kBytes, st>>>(tmQ, tmK, tmV, a);
+  launch_pdl(attn_prefill_tc_kernel<DH>, grid, dim3(kAtThreads), size_t(AtSmem<DH>::kBytes), st, tmQ, tmK, tmV, a);
 }
 
 void launch_attn_prefill_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,

@@ -222,6 +222,15 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 }  // namespace foe
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// pdl_launch_dependents: the next kernel in the stream (launched with programmatic stream serialization) may start
+// being scheduled once every CTA of this grid has said so; pdl_wait: returns when the previous kernel has completed
+// and its writes are visible.  Both are no-ops for kernels launched the ordinary way.
+namespace foe {
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+}  // namespace foe
+
 // ---------------------------------------------------------------- CTA pairs (cluster of 2, tcgen05 cta_group::2)
 namespace foe {
 

@@ -76,6 +76,7 @@ template <int EPI>
 __global__ void __launch_bounds__(kDpThreads, 1)
 decode_proj_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                    const DecodeProjArgs a) {
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kDpStages * kDpStageBytes);
@@ -115,7 +116,17 @@ decode_proj_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       bool ok = true;
       const int w_row = group * a.N + slab * kDpSlab;
       const int x_row = group * a.x_group_stride + chunk * kDpTok;
-      for (int kb = kb0; kb < kb1; ++kb) {
+      // The weights do not depend on anything an earlier kernel wrote: the first ring of weight tiles is requested
+      // before this grid waits for its predecessor (whose tail it overlaps); the activations follow after the wait.
+      const int n_first = min(kb1 - kb0, kDpStages);
+      for (int i = 0; i < n_first; ++i) {
+        mbar_expect_tx(&full_bar[i], kDpStageBytes);
+        tma_load_2d(smem + i * kDpStageBytes, &tmW, &full_bar[i], (kb0 + i) * kDpBK, w_row);
+      }
+      pdl_wait();
+      for (int i = 0; i < n_first; ++i)
+        tma_load_2d(smem + i * kDpStageBytes + kDpWBytes, &tmX, &full_bar[i], (kb0 + i) * kDpBK, x_row);
+      for (int kb = kb0 + n_first; kb < kb1; ++kb) {
         const int i = kb - kb0, s = i % kDpStages;
         if (!mbar_wait(&empty_bar[s], ((i / kDpStages) & 1) ^ 1)) { ok = false; break; }
         uint8_t* dst = smem + s * kDpStageBytes;
@@ -147,6 +158,7 @@ decode_proj_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     // ------------------------------------------------------------ statistics (QKV) and epilogue
     // 16 warps: warp (quarter, tg) reads TMEM lanes 32*quarter.. (the hardware ties a warp to the lane quarter
     // warp % 4) and the 16 accumulator columns (tokens) 16*tg..; four warps per scheduler hide each other's latency.
+    pdl_wait();                                           // everything these warps read or write depends on earlier kernels
     const int quarter = warp & 3, tg = (warp - 2) >> 2;
     const int col = quarter * 32 + lane;                  // 0..127 = accumulator lane = weight row of the slab
     const int etid = tg * 128 + col;                      // 0..511
@@ -306,12 +318,15 @@ void launch_one(const CUtensorMap& tmW, const CUtensorMap& tmX, DecodeProjArgs a
   cfg.blockDim = dim3(kDpThreads, 1, 1);
   cfg.dynamicSmemBytes = kDpSmemBytes;
   cfg.stream = st;
-  cudaLaunchAttribute attr;
+  cudaLaunchAttribute attrs[2];
+  cudaLaunchAttribute& attr = attrs[0];
   attr.id = cudaLaunchAttributeClusterDimension;
   attr.val.clusterDim.y = 1;
   attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
+  attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attrs[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attrs;
+  cfg.numAttrs = g_overlap_launches ? 2 : 1;
   if (max_active[0] < 0) {
     cudaFuncSetAttribute(decode_proj_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kDpSmemBytes));
     for (int i = 0; i < 4; ++i) {

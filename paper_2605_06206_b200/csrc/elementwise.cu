@@ -9,6 +9,8 @@ namespace foe {
 // and the scale is applied in the GEMM epilogue, so the normalised tensor is never written.
 __global__ void row_inv_rms_kernel(const bf16* __restrict__ x, float* __restrict__ inv_rms, int n_rows, int d,
                                    float eps) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (warp >= n_rows) return;
@@ -33,6 +35,8 @@ __global__ void row_inv_rms_kernel(const bf16* __restrict__ x, float* __restrict
 template <int H>
 __global__ void row_inv_rms_xsum_kernel(const bf16* __restrict__ x, float* __restrict__ inv_rms, float* __restrict__ xsum,
                                         int S, int d, float eps) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (s >= S) return;
@@ -71,13 +75,13 @@ bool launch_row_inv_rms_xsum(const bf16* x, float* inv_rms, float* xsum, int S, 
   const int threads = 256;
   const int blocks = (S * 32 + threads - 1) / threads;
   switch (H) {
-    case 2: row_inv_rms_xsum_kernel<2><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
-    case 3: row_inv_rms_xsum_kernel<3><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
-    case 4: row_inv_rms_xsum_kernel<4><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
-    case 5: row_inv_rms_xsum_kernel<5><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
-    case 6: row_inv_rms_xsum_kernel<6><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
-    case 7: row_inv_rms_xsum_kernel<7><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
-    case 8: row_inv_rms_xsum_kernel<8><<<blocks, threads, 0, st>>>(x, inv_rms, xsum, S, d, eps); return true;
+    case 2: launch_pdl(row_inv_rms_xsum_kernel<2>, dim3(blocks), dim3(threads), 0, st, x, inv_rms, xsum, S, d, eps); return true;
+    case 3: launch_pdl(row_inv_rms_xsum_kernel<3>, dim3(blocks), dim3(threads), 0, st, x, inv_rms, xsum, S, d, eps); return true;
+    case 4: launch_pdl(row_inv_rms_xsum_kernel<4>, dim3(blocks), dim3(threads), 0, st, x, inv_rms, xsum, S, d, eps); return true;
+    case 5: launch_pdl(row_inv_rms_xsum_kernel<5>, dim3(blocks), dim3(threads), 0, st, x, inv_rms, xsum, S, d, eps); return true;
+    case 6: launch_pdl(row_inv_rms_xsum_kernel<6>, dim3(blocks), dim3(threads), 0, st, x, inv_rms, xsum, S, d, eps); return true;
+    case 7: launch_pdl(row_inv_rms_xsum_kernel<7>, dim3(blocks), dim3(threads), 0, st, x, inv_rms, xsum, S, d, eps); return true;
+    case 8: launch_pdl(row_inv_rms_xsum_kernel<8>, dim3(blocks), dim3(threads), 0, st, x, inv_rms, xsum, S, d, eps); return true;
     default: return false;
   }
 }
@@ -86,11 +90,13 @@ void launch_row_inv_rms(const bf16* x, float* inv_rms, int n_rows, int d, float 
   if (n_rows <= 0) return;
   const int threads = 256;
   const int blocks = (n_rows * 32 + threads - 1) / threads;
-  row_inv_rms_kernel<<<blocks, threads, 0, st>>>(x, inv_rms, n_rows, d, eps);
+  launch_pdl(row_inv_rms_kernel, dim3(blocks), dim3(threads), 0, st, x, inv_rms, n_rows, d, eps);
 }
 
 // ------------------------------------------------------------------ token -> (sequence, position, cache slot)
 __global__ void cu_q_kernel(const int* __restrict__ q_lens, int n_seqs, int* __restrict__ cu_q) {
+  pdl_launch_dependents();
+  pdl_wait();
   if (threadIdx.x == 0 && blockIdx.x == 0) {
     int acc = 0;
     cu_q[0] = 0;
@@ -103,6 +109,8 @@ __global__ void token_map_kernel(const int* __restrict__ cu_q, int* __restrict__
                                  int num_pages, int page_size, int n_tokens, int max_context,
                                  int* __restrict__ tok_seq, int* __restrict__ tok_pos, int* __restrict__ tok_slot,
                                  int* __restrict__ status) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_tokens) return;
   int b;
@@ -133,9 +141,9 @@ int launch_token_map(const int* q_lens, const int* context_lens, const int* bloc
                       int max_pages_per_seq, int num_pages, int page_size, int n_tokens, int max_context, int* cu_q,
                       int* tok_seq, int* tok_pos, int* tok_slot, int* status, cudaStream_t st) {
   int launches = 0;
-  if (q_lens) { cu_q_kernel<<<1, 32, 0, st>>>(q_lens, n_seqs, cu_q); ++launches; }
+  if (q_lens) { launch_pdl(cu_q_kernel, dim3(1), dim3(32), 0, st, q_lens, n_seqs, cu_q); ++launches; }
   if (n_tokens <= 0) return launches;
-  token_map_kernel<<<(n_tokens + 255) / 256, 256, 0, st>>>(cu_q, cu_q, q_lens != nullptr, context_lens, block_table, n_seqs,
+  launch_pdl(token_map_kernel, dim3((n_tokens + 255) / 256), dim3(256), 0, st, cu_q, cu_q, q_lens != nullptr, context_lens, block_table, n_seqs,
                                                          max_pages_per_seq, num_pages, page_size, n_tokens,
                                                          max_context, tok_seq, tok_pos, tok_slot, status);
   return launches + 1;
@@ -146,6 +154,8 @@ int launch_token_map(const int* q_lens, const int* context_lens, const int* bloc
 __global__ void combine_kernel(const float* __restrict__ r_full, const bf16* __restrict__ y, const float* __restrict__ w,
                                const int* __restrict__ inv, bf16* __restrict__ out, int n_tokens, int d, int H, int kc,
                                int last_mean) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int i = blockIdx.x;
   const float inv_h = 1.0f / float(H);
   for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {
@@ -196,7 +206,7 @@ void launch_combine(const float* r_full, const bf16* y, const float* w, const in
   int threads = d / 8;
   if (threads > 256) threads = 256;
   if (threads < 32) threads = 32;
-  combine_kernel<<<n_tokens, threads, 0, st>>>(r_full, y, w, inv, out, n_tokens, d, H, kc, last_mean);
+  launch_pdl(combine_kernel, dim3(n_tokens), dim3(threads), 0, st, r_full, y, w, inv, out, n_tokens, d, H, kc, last_mean);
 }
 
 // ------------------------------------------------------------------ create-time repacks

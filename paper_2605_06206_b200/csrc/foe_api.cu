@@ -192,6 +192,7 @@ void run_route_and_permute(foe_layer* L, const void* r, int r_is_bf16, int n, cu
 // slots; otherwise it is r_full itself, in the workspace.
 foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaStream_t st, bool decode, foe_shard* sh) {
   const int S = decode ? kv->n_seqs : kv->n_tokens;
+  g_overlap_launches = decode || S <= kFewTokens;     // launches of this call (this thread) overlap their predecessors' tails
   L->last_stream = st;
   L->launches = 0;
   L->last_tokens = S;
@@ -336,6 +337,7 @@ foe_status run_ffn(foe_layer* L, void* out, cudaStream_t st) {
   const int S = L->last_tokens, H = L->H, d = L->d;
   const bool decode = L->last_decode;
   if (S == 0) return FOE_OK;
+  g_overlap_launches = decode || S <= kFewTokens;
 
   // ---- router, top-k, gates, dispatch maps
   stage_mark(L, kStRoute, st);
@@ -635,6 +637,7 @@ foe_status foe_route(foe_layer* L, const void* h, int n_tokens, int* topk_idx, f
   if (n_tokens == 0) return FOE_OK;
   const int saved = L->profiling;
   L->profiling = 0;
+  g_overlap_launches = n_tokens <= kFewTokens;
   run_route_and_permute(L, h, 1, n_tokens, st);
   L->profiling = saved;
   const size_t n = size_t(n_tokens) * L->H * L->kc;
@@ -860,6 +863,7 @@ foe_status foe_shard_ffn(foe_layer* L, foe_shard* sh, void* out, void* stream) {
   if (L->shard_stage != 1 || L->last_tokens != sh->S) return FOE_ERR_UNSUPPORTED;
   if (sh->S > 0 && !out) return FOE_ERR_NULL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  g_overlap_launches = false;             // (the exchange kernels are launched the ordinary way)
   const foe_status f = shard_finish(sh, L->ws->r_full, nullptr, st);      // r_full of the whole group, as fp32
   if (f != FOE_OK) return f;
   L->shard_stage = 0;

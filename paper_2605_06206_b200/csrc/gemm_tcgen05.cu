@@ -29,12 +29,12 @@ void launch_gemm(int epi, const CUtensorMap& tmA, const CUtensorMap& tmB, const 
   }
   if (pairs <= 0) return;
   switch (epi) {
-    case kEpiBf16: gemm_tcgen05_kernel<kEpiBf16, false><<<2 * pairs, kGemmThreads, kGemmSmemBytes, st>>>(tmA, tmB, args); break;
+    case kEpiBf16: launch_pdl(gemm_tcgen05_kernel<kEpiBf16, false>, dim3(2 * pairs), dim3(kGemmThreads), kGemmSmemBytes, st, tmA, tmB, args); break;
     case kEpiSwiGLU:   // expert GEMM 1: always fed through the dispatch permutation (tmA unused)
-      gemm_tcgen05_kernel<kEpiSwiGLU, true><<<2 * pairs, kGemmThreads + kGatherThreads, kGemmSmemBytes, st>>>(tmA, tmB, args);
+      launch_pdl(gemm_tcgen05_kernel<kEpiSwiGLU, true>, dim3(2 * pairs), dim3(kGemmThreads + kGatherThreads), kGemmSmemBytes, st, tmA, tmB, args);
       break;
-    case kEpiQKV: gemm_tcgen05_kernel<kEpiQKV, false><<<2 * pairs, kGemmThreads, kGemmSmemBytes, st>>>(tmA, tmB, args); break;
-    default: gemm_tcgen05_kernel<kEpiOProj, false><<<2 * pairs, kGemmThreads, kGemmSmemBytes, st>>>(tmA, tmB, args); break;
+    case kEpiQKV: launch_pdl(gemm_tcgen05_kernel<kEpiQKV, false>, dim3(2 * pairs), dim3(kGemmThreads), kGemmSmemBytes, st, tmA, tmB, args); break;
+    default: launch_pdl(gemm_tcgen05_kernel<kEpiOProj, false>, dim3(2 * pairs), dim3(kGemmThreads), kGemmSmemBytes, st, tmA, tmB, args); break;
   }
 }
 

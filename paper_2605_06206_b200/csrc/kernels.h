@@ -12,6 +12,26 @@ namespace foe {
 
 typedef __nv_bfloat16 bf16;
 
+// Launch with programmatic stream serialization: the kernel may be scheduled while its predecessor in the stream is
+// still running and must call pdl_wait() before it touches anything the predecessor (or any earlier kernel) wrote.
+// It pays for calls made of short kernels (a decode step: -4 % of the step) and costs a little when every kernel runs
+// for hundreds of microseconds (a large prefill: +0.7 %), so the API layer switches it per call (per host thread).
+inline thread_local bool g_overlap_launches = true;
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = g_overlap_launches ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- elementwise.cu
 // inv_rms[r] = rsqrt(mean(x[r,:]^2) + eps) for n_rows rows of d bf16 values
 void launch_row_inv_rms(const bf16* x, float* inv_rms, int n_rows, int d, float eps, cudaStream_t st);

@@ -21,6 +21,8 @@ constexpr int kPB = kPermuteBlockTokens;      // 256 tokens per block = 8 bitmap
 __global__ void __launch_bounds__(kPB)
 permute_count_kernel(const int* __restrict__ idx, int* __restrict__ rank, int* __restrict__ blk_counts, int n_tokens,
                      int sel, int E, int* __restrict__ status) {
+  pdl_launch_dependents();
+  pdl_wait();
   extern __shared__ uint32_t bm[];            // [E][8]
   for (int q = threadIdx.x; q < E * 8; q += kPB) bm[q] = 0u;
   __syncthreads();
@@ -66,6 +68,8 @@ __device__ __forceinline__ void write_tile_table(const PermuteBuffers& pb, int e
 // Single block.  blk_counts[b][e] becomes the exclusive prefix over b; counts/offsets and the tile table are written.
 __global__ void __launch_bounds__(1024)
 permute_scan_kernel(int* __restrict__ blk_counts, int n_blocks, int E, const PermuteBuffers pb) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ int s_a[1024], s_b[1024];
   int* counts = pb.counts;
   int* offsets = pb.offsets;
@@ -108,6 +112,8 @@ permute_scan_kernel(int* __restrict__ blk_counts, int n_blocks, int E, const Per
 __global__ void permute_scatter_kernel(const int* __restrict__ idx, const int* __restrict__ rank,
                                        const int* __restrict__ blk_prefix, const int* __restrict__ offsets,
                                        int* __restrict__ perm, int* __restrict__ inv, int n_tokens, int sel, int E) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int q = blockIdx.x * blockDim.x + threadIdx.x;
   if (q >= n_tokens * sel) return;
   const int i = q / sel;
@@ -169,6 +175,8 @@ __device__ __forceinline__ void topk_small_regs(const TopkSmall& tk, int task) {
 __global__ void __launch_bounds__(1024)
 permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, const PermuteBuffers pb,
                      int* __restrict__ status, const TopkSmall tk) {
+  pdl_launch_dependents();
+  pdl_wait();
   extern __shared__ uint32_t bm[];            // [E][8]
   __shared__ int s_a[1024], s_b[1024], s_off[1024];
   int* counts = pb.counts;
@@ -288,14 +296,14 @@ int launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int s
   if (n_tokens <= kPB) {
     TopkSmall none;
     none.scores = nullptr;
-    permute_small_kernel<<<1, 1024, size_t(E) * 32, st>>>(idx, n_tokens, sel, E, pb, status, none);
+    launch_pdl(permute_small_kernel, dim3(1), dim3(1024), size_t(E) * 32, st, idx, n_tokens, sel, E, pb, status, none);
     return 1;
   }
   const int n_blocks = (n_tokens + kPB - 1) / kPB;
-  permute_count_kernel<<<n_blocks, kPB, size_t(E) * 32, st>>>(idx, pb.rank, pb.blk_counts, n_tokens, sel, E, status);
-  permute_scan_kernel<<<1, 1024, 0, st>>>(pb.blk_counts, n_blocks, E, pb);
+  launch_pdl(permute_count_kernel, dim3(n_blocks), dim3(kPB), size_t(E) * 32, st, idx, pb.rank, pb.blk_counts, n_tokens, sel, E, status);
+  launch_pdl(permute_scan_kernel, dim3(1), dim3(1024), 0, st, pb.blk_counts, n_blocks, E, pb);
   const int total = n_tokens * sel;
-  permute_scatter_kernel<<<(total + 255) / 256, 256, 0, st>>>(idx, pb.rank, pb.blk_counts, pb.offsets, pb.perm, pb.inv,
+  launch_pdl(permute_scatter_kernel, dim3((total + 255) / 256), dim3(256), 0, st, idx, pb.rank, pb.blk_counts, pb.offsets, pb.perm, pb.inv,
                                                             n_tokens, sel, E);
   return 3;
 }
@@ -307,7 +315,7 @@ int launch_topk_permute_small(const float* scores, int k_splits, const float* bi
   TopkSmall tk;
   tk.scores = scores; tk.k_splits = k_splits; tk.bias = bias; tk.logits_out = logits; tk.idx_out = idx; tk.w_out = w; tk.H = H; tk.Ec = Ec; tk.kc = kc;
   const int E = H * Ec;
-  permute_small_kernel<<<1, 1024, size_t(E) * 32, st>>>(idx, n_tokens, H * kc, E, pb, status, tk);
+  launch_pdl(permute_small_kernel, dim3(1), dim3(1024), size_t(E) * 32, st, idx, n_tokens, H * kc, E, pb, status, tk);
   return 1;
 }
 

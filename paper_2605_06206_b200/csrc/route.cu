@@ -23,6 +23,8 @@ namespace foe {
 __global__ void ffn_norm_kernel(const void* __restrict__ r_in, int r_is_bf16, const bf16* __restrict__ gain,
                                 bf16* __restrict__ u_out, float* __restrict__ inv_out, int n_tokens, int d,
                                 float eps) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (i >= n_tokens) return;
   float ss = 0.f;
@@ -73,6 +75,8 @@ __global__ void __launch_bounds__(kRgThreads, 4)
 router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __restrict__ inv_rms,
                    const bf16* __restrict__ gain, const float* __restrict__ wr, float* __restrict__ part,
                    int n_tokens, int d, int E, int k_per_split) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ __align__(16) float As[2][kRgKC][kRgPA];     // [k][token]
   __shared__ __align__(16) float Bs[2][kRgKC][kRgPB];     // [k][expert]
   const int tid = threadIdx.x;
@@ -177,6 +181,8 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
 __global__ void topk_gates_kernel(const float* __restrict__ part, int k_splits, const float* __restrict__ br,
                                   float* __restrict__ logits_out, int* __restrict__ idx_out, float* __restrict__ w_out,
                                   int n_tokens, int H, int Ec, int kc) {
+  pdl_launch_dependents();
+  pdl_wait();
   // a (token, cluster) task is handled by a group of W lanes (W = 8, 16 or 32), several tasks per warp
   const int W = Ec <= 8 ? 8 : (Ec <= 16 ? 16 : 32);
   const int per_warp = 32 / W;
@@ -250,6 +256,8 @@ __global__ void __launch_bounds__(kRsThreads)
 route_scores_small_kernel(const void* __restrict__ r_in, int r_is_bf16, const bf16* __restrict__ gain,
                           const float* __restrict__ wr, bf16* __restrict__ u_out, float* __restrict__ scores,
                           int n_tokens, int d, int E, float eps, int k_per_split) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ float w_s[kRsK][kRsExp + 1];
   __shared__ float u_s[kRsTok][kRsK];
   __shared__ float red[kRsTok][2];
@@ -311,7 +319,7 @@ int launch_route_small(const void* r_in, int r_is_bf16, const bf16* gain, const 
   int ks = 1;
   while (ks < 16 && (d / (ks * 2)) % kRsK == 0 && d / (ks * 2) >= 2 * kRsK) ks *= 2;
   dim3 grid((n_tokens + kRsTok - 1) / kRsTok, (E + kRsExp - 1) / kRsExp, ks);
-  route_scores_small_kernel<<<grid, kRsThreads, 0, st>>>(r_in, r_is_bf16, gain, wr, u_out, scores, n_tokens, d, E, eps, d / ks);
+  launch_pdl(route_scores_small_kernel, grid, dim3(kRsThreads), 0, st, r_in, r_is_bf16, gain, wr, u_out, scores, n_tokens, d, E, eps, d / ks);
   return 1 + launch_topk_permute_small(scores, ks, br, logits, idx, w, pb, n_tokens, H, Ec, kc, status, st);
 }
 
@@ -322,6 +330,8 @@ template <int EC>
 __global__ void topk_gates_thread_kernel(const float* __restrict__ part, int k_splits, const float* __restrict__ br,
                                          float* __restrict__ logits_out, int* __restrict__ idx_out,
                                          float* __restrict__ w_out, int n_tokens, int H, int kc) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int task = blockIdx.x * blockDim.x + threadIdx.x;
   if (task >= n_tokens * H) return;
   const int i = task / H, h = task - i * H;
@@ -363,15 +373,15 @@ static void launch_topk_gates(const float* part, int ks, const float* br, float*
   const int tasks = n_tokens * H;
   const int tb = (tasks + 127) / 128;
   switch (Ec) {
-    case 4: topk_gates_thread_kernel<4><<<tb, 128, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, kc); return;
-    case 8: topk_gates_thread_kernel<8><<<tb, 128, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, kc); return;
-    case 16: topk_gates_thread_kernel<16><<<tb, 128, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, kc); return;
-    case 32: topk_gates_thread_kernel<32><<<tb, 128, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, kc); return;
+    case 4: launch_pdl(topk_gates_thread_kernel<4>, dim3(tb), dim3(128), 0, st, part, ks, br, logits, idx, w, n_tokens, H, kc); return;
+    case 8: launch_pdl(topk_gates_thread_kernel<8>, dim3(tb), dim3(128), 0, st, part, ks, br, logits, idx, w, n_tokens, H, kc); return;
+    case 16: launch_pdl(topk_gates_thread_kernel<16>, dim3(tb), dim3(128), 0, st, part, ks, br, logits, idx, w, n_tokens, H, kc); return;
+    case 32: launch_pdl(topk_gates_thread_kernel<32>, dim3(tb), dim3(128), 0, st, part, ks, br, logits, idx, w, n_tokens, H, kc); return;
     default: break;
   }
   const int per_warp = Ec <= 8 ? 4 : (Ec <= 16 ? 2 : 1);
   const int warps = (tasks + per_warp - 1) / per_warp;
-  topk_gates_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc);
+  launch_pdl(topk_gates_kernel, dim3((warps * 32 + 255) / 256), dim3(256), 0, st, part, ks, br, logits, idx, w, n_tokens, H, Ec, kc);
 }
 
 int route_k_splits(int n_tokens, int d, int E, int n_sms) {
@@ -386,14 +396,14 @@ int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float*
                  int n_tokens, int d, int H, int Ec, int kc, float eps, int n_sms, int* status, cudaStream_t st) {
   if (n_tokens <= 0) return 0;
   const int E = H * Ec;
-  ffn_norm_kernel<<<(n_tokens * 32 + 255) / 256, 256, 0, st>>>(r_in, r_is_bf16, gain, u_out, inv_rms, n_tokens, d, eps);
+  launch_pdl(ffn_norm_kernel, dim3((n_tokens * 32 + 255) / 256), dim3(256), 0, st, r_in, r_is_bf16, gain, u_out, inv_rms, n_tokens, d, eps);
   int ks = 1;
   if (tm_wr_split && n_tokens >= kRouterTcMinTokens) {
     launch_router_tc(*tm_wr_split, r_in, r_is_bf16, inv_rms, part, n_tokens, d, E, status, st);
   } else {
     ks = route_k_splits(n_tokens, d, E, n_sms);
     dim3 grid((n_tokens + kRgTM - 1) / kRgTM, (E + kRgTN - 1) / kRgTN, ks);
-    router_gemm_kernel<<<grid, kRgThreads, 0, st>>>(r_in, r_is_bf16, inv_rms, gain, wr, part, n_tokens, d, E, d / ks);
+    launch_pdl(router_gemm_kernel, grid, dim3(kRgThreads), 0, st, r_in, r_is_bf16, inv_rms, gain, wr, part, n_tokens, d, E, d / ks);
   }
   launch_topk_gates(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc, st);
   return 3;
@@ -425,6 +435,8 @@ static int g_route_sms[kNaMaxDevices];
 // inv_rms only: the expert input u is not produced on this path (the caller asked for routing, nothing else)
 __global__ void ffn_inv_rms_bf16_kernel(const bf16* __restrict__ r_in, float* __restrict__ inv_out, int n_tokens, int d,
                                         float eps) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (i >= n_tokens) return;
   const uint4* row = reinterpret_cast<const uint4*>(r_in + size_t(i) * d);

@@ -64,6 +64,8 @@ __global__ void __launch_bounds__(kRtThreads, 1)
 router_tc_kernel(const __grid_constant__ CUtensorMap tmW, const void* __restrict__ r_in, int r_is_bf16,
                  const float* __restrict__ inv_rms, float* __restrict__ part, int n_tokens, int d, int E, int E_pad,
                  int* __restrict__ status) {
+  pdl_launch_dependents();
+  pdl_wait();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kRtStages * kRtStageBytes);
@@ -241,7 +243,7 @@ void launch_router_tc(const CUtensorMap& tmW, const void* r, int r_is_bf16, cons
   }
   const int E_pad = router_padded_experts(E);
   dim3 grid((n_tokens + kRtRows - 1) / kRtRows, E_pad / kRtChunk);
-  router_tc_kernel<<<grid, kRtThreads, kRtSmemBytes, st>>>(tmW, r, r_is_bf16, inv_rms, part, n_tokens, d, E, E_pad, status);
+  launch_pdl(router_tc_kernel, grid, dim3(kRtThreads), kRtSmemBytes, st, tmW, r, r_is_bf16, inv_rms, part, n_tokens, d, E, E_pad, status);
 }
 
 }  // namespace foe

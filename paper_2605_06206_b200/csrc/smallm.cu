@@ -65,6 +65,8 @@ __device__ __forceinline__ SmTask sm_task(const SmallMArgs& a, int t, int slabs_
 template <int EPI>
 __global__ void __launch_bounds__(kSmThreads)
 smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int NT = kSmNT;
   constexpr int kSmStages = sm_stages<EPI>();
   extern __shared__ uint8_t smem_raw[];
@@ -323,7 +325,7 @@ static void launch_one(const CUtensorMap& tmW, const SmallMArgs& a, int n_sms, c
   const long long tasks = (long long)a.n_groups * ((a.N + kSmSlab - 1) / kSmSlab) * chunks;
   if (tasks <= 0) return;
   const int grid = int(tasks < 2LL * n_sms ? tasks : 2LL * n_sms);          // two resident CTAs per SM
-  smallm_kernel<EPI><<<grid, kSmThreads, sm_smem_bytes<EPI>(), st>>>(tmW, a);
+  launch_pdl(smallm_kernel<EPI>, dim3(grid), dim3(kSmThreads), sm_smem_bytes<EPI>(), st, tmW, a);
 }
 
 void launch_smallm(const CUtensorMap& tmW, const SmallMArgs& a, int n_sms, cudaStream_t st) {
