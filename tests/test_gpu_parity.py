@@ -283,6 +283,41 @@ def test_repeated_prefill_is_bit_stable_under_timing_noise(dh, q_lens, ctx):
     layer.close()
 
 
+@pytest.mark.parametrize("decode,n", [(True, 64), (True, 9), (False, 100), (False, 1)])
+def test_repeated_small_calls_are_bit_stable_with_overlapping_launches(decode, n):
+    """Decode steps and small prefill calls launch every kernel so that it may start while its predecessor drains
+    (a kernel waits for the predecessor only where it first touches its results).  Back-to-back repeats without any
+    host synchronisation in between, partly with other work queued on the device first, must give the same bits."""
+    shape = synth.LayerShape(512, 8, 2, 2, 128, 4, 2, 256)
+    W = scaled_weights(shape, 31, "cuda", 4.0)
+    if decode:
+        q_lens, ctx = [1] * n, [(53 * i) % 700 + 1 for i in range(n)]
+    else:
+        q_lens, ctx = [n], [70]
+    S = sum(q_lens)
+    x = synth.make_x(shape, 31, S, "cuda")
+    layer = binding.FoeLayer(shape, W, max_tokens=S, max_seqs=len(q_lens), max_context=max(c + q for c, q in zip(ctx, q_lens)))
+    kv = synth.make_paged_cache(shape, 31, ctx, q_lens, "cuda")
+    run = (lambda: layer.decode(x, kv)) if decode else (lambda: layer.prefill(x, kv))
+    first = run().clone()
+    first_aux = layer.aux()
+    k0, v0 = kv.k_pages.clone(), kv.v_pages.clone()
+    outs = []
+    for it in range(150):
+        if it % 7 == 3:
+            torch.empty(160 << 20, dtype=torch.uint8, device="cuda").fill_(1)     # something else in the queue, L2 flushed
+        outs.append(run().clone())                   # (the call rewrites the same K/V slots with the same values)
+    torch.cuda.synchronize()
+    assert layer.poll_status() == 0
+    for it, o in enumerate(outs):
+        assert torch.equal(o, first), f"repeat {it} differs"
+    aux = layer.aux()
+    for k in ("r_full", "topk_idx", "attn_o", "perm"):
+        assert torch.equal(aux[k], first_aux[k]), k
+    assert torch.equal(kv.k_pages, k0) and torch.equal(kv.v_pages, v0)
+    layer.close()
+
+
 # ------------------------------------------------------------------------------------------ error paths (host side)
 def test_host_side_argument_errors():
     shape = shape_small()
