@@ -112,6 +112,7 @@ struct foe_shard {
 namespace {
 
 constexpr int kFewTokens = 256;                  // calls up to this size take the decode-step kernels where they fit
+constexpr int kOverlapTokens = 2048;             // calls up to this size launch their kernels with programmatic dependent launch
 constexpr size_t kShardHeaderBytes = 1024;       // slot counters at 0, gather counters at 128
 
 bool shard_config_ok(const foe_shard_config* c) {
@@ -192,7 +193,7 @@ void run_route_and_permute(foe_layer* L, const void* r, int r_is_bf16, int n, cu
 // slots; otherwise it is r_full itself, in the workspace.
 foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaStream_t st, bool decode, foe_shard* sh) {
   const int S = decode ? kv->n_seqs : kv->n_tokens;
-  g_overlap_launches = decode || S <= kFewTokens;     // launches of this call (this thread) overlap their predecessors' tails
+  g_overlap_launches = decode || S <= kOverlapTokens; // launches of this call (this thread) overlap their predecessors' tails
   L->last_stream = st;
   L->launches = 0;
   L->last_tokens = S;
@@ -337,7 +338,7 @@ foe_status run_ffn(foe_layer* L, void* out, cudaStream_t st) {
   const int S = L->last_tokens, H = L->H, d = L->d;
   const bool decode = L->last_decode;
   if (S == 0) return FOE_OK;
-  g_overlap_launches = decode || S <= kFewTokens;
+  g_overlap_launches = decode || S <= kOverlapTokens;
 
   // ---- router, top-k, gates, dispatch maps
   stage_mark(L, kStRoute, st);
@@ -637,7 +638,7 @@ foe_status foe_route(foe_layer* L, const void* h, int n_tokens, int* topk_idx, f
   if (n_tokens == 0) return FOE_OK;
   const int saved = L->profiling;
   L->profiling = 0;
-  g_overlap_launches = n_tokens <= kFewTokens;
+  g_overlap_launches = n_tokens <= kOverlapTokens;
   run_route_and_permute(L, h, 1, n_tokens, st);
   L->profiling = saved;
   const size_t n = size_t(n_tokens) * L->H * L->kc;
