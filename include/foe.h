@@ -24,7 +24,9 @@
  *    into library-owned device buffers, so the caller may release its copies afterwards.  The
  *    handle owns a workspace sized by max_tokens / max_seqs / max_context.
  *  - Calls are asynchronous on the given stream (a cudaStream_t passed as void*).  A handle is
- *    used from one stream at a time.  Same inputs give bit-identical outputs and maps.
+ *    used from one stream at a time.  Same inputs give bit-identical outputs and maps.  After one
+ *    ordinary call per entry point and call size class (it sets kernel attributes once) a call only
+ *    launches kernels, so it can be captured into a CUDA graph.
  *  - Every function returns a foe_status; argument and shape checks happen on the host before
  *    anything is launched.  Conditions only the device can see (a bounded wait that ran out, an
  *    out-of-range page id) are recorded in a device status word read by foe_poll_status.

@@ -318,6 +318,38 @@ def test_repeated_small_calls_are_bit_stable_with_overlapping_launches(decode, n
     layer.close()
 
 
+@pytest.mark.parametrize("decode", [True, False])
+def test_calls_can_be_captured_into_a_cuda_graph(decode):
+    """After one ordinary call (which does the one-time kernel configuration) a call only launches kernels on the
+    given stream, so it can be captured; replays give the direct call's bits."""
+    shape = synth.LayerShape(512, 8, 2, 2, 128, 4, 2, 256)
+    W = scaled_weights(shape, 33, "cuda", 4.0)
+    if decode:
+        q_lens, ctx = [1] * 20, [(41 * i) % 500 + 3 for i in range(20)]
+    else:
+        q_lens, ctx = [300, 41], [0, 100]
+    S = sum(q_lens)
+    x = synth.make_x(shape, 33, S, "cuda")
+    kv = synth.make_paged_cache(shape, 33, ctx, q_lens, "cuda")
+    layer = binding.FoeLayer(shape, W, max_tokens=S, max_seqs=len(q_lens), max_context=max(c + q for c, q in zip(ctx, q_lens)))
+    out = torch.empty_like(x)
+    mq = max(q_lens)
+    run = (lambda: layer.decode(x, kv, out=out)) if decode else (lambda: layer.prefill(x, kv, n_tokens=S, max_q_len=mq, out=out))
+    run()
+    torch.cuda.synchronize()
+    ref = out.clone()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        run()
+    for _ in range(3):
+        out.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, ref)
+    assert layer.poll_status() == 0
+    layer.close()
+
+
 # ------------------------------------------------------------------------------------------ error paths (host side)
 def test_host_side_argument_errors():
     shape = shape_small()
