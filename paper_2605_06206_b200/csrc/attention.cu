@@ -61,7 +61,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   const int n_tiles = p_end - p_begin;
   const int G = a.n_q / a.n_kv;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tok = a.cu_q[b];
+  const int tok = a.cu_q ? a.cu_q[b] : b;
   const int ld_q = a.n_q * DH;
 
   if (threadIdx.x == 0) {

@@ -228,7 +228,20 @@ decode_proj_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         const int t = t_lo + (q >> 6), p = q & 63;
         if (t >= n_tok) continue;
         const int tok = tok0 + t;
-        const int pos = a.tok_pos[tok];
+        int pos, slot;
+        if (a.tok_pos) {
+          pos = a.tok_pos[tok];
+          slot = a.tok_slot[tok];
+        } else {                                          // decode step: position and cache slot of sequence `tok`
+          pos = a.context_lens[tok];
+          const int lp = pos >> 6;
+          slot = -1;
+          if (lp < a.max_pages_per_seq && pos < a.max_context) {
+            const int page = a.block_table[size_t(tok) * a.max_pages_per_seq + lp];
+            if (page >= 0 && page < a.num_pages) slot = page * 64 + (pos & 63);
+          }
+          if (slot < 0) { atomicExch(a.status, kStatusBounds); pos = min(max(pos, 0), a.max_context - 1); }
+        }
         float2 pv[8];
         float sq[8];
 #pragma unroll
@@ -262,7 +275,6 @@ decode_proj_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         } else {
           const int nn = n - a.q_cols - (is_k ? 0 : a.kv_cols);
           const int kvh = group * (a.kv_cols / a.dh) + nn / a.dh;
-          const int slot = a.tok_slot[tok];
           if (slot >= 0) {
             bf16* o = (is_k ? a.k_pages : a.v_pages) + ((size_t(slot >> 6) * a.n_kv + kvh) * 64 + (slot & 63)) * a.dh;
             o[i] = __float2bfloat16_rn(lo);

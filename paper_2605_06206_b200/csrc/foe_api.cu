@@ -210,7 +210,10 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
 
   // ---- prep: token map and pre-attention RMS statistics
   stage_mark(L, kStPrep, st);
-  L->launches += launch_token_map(decode ? nullptr : kv->q_lens, kv->context_lens, kv->block_table, kv->n_seqs, kv->max_pages_per_seq,
+  // (a decode step whose QKV projection runs on the tensor-core kernel needs no token map: token b is sequence b,
+  //  its position and cache slot are looked up where they are used)
+  const bool inline_map = decode && L->dp_qkv;
+  if (!inline_map) L->launches += launch_token_map(decode ? nullptr : kv->q_lens, kv->context_lens, kv->block_table, kv->n_seqs, kv->max_pages_per_seq,
                    kv->num_pages, 64, S, L->cfg.max_context, L->ws->cu_q, L->ws->tok_seq, L->ws->tok_pos, L->ws->tok_slot, L->ws->status, st);
   const int x_rows = L->first ? S : H * S;
   // Kernel family of the two projections: a call of a few hundred tokens (any decode step, a short prompt chunk, a
@@ -253,6 +256,11 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
     pa.q_cols = L->g * dh; pa.kv_cols = L->c * dh; pa.dh = dh; pa.n_kv = L->n_kv;
     pa.rope_tab = L->rope_tab; pa.tok_pos = L->ws->tok_pos; pa.tok_slot = L->ws->tok_slot;
     pa.k_pages = static_cast<bf16*>(kv->k_pages); pa.v_pages = static_cast<bf16*>(kv->v_pages);
+    if (inline_map) {
+      pa.tok_pos = nullptr; pa.tok_slot = nullptr;
+      pa.context_lens = kv->context_lens; pa.block_table = kv->block_table; pa.max_pages_per_seq = kv->max_pages_per_seq;
+      pa.num_pages = kv->num_pages; pa.max_context = L->cfg.max_context;
+    }
     launch_decode_proj(L->tmt_wqkv, tmX, pa, L->n_sms, st);
   } else {
     SmallMArgs sa;
@@ -273,7 +281,7 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
   stage_mark(L, kStAttn, st);
   AttnArgs aa;
   memset(&aa, 0, sizeof(aa));
-  aa.q = L->ws->qkv; aa.out = L->ws->attn_o; aa.cu_q = L->ws->cu_q; aa.context_lens = kv->context_lens;
+  aa.q = L->ws->qkv; aa.out = L->ws->attn_o; aa.cu_q = inline_map ? nullptr : L->ws->cu_q; aa.context_lens = kv->context_lens;
   aa.q_lens = decode ? nullptr : kv->q_lens; aa.block_table = kv->block_table; aa.n_seqs = kv->n_seqs;
   aa.max_pages_per_seq = kv->max_pages_per_seq; aa.num_pages = kv->num_pages; aa.n_q = L->n_q; aa.n_kv = L->n_kv;
   aa.dh = dh; aa.max_q_len = decode ? 1 : kv->max_q_len; aa.scale_log2 = float(1.4426950408889634 / sqrt(double(dh)));

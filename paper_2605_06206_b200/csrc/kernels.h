@@ -103,7 +103,7 @@ int launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int s
 struct AttnArgs {
   const bf16* q;            // [S][n_q*dh] queries after RoPE
   bf16* out;                // [S][n_q*dh]
-  const int* cu_q;          // [n_seqs+1]
+  const int* cu_q;          // [n_seqs+1]; nullptr in a decode step: sequence b's token is token b
   const int* context_lens;  // [n_seqs]
   const int* q_lens;        // [n_seqs] or nullptr (1 each)
   const int* block_table;   // [n_seqs][max_pages_per_seq]
@@ -167,6 +167,9 @@ struct DecodeProjArgs {
   float rms_eps;
   int q_cols, kv_cols, dh, n_kv, q_head_stride;
   const float2* rope_tab; const int* tok_pos; const int* tok_slot; bf16* k_pages; bf16* v_pages;
+  // kEpiQKV of a decode step (tok_pos == nullptr): token t is the one new token of sequence t; its position is
+  // context_lens[t] and its cache slot comes from the block table, both looked up in the epilogue (no token-map kernel)
+  const int* context_lens; const int* block_table; int max_pages_per_seq, num_pages, max_context;
   // kEpiOProj
   const bf16* xsum; int x_count; size_t x_stride; float out_scale;
 };

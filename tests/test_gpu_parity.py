@@ -370,6 +370,14 @@ def test_host_side_argument_errors():
     layer.prefill(synth.make_x(shape, 27, 8, "cuda"), kv)
     assert layer.poll_status() == -8
     assert layer.poll_status() == 0
+    # the same in a decode step, where position and slot are looked up inside the QKV projection
+    kv = synth.make_paged_cache(shape, 27, [20], [1], "cuda")
+    kv.block_table[0, 0] = -3
+    layer.decode(synth.make_x(shape, 27, 1, "cuda"), kv)
+    assert layer.poll_status() == -8
+    kv = synth.make_paged_cache(shape, 27, [63], [1], "cuda")          # position 63 is fine, position 64 = max_context is not
+    layer.decode(synth.make_x(shape, 27, 1, "cuda"), kv)
+    assert layer.poll_status() == 0
     layer.close()
 
 

@@ -78,8 +78,8 @@ def test_group_prefill_positions_and_sync_modes(position, sync):
 def test_group_decode(position):
     res = run_group(shape_small(position=position), 12, [1] * 9, [5, 64, 127, 128, 300, 1, 77, 640, 63], decode=True,
                     also_one_device=(position == "middle"))
-    # token map, QKV, attention, O-proj, push | gather | two route launches, two expert GEMMs, combine
-    assert all(n == 11 for n in res["launches"])
+    # QKV, attention, O-proj, push | gather | two route launches, two expert GEMMs, combine
+    assert all(n == 10 for n in res["launches"])
 
 
 def test_group_several_tiles_ragged_tail_head_dim_128():
