@@ -42,7 +42,6 @@ template <int DH>
 __global__ void __launch_bounds__(kDcThreads, 2)
 attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
   pdl_launch_dependents();
-  pdl_wait();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int kTileBytes = 64 * DH * 2;
@@ -51,6 +50,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   uint8_t* q_s = smem + kDcStages * 2 * kTileBytes;
   uint64_t* full = reinterpret_cast<uint64_t*>(q_s + kQBytes);
 
+  // Until pdl_wait() only the caller's inputs are read (context lengths, block table, cached pages): this grid may
+  // start while the QKV projection of the same step is still running, and that kernel writes q and the new token's
+  // K / V (into the sequence's last page).
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int ctx = a.context_lens[b];
   const int kv_len = ctx + 1;                                      // cached tokens + the new one
@@ -61,20 +63,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   const int n_tiles = p_end - p_begin;
   const int G = a.n_q / a.n_kv;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tok = a.cu_q ? a.cu_q[b] : b;
   const int ld_q = a.n_q * DH;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kDcStages; ++s) mbar_init(&full[s], 1);
-    mbar_fence_init();
-  }
-  for (int q = threadIdx.x; q < 16 * (DH / 8); q += kDcThreads) {
-    const int r = q / (DH / 8), ch = q - r * (DH / 8);
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (r < G) v = __ldg(reinterpret_cast<const uint4*>(a.q + size_t(tok) * ld_q + (kvh * G + r) * DH + ch * 8));
-    *reinterpret_cast<uint4*>(q_s + tile_off<16>(r, ch * 8)) = v;
-  }
-  __syncthreads();
 
   auto page_row0 = [&](int lp) -> int {
     int page = a.block_table[size_t(b) * a.max_pages_per_seq + min(lp, a.max_pages_per_seq - 1)];
@@ -82,10 +71,28 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     return (page * a.n_kv + kvh) * 64;
   };
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kDcStages && s < n_tiles; ++s)
-      tma_load_page<DH>(kv_s + s * 2 * kTileBytes, kv_s + s * 2 * kTileBytes + kTileBytes, &tmK, &tmV, &full[s],
-                        page_row0(p_begin + s));
+    for (int s = 0; s < kDcStages; ++s) mbar_init(&full[s], 1);
+    mbar_fence_init();
+    for (int s = 0; s < kDcStages && s < n_tiles; ++s)             // the ring's first tiles, except the page being written
+      if (p_begin + s != n_pages - 1)
+        tma_load_page<DH>(kv_s + s * 2 * kTileBytes, kv_s + s * 2 * kTileBytes + kTileBytes, &tmK, &tmV, &full[s],
+                          page_row0(p_begin + s));
   }
+  pdl_wait();
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kDcStages && s < n_tiles; ++s)
+      if (p_begin + s == n_pages - 1)
+        tma_load_page<DH>(kv_s + s * 2 * kTileBytes, kv_s + s * 2 * kTileBytes + kTileBytes, &tmK, &tmV, &full[s],
+                          page_row0(p_begin + s));
+  }
+  const int tok = a.cu_q ? a.cu_q[b] : b;
+  for (int q = threadIdx.x; q < 16 * (DH / 8); q += kDcThreads) {
+    const int r = q / (DH / 8), ch = q - r * (DH / 8);
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (r < G) v = __ldg(reinterpret_cast<const uint4*>(a.q + size_t(tok) * ld_q + (kvh * G + r) * DH + ch * 8));
+    *reinterpret_cast<uint4*>(q_s + tile_off<16>(r, ch * 8)) = v;
+  }
+  __syncthreads();
 
   float o[DH / 8][4];
 #pragma unroll
