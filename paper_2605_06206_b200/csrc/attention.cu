@@ -41,7 +41,6 @@ constexpr int kDcStages = 3;
 template <int DH>
 __global__ void __launch_bounds__(kDcThreads, 2)
 attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
-  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int kTileBytes = 64 * DH * 2;
@@ -50,9 +49,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   uint8_t* q_s = smem + kDcStages * 2 * kTileBytes;
   uint64_t* full = reinterpret_cast<uint64_t*>(q_s + kQBytes);
 
-  // Until pdl_wait() only the caller's inputs are read (context lengths, block table, cached pages): this grid may
-  // start while the QKV projection of the same step is still running, and that kernel writes q and the new token's
-  // K / V (into the sequence's last page).
+  // Until pdl_wait() nothing is read that the previous kernel writes: this grid may start while the QKV projection of
+  // the same step is still running, and that kernel writes q and the new token's K / V (into the sequence's last
+  // page).  Everything older is complete (a kernel lets its successor start only after its own wait).
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int ctx = a.context_lens[b];
   const int kv_len = ctx + 1;                                      // cached tokens + the new one
@@ -79,6 +78,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
                           page_row0(p_begin + s));
   }
   pdl_wait();
+  pdl_launch_dependents();
   if (threadIdx.x == 0) {
     for (int s = 0; s < kDcStages && s < n_tiles; ++s)
       if (p_begin + s == n_pages - 1)

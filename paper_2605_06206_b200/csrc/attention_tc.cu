@@ -62,8 +62,8 @@ template <int DH>
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   using L = AtSmem<DH>;
   constexpr int HN = DH / 64;
   extern __shared__ uint8_t smem_raw[];

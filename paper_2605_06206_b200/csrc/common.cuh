@@ -226,6 +226,9 @@ __device__ __forceinline__ float warp_sum(float v) {
 // pdl_launch_dependents: the next kernel in the stream (launched with programmatic stream serialization) may start
 // being scheduled once every CTA of this grid has said so; pdl_wait: returns when the previous kernel has completed
 // and its writes are visible.  Both are no-ops for kernels launched the ordinary way.
+// Rule of this library: a kernel calls pdl_launch_dependents only AFTER its own pdl_wait.  So when a kernel's code
+// before its wait runs, every kernel but its immediate predecessor has completed, and that code may read anything
+// the predecessor does not write (weights always; cached KV pages other than the one being written).
 namespace foe {
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

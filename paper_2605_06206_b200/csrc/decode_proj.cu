@@ -76,7 +76,6 @@ template <int EPI>
 __global__ void __launch_bounds__(kDpThreads, 1)
 decode_proj_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                    const DecodeProjArgs a) {
-  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kDpStages * kDpStageBytes);
@@ -124,6 +123,7 @@ decode_proj_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         tma_load_2d(smem + i * kDpStageBytes, &tmW, &full_bar[i], (kb0 + i) * kDpBK, w_row);
       }
       pdl_wait();
+      pdl_launch_dependents();
       for (int i = 0; i < n_first; ++i)
         tma_load_2d(smem + i * kDpStageBytes + kDpWBytes, &tmX, &full_bar[i], (kb0 + i) * kDpBK, x_row);
       for (int kb = kb0 + n_first; kb < kb1; ++kb) {

@@ -9,8 +9,8 @@ namespace foe {
 // and the scale is applied in the GEMM epilogue, so the normalised tensor is never written.
 __global__ void row_inv_rms_kernel(const bf16* __restrict__ x, float* __restrict__ inv_rms, int n_rows, int d,
                                    float eps) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (warp >= n_rows) return;
@@ -35,8 +35,8 @@ __global__ void row_inv_rms_kernel(const bf16* __restrict__ x, float* __restrict
 template <int H>
 __global__ void row_inv_rms_xsum_kernel(const bf16* __restrict__ x, float* __restrict__ inv_rms, float* __restrict__ xsum,
                                         int S, int d, float eps) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (s >= S) return;
@@ -95,8 +95,8 @@ void launch_row_inv_rms(const bf16* x, float* inv_rms, int n_rows, int d, float 
 
 // ------------------------------------------------------------------ token -> (sequence, position, cache slot)
 __global__ void cu_q_kernel(const int* __restrict__ q_lens, int n_seqs, int* __restrict__ cu_q) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   if (threadIdx.x == 0 && blockIdx.x == 0) {
     int acc = 0;
     cu_q[0] = 0;
@@ -109,8 +109,8 @@ __global__ void token_map_kernel(const int* __restrict__ cu_q, int* __restrict__
                                  int num_pages, int page_size, int n_tokens, int max_context,
                                  int* __restrict__ tok_seq, int* __restrict__ tok_pos, int* __restrict__ tok_slot,
                                  int* __restrict__ status) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_tokens) return;
   int b;
@@ -154,8 +154,8 @@ int launch_token_map(const int* q_lens, const int* context_lens, const int* bloc
 __global__ void combine_kernel(const float* __restrict__ r_full, const bf16* __restrict__ y, const float* __restrict__ w,
                                const int* __restrict__ inv, bf16* __restrict__ out, int n_tokens, int d, int H, int kc,
                                int last_mean) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int i = blockIdx.x;
   const float inv_h = 1.0f / float(H);
   for (int c = threadIdx.x * 8; c < d; c += blockDim.x * 8) {

@@ -279,7 +279,6 @@ template <int EPI, bool GATHER>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads + (GATHER ? kGatherThreads : 0), 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const GemmArgs args) {
-  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stg_all = smem + kStages * kStageBytes;
@@ -318,6 +317,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();                                            // (barriers, tensor memory and descriptors were set up meanwhile)
+  pdl_launch_dependents();
 
   // tiles: groups are cut into 256-row pair tiles (the device-built table for the ragged experts uses the same size)
   const bool ragged = args.n_mtiles != nullptr;

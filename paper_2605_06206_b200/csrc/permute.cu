@@ -21,8 +21,8 @@ constexpr int kPB = kPermuteBlockTokens;      // 256 tokens per block = 8 bitmap
 __global__ void __launch_bounds__(kPB)
 permute_count_kernel(const int* __restrict__ idx, int* __restrict__ rank, int* __restrict__ blk_counts, int n_tokens,
                      int sel, int E, int* __restrict__ status) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ uint32_t bm[];            // [E][8]
   for (int q = threadIdx.x; q < E * 8; q += kPB) bm[q] = 0u;
   __syncthreads();
@@ -68,8 +68,8 @@ __device__ __forceinline__ void write_tile_table(const PermuteBuffers& pb, int e
 // Single block.  blk_counts[b][e] becomes the exclusive prefix over b; counts/offsets and the tile table are written.
 __global__ void __launch_bounds__(1024)
 permute_scan_kernel(int* __restrict__ blk_counts, int n_blocks, int E, const PermuteBuffers pb) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   __shared__ int s_a[1024], s_b[1024];
   int* counts = pb.counts;
   int* offsets = pb.offsets;
@@ -112,8 +112,8 @@ permute_scan_kernel(int* __restrict__ blk_counts, int n_blocks, int E, const Per
 __global__ void permute_scatter_kernel(const int* __restrict__ idx, const int* __restrict__ rank,
                                        const int* __restrict__ blk_prefix, const int* __restrict__ offsets,
                                        int* __restrict__ perm, int* __restrict__ inv, int n_tokens, int sel, int E) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int q = blockIdx.x * blockDim.x + threadIdx.x;
   if (q >= n_tokens * sel) return;
   const int i = q / sel;
@@ -175,8 +175,8 @@ __device__ __forceinline__ void topk_small_regs(const TopkSmall& tk, int task) {
 __global__ void __launch_bounds__(1024)
 permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, const PermuteBuffers pb,
                      int* __restrict__ status, const TopkSmall tk) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ uint32_t bm[];            // [E][8]
   __shared__ int s_a[1024], s_b[1024], s_off[1024];
   int* counts = pb.counts;

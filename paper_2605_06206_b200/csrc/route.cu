@@ -23,8 +23,8 @@ namespace foe {
 __global__ void ffn_norm_kernel(const void* __restrict__ r_in, int r_is_bf16, const bf16* __restrict__ gain,
                                 bf16* __restrict__ u_out, float* __restrict__ inv_out, int n_tokens, int d,
                                 float eps) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (i >= n_tokens) return;
   float ss = 0.f;
@@ -75,8 +75,8 @@ __global__ void __launch_bounds__(kRgThreads, 4)
 router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __restrict__ inv_rms,
                    const bf16* __restrict__ gain, const float* __restrict__ wr, float* __restrict__ part,
                    int n_tokens, int d, int E, int k_per_split) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   __shared__ __align__(16) float As[2][kRgKC][kRgPA];     // [k][token]
   __shared__ __align__(16) float Bs[2][kRgKC][kRgPB];     // [k][expert]
   const int tid = threadIdx.x;
@@ -181,8 +181,8 @@ router_gemm_kernel(const void* __restrict__ r_in, int r_is_bf16, const float* __
 __global__ void topk_gates_kernel(const float* __restrict__ part, int k_splits, const float* __restrict__ br,
                                   float* __restrict__ logits_out, int* __restrict__ idx_out, float* __restrict__ w_out,
                                   int n_tokens, int H, int Ec, int kc) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   // a (token, cluster) task is handled by a group of W lanes (W = 8, 16 or 32), several tasks per warp
   const int W = Ec <= 8 ? 8 : (Ec <= 16 ? 16 : 32);
   const int per_warp = 32 / W;
@@ -256,8 +256,8 @@ __global__ void __launch_bounds__(kRsThreads)
 route_scores_small_kernel(const void* __restrict__ r_in, int r_is_bf16, const bf16* __restrict__ gain,
                           const float* __restrict__ wr, bf16* __restrict__ u_out, float* __restrict__ scores,
                           int n_tokens, int d, int E, float eps, int k_per_split) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   __shared__ float w_s[kRsK][kRsExp + 1];
   __shared__ float u_s[kRsTok][kRsK];
   __shared__ float red[kRsTok][2];
@@ -330,8 +330,8 @@ template <int EC>
 __global__ void topk_gates_thread_kernel(const float* __restrict__ part, int k_splits, const float* __restrict__ br,
                                          float* __restrict__ logits_out, int* __restrict__ idx_out,
                                          float* __restrict__ w_out, int n_tokens, int H, int kc) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int task = blockIdx.x * blockDim.x + threadIdx.x;
   if (task >= n_tokens * H) return;
   const int i = task / H, h = task - i * H;
@@ -435,8 +435,8 @@ static int g_route_sms[kNaMaxDevices];
 // inv_rms only: the expert input u is not produced on this path (the caller asked for routing, nothing else)
 __global__ void ffn_inv_rms_bf16_kernel(const bf16* __restrict__ r_in, float* __restrict__ inv_out, int n_tokens, int d,
                                         float eps) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (i >= n_tokens) return;
   const uint4* row = reinterpret_cast<const uint4*>(r_in + size_t(i) * d);

@@ -64,8 +64,8 @@ __global__ void __launch_bounds__(kRtThreads, 1)
 router_tc_kernel(const __grid_constant__ CUtensorMap tmW, const void* __restrict__ r_in, int r_is_bf16,
                  const float* __restrict__ inv_rms, float* __restrict__ part, int n_tokens, int d, int E, int E_pad,
                  int* __restrict__ status) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kRtStages * kRtStageBytes);

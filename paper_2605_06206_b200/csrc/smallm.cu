@@ -65,8 +65,8 @@ __device__ __forceinline__ SmTask sm_task(const SmallMArgs& a, int t, int slabs_
 template <int EPI>
 __global__ void __launch_bounds__(kSmThreads)
 smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
   constexpr int NT = kSmNT;
   constexpr int kSmStages = sm_stages<EPI>();
   extern __shared__ uint8_t smem_raw[];
