@@ -384,6 +384,7 @@ foe_status run_ffn(foe_layer* L, void* out, cudaStream_t st) {
     s2.W = L->wd_t; s2.X = L->ws->hmid; s2.ldx = L->I; s2.group_offsets = L->ws->pb.offsets; s2.n_groups = L->E; s2.N = d;
     s2.K = L->I; s2.epi = kEpiBf16; s2.out = L->ws->y; s2.ldo = d;
     s2.status = L->ws->status;
+    s2.early_weights = 1;
     launch_smallm(L->tms_wd, s2, L->n_sms, st);
     L->launches += 2;
   }

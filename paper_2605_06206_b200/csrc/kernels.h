@@ -148,6 +148,8 @@ struct SmallMArgs {
   int q_head_stride;
   const float2* rope_tab; const int* tok_pos; const int* tok_slot; bf16* k_pages; bf16* v_pages;
   const bf16* xsum; int x_count; size_t x_stride; float out_scale;
+  int early_weights;        // kEpiBf16: the previous kernel writes X and nothing else this one reads, so the first weight
+                            // tiles may be requested before waiting for it
   int* status;
 };
 // tmW: tensor map of W as [n_groups*N][K] with 64-column boxes of 64 rows (32 rows for the SwiGLU packing)

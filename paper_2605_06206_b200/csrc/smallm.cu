@@ -65,8 +65,12 @@ __device__ __forceinline__ SmTask sm_task(const SmallMArgs& a, int t, int slabs_
 template <int EPI>
 __global__ void __launch_bounds__(kSmThreads)
 smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
-  pdl_wait();
-  pdl_launch_dependents();
+  // (expert GEMM 2 of a step waits later: its producer first requests the weights of its first ring, see below)
+  const bool early_weights = EPI == kEpiBf16 && a.early_weights != 0;
+  if (!early_weights) {
+    pdl_wait();
+    pdl_launch_dependents();
+  }
   constexpr int NT = kSmNT;
   constexpr int kSmStages = sm_stages<EPI>();
   extern __shared__ uint8_t smem_raw[];
@@ -96,6 +100,29 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
     // row r (gathered through row_index) next to them.
     bool ok = true;
     int it = 0;
+    int pre = 0;                       // leading iterations whose barrier is armed and whose weights are on their way
+    if (early_weights) {
+      // The previous kernel (expert GEMM 1) writes this kernel's activations, nothing else it needs: the dispatch maps
+      // are older and complete.  So the weight tiles of the first ring can be requested while that kernel drains.
+      for (int t = blockIdx.x; t < n_tasks; t += gridDim.x) {
+        const SmTask k = sm_task(a, t, slabs_per_group, chunks);
+        if (k.rows <= 0) continue;
+        if (lane == 0) {
+          const int wrow0 = k.group * a.N + k.slab * kSmSlab;
+          const int rows_pass = min(kSmRows, k.rows);
+          pre = min(kSmStages, k_steps);
+          for (int i = 0; i < pre; ++i) {
+            mbar_expect_tx(&full[i], kSmWBytes + rows_pass * (kSmKStep * 2));
+            tma_load_2d(smem + i * kSmStageBytes, &tmW, &full[i], i * kSmKStep, wrow0);
+            tma_load_2d(smem + i * kSmStageBytes + 8192, &tmW, &full[i], i * kSmKStep + 64, wrow0);
+          }
+        }
+        break;
+      }
+      pre = __shfl_sync(0xffffffffu, pre, 0);
+      pdl_wait();
+      pdl_launch_dependents();
+    }
     for (int t = blockIdx.x; t < n_tasks && ok; t += gridDim.x) {
       const SmTask k = sm_task(a, t, slabs_per_group, chunks);
       if (k.rows <= 0) continue;
@@ -120,10 +147,15 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
         for (int ks = 0; ks < k_steps; ++ks, ++it) {
           const int s = it % kSmStages;
           const uint32_t ph = (it / kSmStages) & 1;
+          uint8_t* dst = smem + s * kSmStageBytes;
+          if (it < pre) {              // armed and weights requested before the wait: only the activations are missing
+            __syncwarp();
+            if (lane < rows_pass) bulk_load(dst + kSmWBytes + lane * kSmXPitch, xsrc + ks * kSmKStep, kSmKStep * 2, &full[s]);
+            continue;
+          }
           if (lane == 0) ok = mbar_wait(&empty[s], ph ^ 1);
           ok = __shfl_sync(0xffffffffu, ok, 0);
           if (!ok) break;
-          uint8_t* dst = smem + s * kSmStageBytes;
           if (lane == 0) {
             mbar_expect_tx(&full[s], kSmWBytes + rows_pass * (kSmKStep * 2));
             const int k0 = ks * kSmKStep;
@@ -147,6 +179,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
   }
 
   // ------------------------------------------------------------------ consumers
+  if (early_weights) pdl_wait();
   const int g = lane >> 2, t4 = lane & 3;
   // shared-memory rows of the two weight rows this thread feeds (MMA rows g and g+8)
   // (QKV: heads are stored with their halves interleaved, so rows 2g and 2g+1 are the two members of a rotary pair)
