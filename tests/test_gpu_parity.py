@@ -110,6 +110,14 @@ def test_one_cluster_baseline_and_wide_topk():
     run_block_parity(shape, 13, [90], [0], wscale=4.0)
 
 
+@pytest.mark.parametrize("H", [3, 6])
+def test_cluster_counts_that_are_not_powers_of_two(H):
+    # (the pre-attention statistics kernel sums the H residual streams with H as a template parameter)
+    shape = synth.LayerShape(384, 2 * H, H, H, 64, 4, 2, 128)
+    run_block_parity(shape, 40 + H, [300, 117], [0, 64], wscale=4.0)
+    run_block_parity(shape, 50 + H, [1] * 5, [3, 64, 200, 65, 130], decode=True, wscale=4.0)
+
+
 def test_head_dim_128_and_ragged_tiles():
     shape = synth.LayerShape(512, 8, 2, 2, 128, 4, 2, 256)
     run_block_parity(shape, 14, [130, 300, 63, 65], [0, 0, 0, 0], wscale=4.0)       # several 128-row tiles + tails
