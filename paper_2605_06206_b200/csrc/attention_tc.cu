@@ -6,14 +6,15 @@
 // pages with the same causal extent.  Per page of 64 keys:
 //     S_t = Q_t K^T        tcgen05.mma  M128 N64  K16 x (d_h/16)   accumulator in tensor memory
 //     P_t = softmax step   one thread per query row: tcgen05.ld, exp2, row max/sum without any shuffle,
-//                          P written to shared memory in the K-major 128-byte-swizzled operand layout
-//     O_t += P_t V         tcgen05.mma  M128 N d_h K16 x 4, V used straight from its page ([key][d_h],
-//                          i.e. an MN-major B operand); O stays in tensor memory for the whole row block
+//                          P written back into tensor memory as bf16 pairs over the scores it came from (tcgen05.st)
+//     O_t += P_t V         tcgen05.mma  M128 N d_h K16 x 4 with the A operand read from tensor memory, V used straight
+//                          from its page ([key][d_h], i.e. an MN-major B operand); O stays in tensor memory for the
+//                          whole row block
 // The running maximum used for the exponentials is only moved when the true maximum has grown by more than
 // 2^8 since it was last moved (the result is mathematically the same, probabilities stay below 256); only
 // then is O rescaled in tensor memory (tcgen05.ld / tcgen05.st), which after the first pages is rare.
-// Warp roles: warp 0 TMA producer (Q once, K/V pages through a 3-stage ring), warp 1 MMA issuer (warps 2-3
-// idle; the first warpgroup gives its registers away with setmaxnreg), warps 4-7 softmax of tile 0, warps 8-11
+// Warp roles: warp 0 TMA producer (Q once, K/V pages through a 5-stage ring), warp 1 MMA issuer (warps 2-3
+// idle), warps 4-7 softmax of tile 0, warps 8-11
 // softmax of tile 1.  While one tile's softmax runs, the tensor core works on
 // the other tile.  All waits are bounded; on expiry the role records a timeout in the status word and the
 // CTA still reaches its teardown (tensor memory is released).
@@ -26,10 +27,8 @@ namespace foe {
 
 constexpr int kAtRows = 128;          // query rows per tile
 constexpr int kAtKeys = 64;           // keys per step = one cache page
-constexpr int kAtStages = 3;
+constexpr int kAtStages = 5;
 constexpr int kAtThreads = 384;        // warpgroup 0: producer + MMA issuer (+2 idle warps); warpgroups 1, 2: softmax
-
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // K-major operand, 128-byte swizzle (rows of 128 bytes, 8-row groups 1024 bytes apart)
 __device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) { return umma_desc_sw128(addr); }
@@ -50,11 +49,9 @@ struct AtSmem {
   static constexpr int kHalves = DH / 64;
   static constexpr int kQTile = kAtRows * DH * 2;              // one query tile
   static constexpr int kKVTile = kAtKeys * DH * 2;             // one K or V page of one head
-  static constexpr int kPTile = kAtRows * kAtKeys * 2;         // probabilities of one tile (bf16)
   static constexpr int kQOff = 0;
   static constexpr int kKVOff = 2 * kQTile;
-  static constexpr int kPOff = kKVOff + kAtStages * 2 * kKVTile;
-  static constexpr int kBarOff = kPOff + 4 * kPTile;           // P is double-buffered per tile
+  static constexpr int kBarOff = kKVOff + kAtStages * 2 * kKVTile;
   static constexpr size_t kBytes = kBarOff + 256 + 1024;
 };
 
@@ -109,7 +106,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   const uint32_t tmem_base = *tmem_slot;
   // tensor-memory columns: scores of tile t, step parity b at 128 t + 64 b (double-buffered so that the next
   // step's Q K^T runs while this step's softmax is still reading); O of tile t at 256 + DH t
-  const uint32_t q_u32 = smem_u32(smem + L::kQOff), kv_u32 = smem_u32(smem + L::kKVOff), p_u32 = smem_u32(smem + L::kPOff);
+  const uint32_t q_u32 = smem_u32(smem + L::kQOff), kv_u32 = smem_u32(smem + L::kKVOff);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -153,11 +150,13 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       };
       auto issue_o = [&](int t, int j) {                      // O_t = P_t V_j
         const int s = j % kAtStages;
-        const uint32_t pb_ = p_u32 + (t * 2 + (j & 1)) * L::kPTile, vb_ = kv_u32 + s * 2 * L::kKVTile + L::kKVTile;
+        // P_t(j) sits in tensor memory, over the first 32 columns of the score buffer it was computed from
+        // (two bf16 per column, 8 columns per K = 16)
+        const uint32_t p_tmem = tmem_base + t * 128 + (j & 1) * 64, vb_ = kv_u32 + s * 2 * L::kKVTile + L::kKVTile;
 #pragma unroll
         for (int kk = 0; kk < kAtKeys / 16; ++kk)
-          umma_bf16(tmem_base + 256 + t * DH, desc_kmajor(pb_ + kk * 32),
-                    desc_mnmajor(vb_ + kk * (16 * 128), kAtKeys * 128, 1024), idesc_o, (j | kk) != 0);
+          umma_bf16_ts(tmem_base + 256 + t * DH, p_tmem + kk * 8,
+                       desc_mnmajor(vb_ + kk * (16 * 128), kAtKeys * 128, 1024), idesc_o, (j | kk) != 0);
         umma_commit(&o_full[t]);
       };
       if (ok && n_tiles > 0) {
@@ -176,7 +175,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           for (int t = 0; t < n_tiles_q; ++t) issue_s(t, j + 1);
         }
         for (int t = 0; t < n_tiles_q && ok; ++t) {
-          if (!mbar_wait(&p_ready[t], ph)) { ok = false; break; }       // P_t(j) is in shared memory
+          if (!mbar_wait(&p_ready[t], ph)) { ok = false; break; }       // P_t(j) is in tensor memory
           tc_fence_after();
           issue_o(t, j);
         }
@@ -195,7 +194,6 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       const uint32_t o_addr = tmem_base + lane_sel + 256 + t * DH;
       const int qpos = ctx + q0 + row;
       const int first_mask_tile = (ctx + q0) / kAtKeys;
-      uint8_t* p_rows = smem + L::kPOff + t * 2 * L::kPTile + row * 128;
       float m_ref = -INFINITY, l_run = 0.f;                  // m_ref: the (possibly stale) maximum the exponentials use
       bool ok = true;
       uint32_t r0[32], r1[32];                               // the 64 scores of this row
@@ -258,7 +256,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         }
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
         // probabilities, written as the bf16 A operand of the PV product (exp2(-inf) = 0 handles the mask)
-        uint8_t* p_row = p_rows + (j & 1) * L::kPTile;
+        const uint32_t p_addr = s_base + (j & 1) * 64;
         // Written in stages over 32 values: all scalings, then all exponentials back to back, then sums and packing.
         float rs4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -275,10 +273,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
             rs4[c & 3] += e[2 * c] + e[2 * c + 1];
             pk[c] = pack_bf16(e[2 * c], e[2 * c + 1]);
           }
-#pragma unroll
-          for (int q = 0; q < 4; ++q)
-            *reinterpret_cast<uint4*>(p_row + (((hf * 4 + q) ^ (row & 7)) << 4)) =
-                make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+          tmem_st16(p_addr + hf * 16, pk);                  // (the scores of this buffer are all in registers by now)
         }
         l_run += (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
         // The scores are used up: if the next step's are already there (they usually are, the issuer runs a step
@@ -298,8 +293,8 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         // (before this warp's arrival below: P V of step j cannot have been issued yet, so the barrier is at most one
         // phase ahead of what is waited for)
         if (!o_seen && !mbar_wait(&o_full[t], ph ^ 1)) { ok = false; break; }
+        tmem_st_wait();                                      // P is in tensor memory
         tc_fence_before();
-        fence_async_smem();                                  // P visible to the tensor core's shared-memory reads
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_ready[t]);
       }
