@@ -30,6 +30,30 @@ constexpr int kAtKeys = 64;           // keys per step = one cache page
 constexpr int kAtStages = 5;
 constexpr int kAtThreads = 384;        // warpgroup 0: producer + MMA issuer (+2 idle warps); warpgroups 1, 2: softmax
 
+// two fp32 values in one 64-bit register and the packed instructions on them
+__device__ __forceinline__ uint64_t pack_b32x2(uint32_t lo, uint32_t hi) {
+  uint64_t v;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "r"(lo), "r"(hi));
+  return v;
+}
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) { return pack_b32x2(__float_as_uint(lo), __float_as_uint(hi)); }
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+  uint32_t a, b;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+  lo = __uint_as_float(a);
+  hi = __uint_as_float(b);
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 // K-major operand, 128-byte swizzle (rows of 128 bytes, 8-row groups 1024 bytes apart)
 __device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) { return umma_desc_sw128(addr); }
 // MN-major operand, 128-byte swizzle: 64 contiguous elements of the M/N dimension per 128-byte row, one row
@@ -258,23 +282,32 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         // probabilities, written as the bf16 A operand of the PV product (exp2(-inf) = 0 handles the mask)
         const uint32_t p_addr = s_base + (j & 1) * 64;
         // Written in stages over 32 values: all scalings, then all exponentials back to back, then sums and packing.
-        float rs4[4] = {0.f, 0.f, 0.f, 0.f};
+        // Packed fp32 arithmetic (two values per instruction) for the scaling and the row sums: the step is bound by
+        // the softmax warps' instruction stream, not by any one unit.
+        uint64_t rs2[4] = {0ull, 0ull, 0ull, 0ull};           // four independent chains of (even, odd) partial sums
+        const uint64_t sc2 = pack_f32x2(a.scale_log2, a.scale_log2), nm2 = pack_f32x2(-m_use, -m_use);
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
           uint32_t (&rr)[32] = hf ? r1 : r0;
           float e[32];
 #pragma unroll
-          for (int c = 0; c < 32; ++c) e[c] = fmaf(__uint_as_float(rr[c]), a.scale_log2, -m_use);
+          for (int c = 0; c < 16; ++c) {
+            const uint64_t v = fma_f32x2(pack_b32x2(rr[2 * c], rr[2 * c + 1]), sc2, nm2);
+            unpack_f32x2(v, e[2 * c], e[2 * c + 1]);
+          }
 #pragma unroll
           for (int c = 0; c < 32; ++c) asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(e[c]) : "f"(e[c]));
           uint32_t pk[16];
 #pragma unroll
           for (int c = 0; c < 16; ++c) {
-            rs4[c & 3] += e[2 * c] + e[2 * c + 1];
+            rs2[c & 3] = add_f32x2(rs2[c & 3], pack_f32x2(e[2 * c], e[2 * c + 1]));
             pk[c] = pack_bf16(e[2 * c], e[2 * c + 1]);
           }
           tmem_st16(p_addr + hf * 16, pk);                  // (the scores of this buffer are all in registers by now)
         }
+        float rs4[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { float lo, hi; unpack_f32x2(rs2[q], lo, hi); rs4[q] = lo + hi; }
         l_run += (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
         // The scores are used up: if the next step's are already there (they usually are, the issuer runs a step
         // ahead), start loading them now, so that the load's latency passes behind the stores and arrivals below.
