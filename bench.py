@@ -402,10 +402,21 @@ def run_serve(args):
     num_pages = 4096                                        # 262,144 tokens of KV per layer
     runner = sv.FoeStackRunner(shape, n_layers, seed=2, num_pages=num_pages, max_batch_tokens=max_batch_tokens,
                                max_seqs=max_seqs, max_context=max_context)
-    warm = sv.synthetic_trace(3, rate=1e6, seed=12, prompt_range=(512, 4096), output_range=(2, 4))
-    sv.Engine(sv.Scheduler(sv.PagePool(num_pages), max_batch_tokens, max_seqs, chunk), runner.forward).run(warm)
+    # Warm-up: every kernel family the run can launch (large and small prefill chunks, mixed batches, decode steps of
+    # several sizes) once, so that no one-time cost of a first launch (module loading, kernel attributes) lands inside
+    # an iteration whose device time is charged to the requests waiting on it.  The collector is off during the run for
+    # the same reason: an iteration's time is taken between two events and includes any pause of the launching thread.
+    import gc
+    for seed, n, pr, orr in ((12, 3, (512, 4096), (2, 4)), (13, 12, (64, 9000), (2, 12))):
+        warm = sv.synthetic_trace(n, rate=1e6, seed=seed, prompt_range=pr, output_range=orr)
+        sv.Engine(sv.Scheduler(sv.PagePool(num_pages), max_batch_tokens, max_seqs, chunk), runner.forward).run(warm)
     eng = sv.Engine(sv.Scheduler(sv.PagePool(num_pages), max_batch_tokens, max_seqs, chunk), runner.forward)
-    done = eng.run(reqs)
+    gc.collect()
+    gc.disable()
+    try:
+        done = eng.run(reqs)
+    finally:
+        gc.enable()
     runner.close()
     rep = sv.latency_report(done)
     toks = sum(r.prompt_len + r.output_len - 1 for r in done)
