@@ -153,3 +153,38 @@ def test_workload5_foe_stack_prefill_and_128_decode_steps():
 
 def test_workload5_one_cluster_moe_baseline_stack():
     _run_workload5(1, checked_layers=(0, 15), rows_per_seq=8, decode_steps=128, checked_steps=(127,))
+
+
+def test_package_stack_helper_matches_layer_by_layer_calls():
+    """paper_2605_06206_b200.stack.FoeStack (used by bench.py --stack) is plumbing over the same layer calls: its
+    prefill and decode outputs equal those of hand-driven layers built from the same seeds, bit for bit."""
+    from paper_2605_06206_b200.stack import FoeStack
+    base = synth.LayerShape(256, 8, 4, 4, 64, 8, 2, 128)
+    q_lens, L, extra = [150, 77], 3, 2
+    st = FoeStack(base, L, 9, q_lens, extra)
+    S = sum(q_lens)
+    x = synth.make_x(st.shapes[0], 9, S, "cuda")
+    out_p = st.forward(x, [0, 0], decode=False).clone()
+    xs = synth.make_x(st.shapes[0], 9, len(q_lens), "cuda", tid=synth.TID["x_step"])
+    out_d = st.forward(xs, q_lens, decode=True).clone()
+    assert st.status() == 0
+    st.close()
+    # by hand
+    layers, kvs = [], []
+    for l in range(L):
+        sh = dataclasses.replace(base, position=("first", "middle", "last")[l])
+        W = synth.make_weights(sh, 9, "cuda", layer=l + 1)
+        layers.append(binding.FoeLayer(sh, W, max_tokens=S, max_seqs=len(q_lens), max_context=max(q_lens) + extra))
+        kvs.append(synth.make_paged_cache(base, 9, [0, 0], [q + extra for q in q_lens], "cuda", fill_random=False))
+    h = x
+    for layer, kv in zip(layers, kvs):
+        kv.q_lens = torch.tensor(q_lens, dtype=torch.int32, device="cuda")
+        h = layer.prefill(h, kv)
+    assert torch.equal(h, out_p)
+    h = xs
+    for layer, kv in zip(layers, kvs):
+        kv.context_lens = torch.tensor(q_lens, dtype=torch.int32, device="cuda")
+        h = layer.decode(h, kv)
+    assert torch.equal(h, out_d)
+    for layer in layers:
+        layer.close()
