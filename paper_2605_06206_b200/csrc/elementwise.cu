@@ -200,12 +200,97 @@ __global__ void combine_kernel(const float* __restrict__ r_full, const bf16* __r
   }
 }
 
+// The same for calls of a few hundred tokens, where the kernel is a chain of dependent loads rather than a stream: the
+// token's slots and gates (and the residual) are fetched before the wait for the expert GEMM -- they are older than
+// that kernel -- and the expert rows are requested eight at a time instead of one after the other.  Same sums in the
+// same order as combine_kernel.
+__global__ void combine_small_kernel(const float* __restrict__ r_full, const bf16* __restrict__ y, const float* __restrict__ w,
+                                     const int* __restrict__ inv, bf16* __restrict__ out, int n_tokens, int d, int H, int kc,
+                                     int last_mean) {
+  __shared__ int s_slot[256];                 // H <= 8, k_c <= 32
+  __shared__ float s_gate[256];
+  const int i = blockIdx.x;
+  const int n_sel = H * kc;
+  for (int t = threadIdx.x; t < n_sel; t += blockDim.x) {
+    s_slot[t] = __ldg(inv + size_t(i) * n_sel + t);
+    s_gate[t] = __ldg(w + size_t(i) * n_sel + t);
+  }
+  const int c0 = threadIdx.x * 8;
+  float r0[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (c0 < d) {
+    const float4 a = *reinterpret_cast<const float4*>(r_full + size_t(i) * d + c0);
+    const float4 b = *reinterpret_cast<const float4*>(r_full + size_t(i) * d + c0 + 4);
+    r0[0] = a.x; r0[1] = a.y; r0[2] = a.z; r0[3] = a.w; r0[4] = b.x; r0[5] = b.y; r0[6] = b.z; r0[7] = b.w;
+  }
+  pdl_wait();                                 // the expert rows come from the kernel before this one
+  pdl_launch_dependents();
+  __syncthreads();
+  const float inv_h = 1.0f / float(H);
+  for (int c = c0; c < d; c += blockDim.x * 8) {
+    float r[8];
+    if (c == c0) {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) r[t] = r0[t];
+    } else {
+      const float4 a = *reinterpret_cast<const float4*>(r_full + size_t(i) * d + c);
+      const float4 b = *reinterpret_cast<const float4*>(r_full + size_t(i) * d + c + 4);
+      r[0] = a.x; r[1] = a.y; r[2] = a.z; r[3] = a.w; r[4] = b.x; r[5] = b.y; r[6] = b.z; r[7] = b.w;
+    }
+    float mean[8], acc[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { mean[t] = 0.f; acc[t] = r[t]; }
+    int j = 0, h = 0;                         // position of the next selection inside its cluster
+    for (int s0 = 0; s0 < n_sel; s0 += 8) {
+      uint4 q[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        q[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (s0 + u < n_sel) q[u] = __ldcg(reinterpret_cast<const uint4*>(y + size_t(s_slot[s0 + u]) * d + c));
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (s0 + u >= n_sel) break;
+        const float g = s_gate[s0 + u];
+        const uint32_t v[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          acc[2 * t] += g * bf16_lo(v[t]);
+          acc[2 * t + 1] += g * bf16_hi(v[t]);
+        }
+        if (++j == kc) {                      // cluster h is complete
+          if (last_mean) {
+#pragma unroll
+            for (int t = 0; t < 8; ++t) mean[t] += acc[t];
+          } else {
+            *reinterpret_cast<uint4*>(out + (size_t(h) * n_tokens + i) * d + c) =
+                make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
+                           pack_bf16(acc[6], acc[7]));
+          }
+#pragma unroll
+          for (int t = 0; t < 8; ++t) acc[t] = r[t];
+          j = 0;
+          ++h;
+        }
+      }
+    }
+    if (last_mean) {
+      *reinterpret_cast<uint4*>(out + size_t(i) * d + c) =
+          make_uint4(pack_bf16(mean[0] * inv_h, mean[1] * inv_h), pack_bf16(mean[2] * inv_h, mean[3] * inv_h),
+                     pack_bf16(mean[4] * inv_h, mean[5] * inv_h), pack_bf16(mean[6] * inv_h, mean[7] * inv_h));
+    }
+  }
+}
+
 void launch_combine(const float* r_full, const bf16* y, const float* w, const int* inv, bf16* out, int n_tokens, int d,
                     int H, int kc, int last_mean, cudaStream_t st) {
   if (n_tokens <= 0) return;
   int threads = d / 8;
   if (threads > 256) threads = 256;
   if (threads < 32) threads = 32;
+  if (n_tokens <= 1024) {
+    launch_pdl(combine_small_kernel, dim3(n_tokens), dim3(threads), 0, st, r_full, y, w, inv, out, n_tokens, d, H, kc, last_mean);
+    return;
+  }
   launch_pdl(combine_kernel, dim3(n_tokens), dim3(threads), 0, st, r_full, y, w, inv, out, n_tokens, d, H, kc, last_mean);
 }
 
