@@ -193,7 +193,12 @@ void run_route_and_permute(foe_layer* L, const void* r, int r_is_bf16, int n, cu
 // slots; otherwise it is r_full itself, in the workspace.
 foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaStream_t st, bool decode, foe_shard* sh) {
   const int S = decode ? kv->n_seqs : kv->n_tokens;
-  g_overlap_launches = decode || S <= kOverlapTokens; // launches of this call (this thread) overlap their predecessors' tails
+  // Launches of this call (this thread) overlap their predecessors' tails when the call is small; kernels that follow
+  // a SHORT kernel do so at any size (the token map and statistics at the start of a call, the QKV projection after
+  // them, the routing chain, expert GEMM 1 after the dispatch scatter): what costs at large sizes is a kernel's CTAs
+  // sitting resident beside a long, power-bound predecessor.
+  const bool overlap_call = decode || S <= kOverlapTokens;
+  g_overlap_launches = true;
   L->last_stream = st;
   L->launches = 0;
   L->last_tokens = S;
@@ -278,6 +283,7 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
   L->launches += 1;
 
   // ---- attention core over the paged cache
+  g_overlap_launches = overlap_call;     // (attention follows the long QKV projection)
   stage_mark(L, kStAttn, st);
   AttnArgs aa;
   memset(&aa, 0, sizeof(aa));
@@ -350,7 +356,13 @@ foe_status run_ffn(foe_layer* L, void* out, cudaStream_t st) {
 
   // ---- router, top-k, gates, dispatch maps
   stage_mark(L, kStRoute, st);
-  run_route_and_permute(L, L->ws->r_full, 0, S, st);
+  {
+    // the routing and dispatch-map kernels are short at any call size: they always overlap their predecessors' tails
+    const bool saved = g_overlap_launches;
+    g_overlap_launches = true;
+    run_route_and_permute(L, L->ws->r_full, 0, S, st);
+    g_overlap_launches = saved;
+  }
   const int R = S * H * L->kc;
   // experts: the weight-streaming kernels take 16 rows of an expert per pass over its weights; up to 8 rows per
   // expert on average (few experts need a second pass) they beat the tiled GEMMs, at 16 they no longer do
@@ -363,7 +375,12 @@ foe_status run_ffn(foe_layer* L, void* out, cudaStream_t st) {
     g1.n_groups = L->E; g1.mt_group = L->ws->pb.mt_group; g1.mt_row0 = L->ws->pb.mt_row0; g1.group_end = L->ws->pb.offsets + 1;
     g1.n_mtiles = L->ws->pb.n_mtiles; g1.N = 2 * L->I; g1.K = d; g1.status = L->ws->status; g1.out = L->ws->hmid; g1.ldo = L->I;
     g1.a_gather = L->ws->u; g1.a_row_index = L->ws->pb.perm;      // rows of u gathered through the dispatch map
-    launch_gemm(kEpiSwiGLU, L->ws->tm_hmid, L->tm_wgu, g1, L->n_sms, st);   // the A map is unused with a gathered A
+    {
+      const bool saved = g_overlap_launches;
+      g_overlap_launches = true;          // its predecessor (the dispatch scatter) is short: set up while it runs
+      launch_gemm(kEpiSwiGLU, L->ws->tm_hmid, L->tm_wgu, g1, L->n_sms, st);   // the A map is unused with a gathered A
+      g_overlap_launches = saved;
+    }
     stage_mark(L, kStGemm2, st);
     GemmArgs g2 = g1;
     g2.a_gather = nullptr; g2.a_row_index = nullptr;
