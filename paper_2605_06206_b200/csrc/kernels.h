@@ -13,10 +13,12 @@ namespace foe {
 typedef __nv_bfloat16 bf16;
 
 // Launch with programmatic stream serialization: the kernel may be scheduled while its predecessor in the stream is
-// still running and must call pdl_wait() before it touches anything the predecessor (or any earlier kernel) wrote.
-// It pays for calls made of short kernels (a decode step: -4 % of the step, a 1024-token block: -8 %) and costs a
-// little when every kernel runs for hundreds of microseconds (a 16k-token prefill: +0.7 %), so the API layer switches
-// it per call (per host thread).
+// still running and must call pdl_wait() before it touches anything the predecessor wrote (everything older is complete
+// by then, because every kernel of the library triggers its successor only after its own wait).
+// It pays for calls made of short kernels (a decode step: -6 % of the step, a 1024-token block: -8 %) and costs a
+// little when a kernel's CTAs sit resident beside a predecessor that runs for hundreds of microseconds (a 16k-token
+// prefill with the attribute on every launch: +0.7 %), so the API layer switches it per call and, inside large calls,
+// per launch (this flag, per host thread).
 inline thread_local bool g_overlap_launches = true;
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
