@@ -20,6 +20,37 @@
 namespace foe {
 
 // ------------------------------------------------------------------------------------------------ 1
+// The same for an fp32 input whose row fits in registers (d = 128 * NV, NV float4 per lane): the row is read once.
+// Same arithmetic in the same order as ffn_norm_kernel.
+template <int NV>
+__global__ void ffn_norm_f32_kernel(const float* __restrict__ r_in, const bf16* __restrict__ gain, bf16* __restrict__ u_out,
+                                    float* __restrict__ inv_out, int n_tokens, float eps) {
+  pdl_wait();
+  pdl_launch_dependents();
+  constexpr int d = NV * 128;
+  const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (i >= n_tokens) return;
+  const float4* row = reinterpret_cast<const float4*>(r_in + size_t(i) * d);
+  float4 q[NV];
+#pragma unroll
+  for (int j = 0; j < NV; ++j) q[j] = __ldg(row + lane + 32 * j);
+  float ss = 0.f;
+#pragma unroll
+  for (int j = 0; j < NV; ++j) ss += q[j].x * q[j].x + q[j].y * q[j].y + q[j].z * q[j].z + q[j].w * q[j].w;
+  ss = warp_sum(ss);
+  const float inv = rsqrtf(ss / float(d) + eps);
+  if (lane == 0) inv_out[i] = inv;
+  // lane's float4 j covers columns 4 * (lane + 32 j) ..: written as 8-byte bf16 quadruples
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    const int c4 = lane + 32 * j;
+    const uint2 gq = __ldg(reinterpret_cast<const uint2*>(gain) + c4);
+    const float v0 = q[j].x * inv * bf16_lo(gq.x), v1 = q[j].y * inv * bf16_hi(gq.x);
+    const float v2 = q[j].z * inv * bf16_lo(gq.y), v3 = q[j].w * inv * bf16_hi(gq.y);
+    *reinterpret_cast<uint2*>(u_out + size_t(i) * d + c4 * 4) = make_uint2(pack_bf16(v0, v1), pack_bf16(v2, v3));
+  }
+}
+
 __global__ void ffn_norm_kernel(const void* __restrict__ r_in, int r_is_bf16, const bf16* __restrict__ gain,
                                 bf16* __restrict__ u_out, float* __restrict__ inv_out, int n_tokens, int d,
                                 float eps) {
@@ -396,7 +427,11 @@ int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float*
                  int n_tokens, int d, int H, int Ec, int kc, float eps, int n_sms, int* status, cudaStream_t st) {
   if (n_tokens <= 0) return 0;
   const int E = H * Ec;
-  launch_pdl(ffn_norm_kernel, dim3((n_tokens * 32 + 255) / 256), dim3(256), 0, st, r_in, r_is_bf16, gain, u_out, inv_rms, n_tokens, d, eps);
+  const dim3 ngrid((n_tokens * 32 + 255) / 256);
+  const float* rf = static_cast<const float*>(r_in);
+  if (!r_is_bf16 && d == 1024) launch_pdl(ffn_norm_f32_kernel<8>, ngrid, dim3(256), 0, st, rf, gain, u_out, inv_rms, n_tokens, eps);
+  else if (!r_is_bf16 && d == 2048) launch_pdl(ffn_norm_f32_kernel<16>, ngrid, dim3(256), 0, st, rf, gain, u_out, inv_rms, n_tokens, eps);
+  else launch_pdl(ffn_norm_kernel, ngrid, dim3(256), 0, st, r_in, r_is_bf16, gain, u_out, inv_rms, n_tokens, d, eps);
   int ks = 1;
   if (tm_wr_split && n_tokens >= kRouterTcMinTokens) {
     launch_router_tc(*tm_wr_split, r_in, r_is_bf16, inv_rms, part, n_tokens, d, E, status, st);
