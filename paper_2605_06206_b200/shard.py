@@ -71,8 +71,11 @@ def load_library() -> ctypes.CDLL:
 
 def cluster_shape(shape, h: int):
     """Layer description of cluster h alone (the handle rank h creates): one cluster with the cluster's heads
-    and experts.  Position and sync keep their meaning."""
+    and experts.  Position and sync keep their meaning.  The cluster's own query width (query heads per cluster x
+    head width) must be a multiple of 128, as for any layer handle."""
     assert 0 <= h < shape.n_clusters
+    if (shape.q_per_cluster * shape.head_dim) % 128:
+        raise ValueError("one cluster per rank needs a per-cluster query width that is a multiple of 128")
     return dataclasses.replace(shape, n_clusters=1, n_q_heads=shape.q_per_cluster, n_kv_heads=shape.kv_per_cluster)
 
 

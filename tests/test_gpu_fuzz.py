@@ -1,0 +1,63 @@
+"""Seeded random layer shapes and batches against the oracle: every draw is reproducible from its case number.
+The draws cover what the fixed cases do not pair up: head widths with group sizes, cluster counts with expert counts,
+token counts on both sides of the sizes at which the library changes kernels, cached context with ragged chunks."""
+import random
+
+import pytest
+
+from paper_2605_06206_b200 import synth
+
+from parity import run_block_parity
+from test_gpu_shard import run_group
+
+pytestmark = pytest.mark.gpu
+
+
+def draw_shape(rng: random.Random) -> synth.LayerShape:
+    while True:
+        H = rng.choice([1, 2, 3, 4, 5, 8])
+        dh = rng.choice([64, 96, 128])
+        c = rng.choice([1, 2])                      # KV heads per cluster
+        group = rng.choice([1, 2, 4])               # query heads per KV head
+        n_kv, n_q = H * c, H * c * group
+        if (n_q * dh) % 128 or n_q * dh > 2048:
+            continue
+        hidden = 128 * rng.choice([1, 2, 3, 4, 8])
+        Ec = rng.choice([1, 2, 4, 8, 16])
+        k = rng.randint(1, min(Ec, 4))
+        inter = 128 * rng.choice([1, 2, 3])
+        position = rng.choice(["middle", "middle", "first", "last", "single"] if H > 1 else ["middle", "single"])
+        sync = rng.choice(["mean", "sum"])
+        return synth.LayerShape(hidden, n_q, n_kv, H, dh, Ec, k, inter, position=position, sync=sync)
+
+
+def draw_batch(rng: random.Random, decode: bool):
+    if decode:
+        n = rng.choice([1, 2, 7, 64, 65, 150])
+        return [1] * n, [rng.choice([0, 1, 63, 64, 65, 127, 200, 513]) for _ in range(n)]
+    n = rng.randint(1, 4)
+    q = [rng.choice([1, 5, 63, 64, 65, 130, 257, 300]) for _ in range(n)]
+    ctx = [rng.choice([0, 0, 64, 130, 191]) for _ in range(n)]
+    return q, ctx
+
+
+@pytest.mark.parametrize("case", range(64))
+def test_random_shape_and_batch(case):
+    rng = random.Random(7000 + case)
+    shape = draw_shape(rng)
+    decode = rng.random() < 0.4
+    q_lens, ctx_lens = draw_batch(rng, decode)
+    run_block_parity(shape, 7000 + case, q_lens, ctx_lens, decode=decode)
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_random_shape_and_batch_one_cluster_per_rank(case):
+    rng = random.Random(9000 + case)
+    while True:
+        shape = draw_shape(rng)
+        if (shape.n_clusters > 1 and shape.hidden % (32 * shape.n_clusters) == 0
+                and (shape.q_per_cluster * shape.head_dim) % 128 == 0):
+            break
+    decode = rng.random() < 0.4
+    q_lens, ctx_lens = draw_batch(rng, decode)
+    run_group(shape, 9000 + case, q_lens, ctx_lens, decode=decode)

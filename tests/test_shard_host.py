@@ -78,6 +78,8 @@ def test_cluster_slices_of_shape_and_weights():
         assert w["attn_norm_g"] is W["attn_norm_g"] and w["ffn_norm_g"] is W["ffn_norm_g"]
         # views, not copies
         assert w["w_up"].data_ptr() == W["w_up"][h * 8].data_ptr()
+    with pytest.raises(ValueError):                 # 1 query head of width 64 per cluster: no 128-wide O-proj block
+        shard.cluster_shape(synth.LayerShape(256, 4, 4, 4, 64, 8, 2, 128), 0)
     cfg = shard.exchange_config(s, 3, 77, 5)
     assert (cfg.rank, cfg.n_ranks, cfg.hidden, cfg.max_tokens, cfg.wait_limit_ms) == (3, 4, 256, 77, 5)
 
