@@ -61,3 +61,28 @@ def test_random_shape_and_batch_one_cluster_per_rank(case):
     decode = rng.random() < 0.4
     q_lens, ctx_lens = draw_batch(rng, decode)
     run_group(shape, 9000 + case, q_lens, ctx_lens, decode=decode)
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_random_wide_expert_sets_with_skewed_routing(case):
+    """Many experts per cluster (up to the 128 the library takes), wider top-k, a popularity-skewed router bias with
+    dead experts on every other case, scaled weights so that the routing logits spread."""
+    rng = random.Random(11000 + case)
+    H = rng.choice([1, 2, 4, 8])
+    Ec = rng.choice([32, 64, 128])
+    k = rng.choice([1, 2, 4, 8])
+    hidden = 128 * rng.choice([2, 4, 8])
+    shape = synth.LayerShape(hidden, 2 * H, H, H, rng.choice([64, 128]), Ec, k, 128 * rng.choice([1, 2]),
+                             position=rng.choice(["middle", "first", "last"]) if H > 1 else "single")
+    bias = synth.zipf_router_bias(shape, 11000 + case, 1.0, 1.2, dead_per_cluster=rng.choice([0, 5])) if case % 2 else None
+    decode = rng.random() < 0.4
+    if decode:
+        n = rng.choice([3, 64, 200])
+        q_lens, ctx_lens = [1] * n, [rng.choice([0, 63, 64, 300]) for _ in range(n)]
+    else:
+        q_lens = [rng.choice([20, 257, 700, 1500]) for _ in range(rng.randint(1, 2))]
+        ctx_lens = [rng.choice([0, 64, 100]) for _ in q_lens]
+    # wider layers take a smaller factor: attention logits grow with the square of the factor and with the width,
+    # and past a point the softmax turns bf16 noise in q and k into errors beyond the stress bounds
+    run_block_parity(shape, 11000 + case, q_lens, ctx_lens, decode=decode, wscale=4.0 if hidden <= 512 else 2.0,
+                     router_bias=bias)
