@@ -140,6 +140,17 @@ def compare_with_oracle(shape, W, x, q_lens, ctx_lens, cache, kv, out, aux, rows
         if ctx_lens[b]:
             assert np.array_equal(newc[b][0][:ctx_lens[b]], cache[b][0]) and np.array_equal(newc[b][1][:ctx_lens[b]], cache[b][1])
     assert_close(adapter.to_np(aux["attn_o"])[rsel], ref["o"], "attention output", STAGE_MAX_TOL, STAGE_REL_TOL)
+    # the attention stage by itself: the oracle's attend() on the GPU's own q and on the pages as the call left them
+    # (both already bf16), so only the kernel's softmax and its two contractions are compared; the task's bounds
+    qg = q_gpu[rsel].reshape(len(rsel), nq, dh).astype(np.float64)
+    seq_of = np.repeat(np.arange(len(q_lens)), q_lens)
+    o_iso = np.zeros((len(rsel), nq, dh))
+    for b in range(len(q_lens)):
+        sel = np.nonzero(seq_of[rsel] == b)[0]
+        if len(sel):
+            o_iso[sel] = orc.attend(qg[sel], ref["pos"][rsel[sel]], newc[b][0].astype(np.float64),
+                                    newc[b][1].astype(np.float64), nq // nkv)
+    assert_close(adapter.to_np(aux["attn_o"])[rsel], o_iso.reshape(len(rsel), -1), "attention on the GPU's q and pages")
     assert_close(adapter.to_np(aux["r_full"])[rsel], ref["r_full"], "r_full", STAGE_MAX_TOL, STAGE_REL_TOL)
 
     # tier (ii)/(iii): routing flips must be explained by the noise of the router input
