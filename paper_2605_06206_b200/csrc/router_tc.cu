@@ -10,13 +10,13 @@
 // the three dropped ones are below 2^-24.  Eight accumulators take the k-blocks in turn and are summed in fp32 by the
 // epilogue, so that no tensor-core accumulation chain is longer than 96 steps.
 //
-// The weights are split when the layer is created (gain folded in); the residual r is split on the fly: eight
+// The weights are split when the layer is created (gain folded in); the residual r is split on the fly: sixteen
 // converter warps read a 128 x 64 fp32 tile per k-block straight from global memory (coalesced, 512 bytes per warp
 // instruction), split it in registers and store the three bf16 tiles in the 128-byte-swizzled operand layout, then
 // cross to the async proxy and arrive on the stage's barrier.  r is read exactly once and the kernel runs at the rate
 // r streams in.  One CTA per 128 tokens x 64 experts.
 //
-// Warp roles: 0 TMA producer (weight planes), 1 MMA issuer, 2-5 epilogue, 6-13 converters.  All waits are bounded.
+// Warp roles: 0 TMA producer (weight planes), 1 MMA issuer, 2-5 epilogue, 6-21 converters.  All waits are bounded.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -26,8 +26,9 @@ constexpr int kRtRows = 128, kRtChunk = kRouterChunk, kRtBK = 64, kRtStages = 3;
 constexpr int kRtATile = kRtRows * kRtBK * 2;       // 16 KB: one bf16 term of the A tile
 constexpr int kRtBTile = kRtChunk * kRtBK * 2;      // 8 KB: one bf16 term of the B tile
 constexpr int kRtStageBytes = 3 * kRtATile + 3 * kRtBTile;   // 72 KB
-constexpr int kRtConvWarps = 8;
+constexpr int kRtConvWarps = 16;
 constexpr int kRtThreads = (6 + kRtConvWarps) * 32;
+constexpr int kRtRowsPerLane = kRtRows / (2 * kRtConvWarps);   // tile rows one converter lane handles per k-block
 constexpr int kRtAccs = 8;                          // accumulators of 64 columns: all 512 TMEM columns
 constexpr size_t kRtSmemBytes = size_t(kRtStages) * kRtStageBytes + 1024 + 256;
 
@@ -134,11 +135,12 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmW, const void* __restrict
     const int cw = warp - 6;
     const int sub = lane >> 4, c4 = lane & 15;             // row inside the pair; float4 column (4 k values)
     const int chunk16 = c4 >> 1, half8 = (c4 & 1) * 8;      // 16-byte chunk of the bf16 row and offset inside it
-    size_t src[8];                                          // element offset of this lane's four values in k-block 0
-    int trow[8];
+    constexpr int NR = kRtRowsPerLane;
+    size_t src[NR];                                         // element offset of this lane's four values in k-block 0
+    int trow[NR];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      trow[i] = cw * 16 + 2 * i + sub;                      // row of the tile
+    for (int i = 0; i < NR; ++i) {
+      trow[i] = cw * (2 * NR) + 2 * i + sub;                // row of the tile
       src[i] = size_t(min(row0 + trow[i], n_tokens - 1)) * d + c4 * 4;          // rows past the end repeat the last one
     }
     // the residual comes as fp32 (inside a block) or as bf16 (routing call on a caller's tensor)
@@ -149,14 +151,19 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmW, const void* __restrict
       }
       return __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(r_in) + off));
     };
+    // two k-blocks of loads stay in flight per lane while a third is converted
     bool ok = true;
-    float4 cur[8], nxt[8];
+    float4 cur[NR], nxt[NR], nx2[NR];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) cur[i] = load4(src[i]);
+    for (int i = 0; i < NR; ++i) cur[i] = load4(src[i]);
+    if (kblocks > 1) {
+#pragma unroll
+      for (int i = 0; i < NR; ++i) nxt[i] = load4(src[i] + size_t(kRtBK));
+    }
     for (int kb = 0; kb < kblocks; ++kb) {
-      if (kb + 1 < kblocks) {
+      if (kb + 2 < kblocks) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) nxt[i] = load4(src[i] + size_t(kb + 1) * kRtBK);
+        for (int i = 0; i < NR; ++i) nx2[i] = load4(src[i] + size_t(kb + 2) * kRtBK);
       }
       const int s = kb % kRtStages;
       if (lane == 0) ok = mbar_wait(&empty_bar[s], ((kb / kRtStages) & 1) ^ 1);
@@ -164,7 +171,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmW, const void* __restrict
       if (!ok) break;
       uint8_t* sa = smem + s * kRtStageBytes;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < NR; ++i) {
         uint32_t h0, m0, l0, h1, m1, l1;
         split3(cur[i].x, cur[i].y, h0, m0, l0);
         split3(cur[i].z, cur[i].w, h1, m1, l1);
@@ -177,7 +184,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmW, const void* __restrict
       __syncwarp();
       if (lane == 0) mbar_arrive(&full_bar[s]);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) cur[i] = nxt[i];
+      for (int i = 0; i < NR; ++i) { cur[i] = nxt[i]; nxt[i] = nx2[i]; }
     }
     if (!ok && lane == 0) atomicExch(status, kStatusTimeout);
   } else {
