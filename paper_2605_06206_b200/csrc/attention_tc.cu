@@ -99,11 +99,17 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_full + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = blockIdx.z;
+  // Blocks start in the order of their linear index.  The work of a block grows with its query block (causal
+  // extent), so the index runs over (sequence, head pair) fastest and over the query block slowest, late query
+  // blocks first: every long block of the whole call starts before any short one, and the short ones fill the tail.
+  const int lin = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+  const int per_qb = gridDim.y * gridDim.z;
+  const int qb = gridDim.x - 1 - lin / per_qb;
+  const int pair = (lin % per_qb) % gridDim.y;
+  const int b = (lin % per_qb) / gridDim.y;
   const int G = a.n_q / a.n_kv;
   const int n_tiles_q = (G % 2 == 0) ? 2 : 1;              // heads per CTA
-  const int head0 = blockIdx.y * n_tiles_q;
-  const int qb = gridDim.x - 1 - blockIdx.x;               // heavy (late) query blocks first
+  const int head0 = pair * n_tiles_q;
   const int q_len = a.q_lens ? a.q_lens[b] : 1;
   const int q0 = qb * kAtRows;
   if (q0 >= q_len) return;
