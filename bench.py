@@ -33,7 +33,7 @@ from paper_2605_06206_b200 import replicas, synth  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernels, from the committed ncu captures
 # of these same workloads (profiles/): not re-measured by a plain bench run
-NCU_TRAFFIC = dict(expert_gemm1_prefill=972.1e6 + 256.5e6, attn_decode=1349.4e6 + 8.9e6)
+NCU_TRAFFIC = dict(expert_gemm1_prefill=973.5e6 + 258.0e6, attn_decode=1349.4e6 + 8.9e6)
 
 
 # ----------------------------------------------------------------------------------------------
