@@ -153,6 +153,22 @@ foe_status foe_prefill(foe_layer* layer, const void* x, const foe_kv_cache* kv, 
  * x_step: [H][n_seqs][hidden] bf16 ([n_seqs][hidden] on a first layer). */
 foe_status foe_decode(foe_layer* layer, const void* x_step, const foe_kv_cache* kv, void* out, void* stream);
 
+/* A stack of layers (Section 3.1 "Layer boundaries": a first layer, middle layers, a last layer) in ONE host call:
+ * layer l runs foe_prefill (decode == 0) or foe_decode (decode != 0) on the output of layer l-1 with its own cache
+ * kvs[l] (host array of n_layers structs; they normally share block_table / context_lens / q_lens and differ in the
+ * pages).  x is the first layer's input, out the last layer's output; work0 and work1 are two caller-owned device
+ * buffers of n_clusters * S * hidden bf16 each for the activations between layers (work0 may be NULL for one layer,
+ * work1 for up to two); none of x, out, work0, work1 may alias another.  Every layer's arguments are checked before
+ * anything is launched; consecutive layers must fit (FOE_ERR_CONFIG: a first layer after another layer, a layer after
+ * a last layer, different hidden sizes or cluster counts).  The layers may share one workspace.  Exactly the launches
+ * of the single-layer calls, issued back to back: results are bit-identical to calling the layers one by one. */
+foe_status foe_stack_forward(foe_layer* const* layers, int n_layers, const void* x, const foe_kv_cache* kvs, void* out,
+                             void* work0, void* work1, int decode, void* stream);
+
+/* context_lens[i] += by for i < n_seqs, on the stream (device array): after a decode step (by = 1) or a prompt chunk,
+ * so that a generation loop keeps the lengths on the device and its steps can be replayed from a CUDA graph. */
+foe_status foe_context_advance(int* context_lens, int n_seqs, int by, void* stream);
+
 /* Section 3.1 "Routing": FFN RMSNorm, fp32 router scores, per-cluster top-k (larger score first, equal
  * scores -> lower expert id) and gates (softmax over the selected scores) for n_tokens rows of
  * h = r_full given as [n_tokens][hidden] bf16.  topk_idx: [n_tokens][H][k_c] int32 global expert ids;
@@ -172,8 +188,13 @@ foe_status foe_route(foe_layer* layer, const void* h, int n_tokens, int* topk_id
  *   device pointers owned by the caller.  The dispatch maps and the expert input are not produced.
  * Limits: n_tokens <= 8192 and n_tokens * n_clusters * experts_per_cluster <= 524288; larger calls return
  * FOE_ERR_SHAPE and launch nothing.  Shape rules as for the layer description (FOE_ERR_CONFIG otherwise).
+ * Alignment: h and router_w on 16 bytes, ffn_norm_g on 8, router_b / topk_idx / topk_w on 4 (FOE_ERR_SHAPE otherwise,
+ * nothing launched): a sliced view that starts in the middle of a row group does not qualify.
  * The first call on each device looks up the device address of the scratch array (with that device current);
- * make that first call before any stream capture begins.  Every call on a device uses the same scratch, which
+ * make that first call before any stream capture begins.  With lazy module loading that first call is also the
+ * moment the driver places the library's code and this array on the device, so make it before your own pool takes
+ * the memory that is left (it returns FOE_ERR_CUDA if the image cannot be loaded).  First calls from several host
+ * threads at once are safe.  Every call on a device uses the same scratch, which
  * simply keeps the previous call's contents (nothing in it needs clearing: each call writes what it reads);
  * two calls that overlap on the GPU -- different streams, or different host threads -- race on it, so run
  * them one after the other. */
@@ -194,11 +215,24 @@ int foe_last_launch_count(const foe_layer* layer);
 /* Per-stage device timing of prefill/decode calls.  When enabled, every call records CUDA events on its
  * stream between the stages of the block; foe_get_stage_ms waits for the last call and writes the
  * foe_num_stages() elapsed times (milliseconds) into ms[0..n), n >= foe_num_stages().  foe_stage_name(i)
- * names stage i.  FOE_ERR_UNSUPPORTED if the last call was not recorded. */
+ * names stage i.  FOE_ERR_UNSUPPORTED if the last call was not recorded.
+ * `enabled` is the number of most recent calls whose events are kept (0 = off, 1 = the last call, at most 256):
+ * with enabled > 1 the calls can be issued back to back without reading anything in between, and foe_get_stage_ms
+ * returns the mean over the calls recorded since it was last read (the most recent `enabled` of them), so that stage
+ * times can be taken deep inside a long run of steps, at the clocks the GPU settles to. */
 foe_status foe_set_profiling(foe_layer* layer, int enabled);
 int foe_num_stages(void);
 const char* foe_stage_name(int i);
 foe_status foe_get_stage_ms(foe_layer* layer, float* ms, int n);
+
+/* Host-only arithmetic, no device work (used by the tests; Section 3.1 "Routing" is the step they size).
+ * The fp32 score kernels cut the hidden dimension into k_splits slices when a call has too few tokens to fill the
+ * GPU; the slices' partial scores ([k_splits][n_tokens][n_experts] floats) go to a workspace buffer and are summed
+ * in a fixed order.  foe_route_partial_capacity: floats of that buffer in a handle created with these sizes.
+ * foe_route_partial_floats: floats a routing call of n_tokens tokens writes there on a device with n_sms SMs when
+ * the buffer holds `capacity` floats (the number of slices is halved until they fit; 0 for n_tokens <= 0). */
+size_t foe_route_partial_capacity(int max_tokens, int max_seqs, int n_experts);
+size_t foe_route_partial_floats(int hidden, int n_experts, int n_tokens, int n_sms, size_t capacity);
 
 /* Static description of a status code. */
 const char* foe_status_string(int status);

@@ -21,7 +21,8 @@ SYNCS = {"mean": 0, "sum": 1}
 
 EXPORTS = ["foe_layer_create", "foe_layer_destroy", "foe_prefill", "foe_decode", "foe_route", "foe_get_aux",
            "foe_poll_status", "foe_last_launch_count", "foe_status_string", "foe_set_profiling", "foe_num_stages",
-           "foe_stage_name", "foe_get_stage_ms", "foe_route_noalloc", "foe_layer_create_shared"]
+           "foe_stage_name", "foe_get_stage_ms", "foe_route_noalloc", "foe_layer_create_shared",
+           "foe_route_partial_capacity", "foe_route_partial_floats", "foe_stack_forward", "foe_context_advance"]
 
 
 class FoeConfig(ctypes.Structure):
@@ -94,6 +95,14 @@ def load_library() -> ctypes.CDLL:
     lib.foe_get_stage_ms.restype = ci
     lib.foe_route_noalloc.argtypes = [ci, ci, ci, ci, ctypes.c_float, vp, vp, vp, vp, ci, vp, vp, vp]
     lib.foe_route_noalloc.restype = ci
+    lib.foe_route_partial_capacity.argtypes = [ci, ci, ci]
+    lib.foe_route_partial_capacity.restype = ctypes.c_size_t
+    lib.foe_route_partial_floats.argtypes = [ci, ci, ci, ci, ctypes.c_size_t]
+    lib.foe_route_partial_floats.restype = ctypes.c_size_t
+    lib.foe_stack_forward.argtypes = [ctypes.POINTER(vp), ci, vp, ctypes.POINTER(FoeKvCache), vp, vp, vp, ci, vp]
+    lib.foe_stack_forward.restype = ci
+    lib.foe_context_advance.argtypes = [vp, ci, ci, vp]
+    lib.foe_context_advance.restype = ci
     _lib = lib
     return lib
 
@@ -250,8 +259,9 @@ class FoeLayer:
     def last_launch_count(self) -> int:
         return self.lib.foe_last_launch_count(self.handle)
 
-    def set_profiling(self, on: bool) -> None:
-        _check(self.lib.foe_set_profiling(self.handle, 1 if on else 0), "foe_set_profiling")
+    def set_profiling(self, on) -> None:
+        """False / 0: off; True / 1: the last call; n > 1: the n most recent calls (stage_ms returns their mean)."""
+        _check(self.lib.foe_set_profiling(self.handle, int(on)), "foe_set_profiling")
 
     def stage_ms(self) -> Dict[str, float]:
         n = self.lib.foe_num_stages()

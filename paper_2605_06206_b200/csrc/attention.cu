@@ -8,7 +8,7 @@
 // two 64 x 64 boxes written with the 128-byte swizzle, the bank-conflict-free layout ldmatrix wants.  One CTA
 // per (sequence, KV head, split of the context); the g query heads of the KV head are the rows of mma.sync
 // m16n8k16 tiles (fp32 accumulate, online softmax in the exp2 domain); each of 4 warps takes 16 keys of every
-// page; partial (m, l, o) per split are merged by a second kernel.
+// page; partial (m, l, o) per split are merged by whichever CTA of the (sequence, KV head) finishes last.
 #include <math.h>
 
 #include "common.cuh"
@@ -48,12 +48,13 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   uint8_t* kv_s = smem;                                            // [stage][K | V]; reused for the merge
   uint8_t* q_s = smem + kDcStages * 2 * kTileBytes;
   uint64_t* full = reinterpret_cast<uint64_t*>(q_s + kQBytes);
+  int* abort_s = reinterpret_cast<int*>(full + kDcStages);         // [2]: a wait ran out in an (even, odd) iteration
 
   // Until pdl_wait() nothing is read that the previous kernel writes: this grid may start while the QKV projection of
   // the same step is still running, and that kernel writes q and the new token's K / V (into the sequence's last
   // page).  Everything older is complete (a kernel lets its successor start only after its own wait).
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
-  const int ctx = a.context_lens[b];
+  const int ctx = min(max(a.context_lens[b], 0), a.max_pages_per_seq * 64 - 1);     // (out-of-range values are reported by the QKV step)
   const int kv_len = ctx + 1;                                      // cached tokens + the new one
   const int n_pages = (kv_len + 63) >> 6;
   const int p_begin = split * a.pages_per_split;
@@ -71,6 +72,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   };
   if (threadIdx.x == 0) {
     for (int s = 0; s < kDcStages; ++s) mbar_init(&full[s], 1);
+    abort_s[0] = abort_s[1] = 0;
     mbar_fence_init();
     for (int s = 0; s < kDcStages && s < n_tiles; ++s)             // the ring's first tiles, except the page being written
       if (p_begin + s != n_pages - 1)
@@ -104,11 +106,15 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
 
   for (int j = 0; j < n_tiles; ++j) {
     const int st = j % kDcStages;
-    if (!mbar_wait(&full[st], (j / kDcStages) & 1)) { ok = false; break; }
+    // A wait that runs out is announced through shared memory and the whole CTA leaves the loop together after the
+    // barrier below (the flag alternates with the iteration's parity, so a thread that is already one iteration ahead
+    // cannot change what a slower one reads).
+    const bool landed = mbar_wait(&full[st], (j / kDcStages) & 1);
+    if (!landed) abort_s[j & 1] = 1;
     const uint32_t k_base = smem_u32(kv_s + st * 2 * kTileBytes);
     const uint32_t v_base = k_base + kTileBytes;
     const int key0 = (p_begin + j) * 64 + warp * 16;               // this warp's 16 keys of the page
-    if (key0 < kv_len) {
+    if (landed && key0 < kv_len) {
       float s[2][4];
       s[0][0] = s[0][1] = s[0][2] = s[0][3] = s[1][0] = s[1][1] = s[1][2] = s[1][3] = 0.f;
 #pragma unroll
@@ -170,14 +176,14 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
       }
     }
     __syncthreads();
+    if (abort_s[j & 1]) { ok = false; break; }
     if (threadIdx.x == 0 && j + kDcStages < n_tiles)
       tma_load_page<DH>(kv_s + st * 2 * kTileBytes, kv_s + st * 2 * kTileBytes + kTileBytes, &tmK, &tmV, &full[st],
                         page_row0(p_begin + j + kDcStages));
   }
-  if (!ok) {
-    if (lane == 0) atomicExch(a.status, kStatusTimeout);
-    return;
-  }
+  // A split whose wait ran out records the timeout and writes no partial state, but still takes its ticket below: the
+  // counter of its (sequence, KV head) returns to zero and the handle stays usable (this call's output is not).
+  if (!ok && threadIdx.x == 0) atomicExch(a.status, kStatusTimeout);
 
   // merge the four warps' partial states (each saw a different quarter of every page)
   float* mo = reinterpret_cast<float*>(kv_s);                      // [4][16][DH]
@@ -193,7 +199,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     ml[warp * 16 + g] = l_run[0]; ml[warp * 16 + g + 8] = l_run[1];
   }
   __syncthreads();
-  for (int q = threadIdx.x; q < G * DH; q += kDcThreads) {
+  for (int q = threadIdx.x; ok && q < G * DH; q += kDcThreads) {
     const int r = q / DH, c = q - r * DH;
     float m = -INFINITY;
 #pragma unroll
@@ -245,14 +251,19 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
 }
 
 template <int DH>
+constexpr size_t decode_smem_bytes() { return kDcStages * 2 * 64 * DH * 2 + 16 * DH * 2 + 1024 + 64; }   // ... + barriers and abort flags
+
+// opt in to the dynamic shared memory of the decode kernels on the current device (every layer creation calls this)
+cudaError_t attn_decode_configure() {
+  cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(decode_smem_bytes<64>()));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attn_decode_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(decode_smem_bytes<128>()));
+}
+
+template <int DH>
 static void launch_decode_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st) {
-  constexpr size_t smem = kDcStages * 2 * 64 * DH * 2 + 16 * DH * 2 + 1024 + 64;
+  constexpr size_t smem = decode_smem_bytes<DH>();
   static_assert(kDcStages * 2 * 64 * DH * 2 >= (4 * 16 * DH + 128 + 4) * 4, "merge buffer must fit in the stages");
-  static bool configured = false;
-  if (!configured) {
-    cudaFuncSetAttribute(attn_decode_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    configured = true;
-  }
   dim3 grid(a.max_splits, a.n_kv, a.n_seqs);
   launch_pdl(attn_decode_kernel<DH>, grid, dim3(kDcThreads), smem, st, tmK, tmV, a);
 }

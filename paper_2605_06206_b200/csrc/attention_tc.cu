@@ -113,10 +113,13 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   const int q_len = a.q_lens ? a.q_lens[b] : 1;
   const int q0 = qb * kAtRows;
   if (q0 >= q_len) return;
-  const int ctx = a.context_lens[b];
   const int tok0 = a.cu_q[b] + q0;
+  if (tok0 < 0 || tok0 >= a.n_tokens) return;              // q_lens that disagree with the call's token count (reported by the token map)
   const int kvh = head0 / G;
-  const int rows_here = min(kAtRows, q_len - q0);
+  const int rows_here = min(min(kAtRows, q_len - q0), a.n_tokens - tok0);
+  // a context length outside what the block table can describe is reported by the token map; here it is only kept
+  // from driving the loop bounds
+  const int ctx = min(max(a.context_lens[b], 0), max(a.max_pages_per_seq * kAtKeys - (q0 + rows_here), 0));
   const int kv_len = ctx + q0 + rows_here;
   const int n_tiles = (kv_len + kAtKeys - 1) / kAtKeys;
 
@@ -383,14 +386,15 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   }
 }
 
+cudaError_t attn_prefill_configure() {
+  cudaError_t e = cudaFuncSetAttribute(attn_prefill_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(AtSmem<64>::kBytes));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attn_prefill_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(AtSmem<128>::kBytes));
+}
+
 template <int DH>
 static void launch_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
                       cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaFuncSetAttribute(attn_prefill_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(AtSmem<DH>::kBytes));
-    configured = true;
-  }
   const int G = a.n_q / a.n_kv;
   const int heads_per_cta = (G % 2 == 0) ? 2 : 1;
   dim3 grid((a.max_q_len + kAtRows - 1) / kAtRows, a.n_q / heads_per_cta, a.n_seqs);

@@ -236,7 +236,7 @@ decode_proj_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
           pos = a.context_lens[tok];
           const int lp = pos >> 6;
           slot = -1;
-          if (lp < a.max_pages_per_seq && pos < a.max_context) {
+          if (pos >= 0 && lp < a.max_pages_per_seq && pos < a.max_context) {
             const int page = a.block_table[size_t(tok) * a.max_pages_per_seq + lp];
             if (page >= 0 && page < a.num_pages) slot = page * 64 + (pos & 63);
           }
@@ -322,9 +322,40 @@ decode_proj_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 
 namespace {
 
+// clusters of 1, 2, 4, 8 CTAs of each kernel the device holds at once (a property of the GPU model, refreshed by
+// every decode_proj_configure)
+template <int EPI>
+struct DpOccupancy { static int max_active[4]; };
+template <int EPI>
+int DpOccupancy<EPI>::max_active[4] = {0, 0, 0, 0};
+
+template <int EPI>
+cudaError_t configure_one() {
+  const cudaError_t e = cudaFuncSetAttribute(decode_proj_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kDpSmemBytes));
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.blockDim = dim3(kDpThreads, 1, 1);
+  cfg.dynamicSmemBytes = kDpSmemBytes;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  for (int i = 0; i < 4; ++i) {
+    int n = 0;
+    attr.val.clusterDim.x = 1 << i;
+    cfg.gridDim = dim3(1 << i, 1, 1);
+    if (cudaOccupancyMaxActiveClusters(&n, decode_proj_kernel<EPI>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+    DpOccupancy<EPI>::max_active[i] = n;
+  }
+  return cudaSuccess;
+}
+
 template <int EPI>
 void launch_one(const CUtensorMap& tmW, const CUtensorMap& tmX, DecodeProjArgs a, int tiles, cudaStream_t st) {
-  static int max_active[4] = {-1, -1, -1, -1};   // clusters of 1, 2, 4, 8 of these CTAs the device holds at once (asked once)
+  const int* max_active = DpOccupancy<EPI>::max_active;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.blockDim = dim3(kDpThreads, 1, 1);
@@ -339,16 +370,6 @@ void launch_one(const CUtensorMap& tmW, const CUtensorMap& tmX, DecodeProjArgs a
   attrs[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attrs;
   cfg.numAttrs = g_overlap_launches ? 2 : 1;
-  if (max_active[0] < 0) {
-    cudaFuncSetAttribute(decode_proj_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kDpSmemBytes));
-    for (int i = 0; i < 4; ++i) {
-      int n = 0;
-      attr.val.clusterDim.x = 1 << i;
-      cfg.gridDim = dim3(1 << i, 1, 1);
-      if (cudaOccupancyMaxActiveClusters(&n, decode_proj_kernel<EPI>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
-      max_active[i] = n;
-    }
-  }
   // all clusters of a launch should be resident together: a cluster that has to wait for a free group of SMs
   // doubles the kernel's time
   while (a.k_splits > 1) {
@@ -363,6 +384,11 @@ void launch_one(const CUtensorMap& tmW, const CUtensorMap& tmX, DecodeProjArgs a
 }
 
 }  // namespace
+
+cudaError_t decode_proj_configure() {
+  const cudaError_t e = configure_one<kEpiQKV>();
+  return e != cudaSuccess ? e : configure_one<kEpiOProj>();
+}
 
 bool decode_proj_supported(int epi, int N, int K, int dh) {
   if (N <= 0 || N % kDpSlab || K <= 0 || K % kDpBK) return false;

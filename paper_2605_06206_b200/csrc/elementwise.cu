@@ -106,7 +106,7 @@ __global__ void cu_q_kernel(const int* __restrict__ q_lens, int n_seqs, int* __r
 
 __global__ void token_map_kernel(const int* __restrict__ cu_q, int* __restrict__ cu_q_out, int has_q_lens, const int* __restrict__ context_lens,
                                  const int* __restrict__ block_table, int n_seqs, int max_pages_per_seq,
-                                 int num_pages, int page_size, int n_tokens, int max_context,
+                                 int num_pages, int page_size, int n_tokens, int max_context, int max_q_len,
                                  int* __restrict__ tok_seq, int* __restrict__ tok_pos, int* __restrict__ tok_slot,
                                  int* __restrict__ status) {
   pdl_wait();
@@ -124,29 +124,49 @@ __global__ void token_map_kernel(const int* __restrict__ cu_q, int* __restrict__
     b = lo;
   }
   const int local = has_q_lens ? i - cu_q[b] : 0;
+  const int q_len = has_q_lens ? cu_q[b + 1] - cu_q[b] : 1;
   const int pos = context_lens[b] + local;
-  const int lp = pos / page_size;
   int slot = -1;
-  if (lp < max_pages_per_seq && pos < max_context) {
-    const int page = block_table[size_t(b) * max_pages_per_seq + lp];
-    if (page >= 0 && page < num_pages) slot = page * page_size + (pos - lp * page_size);
+  // a position outside [0, max_context) never reaches the block table; a sequence longer than the call's stated
+  // bound, or a prefix sum that disagrees with the call's token count, is an error of the whole call
+  bool ok = pos >= 0 && pos < max_context && q_len <= max_q_len;
+  if (has_q_lens && i == n_tokens - 1 && cu_q[n_seqs] != n_tokens) ok = false;
+  if (ok) {
+    const int lp = pos / page_size;
+    if (lp < max_pages_per_seq) {
+      const int page = block_table[size_t(b) * max_pages_per_seq + lp];
+      if (page >= 0 && page < num_pages) slot = page * page_size + (pos - lp * page_size);
+    }
   }
   if (slot < 0) atomicExch(status, kStatusBounds);
   tok_seq[i] = b;
-  tok_pos[i] = pos;
+  // consumers index the rotary table with this: keep it inside the table whatever the caller passed
+  tok_pos[i] = min(max(pos, 0), max_context - 1);
   tok_slot[i] = slot;
 }
 
 int launch_token_map(const int* q_lens, const int* context_lens, const int* block_table, int n_seqs,
-                      int max_pages_per_seq, int num_pages, int page_size, int n_tokens, int max_context, int* cu_q,
-                      int* tok_seq, int* tok_pos, int* tok_slot, int* status, cudaStream_t st) {
+                      int max_pages_per_seq, int num_pages, int page_size, int n_tokens, int max_context, int max_q_len,
+                      int* cu_q, int* tok_seq, int* tok_pos, int* tok_slot, int* status, cudaStream_t st) {
   int launches = 0;
   if (q_lens) { launch_pdl(cu_q_kernel, dim3(1), dim3(32), 0, st, q_lens, n_seqs, cu_q); ++launches; }
   if (n_tokens <= 0) return launches;
   launch_pdl(token_map_kernel, dim3((n_tokens + 255) / 256), dim3(256), 0, st, cu_q, cu_q, q_lens != nullptr, context_lens, block_table, n_seqs,
                                                          max_pages_per_seq, num_pages, page_size, n_tokens,
-                                                         max_context, tok_seq, tok_pos, tok_slot, status);
+                                                         max_context, max_q_len, tok_seq, tok_pos, tok_slot, status);
   return launches + 1;
+}
+
+// v[i] += by: the caller's context lengths after a step, bumped on the device so that a decode loop never touches them
+// from the host.  An ordinary launch (no early start): it follows kernels that still read the old values.
+__global__ void add_to_ints_kernel(int* __restrict__ v, int n, int by) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) v[i] += by;
+}
+
+void launch_add_to_ints(int* v, int n, int by, cudaStream_t st) {
+  if (n <= 0) return;
+  add_to_ints_kernel<<<(n + 255) / 256, 256, 0, st>>>(v, n, by);
 }
 
 // ------------------------------------------------------------------ combine (+ residual, + last-layer mean)

@@ -59,6 +59,8 @@ struct foe_workspace {
   float *inv_rms, *inv_rms_f, *route_part, *r_full, *logits, *topk_w, *part_o, *part_ml;
   bf16 *qkv, *attn_o, *u, *hmid, *y;
   int *topk_idx, *cu_q, *tok_seq, *tok_pos, *tok_slot, *status, *split_done;
+  size_t route_part_cap;                        // floats in route_part
+  size_t split_done_count;                      // ints in split_done
   PermuteBuffers pb;
   CUtensorMap tm_attn_o, tm_hmid, tm_qkv;       // maps of workspace buffers (A operands, attention Q)
   CUtensorMap tm_attn_o64;                       // attention output with 64-row boxes (decode O-projection)
@@ -88,8 +90,9 @@ struct foe_layer {
   int last_tokens, launches;
   bool last_decode;
   int shard_stage;       // 0: no sharded call in flight; 1: foe_shard_attend done, foe_shard_ffn owed
-  int profiling;
-  cudaEvent_t ev[kNumStages + 1];
+  int profiling;                       // 0 off, else the number of recent calls whose stage events are kept
+  std::vector<cudaEvent_t> ev;         // [profiling][kNumStages + 1]
+  int prof_calls;                      // calls recorded since the times were last read
   bool ev_valid;
 };
 
@@ -120,6 +123,9 @@ bool shard_config_ok(const foe_shard_config* c) {
          c->hidden % (32 * c->n_ranks) == 0 && c->max_tokens > 0 && c->wait_limit_ms >= 0;
 }
 size_t shard_slots_bytes(const foe_shard_config* c) { return size_t(2) * c->max_tokens * c->hidden * sizeof(bf16); }
+
+// floats of the split-K partial-score buffer of a workspace for calls of up to S tokens
+size_t route_part_capacity(size_t S, size_t E) { return S * E > (size_t(1) << 21) ? S * E : (size_t(1) << 21); }
 
 template <typename T>
 bool dalloc(foe_layer* L, T** p, size_t count) {
@@ -168,7 +174,7 @@ foe_status validate(const foe_config* c) {
 }
 
 void stage_mark(foe_layer* L, int i, cudaStream_t st) {
-  if (L->profiling) cudaEventRecord(L->ev[i], st);
+  if (L->profiling) cudaEventRecord(L->ev[size_t(L->prof_calls % L->profiling) * (kNumStages + 1) + i], st);
 }
 
 foe_status check_launch() { return cudaGetLastError() == cudaSuccess ? FOE_OK : FOE_ERR_CUDA; }
@@ -177,13 +183,13 @@ foe_status check_launch() { return cudaGetLastError() == cudaSuccess ? FOE_OK : 
 void run_route_and_permute(foe_layer* L, const void* r, int r_is_bf16, int n, cudaStream_t st) {
   if (n <= kRouteSmallMaxTokens) {          // a decode step: two launches for norm, scores, top-k, gates and maps
     L->launches += launch_route_small(r, r_is_bf16, L->ffn_gain, L->router_w, L->router_b, L->ws->u, L->ws->route_part,
-                                      L->ws->logits, L->ws->topk_idx, L->ws->topk_w, L->ws->pb, n, L->d, L->H, L->Ec,
+                                      L->ws->route_part_cap, L->ws->logits, L->ws->topk_idx, L->ws->topk_w, L->ws->pb, n, L->d, L->H, L->Ec,
                                       L->kc, L->cfg.rms_eps, L->ws->status, st);
     stage_mark(L, kStPermute, st);
     return;
   }
   L->launches += launch_route(r, r_is_bf16, L->ffn_gain, L->router_w, &L->tm_router, L->router_b, L->ws->u, L->ws->inv_rms_f, L->ws->route_part,
-                              L->ws->logits, L->ws->topk_idx, L->ws->topk_w, n, L->d, L->H, L->Ec, L->kc, L->cfg.rms_eps, L->n_sms, L->ws->status, st);
+                              L->ws->route_part_cap, L->ws->logits, L->ws->topk_idx, L->ws->topk_w, n, L->d, L->H, L->Ec, L->kc, L->cfg.rms_eps, L->n_sms, L->ws->status, st);
   stage_mark(L, kStPermute, st);
   L->launches += launch_permute(L->ws->topk_idx, L->ws->pb, n, L->H * L->kc, L->E, L->ws->status, st);
 }
@@ -203,7 +209,7 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
   L->launches = 0;
   L->last_tokens = S;
   L->last_decode = decode;
-  L->ev_valid = false;
+  if (L->profiling <= 1) { L->ev_valid = false; L->prof_calls = 0; }
   if (S == 0) return FOE_OK;
   const int H = L->H, d = L->d, dh = L->dh;
   const bf16* xb = static_cast<const bf16*>(x);
@@ -219,7 +225,7 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
   //  its position and cache slot are looked up where they are used)
   const bool inline_map = decode && L->dp_qkv;
   if (!inline_map) L->launches += launch_token_map(decode ? nullptr : kv->q_lens, kv->context_lens, kv->block_table, kv->n_seqs, kv->max_pages_per_seq,
-                   kv->num_pages, 64, S, L->cfg.max_context, L->ws->cu_q, L->ws->tok_seq, L->ws->tok_pos, L->ws->tok_slot, L->ws->status, st);
+                   kv->num_pages, 64, S, L->cfg.max_context, decode ? 1 : kv->max_q_len, L->ws->cu_q, L->ws->tok_seq, L->ws->tok_pos, L->ws->tok_slot, L->ws->status, st);
   const int x_rows = L->first ? S : H * S;
   // Kernel family of the two projections: a call of a few hundred tokens (any decode step, a short prompt chunk, a
   // small mixed batch) is a weight-streaming problem and takes the decode kernels, whatever entry point it came by.
@@ -289,7 +295,7 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
   memset(&aa, 0, sizeof(aa));
   aa.q = L->ws->qkv; aa.out = L->ws->attn_o; aa.cu_q = inline_map ? nullptr : L->ws->cu_q; aa.context_lens = kv->context_lens;
   aa.q_lens = decode ? nullptr : kv->q_lens; aa.block_table = kv->block_table; aa.n_seqs = kv->n_seqs;
-  aa.max_pages_per_seq = kv->max_pages_per_seq; aa.num_pages = kv->num_pages; aa.n_q = L->n_q; aa.n_kv = L->n_kv;
+  aa.max_pages_per_seq = kv->max_pages_per_seq; aa.num_pages = kv->num_pages; aa.n_tokens = S; aa.n_q = L->n_q; aa.n_kv = L->n_kv;
   aa.dh = dh; aa.max_q_len = decode ? 1 : kv->max_q_len; aa.scale_log2 = float(1.4426950408889634 / sqrt(double(dh)));
   aa.status = L->ws->status; aa.part_o = L->ws->part_o; aa.part_ml = L->ws->part_ml; aa.max_splits = L->max_splits;
   aa.pages_per_split = L->pages_per_split; aa.split_done = L->ws->split_done;
@@ -410,7 +416,7 @@ foe_status run_ffn(foe_layer* L, void* out, cudaStream_t st) {
   stage_mark(L, kStCombine, st);
   launch_combine(L->ws->r_full, L->ws->y, L->ws->topk_w, L->ws->pb.inv, static_cast<bf16*>(out), S, d, H, L->kc, L->last ? 1 : 0, st);
   L->launches += 1;
-  if (L->profiling) { cudaEventRecord(L->ev[kNumStages], st); L->ev_valid = true; }
+  if (L->profiling) { stage_mark(L, kNumStages, st); L->prof_calls += 1; L->ev_valid = true; }
   return check_launch();
 }
 
@@ -458,8 +464,7 @@ foe_status foe_layer_destroy(foe_layer* L) {
   if (!L) return FOE_OK;
   for (void* p : L->allocs) cudaFree(p);
   ws_release(L->ws);
-  for (int i = 0; i <= kNumStages; ++i)
-    if (L->ev[i]) cudaEventDestroy(L->ev[i]);
+  for (cudaEvent_t e : L->ev) cudaEventDestroy(e);
   delete L;
   return FOE_OK;
 }
@@ -482,7 +487,11 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return FOE_ERR_CUDA;
   if (prop.major != 10) return FOE_ERR_UNSUPPORTED;       // tcgen05/TMEM kernels: sm_100 only
-  if (gemm_configure() != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  if (gemm_configure() != cudaSuccess || attn_decode_configure() != cudaSuccess || attn_prefill_configure() != cudaSuccess ||
+      router_tc_configure() != cudaSuccess || smallm_configure() != cudaSuccess || decode_proj_configure() != cudaSuccess) {
+    cudaGetLastError();
+    return FOE_ERR_CUDA;
+  }
   if (donor) {   // a shared workspace must have been sized for exactly these shapes
     const foe_config& a = donor->cfg;
     if (a.hidden != cfg->hidden || a.n_q_heads != cfg->n_q_heads || a.n_kv_heads != cfg->n_kv_heads ||
@@ -536,7 +545,8 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     ok = ok && walloc(W, &W->r_full, size_t(S) * d);
     ok = ok && walloc(W, &W->logits, size_t(S) * E);
     ok = ok && walloc(W, &W->inv_rms_f, size_t(S));
-    ok = ok && walloc(W, &W->route_part, size_t(S) * E > (size_t(1) << 21) ? size_t(S) * E : (size_t(1) << 21));
+    W->route_part_cap = route_part_capacity(size_t(S), size_t(E));
+    ok = ok && walloc(W, &W->route_part, W->route_part_cap);
     ok = ok && walloc(W, &W->topk_w, size_t(R));
     ok = ok && walloc(W, &W->topk_idx, size_t(R));
     ok = ok && walloc(W, &W->qkv, size_t(S + 128) * L->n_q * L->dhp);      // q after RoPE (k, v go to the pages)
@@ -551,7 +561,8 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
     ok = ok && walloc(W, &W->status, size_t(1));
     ok = ok && walloc(W, &W->part_o, size_t(cfg->max_seqs) * L->n_q * L->max_splits * L->dhp);
     ok = ok && walloc(W, &W->part_ml, size_t(cfg->max_seqs) * L->n_q * L->max_splits * 2);
-    ok = ok && walloc(W, &W->split_done, size_t(cfg->max_seqs) * L->n_kv);
+    W->split_done_count = size_t(cfg->max_seqs) * L->n_kv;
+    ok = ok && walloc(W, &W->split_done, W->split_done_count);
     ok = ok && walloc(W, &W->pb.counts, size_t(E));
     ok = ok && walloc(W, &W->pb.offsets, size_t(E) + 1);
     ok = ok && walloc(W, &W->pb.perm, size_t(R));
@@ -626,7 +637,6 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
   L->dp_qkv = decode_proj_supported(kEpiQKV, qkvN, d, dh);
   L->dp_oproj = decode_proj_supported(kEpiOProj, d, L->n_q * dh, dh);
   if (!ok) { foe_layer_destroy(L); return FOE_ERR_CUDA; }
-  for (int i = 0; i <= kNumStages; ++i) cudaEventCreate(&L->ev[i]);
   *out = L;
   return FOE_OK;
 }
@@ -651,6 +661,52 @@ foe_status foe_decode(foe_layer* L, const void* x, const foe_kv_cache* kv, void*
   if (c != FOE_OK) return c;
   if (x == out) return FOE_ERR_UNSUPPORTED;
   return run_block(L, x, kv, out, static_cast<cudaStream_t>(stream), true);
+}
+
+foe_status foe_stack_forward(foe_layer* const* layers, int n_layers, const void* x, const foe_kv_cache* kvs, void* out,
+                             void* work0, void* work1, int decode, void* stream) {
+  if (!layers || !kvs || n_layers <= 0) return n_layers <= 0 && layers && kvs ? FOE_ERR_SHAPE : FOE_ERR_NULL;
+  for (int l = 0; l < n_layers; ++l)
+    if (!layers[l]) return FOE_ERR_NULL;
+  if (n_layers > 1 && !work0) return FOE_ERR_NULL;
+  if (n_layers > 2 && !work1) return FOE_ERR_NULL;
+  if (work0 && (work0 == work1 || work0 == x || work0 == out)) return FOE_ERR_UNSUPPORTED;
+  if (work1 && (work1 == x || work1 == out)) return FOE_ERR_UNSUPPORTED;
+  // every layer's arguments are checked before the first one is launched
+  for (int l = 0; l < n_layers; ++l) {
+    const foe_kv_cache* kv = &kvs[l];
+    if (kv->n_tokens < 0 || kv->n_seqs < 0) return FOE_ERR_SHAPE;
+    const int S = decode ? kv->n_seqs : kv->n_tokens;
+    const int S0 = decode ? kvs[0].n_seqs : kvs[0].n_tokens;
+    if (S != S0) return FOE_ERR_SHAPE;
+    if (S == 0) continue;
+    const foe_status c = check_call(layers[l], kv, decode != 0);
+    if (c != FOE_OK) return c;
+    if (l > 0 && (layers[l]->first || layers[l]->d != layers[l - 1]->d ||
+                  (layers[l - 1]->last ? 1 : layers[l - 1]->H) != layers[l]->H))
+      return FOE_ERR_CONFIG;             // layer l must take what layer l-1 produces
+  }
+  const int S = decode ? kvs[0].n_seqs : kvs[0].n_tokens;
+  if (S > 0 && (!x || !out)) return FOE_ERR_NULL;
+  if (S > 0 && x == out) return FOE_ERR_UNSUPPORTED;
+  void* bufs[2] = {work0, work1};
+  const void* in = x;
+  for (int l = 0; l < n_layers; ++l) {
+    void* dst = l == n_layers - 1 ? out : bufs[l & 1];
+    if (S == 0) { layers[l]->launches = 0; layers[l]->last_tokens = 0; continue; }
+    const foe_status r = run_block(layers[l], in, &kvs[l], dst, static_cast<cudaStream_t>(stream), decode != 0);
+    if (r != FOE_OK) return r;
+    in = dst;
+  }
+  return FOE_OK;
+}
+
+foe_status foe_context_advance(int* context_lens, int n_seqs, int by, void* stream) {
+  if (!context_lens) return FOE_ERR_NULL;
+  if (n_seqs < 0) return FOE_ERR_SHAPE;
+  if (n_seqs == 0 || by == 0) return FOE_OK;
+  launch_add_to_ints(context_lens, n_seqs, by, static_cast<cudaStream_t>(stream));
+  return check_launch();
 }
 
 foe_status foe_route(foe_layer* L, const void* h, int n_tokens, int* topk_idx, float* topk_w, void* stream) {
@@ -682,10 +738,29 @@ foe_status foe_route_noalloc(int hidden, int n_clusters, int experts_per_cluster
       n_clusters * experts_per_cluster > 1024 || !(rms_eps >= 0.f))
     return FOE_ERR_CONFIG;
   if (n_tokens < 0) return FOE_ERR_SHAPE;
+  // the kernels read h and router_w 16 bytes at a time, the gain 8, the outputs 4: a misaligned view is refused here
+  // instead of faulting on the device
+  auto misaligned = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; };
+  if (misaligned(h, 16) || misaligned(router_w, 16) || misaligned(ffn_norm_g, 8) || misaligned(topk_idx, 4) ||
+      misaligned(topk_w, 4) || (router_b && misaligned(router_b, 4)))
+    return FOE_ERR_SHAPE;
   const int rc = launch_route_noalloc(static_cast<const bf16*>(h), static_cast<const bf16*>(ffn_norm_g), router_w, router_b,
                                       topk_idx, topk_w, n_tokens, hidden, n_clusters, experts_per_cluster,
                                       top_k_per_cluster, rms_eps, static_cast<cudaStream_t>(stream));
   return rc == 0 ? FOE_OK : (rc == -3 ? FOE_ERR_SHAPE : FOE_ERR_CUDA);
+}
+
+size_t foe_route_partial_capacity(int max_tokens, int max_seqs, int n_experts) {
+  if (max_tokens <= 0 || max_seqs <= 0 || n_experts <= 0) return 0;
+  return route_part_capacity(size_t(max_tokens > max_seqs ? max_tokens : max_seqs), size_t(n_experts));
+}
+
+size_t foe_route_partial_floats(int hidden, int n_experts, int n_tokens, int n_sms, size_t capacity) {
+  if (hidden <= 0 || n_experts <= 0 || n_tokens <= 0 || n_sms <= 0) return 0;
+  int ks = 1;                                             // the tensor-core score kernel does not split
+  if (n_tokens <= kRouteSmallMaxTokens) ks = clamp_k_splits(route_small_k_splits(hidden), n_tokens, n_experts, capacity);
+  else if (n_tokens < kRouterTcMinTokens) ks = clamp_k_splits(route_k_splits(n_tokens, hidden, n_experts, n_sms), n_tokens, n_experts, capacity);
+  return size_t(ks) * size_t(n_tokens) * size_t(n_experts);
 }
 
 foe_status foe_get_aux(foe_layer* L, foe_aux* a) {
@@ -703,7 +778,11 @@ foe_status foe_poll_status(foe_layer* L, int* device_status) {
   int v = 0;
   if (cudaMemcpy(&v, L->ws->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FOE_ERR_CUDA;
   *device_status = v;
-  if (v != 0) cudaMemset(L->ws->status, 0, sizeof(int));
+  if (v != 0) {
+    cudaMemset(L->ws->status, 0, sizeof(int));
+    // the split counters of the decode attention re-arm themselves; after a reported failure make sure of it
+    cudaMemset(L->ws->split_done, 0, L->ws->split_done_count * sizeof(int));
+  }
   return FOE_OK;
 }
 
@@ -711,7 +790,16 @@ int foe_last_launch_count(const foe_layer* L) { return L ? L->launches : 0; }
 
 foe_status foe_set_profiling(foe_layer* L, int enabled) {
   if (!L) return FOE_ERR_NULL;
-  L->profiling = enabled ? 1 : 0;
+  const int ring = enabled < 0 ? 0 : (enabled > 256 ? 256 : enabled);
+  const size_t want = size_t(ring) * (kNumStages + 1);
+  while (L->ev.size() < want) {
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+    L->ev.push_back(e);
+  }
+  L->profiling = ring;
+  L->prof_calls = 0;
+  L->ev_valid = false;
   return FOE_OK;
 }
 
@@ -721,10 +809,23 @@ const char* foe_stage_name(int i) { return (i >= 0 && i < kNumStages) ? kStageNa
 
 foe_status foe_get_stage_ms(foe_layer* L, float* ms, int n) {
   if (!L || !ms) return FOE_ERR_NULL;
-  if (!L->ev_valid || n < kNumStages) return FOE_ERR_UNSUPPORTED;
-  if (cudaEventSynchronize(L->ev[kNumStages]) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
-  for (int i = 0; i < kNumStages; ++i)
-    if (cudaEventElapsedTime(&ms[i], L->ev[i], L->ev[i + 1]) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  if (!L->ev_valid || n < kNumStages || L->profiling <= 0 || L->prof_calls <= 0) return FOE_ERR_UNSUPPORTED;
+  const int ring = L->profiling;
+  const int sets = L->prof_calls < ring ? L->prof_calls : ring;          // the most recent calls still in the ring
+  const int last = (L->prof_calls - 1) % ring;
+  if (cudaEventSynchronize(L->ev[size_t(last) * (kNumStages + 1) + kNumStages]) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+  for (int i = 0; i < kNumStages; ++i) ms[i] = 0.f;
+  for (int c = 0; c < sets; ++c) {
+    const size_t base = size_t((L->prof_calls - 1 - c) % ring) * (kNumStages + 1);
+    for (int i = 0; i < kNumStages; ++i) {
+      float t = 0.f;
+      if (cudaEventElapsedTime(&t, L->ev[base + i], L->ev[base + i + 1]) != cudaSuccess) { cudaGetLastError(); return FOE_ERR_CUDA; }
+      ms[i] += t;
+    }
+  }
+  for (int i = 0; i < kNumStages; ++i) ms[i] /= float(sets);
+  L->prof_calls = 0;
+  L->ev_valid = false;
   return FOE_OK;
 }
 

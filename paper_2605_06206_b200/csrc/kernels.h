@@ -40,11 +40,13 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 void launch_row_inv_rms(const bf16* x, float* inv_rms, int n_rows, int d, float eps, cudaStream_t st);
 // the same for x = [H][S][d], plus xsum[s][:] = sum_h x[h][s][:] in fp32; false (nothing launched) unless 2 <= H <= 8
 bool launch_row_inv_rms_xsum(const bf16* x, float* inv_rms, float* xsum, int S, int d, int H, float eps, cudaStream_t st);
-// per-token position / sequence / cache slot from q_lens and context_lens (device arrays)
+// per-token position / sequence / cache slot from q_lens and context_lens (device arrays); positions outside
+// [0, max_context), a q_len above max_q_len or sum(q_lens) != n_tokens set the bounds status (slot -1, position clamped)
 // returns the number of kernels launched
 int launch_token_map(const int* q_lens, const int* context_lens, const int* block_table, int n_seqs,
-                      int max_pages_per_seq, int num_pages, int page_size, int n_tokens, int max_context, int* cu_q,
-                      int* tok_seq, int* tok_pos, int* tok_slot, int* status, cudaStream_t st);
+                      int max_pages_per_seq, int num_pages, int page_size, int n_tokens, int max_context, int max_q_len,
+                      int* cu_q, int* tok_seq, int* tok_pos, int* tok_slot, int* status, cudaStream_t st);
+void launch_add_to_ints(int* v, int n, int by, cudaStream_t st);
 // combine: out = r_full + sum_j w * y[inv]  (per cluster), optional mean over clusters
 void launch_combine(const float* r_full, const bf16* y, const float* w, const int* inv, bf16* out, int n_tokens,
                     int d, int H, int kc, int last_mean, cudaStream_t st);
@@ -55,16 +57,20 @@ void launch_pack_gate_up(const bf16* wg, const bf16* wu, bf16* dst, int E, int d
 
 // ---- route.cu
 // FFN norm + fp32 router + per-cluster top-k + gates.  r_in is fp32 or bf16 [S][d].
-// Returns the number of kernels launched.  inv_rms: [S] scratch; part: scratch for the split-K partial scores
-// (at least max(S*E, 2^21) floats).
+// Returns the number of kernels launched.  inv_rms: [S] scratch; part: scratch of part_cap floats (at least S*E) for the
+// split-K partial scores [k_splits][S][E]; the number of splits is reduced until they fit.
 // tm_wr_split: map of the split router weights (launch_split_router_weights; box 64 x 64), or null: plain-ALU scores
 // at every size.
 constexpr int kRouterTcMinTokens = 2048;
 constexpr int kRouterChunk = 64;              // experts per CTA of the tensor-core score kernel
 inline int router_padded_experts(int E) { return (E + kRouterChunk - 1) / kRouterChunk * kRouterChunk; }
 int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const CUtensorMap* tm_wr_split,
-                 const float* br, bf16* u_out, float* inv_rms, float* part, float* logits, int* idx, float* w,
-                 int n_tokens, int d, int H, int Ec, int kc, float eps, int n_sms, int* status, cudaStream_t st);
+                 const float* br, bf16* u_out, float* inv_rms, float* part, size_t part_cap, float* logits, int* idx,
+                 float* w, int n_tokens, int d, int H, int Ec, int kc, float eps, int n_sms, int* status, cudaStream_t st);
+// split-K factors the two score kernels would like for a call (before the clamp to the partial-score buffer) and the clamp
+int route_k_splits(int n_tokens, int d, int E, int n_sms);
+int route_small_k_splits(int d);
+int clamp_k_splits(int ks, int n_tokens, int E, size_t part_cap);
 // planes: [3][router_padded_experts(E)][d] bf16 terms of gain * W
 void launch_split_router_weights(const float* wr, const bf16* gain, bf16* planes, int E, int d, cudaStream_t st);
 void launch_router_tc(const CUtensorMap& tmW, const void* r, int r_is_bf16, const float* inv_rms, float* part,
@@ -75,8 +81,8 @@ void launch_router_tc(const CUtensorMap& tmW, const void* r, int r_is_bf16, cons
 constexpr int kRouteSmallMaxTokens = 256;
 struct PermuteBuffers;
 int launch_route_small(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const float* br, bf16* u_out,
-                       float* scores, float* logits, int* idx, float* w, const PermuteBuffers& pb, int n_tokens, int d,
-                       int H, int Ec, int kc, float eps, int* status, cudaStream_t st);
+                       float* scores, size_t scores_cap, float* logits, int* idx, float* w, const PermuteBuffers& pb,
+                       int n_tokens, int d, int H, int Ec, int kc, float eps, int* status, cudaStream_t st);
 int launch_topk_permute_small(const float* scores, int k_splits, const float* bias, float* logits, int* idx, float* w,
                               const PermuteBuffers& pb, int n_tokens, int H, int Ec, int kc, int* status, cudaStream_t st);
 
@@ -110,6 +116,7 @@ struct AttnArgs {
   const int* q_lens;        // [n_seqs] or nullptr (1 each)
   const int* block_table;   // [n_seqs][max_pages_per_seq]
   int n_seqs, max_pages_per_seq, num_pages;
+  int n_tokens;             // tokens of the call (prefill)
   int n_q, n_kv, dh;        // dh: the real head_dim (64, 96 or 128); kernels are instantiated for 64 and 128 and read
                             // a 96-wide head zero-padded: q with a head stride of 128, K/V through the tensor maps
   int max_q_len;
@@ -131,6 +138,13 @@ void launch_attn_decode(const CUtensorMap& tmK, const CUtensorMap& tmV, const At
 void launch_gemm(int epi, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args, int n_sms,
                  cudaStream_t st);
 cudaError_t gemm_configure();   // opt in to the dynamic shared memory the kernels need
+// The same for the other kernel families.  Kernel attributes belong to the device that is current when they are set, so
+// every layer creation calls all of these (a process may create layers on several GPUs, from several host threads).
+cudaError_t attn_decode_configure();
+cudaError_t attn_prefill_configure();
+cudaError_t router_tc_configure();
+cudaError_t smallm_configure();
+cudaError_t decode_proj_configure();
 
 // ---- smallm.cu  (weight-streaming GEMMs for a handful of rows per group)
 struct SmallMArgs {

@@ -14,6 +14,8 @@
 //                   softmax over the selected scores.
 #include <float.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "kernels.h"
 
@@ -340,15 +342,20 @@ route_scores_small_kernel(const void* __restrict__ r_in, int r_is_bf16, const bf
     scores[(size_t(blockIdx.z) * n_tokens + tok) * E + e0 + el] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
 }
 
+int route_small_k_splits(int d) {
+  int ks = 1;
+  while (ks < 16 && (d / (ks * 2)) % kRsK == 0 && d / (ks * 2) >= 2 * kRsK) ks *= 2;
+  return ks;
+}
+
 int launch_route_small(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const float* br, bf16* u_out,
-                       float* scores, float* logits, int* idx, float* w, const PermuteBuffers& pb, int n_tokens, int d,
-                       int H, int Ec, int kc, float eps, int* status, cudaStream_t st) {
+                       float* scores, size_t scores_cap, float* logits, int* idx, float* w, const PermuteBuffers& pb,
+                       int n_tokens, int d, int H, int Ec, int kc, float eps, int* status, cudaStream_t st) {
   if (n_tokens <= 0) return 0;
   const int E = H * Ec;
   // K is cut into slices so that a few dozen tokens still spread over the GPU; the partial scores are summed in a
   // fixed order by the second kernel
-  int ks = 1;
-  while (ks < 16 && (d / (ks * 2)) % kRsK == 0 && d / (ks * 2) >= 2 * kRsK) ks *= 2;
+  const int ks = clamp_k_splits(route_small_k_splits(d), n_tokens, E, scores_cap);
   dim3 grid((n_tokens + kRsTok - 1) / kRsTok, (E + kRsExp - 1) / kRsExp, ks);
   launch_pdl(route_scores_small_kernel, grid, dim3(kRsThreads), 0, st, r_in, r_is_bf16, gain, wr, u_out, scores, n_tokens, d, E, eps, d / ks);
   return 1 + launch_topk_permute_small(scores, ks, br, logits, idx, w, pb, n_tokens, H, Ec, kc, status, st);
@@ -415,6 +422,12 @@ static void launch_topk_gates(const float* part, int ks, const float* br, float*
   launch_pdl(topk_gates_kernel, dim3((warps * 32 + 255) / 256), dim3(256), 0, st, part, ks, br, logits, idx, w, n_tokens, H, Ec, kc);
 }
 
+// the partial scores of all splits ([ks][n_tokens][E] floats) must fit the buffer they go to
+int clamp_k_splits(int ks, int n_tokens, int E, size_t part_cap) {
+  while (ks > 1 && size_t(ks) * size_t(n_tokens) * size_t(E) > part_cap) ks >>= 1;
+  return ks;
+}
+
 int route_k_splits(int n_tokens, int d, int E, int n_sms) {
   const int ctas = ((n_tokens + kRgTM - 1) / kRgTM) * ((E + kRgTN - 1) / kRgTN);
   int ks = 1;
@@ -423,8 +436,8 @@ int route_k_splits(int n_tokens, int d, int E, int n_sms) {
 }
 
 int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float* wr, const CUtensorMap* tm_wr_split,
-                 const float* br, bf16* u_out, float* inv_rms, float* part, float* logits, int* idx, float* w,
-                 int n_tokens, int d, int H, int Ec, int kc, float eps, int n_sms, int* status, cudaStream_t st) {
+                 const float* br, bf16* u_out, float* inv_rms, float* part, size_t part_cap, float* logits, int* idx,
+                 float* w, int n_tokens, int d, int H, int Ec, int kc, float eps, int n_sms, int* status, cudaStream_t st) {
   if (n_tokens <= 0) return 0;
   const int E = H * Ec;
   const dim3 ngrid((n_tokens * 32 + 255) / 256);
@@ -436,7 +449,7 @@ int launch_route(const void* r_in, int r_is_bf16, const bf16* gain, const float*
   if (tm_wr_split && n_tokens >= kRouterTcMinTokens) {
     launch_router_tc(*tm_wr_split, r_in, r_is_bf16, inv_rms, part, n_tokens, d, E, status, st);
   } else {
-    ks = route_k_splits(n_tokens, d, E, n_sms);
+    ks = clamp_k_splits(route_k_splits(n_tokens, d, E, n_sms), n_tokens, E, part_cap);
     dim3 grid((n_tokens + kRgTM - 1) / kRgTM, (E + kRgTN - 1) / kRgTN, ks);
     launch_pdl(router_gemm_kernel, grid, dim3(kRgThreads), 0, st, r_in, r_is_bf16, inv_rms, gain, wr, part, n_tokens, d, E, d / ks);
   }
@@ -464,8 +477,11 @@ constexpr int kNaMaxDevices = 64;
 
 static __device__ __align__(256) float g_route_scratch[kNaMaxTokens + kNaMaxScores + kNaMaxPartial];
 
-static float* g_route_scratch_dev[kNaMaxDevices];     // device address of the array, per device
-static int g_route_sms[kNaMaxDevices];
+// Device address of the array and SM count, per device.  Host threads may make their first calls at the same time:
+// each resolves the same two values, stores the SM count first and then publishes the address with release order, so a
+// thread that sees a non-null address also sees the SM count.
+static std::atomic<float*> g_route_scratch_dev[kNaMaxDevices];
+static std::atomic<int> g_route_sms[kNaMaxDevices];
 
 // inv_rms only: the expert input u is not produced on this path (the caller asked for routing, nothing else)
 __global__ void ffn_inv_rms_bf16_kernel(const bf16* __restrict__ r_in, float* __restrict__ inv_out, int n_tokens, int d,
@@ -494,7 +510,8 @@ int launch_route_noalloc(const bf16* h, const bf16* gain, const float* wr, const
   if (size_t(n_tokens) > kNaMaxTokens || size_t(n_tokens) * E > kNaMaxScores) return -3;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNaMaxDevices) return -6;
-  if (!g_route_scratch_dev[dev]) {
+  float* inv = g_route_scratch_dev[dev].load(std::memory_order_acquire);
+  if (!inv) {
     float* p = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_route_scratch) != cudaSuccess || !p) {
       cudaGetLastError();
@@ -502,17 +519,16 @@ int launch_route_noalloc(const bf16* h, const bf16* gain, const float* wr, const
     }
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return -6;
-    g_route_sms[dev] = sms;
-    g_route_scratch_dev[dev] = p;
+    g_route_sms[dev].store(sms, std::memory_order_relaxed);
+    g_route_scratch_dev[dev].store(p, std::memory_order_release);
+    inv = p;
   }
-  float* inv = g_route_scratch_dev[dev];
   float* logits = inv + kNaMaxTokens;
   float* part = logits + kNaMaxScores;
   if (n_tokens <= 0) return 0;
   // Nothing in the scratch has to start at zero: every entry that is read below is written first by this call.
   ffn_inv_rms_bf16_kernel<<<(n_tokens * 32 + 255) / 256, 256, 0, st>>>(h, inv, n_tokens, d, eps);
-  int ks = route_k_splits(n_tokens, d, E, g_route_sms[dev]);
-  while (ks > 1 && size_t(ks) * n_tokens * E > kNaMaxPartial) ks >>= 1;
+  const int ks = clamp_k_splits(route_k_splits(n_tokens, d, E, g_route_sms[dev].load(std::memory_order_relaxed)), n_tokens, E, kNaMaxPartial);
   dim3 grid((n_tokens + kRgTM - 1) / kRgTM, (E + kRgTN - 1) / kRgTN, ks);
   router_gemm_kernel<<<grid, kRgThreads, 0, st>>>(h, 1, inv, gain, wr, part, n_tokens, d, E, d / ks);
   launch_topk_gates(part, ks, br, logits, idx, w, n_tokens, H, Ec, kc, st);

@@ -241,13 +241,12 @@ void launch_split_router_weights(const float* wr, const bf16* gain, bf16* planes
   split_router_weights_kernel<<<unsigned((total + 255) / 256), 256, 0, st>>>(wr, gain, planes, E, E_pad, d);
 }
 
+cudaError_t router_tc_configure() {
+  return cudaFuncSetAttribute(router_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kRtSmemBytes));
+}
+
 void launch_router_tc(const CUtensorMap& tmW, const void* r, int r_is_bf16, const float* inv_rms, float* part,
                       int n_tokens, int d, int E, int* status, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaFuncSetAttribute(router_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kRtSmemBytes));
-    configured = true;
-  }
   const int E_pad = router_padded_experts(E);
   dim3 grid((n_tokens + kRtRows - 1) / kRtRows, E_pad / kRtChunk);
   launch_pdl(router_tc_kernel, grid, dim3(kRtThreads), kRtSmemBytes, st, tmW, r, r_is_bf16, inv_rms, part, n_tokens, d, E, E_pad, status);

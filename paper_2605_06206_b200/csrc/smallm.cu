@@ -349,16 +349,24 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
 
 template <int EPI>
 static void launch_one(const CUtensorMap& tmW, const SmallMArgs& a, int n_sms, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaFuncSetAttribute(smallm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sm_smem_bytes<EPI>()));
-    configured = true;
-  }
   const int chunks = a.group_offsets ? 1 : (a.rows_per_group + kSmRows - 1) / kSmRows;
   const long long tasks = (long long)a.n_groups * ((a.N + kSmSlab - 1) / kSmSlab) * chunks;
   if (tasks <= 0) return;
   const int grid = int(tasks < 2LL * n_sms ? tasks : 2LL * n_sms);          // two resident CTAs per SM
   launch_pdl(smallm_kernel<EPI>, dim3(grid), dim3(kSmThreads), sm_smem_bytes<EPI>(), st, tmW, a);
+}
+
+template <int EPI>
+static cudaError_t configure_one() {
+  return cudaFuncSetAttribute(smallm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sm_smem_bytes<EPI>()));
+}
+
+cudaError_t smallm_configure() {
+  cudaError_t e = configure_one<kEpiSwiGLU>();
+  if (e == cudaSuccess) e = configure_one<kEpiBf16>();
+  if (e == cudaSuccess) e = configure_one<kEpiQKV>();
+  if (e == cudaSuccess) e = configure_one<kEpiOProj>();
+  return e;
 }
 
 void launch_smallm(const CUtensorMap& tmW, const SmallMArgs& a, int n_sms, cudaStream_t st) {

@@ -194,3 +194,50 @@ def compare_with_oracle(shape, W, x, q_lens, ctx_lens, cache, kv, out, aux, rows
     else:
         mx, rel = assert_close(got, ref_g["out"], "block output (scaled weights)", STAGE_MAX_TOL, STAGE_REL_TOL)
     return dict(max_abs=mx, rel_l1=rel, flips=int(flips.sum()), counts=counts, ref=ref)
+
+
+def check_every_row(shape, W, out, aux, kv, q_lens, ctx_lens, attn_seqs: Sequence[int], chunk: int = 4096) -> Dict:
+    """Full-size parity over EVERY output row of one finished call, stage by stage, at the task's bounds.
+
+    Experts stage: the oracle's moe_stage on the GPU's own fp32 r_full and expert ids, for all tokens (in chunks of
+    tokens: the stage is per token, so chunking changes nothing), against the block output -- every row of every
+    256-row tile of every expert's grouped GEMM enters the maximum.  Attention stage: the oracle's attend() on the
+    GPU's q and on the pages as the call left them, for all rows of the sequences in `attn_seqs`, against the
+    attention output -- every 128-row query block of those sequences."""
+    q_lens, ctx_lens = list(q_lens), list(ctx_lens)
+    S = sum(q_lens)
+    cfg = adapter.cfg_from_shape(shape)
+    Wn = adapter.weights_to_numpy(W)
+    r_gpu = adapter.to_np(aux["r_full"])
+    idx_gpu = aux["topk_idx"].cpu().numpy()
+    got = adapter.to_np(out)
+    max_err = max_ref = sum_err = sum_ref = 0.0
+    worst_tok = -1
+    for t0 in range(0, S, chunk):
+        t1 = min(S, t0 + chunk)
+        iso = orc.moe_stage(cfg, Wn, r_gpu[t0:t1].astype(np.float64), idx_override=idx_gpu[t0:t1])["out"]
+        g = (got[:, t0:t1] if shape.grouped_output else got[t0:t1]).astype(np.float64)
+        err = np.abs(g - iso)
+        if err.max() > max_err:
+            max_err = float(err.max())
+            worst_tok = t0 + int(np.unravel_index(err.argmax(), err.shape)[-2])
+        max_ref = max(max_ref, float(np.abs(iso).max()))
+        sum_err += float(err.sum())
+        sum_ref += float(np.abs(iso).sum())
+    e_max, e_rel = max_err / max_ref, sum_err / sum_ref
+    assert e_max <= MAX_ABS_TOL and e_rel <= MEAN_REL_TOL, \
+        f"experts stage over all {S} tokens: max_abs/max_ref={e_max:.3e} at token {worst_tok}, rel_l1={e_rel:.3e}"
+
+    nq, nkv, dh = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    starts = np.concatenate([[0], np.cumsum(q_lens)])
+    full = [c + q for c, q in zip(ctx_lens, q_lens)]
+    a_stats = []
+    for b in attn_seqs:
+        lo, hi = int(starts[b]), int(starts[b + 1])
+        newc = adapter.logical_cache(kv.k_pages, kv.v_pages, kv.block_table[b:b + 1], [full[b]], 64)[0]
+        qg = adapter.to_np(aux["q"][lo:hi]).reshape(hi - lo, nq, dh).astype(np.float64)
+        pos = ctx_lens[b] + np.arange(hi - lo)
+        o_iso = orc.attend(qg, pos, newc[0].astype(np.float64), newc[1].astype(np.float64), nq // nkv)
+        a_stats.append(assert_close(adapter.to_np(aux["attn_o"][lo:hi]), o_iso.reshape(hi - lo, -1),
+                                    f"attention, every row of sequence {b}"))
+    return dict(experts_max=e_max, experts_rel=e_rel, attention=a_stats)

@@ -63,6 +63,29 @@ def test_null_and_config_errors_need_no_device(lib):
     assert lib.foe_num_stages() == 9 and lib.foe_stage_name(6).decode() == "expert_gemm1_swiglu"
 
 
+def test_split_k_partial_scores_fit_their_buffer_at_every_call_size(lib):
+    """The fp32 score kernels write [k_splits][n_tokens][E] partial scores into a workspace buffer whose size is fixed
+    when the handle is created: for every call size up to the largest that splits, on the five workloads' layer
+    shapes (and the widest layer the configuration rules allow) and several max_tokens, what a call writes must fit.
+    Without the clamp on the number of splits this fails (e.g. E = 128, d = 4096, 1025..1152 tokens: 16 splits)."""
+    from paper_2605_06206_b200 import synth
+    shapes = [(synth.workload(i)[0].hidden, synth.workload(i)[0].n_experts) for i in range(1, 6)]
+    shapes += [(4096, 128), (2048, 1024), (8192, 1024), (128, 1)]
+    worst = 0.0
+    for d, E in shapes:
+        for max_tokens in (1, 64, 300, 2047, 8192, 16384, 32768):
+            cap = lib.foe_route_partial_capacity(max_tokens, 64, E)
+            assert cap >= max(max_tokens, 64) * E
+            for n in range(1, min(max_tokens, 2047) + 1):
+                wrote = lib.foe_route_partial_floats(d, E, n, 148, cap)
+                assert n * E <= wrote <= cap, (d, E, max_tokens, n, wrote, cap)
+                worst = max(worst, wrote / cap)
+    assert worst > 0.5          # the sweep does reach cases where the clamp is what keeps the call inside
+    assert lib.foe_route_partial_floats(2048, 64, 0, 148, 1 << 21) == 0
+    # the tensor-core score kernel (2048 tokens and more) writes one slice
+    assert lib.foe_route_partial_floats(2048, 64, 16384, 148, 1 << 21) == 16384 * 64
+
+
 def test_product_path_fails_loudly_without_a_gpu():
     import torch
     from paper_2605_06206_b200 import binding, synth

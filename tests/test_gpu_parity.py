@@ -8,7 +8,7 @@ from oracle import adapter
 from oracle import foe_oracle as orc
 from paper_2605_06206_b200 import binding, synth
 
-from parity import (assert_close, check_maps, check_routing, run_block_parity, scaled_weights)
+from parity import (assert_close, check_every_row, check_maps, check_routing, run_block_parity, scaled_weights)
 
 pytestmark = pytest.mark.gpu
 
@@ -72,6 +72,44 @@ def test_route_bit_exact_tensor_core_scores_odd_k_blocks():
     assert exempt <= n_tok // 200
     assert np.abs(adapter.to_np(aux["logits"]) - rt["logits"]).max() <= 2e-5 * max(1.0, np.abs(rt["logits"]).max())
     check_maps(shape, aux, idx.cpu().numpy())
+
+
+@pytest.mark.parametrize("wl,n_tok,max_tokens", [(5, 1088, 1088), (5, 1100, 16384), (4, 560, 8192), (4, 1152, 4096)])
+def test_route_bit_exact_where_split_k_partials_would_outgrow_their_buffer(wl, n_tok, max_tokens):
+    """Call sizes at which the fp32 score kernel would like 16 slices of the hidden dimension while the partial-score
+    buffer of the handle holds fewer: the number of slices is reduced, the scores still agree with the oracle's."""
+    shape, info = synth.workload(wl)
+    W = dict(ffn_norm_g=synth.normal_bf16(info["seed"], synth.TID["ffn_norm_g"], (shape.hidden,), 0.02, 1.0, "cuda"),
+             router_w=synth.normal_bf16(info["seed"], synth.TID["router_w"], (shape.n_experts, shape.hidden), 0.02, 0.0, "cuda").float())
+    h = synth.normal_bf16(info["seed"], 77, (n_tok, shape.hidden), 1.5, 0.0, "cuda")
+    lib = binding.load_library()
+    cap = lib.foe_route_partial_capacity(max_tokens, 1, shape.n_experts)
+    assert 16 * n_tok * shape.n_experts > cap                                       # the case is the one meant
+    layer = binding.FoeLayer(shape, _route_only_weights(shape, W), max_tokens=max_tokens, max_seqs=1, max_context=64)
+    idx, w = layer.route(h)
+    assert layer.poll_status() == 0
+    aux = layer.aux()
+    layer.close()
+    cfg = adapter.cfg_from_shape(shape)
+    Wn = {k: adapter.to_np(W[k]) for k in ("ffn_norm_g", "router_w")}
+    Wn["router_b"] = None
+    rt = orc.route(cfg, Wn, adapter.to_np(h))
+    exempt = check_routing(shape, idx.cpu().numpy(), w.cpu().numpy().astype(np.float64), rt["logits"], rt["idx"], rt["w"])
+    assert exempt <= max(2, n_tok // 200)
+    assert np.abs(adapter.to_np(aux["logits"]) - rt["logits"]).max() <= 2e-5 * max(1.0, np.abs(rt["logits"]).max())
+    check_maps(shape, aux, idx.cpu().numpy())
+
+
+def _route_only_weights(shape, W):
+    """A full weight set for foe_layer_create in which everything but the router and the FFN-norm gain is a small
+    shared zero buffer of the right size class (routing reads nothing else)."""
+    s = shape
+    dev = "cuda"
+    H, g, c, dh, d, I, E = s.n_clusters, s.n_q_heads // s.n_clusters, s.n_kv_heads // s.n_clusters, s.head_dim, s.hidden, s.ffn_inter, s.n_experts
+    z = lambda *shp: torch.zeros(shp, dtype=torch.bfloat16, device=dev)
+    return dict(attn_norm_g=z(d), wq=z(H, d, g * dh), wk=z(H, d, c * dh), wv=z(H, d, c * dh), wo=z(s.n_q_heads * dh, d),
+                ffn_norm_g=W["ffn_norm_g"], w_gate=z(E, d, I), w_up=z(E, d, I), w_down=z(E, I, d),
+                router_w=W["router_w"], router_b=None)
 
 
 def test_route_is_deterministic():
@@ -386,6 +424,33 @@ def test_host_side_argument_errors():
     kv = synth.make_paged_cache(shape, 27, [63], [1], "cuda")          # position 63 is fine, position 64 = max_context is not
     layer.decode(synth.make_x(shape, 27, 1, "cuda"), kv)
     assert layer.poll_status() == 0
+    kv = synth.make_paged_cache(shape, 27, [64], [1], "cuda")
+    layer.decode(synth.make_x(shape, 27, 1, "cuda"), kv)
+    assert layer.poll_status() == -8
+    kv.context_lens[0] = -5                                            # a negative context length never reaches the block table
+    layer.decode(synth.make_x(shape, 27, 1, "cuda"), kv)
+    assert layer.poll_status() == -8
+    # prefill: context + new tokens one past max_context (the rotary table ends there), reported, nothing faults
+    kv = synth.make_paged_cache(shape, 27, [57], [8], "cuda")          # positions 57..64
+    x8 = synth.make_x(shape, 27, 8, "cuda")
+    layer.prefill(x8, kv)
+    assert layer.poll_status() == -8
+    kv = synth.make_paged_cache(shape, 27, [56], [8], "cuda")          # positions 56..63: fine
+    layer.prefill(x8, kv)
+    assert layer.poll_status() == 0
+    kv.context_lens[0] = -60
+    layer.prefill(x8, kv)
+    assert layer.poll_status() == -8
+    # q_lens that do not add up to the call's token count, or exceed the stated bound
+    kv = synth.make_paged_cache(shape, 27, [0], [8], "cuda")
+    kv.q_lens[0] = 5
+    layer.prefill(x8, kv, n_tokens=8, max_q_len=8)
+    assert layer.poll_status() == -8
+    kv.q_lens[0] = 8
+    layer.prefill(x8, kv, n_tokens=8, max_q_len=4)
+    assert layer.poll_status() == -8
+    layer.prefill(x8, kv, n_tokens=8, max_q_len=8)                     # and the handle is fine afterwards
+    assert layer.poll_status() == 0
     layer.close()
 
 
@@ -400,13 +465,17 @@ def _sample_rows(q_lens, per_seq, seed):
     return np.array(rows, dtype=np.int64)
 
 
-def test_workload2_full_size_prefill_sampled():
+def test_workload2_full_size_prefill_sampled_end_to_end_and_every_row_per_stage():
+    """End to end (every stage chained) on sampled tokens; then the experts stage over all 16,384 tokens and the
+    attention stage over every row of the last sequence, each against the oracle fed the GPU's own stage input."""
     shape, info = synth.workload(2)
     rows = _sample_rows(info["q_lens"], 40, 2)
-    r = run_block_parity(shape, info["seed"], info["q_lens"], info["context_lens"], rows=rows)
+    r = run_block_parity(shape, info["seed"], info["q_lens"], info["context_lens"], rows=rows, return_all=True)
     print("workload 2:", {k: r[k] for k in ("max_abs", "rel_l1", "flips", "launches")})
     c = r["counts"]
     assert c.min() > 1500 and c.max() < 2700                                       # near-uniform load, ~2048 rows/expert
+    e = check_every_row(shape, r["W"], r["out"], r["aux"], r["kv"], info["q_lens"], info["context_lens"], attn_seqs=[3])
+    print("workload 2, every row:", e)
 
 
 def test_workload3_full_size_decode_all_tokens():
@@ -415,7 +484,7 @@ def test_workload3_full_size_decode_all_tokens():
     print("workload 3:", {k: r[k] for k in ("max_abs", "rel_l1", "flips", "launches")})
 
 
-def test_workload4_skewed_routing_sampled():
+def test_workload4_skewed_routing_sampled_end_to_end_and_every_row_per_stage():
     shape, info = synth.workload(4)
     dev = "cuda"
     W = synth.make_weights(shape, info["seed"], dev)
@@ -428,10 +497,14 @@ def test_workload4_skewed_routing_sampled():
     bias = synth.zipf_router_bias(shape, info["seed"], sigma, info["zipf"], dead_per_cluster=2)
     rows = _sample_rows(info["q_lens"], 12, 4)
     r = run_block_parity(shape, info["seed"], info["q_lens"], info["context_lens"], rows=rows, router_bias=bias,
-                         weights=W)
+                         weights=W, return_all=True)
     c = r["counts"].reshape(shape.n_clusters, shape.experts_per_cluster)
     print("workload 4:", {k: r[k] for k in ("max_abs", "rel_l1", "flips")}, "max/mean rows", c.max() / c.mean())
     assert (c == 0).sum() >= 2 * shape.n_clusters and c.max() > 3 * c.mean()       # empty and overfull experts
+    # every row of every expert's tiles (the hottest expert's ~13 k rows and the empty ones included), and every
+    # query block of the first and the last sequence
+    e = check_every_row(shape, r["W"], r["out"], r["aux"], r["kv"], info["q_lens"], info["context_lens"], attn_seqs=[0, 7])
+    print("workload 4, every row:", e, "hottest expert rows", int(c.max()))
 
 
 # ------------------------------------------------------------------------------------------ the paper's own model shape

@@ -212,6 +212,38 @@ def test_topk_matches_library_and_tie_rule():
     np.testing.assert_allclose(w[0, 0], e / e.sum(), atol=1e-12)
 
 
+def test_topk_margin_on_hand_written_scores_and_by_brute_force():
+    """The margin decides which (token, cluster) pairs the bit-exact routing check may skip, so it is pinned by
+    itself: hand-written scores whose adjacent gaps all differ (an off-by-one in the position picks another gap),
+    an unsorted row, a cluster with exactly k_c experts, and a definition that does not sort."""
+    s = small_shape(H=2, nq=4, nkv=2, Ec=4, kc=2)
+    cfg = to_cfg(s)
+    # cluster 0: sorted gaps 2, 0.5, 1.5 -> k_c = 2 gives 3 - 2.5; cluster 1 is given unsorted: sorted 9, 4, 3, -1 -> 4 - 3
+    logits = np.array([[5.0, 3.0, 2.5, 1.0, 3.0, -1.0, 9.0, 4.0]], dtype=np.float32)
+    m = orc.topk_margin(cfg, logits)
+    assert m.shape == (1, 2)
+    assert m[0, 0] == 0.5 and m[0, 1] == 1.0
+    # k_c = 1 and k_c = 3 on the same scores pick the other gaps
+    assert orc.topk_margin(to_cfg(small_shape(H=2, nq=4, nkv=2, Ec=4, kc=1)), logits)[0].tolist() == [2.0, 5.0]
+    assert orc.topk_margin(to_cfg(small_shape(H=2, nq=4, nkv=2, Ec=4, kc=3)), logits)[0].tolist() == [1.5, 4.0]
+    # as many experts as selections: nothing can flip
+    assert np.all(np.isinf(orc.topk_margin(to_cfg(small_shape(H=2, nq=4, nkv=2, Ec=4, kc=4)), logits)))
+    # definition without sorting: the smallest selected score minus the largest score left out, with the selection
+    # taken from topk_per_cluster
+    s3 = small_shape(H=3, nq=6, nkv=3, Ec=7, kc=3)
+    cfg3 = to_cfg(s3)
+    rng = np.random.default_rng(5)
+    lg = rng.standard_normal((300, s3.n_experts)).astype(np.float32)
+    idx, _ = orc.topk_per_cluster(cfg3, lg)
+    m3 = orc.topk_margin(cfg3, lg)
+    for i in range(300):
+        for h in range(3):
+            chosen = set(idx[i, h].tolist())
+            rest = [e for e in range(h * 7, (h + 1) * 7) if e not in chosen]
+            want = float(min(lg[i, e] for e in chosen)) - float(max(lg[i, e] for e in rest))
+            assert m3[i, h] == want and want >= 0.0
+
+
 def test_dispatch_invariants():
     s = small_shape(H=4, Ec=8, kc=2)
     cfg = to_cfg(s)

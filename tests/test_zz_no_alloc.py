@@ -10,7 +10,11 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import adapter
+from oracle import foe_oracle as orc
 from paper_2605_06206_b200 import binding, synth
+
+from parity import check_routing
 
 pytestmark = pytest.mark.gpu
 
@@ -51,6 +55,33 @@ def test_noalloc_route_matches_handle_route_twice_in_a_row():
         wb = torch.gather(w_ref, -1, torch.argsort(idx_ref, -1))
         assert float((wa - wb).abs()[same].max()) <= 1e-5
         np.testing.assert_allclose(w.sum(-1).cpu().numpy(), 1.0, atol=1e-5)
+        # and directly against the oracle's routing of the same rows (ids bit-exact outside near-ties, gates to 1e-5)
+        Wn = {k: adapter.to_np(W[k]) for k in ("ffn_norm_g", "router_w", "router_b")}
+        rt = orc.route(adapter.cfg_from_shape(shape), Wn, adapter.to_np(h))
+        check_routing(shape, idx.cpu().numpy(), w.cpu().numpy().astype(np.float64), rt["logits"], rt["idx"], rt["w"])
+
+
+def test_noalloc_route_refuses_misaligned_views_without_launching():
+    """The kernels read h and the router weights 16 bytes at a time: a view that starts in the middle of such a group
+    is refused on the host (a caller without an allocator of its own tends to carve tensors out of one big buffer)."""
+    shape, _ = synth.workload(1)
+    dev = "cuda"
+    W = synth.make_weights(shape, 1, dev)
+    n = 16
+    big = torch.zeros(n * shape.hidden + 8, dtype=torch.bfloat16, device=dev)
+    h_bad = big[1:1 + n * shape.hidden].view(n, shape.hidden)          # 2 bytes past a 16-byte boundary
+    idx = torch.full((n, shape.n_clusters, shape.top_k_per_cluster), -7, dtype=torch.int32, device=dev)
+    w = torch.zeros((n, shape.n_clusters, shape.top_k_per_cluster), dtype=torch.float32, device=dev)
+    with pytest.raises(binding.FoeError) as e:
+        binding.route_noalloc(shape, W["ffn_norm_g"], W["router_w"], None, h_bad, idx, w)
+    assert e.value.code == -3
+    rw = torch.zeros(W["router_w"].numel() + 4, dtype=torch.float32, device=dev)
+    rw_bad = rw[1:1 + W["router_w"].numel()].view_as(W["router_w"])    # 4 bytes past
+    with pytest.raises(binding.FoeError) as e:
+        binding.route_noalloc(shape, W["ffn_norm_g"], rw_bad, None, big[:n * shape.hidden].view(n, shape.hidden), idx, w)
+    assert e.value.code == -3
+    torch.cuda.synchronize()
+    assert int((idx != -7).sum()) == 0
 
 
 def test_noalloc_route_rejects_oversized_calls_without_launching():
