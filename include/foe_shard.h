@@ -18,6 +18,10 @@
  * arrival counters; no kernel of this library is given another GPU's memory through a tensor map.
  * foe_shard_push / foe_shard_reduce / foe_shard_gather run the same exchange on a tensor that already sits in
  * memory (the mean over clusters that ends the last layer, Section 3.1).
+ * Precision: every partial and the reduced r_full cross the links as bf16, so the r_full a rank's routing and experts
+ * see is the fp32 sum of bf16-rounded partials, rounded to bf16 once more.  The one-device block (foe_prefill /
+ * foe_decode) keeps r_full in fp32 from the O-projection to the combine; the two ways of running a block therefore
+ * agree within the output tolerance but not bit for bit.
  *
  * Exchange buffers.  Every rank allocates one buffer with foe_shard_buffer_alloc and makes it visible to the other
  * ranks: in one process driving several devices the pointers are used directly (with peer access enabled by the

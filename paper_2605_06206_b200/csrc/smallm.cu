@@ -28,7 +28,9 @@ constexpr int kSmXPitch = kSmKStep * 2 + 16;             // padded activation ro
 constexpr int kSmStageBytes = ((kSmWBytes + kSmRows * kSmXPitch + 1023) / 1024) * 1024;
 // ring depth: 5 stages of 21 KB, two CTAs per SM
 template <int EPI> __host__ __device__ constexpr int sm_stages() { return 5; }
-template <int EPI> constexpr size_t sm_smem_bytes() { return size_t(sm_stages<EPI>()) * kSmStageBytes + 1024 + 256 + 4 * kSmRows * 4; }
+constexpr int kSmMaxGroups = 1024;              // ragged problems: experts of a layer
+// stages | barriers + statistics scratch (512 B) | list of the groups that have rows (2 KB) ; + alignment slack
+template <int EPI> constexpr size_t sm_smem_bytes() { return size_t(sm_stages<EPI>()) * kSmStageBytes + 1024 + 512 + kSmMaxGroups * 2; }
 
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -42,11 +44,14 @@ struct SmTask {
 
 // task t of the persistent loop -> (group, slab, rows).  A ragged group takes all its rows (in passes of 16);
 // a uniform group is cut into 16-row chunks so that the few slabs of a small projection still spread out.
-__device__ __forceinline__ SmTask sm_task(const SmallMArgs& a, int t, int slabs_per_group, int chunks) {
+// Ragged problems number their tasks over the groups that HAVE rows only (`live`, built by every CTA when it starts):
+// with a quarter of the experts touched, tasks numbered over all groups leave some CTAs with twice the work of others.
+__device__ __forceinline__ SmTask sm_task(const SmallMArgs& a, int t, int slabs_per_group, int chunks, const uint16_t* live) {
   SmTask k;
   const int sc = slabs_per_group * chunks;
   k.group = t / sc;
   const int r = t - k.group * sc;
+  if (a.group_offsets) k.group = live[k.group];
   k.slab = r / chunks;
   const int chunk = r - k.slab * chunks;
   if (a.group_offsets) {
@@ -81,14 +86,29 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int slabs_per_group = (a.N + kSmSlab - 1) / kSmSlab;    // the last slab of a group may be partly past its rows
   const int chunks = a.group_offsets ? 1 : (a.rows_per_group + kSmRows - 1) / kSmRows;
-  const int n_tasks = a.n_groups * slabs_per_group * chunks;
   const int k_steps = a.K / kSmKStep;
+  uint16_t* live = reinterpret_cast<uint16_t*>(smem + kSmStages * kSmStageBytes + 512);
+  int* n_live_s = reinterpret_cast<int*>(smem + kSmStages * kSmStageBytes + 512 - 16);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSmStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kSmConsumers); }
     mbar_fence_init();
   }
+  if (a.group_offsets && warp == 0) {
+    // the groups with rows, in ascending order (the offsets are complete: they are older than this kernel's
+    // predecessor when it starts before its wait, see early_weights)
+    int n = 0;
+    for (int g0 = 0; g0 < a.n_groups; g0 += 32) {
+      const int g = g0 + lane;
+      const bool has = g < a.n_groups && a.group_offsets[g + 1] > a.group_offsets[g];
+      const uint32_t m = __ballot_sync(0xffffffffu, has);
+      if (has) live[n + __popc(m & ((1u << lane) - 1u))] = uint16_t(g);
+      n += __popc(m);
+    }
+    if (lane == 0) *n_live_s = n;
+  }
   __syncthreads();
+  const int n_tasks = (a.group_offsets ? *n_live_s : a.n_groups) * slabs_per_group * chunks;
 
   // The CTA is persistent: it walks tasks blockIdx.x, blockIdx.x + gridDim.x, ... and the stage ring keeps
   // running across task boundaries, so the producer is already streaming the next slab while the consumers
@@ -105,7 +125,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
       // The previous kernel (expert GEMM 1) writes this kernel's activations, nothing else it needs: the dispatch maps
       // are older and complete.  So the weight tiles of the first ring can be requested while that kernel drains.
       for (int t = blockIdx.x; t < n_tasks; t += gridDim.x) {
-        const SmTask k = sm_task(a, t, slabs_per_group, chunks);
+        const SmTask k = sm_task(a, t, slabs_per_group, chunks, live);
         if (k.rows <= 0) continue;
         if (lane == 0) {
           const int wrow0 = k.group * a.N + k.slab * kSmSlab;
@@ -124,7 +144,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
       pdl_launch_dependents();
     }
     for (int t = blockIdx.x; t < n_tasks && ok; t += gridDim.x) {
-      const SmTask k = sm_task(a, t, slabs_per_group, chunks);
+      const SmTask k = sm_task(a, t, slabs_per_group, chunks, live);
       if (k.rows <= 0) continue;
       // first weight row of the slab inside the [n_groups * N][K] matrix.  SwiGLU slabs are 32 gate rows and
       // their 32 up rows (128 rows further in the packed layout), everything else 64 consecutive rows.
@@ -198,7 +218,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
   };
 
   for (int t = blockIdx.x; t < n_tasks && ok; t += gridDim.x) {
-    const SmTask k = sm_task(a, t, slabs_per_group, chunks);
+    const SmTask k = sm_task(a, t, slabs_per_group, chunks, live);
     if (k.rows <= 0) continue;
     const int group = k.group, rows = k.rows, out_row0 = k.out_row0;
     // global output columns of this thread's two weight rows
