@@ -235,9 +235,9 @@ def test_workload5_shapes_reduced_stack_free_running_against_the_float64_oracle_
     the rounding noise, and in this random-weight network an expert's output is as large as the residual it is added
     to, so with each side choosing for itself the comparison measures those coin flips (measured once: median token
     1.0e-1 relative L1, 90 % below 2.1e-1), not the arithmetic.  How many decisions the oracle would have taken
-    differently on its own state is reported.  Bounds on the per-token relative L1 error of the last layer's output:
-    median 2e-2 (16 layers x the ~2e-3 of a teacher-forced layer, added linearly: the pessimistic case), 99 % of the
-    tokens within 5e-2; nothing non-finite."""
+    differently on its own state is reported (measured: 803 of 131,072).  Bounds on the per-token relative L1 error of
+    the last layer's output: median 1e-2, 99 % of the tokens within 2e-2 (16 layers x the ~2e-3 of a teacher-forced
+    layer would be 3e-2 if the errors added linearly; measured: median 5.3e-3, maximum 6.4e-3); nothing non-finite."""
     import time
     shape, info = synth.workload(5)
     L, seed, q_lens = info["layers"], info["seed"], [512, 512]
@@ -277,7 +277,7 @@ def test_workload5_shapes_reduced_stack_free_running_against_the_float64_oracle_
           "p90 %.3e p99 %.3e max %.3e; whole tensor %.3e; %d of %d (token, cluster, layer) choices differ from the "
           "oracle's own (oracle %.0f s)" % (q[0], q[1], q[2], tok.max(), overall, differing, S * shape.n_clusters * L,
                                             time.time() - t0))
-    assert q[0] < 2e-2 and q[2] < 5e-2
+    assert q[0] < 1e-2 and q[2] < 2e-2
 
 
 def test_package_stack_helper_matches_layer_by_layer_calls():
