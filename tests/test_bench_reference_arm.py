@@ -30,3 +30,22 @@ def test_other_ranks_of_the_reference_arm_exit_without_work():
                         "--warmup", "0"], env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True, timeout=120, cwd=ROOT)
     assert p.returncode == 0, p.stderr[-2000:]
     assert not [l for l in p.stdout.strip().splitlines() if l.startswith("{")]
+
+
+def test_roofline_traffic_is_read_from_the_committed_profiles():
+    """The `traffic` figure of the bench line is parsed out of the ncu summary the line names, not kept in the source:
+    the committed summaries must hold the two kernels' DRAM byte rows, and the figures must be near the algorithmic
+    bytes they are compared with (1.0-1.5 x: a smaller or far larger value means the wrong section was read)."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("bench_mod", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    t, src = bench.profile_traffic("ncu_full_prefill_kernels_workload2.md", "gemm_tcgen05_kernel<1, 1>")
+    assert t is not None and "profiles/ncu_full_prefill_kernels_workload2.md" in src
+    assert 0.872e9 <= t <= 1.5 * 0.872e9               # weights 537 MB + output 268 MB + distinct activations 67 MB
+    t, src = bench.profile_traffic("ncu_full_decode_kernels_workload3.md", "attn_decode_kernel")
+    assert t is not None and 1.34e9 <= t <= 1.1 * 1.344e9
+    t, src = bench.profile_traffic("ncu_full_decode_kernels_workload3.md", "no_such_kernel")
+    assert t is None and "not found" in src
+    t, src = bench.profile_traffic("no_such_file.md", "x")
+    assert t is None and "missing" in src
