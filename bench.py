@@ -192,6 +192,36 @@ def sustained_profile(layer, fn, ms_per_step, seconds=1.2, ring=64):
     return e0.elapsed_time(e1) / n, stages, n
 
 
+def library_gemm_same_shape(R, K, N, seconds=0.6):
+    """Context for the tensor roofline, not part of the path: the vendor library's bf16 GEMM (torch.matmul) on ONE dense
+    problem with the row count, reduction length and output width of an expert GEMM launch ([R, K] x [K, N]), run
+    back to back for `seconds` so that it meets the same power cap.  The measured peak in MEASURED_PEAKS.json is an
+    8192^3 problem, whose reduction is four to eight times longer per output element than an expert GEMM's."""
+    a = torch.randn(R, K, device="cuda", dtype=torch.bfloat16)
+    b = torch.randn(K, N, device="cuda", dtype=torch.bfloat16)
+    c = torch.empty(R, N, device="cuda", dtype=torch.bfloat16)
+    for _ in range(3):
+        torch.matmul(a, b, out=c)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    torch.matmul(a, b, out=c)
+    e1.record()
+    torch.cuda.synchronize()
+    n = max(4, int(seconds * 1e3 / max(e0.elapsed_time(e1), 1e-3)))
+    for _ in range(n // 2):                       # settle to the sustained clock, then time the second half
+        torch.matmul(a, b, out=c)
+    e0.record()
+    for _ in range(n - n // 2):
+        torch.matmul(a, b, out=c)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / (n - n // 2)
+    del a, b, c
+    return dict(tflops=2.0 * R * K * N / (ms * 1e-3) / 1e12, ms=ms, shape=[R, K, N], seconds=seconds,
+                note="torch.matmul (vendor library) on one dense problem of the launch's size, sustained; context only")
+
+
 def expert_row_histogram(counts):
     """Rows per expert of the last call: how ragged the grouped GEMMs' tiles were."""
     c = counts.double()
@@ -407,6 +437,11 @@ def measure(kind, args, dist_on, rank, world, peaks, with_cpu):
                               note="the same step back to back for about a second; stages_ms are the mean of the 64 steps that follow it without a pause"),
                clocks=clocks, tokens_per_step=S, expert_rows=expert_row_histogram(wl["layer"].aux()["counts"].cpu()))
     res["roofline"] = roofline_of(kind, work, stages, sus_ms, peaks, wl["n"])
+    if kind == "prefill" and rank == 0:
+        sh = wl["shape"]
+        res["roofline"]["library_gemm_same_shape"] = dict(
+            gemm1=library_gemm_same_shape(work["rows"], sh.hidden, 2 * sh.ffn_inter),
+            gemm2=library_gemm_same_shape(work["rows"], sh.ffn_inter, sh.hidden))
     res["work"] = {k: v for k, v in work.items()}
     e_ms, h2d, d2h = e2e_loop(wl, max(4, min(args.steps, 10)), 3)
     res["e2e"] = dict(value=world * S / (e_ms * 1e-3), unit="tokens/s", ms_per_step=e_ms, h2d_bytes_per_step=h2d,
@@ -494,12 +529,16 @@ def stack_decode_bytes(st, shape, xs, ctx0):
     return sum(per_layer), touched
 
 
-def measure_stack(args, peaks, clock_index):
+def measure_stack(args, peaks, clock_index, one_cluster=False):
     """Workload 5 as FoE: 16 layers (hidden 4096, 32q/8kv heads, 8 clusters x 16 experts top-2, inter 1408; 72 GB of
     weights), prefill of 2 x 16,384 tokens, then 128 decode steps on the caches it wrote.  A decode step is one
-    foe_stack_forward + foe_context_advance; it is timed issued directly and replayed from a CUDA graph."""
+    foe_stack_forward + foe_context_advance; it is timed issued directly and replayed from a CUDA graph.
+    one_cluster: the equal-size MoE baseline on the same kernels (1 cluster x 128 experts, top-16)."""
+    import dataclasses
     from paper_2605_06206_b200.stack import FoeStack
     shape, info = synth.workload(5)
+    if one_cluster:
+        shape = dataclasses.replace(shape, n_clusters=1, experts_per_cluster=128, top_k_per_cluster=16)
     q_lens, L, steps = info["q_lens"], info["layers"], info.get("decode_steps", 128)
     st = FoeStack(shape, L, info["seed"], q_lens, steps + 8)
     S, B = sum(q_lens), len(q_lens)
@@ -569,8 +608,9 @@ def measure_stack(args, peaks, clock_index):
     best = min(direct_ms, graph_ms)
     gbs = step_bytes / (best * 1e-3) / 1e9
     pf = L * flops_layer / (prefill_ms * 1e-3) / 1e12
-    return dict(workload="workload 5: 16-layer FoE stack, hidden 4096, 32q/8kv heads, 8 clusters x 16 experts top-2, inter 1408; "
-                         "prefill 2 x 16384 tokens, then 128 decode steps of 2 tokens",
+    return dict(workload="workload 5: 16-layer stack, hidden 4096, 32q/8kv heads, "
+                         + ("1 cluster x 128 experts top-16 (the equal-size MoE baseline)" if one_cluster else "8 clusters x 16 experts top-2")
+                         + ", inter 1408; prefill 2 x 16384 tokens, then 128 decode steps of 2 tokens",
                 prefill_ms=prefill_ms, prefill_tokens_per_s=S / (prefill_ms * 1e-3), prefill_tflops=pf,
                 prefill_frac_of_sustained=pf / peaks["bf16_tflops_sustained"], prefill_frac_of_burst=pf / peaks["bf16_tflops"],
                 decode_ms_per_step=best, decode_ms_per_step_direct=direct_ms, decode_ms_per_step_graph=graph_ms,
@@ -651,52 +691,13 @@ def run_serve(args):
 
 
 def run_stack(args):
-    """The 16-layer stack (first, 14 middle, last layer; hidden 4096, 32q/8kv heads, 8 clusters x 16 experts top-2,
-    inter 1408; 72 GB of weights): prefill of 2 x 16,384 tokens, then 128 decode steps on the caches it wrote, once as
-    FoE and once as the equal-size one-cluster MoE (128 experts, top-16) on the same kernels."""
-    import dataclasses
-    from paper_2605_06206_b200.stack import FoeStack
-    shape, info = synth.workload(5)
-    q_lens, L, steps = info["q_lens"], info["layers"], info.get("decode_steps", 128)
-    rows = []
-    for H in (shape.n_clusters, 1):
-        sh = shape if H != 1 else dataclasses.replace(shape, n_clusters=1, experts_per_cluster=128, top_k_per_cluster=16)
-        st = FoeStack(sh, L, info["seed"], q_lens, steps)
-        S = sum(q_lens)
-        x0 = synth.make_x(st.shapes[0], info["seed"], S, "cuda")
-        st.forward(x0, [0] * len(q_lens), decode=False)                      # warm-up (also writes the caches)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = 3
-        e0.record()
-        for _ in range(reps):
-            st.forward(x0, [0] * len(q_lens), decode=False)
-        e1.record()
-        torch.cuda.synchronize()
-        prefill_ms = e0.elapsed_time(e1) / reps
-        xs = [synth.make_x(st.shapes[0], info["seed"], len(q_lens), "cuda", tid=synth.TID["x_step"] + s) for s in range(steps)]
-        ctx = list(q_lens)
-        for s in range(3):                                                   # warm-up steps (not counted)
-            st.forward(xs[s], ctx, decode=True)
-        torch.cuda.synchronize()
-        e0.record()
-        for s in range(steps):
-            st.forward(xs[s], ctx, decode=True)
-            ctx = [c + 1 for c in ctx]
-        e1.record()
-        torch.cuda.synchronize()
-        decode_ms = e0.elapsed_time(e1) / steps
-        assert st.status() == 0
-        rows.append(dict(n_clusters=H, prefill_ms=prefill_ms, prefill_tokens_per_s=S / (prefill_ms * 1e-3),
-                         decode_ms_per_step=decode_ms, decode_tokens_per_s=len(q_lens) / (decode_ms * 1e-3)))
-        st.close()
-        del st, x0, xs
-        torch.cuda.empty_cache()
+    """The 16-layer stack (workload 5) once as FoE and once as the equal-size one-cluster MoE (128 experts, top-16) on
+    the same kernels: prefill of 2 x 16,384 tokens, then 128 decode steps on the caches it wrote."""
+    peaks = measured_peaks()
+    dev = torch.cuda.current_device()
+    rows = [measure_stack(args, peaks, dev, one_cluster=False), measure_stack(args, peaks, dev, one_cluster=True)]
     print(json.dumps(dict(metric="foe_stack_tokens_per_s", unit="tokens/s", data="synthetic", dtype="bf16",
-                          config=dict(workload="workload 5: 16-layer stack, hidden 4096, 32q/8kv heads, 8 clusters x 16 experts "
-                                               "top-2 (and 1 cluster x 128 experts top-16), inter 1408; prefill 2 x 16384 tokens, "
-                                               "then 128 decode steps (host tensor set-up of every step included)"),
-                          stacks=rows)))
+                          config=dict(workload="workload 5, FoE and its one-cluster MoE twin"), stacks=rows)))
 
 
 def run_shard(args):
