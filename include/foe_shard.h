@@ -58,8 +58,9 @@ typedef struct {
 
 typedef struct foe_shard foe_shard;
 
-/* Bytes of one rank's exchange buffer: 1 KB of counters, receive slots [2][H][max_tokens][d/H] bf16 and the gather
- * buffer [2][max_tokens][d] bf16.  0 if the description is invalid. */
+/* Bytes of one rank's exchange buffer: a header of arrival counters (per owner for the gather buffer; per exchange
+ * parity, source rank and block of 256 rows for the receive slots), receive slots [2][H][max_tokens][d/H] bf16 and the
+ * gather buffer [2][max_tokens][d] bf16.  0 if the description is invalid. */
 size_t foe_shard_buffer_bytes(const foe_shard_config* config);
 
 /* Allocates (cudaMalloc on the current device) and zeroes one exchange buffer; synchronises.  The buffer belongs to the

@@ -306,11 +306,32 @@ decode_proj_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
           sum.x += bf16_lo(xr[r].x); sum.y += bf16_hi(xr[r].x); sum.z += bf16_lo(xr[r].y); sum.w += bf16_hi(xr[r].y);
         }
         const float sc = a.out_scale;
-        *reinterpret_cast<float4*>(static_cast<float*>(a.out) + off) = make_float4(sum.x * sc, sum.y * sc, sum.z * sc, sum.w * sc);
+        if (a.push_span) {
+          // one rank of a cluster-per-GPU group: the slab's 128 columns lie inside one owner's span; bf16 to its slot
+          const int col = n0 + c4 * 4, owner = col / a.push_span;
+          bf16* dst = a.push_base[owner] + a.push_slot_off + size_t(tok0 + t) * a.push_span + (col - owner * a.push_span);
+          *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(sum.x * sc, sum.y * sc), pack_bf16(sum.z * sc, sum.w * sc));
+        } else {
+          *reinterpret_cast<float4*>(static_cast<float*>(a.out) + off) = make_float4(sum.x * sc, sum.y * sc, sum.z * sc, sum.w * sc);
+        }
       }
+      if (a.push_span) __threadfence_system();               // every storing thread: its stores before the count below
     }
   }
   cluster_sync_all();                                       // nobody leaves while a peer may still read its tile
+  if constexpr (EPI == kEpiOProj) {
+    if (a.push_span && threadIdx.x == 64) {
+      // this CTA finished the tokens [t_lo, t_lo + share) of the tile: their element count goes to the owner's counter
+      // of the tile's row block (a tile's 64 tokens lie inside one block of 256)
+      const int share = kDpTok / ks, tok0 = chunk * kDpTok;
+      const int n_tok = min(kDpTok, a.rows_per_group - tok0);
+      const int mine = max(0, min(share, n_tok - z * share));
+      if (mine > 0) {
+        const int owner = slab * kDpSlab / a.push_span;
+        atomicAdd_system(a.push_cnt[owner] + tok0 / kShardBlockRows, unsigned(mine) * unsigned(kDpSlab));
+      }
+    }
+  }
 
   tc_fence_before();
   __syncthreads();

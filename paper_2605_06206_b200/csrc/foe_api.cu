@@ -104,7 +104,8 @@ struct foe_shard {
   uint8_t* buf[8];                  // every rank's exchange buffer as seen from here
   ShardPeerTable table;
   unsigned int epoch;               // exchanges started
-  unsigned int slot_expect, gather_expect;   // running totals the counters must reach for the current exchange
+  unsigned int gather_expect;       // running total the gather counters must reach for the current exchange
+  int n_blk;                        // row blocks (of kShardBlockRows rows) that have slot counters
   int S;                            // tokens of the current exchange
   int stage;                        // 0 idle, 1 pushed, 2 reduced
   int* status;
@@ -116,7 +117,11 @@ namespace {
 
 constexpr int kFewTokens = 256;                  // calls up to this size take the decode-step kernels where they fit
 constexpr int kOverlapTokens = 2048;             // calls up to this size launch their kernels with programmatic dependent launch
-constexpr size_t kShardHeaderBytes = 1024;       // slot counters at 0, gather counters at 128
+// header of an exchange buffer: gather counters [8] at 0; slot counters [2 parities][8 sources][n_blk] from 128 on
+int shard_blocks(const foe_shard_config* c) { return (c->max_tokens + kShardBlockRows - 1) / kShardBlockRows; }
+size_t shard_header_bytes(const foe_shard_config* c) {
+  return (128 + size_t(2) * 8 * shard_blocks(c) * sizeof(unsigned int) + 1023) / 1024 * 1024;
+}
 
 bool shard_config_ok(const foe_shard_config* c) {
   return c && c->n_ranks >= 1 && c->n_ranks <= 8 && c->rank >= 0 && c->rank < c->n_ranks && c->hidden > 0 &&
@@ -313,6 +318,7 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
     x_count = (L->first && sh->cfg.rank != 0) ? 0 : 1;
   }
   const long long slot_off = sh ? (long long)((size_t(sh->epoch & 1) * sh->cfg.n_ranks + sh->cfg.rank) * sh->S_cap * sh->span) : 0;
+  const int cnt_off = sh ? int(sh->epoch & 1) * 8 * sh->n_blk : 0;          // this exchange's half of the slot counters
   if (oproj_gemm) {
     GemmArgs ga;
     memset(&ga, 0, sizeof(ga));
@@ -321,7 +327,7 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
     ga.out_scale = out_scale;
     if (x_summed) { ga.x_count = 0; ga.x_in_out = 1; }
     if (sh) {     // the epilogue stores each tile straight into the owners' slots
-      for (int o = 0; o < sh->cfg.n_ranks; ++o) { ga.push_base[o] = sh->table.slots[o]; ga.push_cnt[o] = sh->table.slot_cnt[o]; }
+      for (int o = 0; o < sh->cfg.n_ranks; ++o) { ga.push_base[o] = sh->table.slots[o]; ga.push_cnt[o] = sh->table.slot_cnt[o] + cnt_off; }
       ga.push_span = sh->span;
       ga.push_slot_off = slot_off;
     }
@@ -332,9 +338,15 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
     pa.n_groups = 1; pa.rows_per_group = S; pa.x_group_stride = 0; pa.N = d; pa.K = L->n_q * dh; pa.epi = kEpiOProj;
     pa.status = L->ws->status;
     pa.out = L->ws->r_full; pa.ldo = d; pa.xsum = xb; pa.x_count = x_count; pa.x_stride = size_t(S) * d; pa.out_scale = out_scale;
+    const bool fused_push = sh && sh->span % 128 == 0;      // a 128-row weight slab then lies inside one owner's columns
+    if (fused_push) {
+      for (int o = 0; o < sh->cfg.n_ranks; ++o) { pa.push_base[o] = sh->table.slots[o]; pa.push_cnt[o] = sh->table.slot_cnt[o] + cnt_off; }
+      pa.push_span = sh->span;
+      pa.push_slot_off = slot_off;
+    }
     launch_decode_proj(L->tmt_wo, L->ws->tm_attn_o64, pa, L->n_sms, st);
-    if (sh) {
-      launch_shard_push(L->ws->r_full, 1, 1.0f, S, d, sh->cfg.n_ranks, sh->table, slot_off, st);
+    if (sh && !fused_push) {
+      launch_shard_push(L->ws->r_full, 1, 1.0f, S, d, sh->cfg.n_ranks, sh->table, slot_off, cnt_off, st);
       L->launches += 1;
     }
   } else {
@@ -345,7 +357,7 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
     sa.x_stride = size_t(S) * d; sa.out_scale = out_scale; sa.status = L->ws->status;
     launch_smallm(L->tms_wo, sa, L->n_sms, st);
     if (sh) {     // a decode step's partial is a few hundred KB: one more launch pushes it
-      launch_shard_push(L->ws->r_full, 1, 1.0f, S, d, sh->cfg.n_ranks, sh->table, slot_off, st);
+      launch_shard_push(L->ws->r_full, 1, 1.0f, S, d, sh->cfg.n_ranks, sh->table, slot_off, cnt_off, st);
       L->launches += 1;
     }
   }
@@ -833,7 +845,7 @@ foe_status foe_get_stage_ms(foe_layer* L, float* ms, int n) {
 
 size_t foe_shard_buffer_bytes(const foe_shard_config* c) {
   if (!shard_config_ok(c)) return 0;
-  return kShardHeaderBytes + 2 * shard_slots_bytes(c);       // slots and gather buffer have the same size
+  return shard_header_bytes(c) + 2 * shard_slots_bytes(c);       // slots and gather buffer have the same size
 }
 
 foe_status foe_shard_buffer_alloc(const foe_shard_config* c, void** buffer) {
@@ -892,15 +904,16 @@ foe_status foe_shard_create(const foe_shard_config* c, void* const* buffers, foe
   if (!sh) return FOE_ERR_OOM;
   sh->cfg = *c;
   sh->span = c->hidden / c->n_ranks;
+  sh->n_blk = shard_blocks(c);
   sh->S_cap = size_t(c->max_tokens);
   sh->limit_ns = (unsigned long long)(c->wait_limit_ms > 0 ? c->wait_limit_ms : 2000) * 1000000ull;
   for (int r = 0; r < c->n_ranks; ++r) {
     uint8_t* b = static_cast<uint8_t*>(buffers[r]);
     sh->buf[r] = b;
-    sh->table.slots[r] = reinterpret_cast<bf16*>(b + kShardHeaderBytes);
-    sh->table.gather[r] = reinterpret_cast<bf16*>(b + kShardHeaderBytes + shard_slots_bytes(c));
-    sh->table.slot_cnt[r] = reinterpret_cast<unsigned int*>(b) + c->rank;        // rank r's counter of MY pushes
-    sh->table.gather_cnt[r] = reinterpret_cast<unsigned int*>(b + 128);          // rank r's counters, one per owner
+    sh->table.slots[r] = reinterpret_cast<bf16*>(b + shard_header_bytes(c));
+    sh->table.gather[r] = reinterpret_cast<bf16*>(b + shard_header_bytes(c) + shard_slots_bytes(c));
+    sh->table.slot_cnt[r] = reinterpret_cast<unsigned int*>(b + 128) + size_t(c->rank) * sh->n_blk;   // rank r's counters of MY pushes
+    sh->table.gather_cnt[r] = reinterpret_cast<unsigned int*>(b);                // rank r's counters, one per owner
   }
   if (cudaMalloc(reinterpret_cast<void**>(&sh->status), sizeof(int)) != cudaSuccess) { cudaGetLastError(); delete sh; return FOE_ERR_OOM; }
   cudaMemset(sh->status, 0, sizeof(int));
@@ -921,7 +934,6 @@ static foe_status shard_begin(foe_shard* sh, int S, cudaStream_t st) {
   if (S < 0 || S > sh->cfg.max_tokens) return FOE_ERR_SHAPE;
   sh->epoch += 1;
   sh->S = S;
-  sh->slot_expect += unsigned(S) * unsigned(sh->span);
   sh->gather_expect += unsigned(S) * unsigned(sh->span);
   sh->stage = 1;
   sh->last_stream = st;
@@ -954,7 +966,8 @@ foe_status foe_shard_push(foe_shard* sh, const void* src, int n_tokens, float sc
   if (b != FOE_OK) return b;
   if (n_tokens == 0) return FOE_OK;
   const long long slot_off = (long long)((size_t(sh->epoch & 1) * sh->cfg.n_ranks + sh->cfg.rank) * sh->S_cap * sh->span);
-  launch_shard_push(src, 0, scale, n_tokens, sh->cfg.hidden, sh->cfg.n_ranks, sh->table, slot_off, st);
+  launch_shard_push(src, 0, scale, n_tokens, sh->cfg.hidden, sh->cfg.n_ranks, sh->table, slot_off,
+                    int(sh->epoch & 1) * 8 * sh->n_blk, st);
   return check_launch();
 }
 
@@ -968,8 +981,8 @@ foe_status foe_shard_reduce(foe_shard* sh, void* stream) {
   const int H = sh->cfg.n_ranks, me = sh->cfg.rank;
   const size_t half = size_t(sh->epoch & 1);
   const bf16* my_slots = sh->table.slots[me] + half * H * sh->S_cap * sh->span;
-  const unsigned int* my_cnt = reinterpret_cast<const unsigned int*>(sh->buf[me]);
-  launch_shard_reduce(my_slots, my_cnt, sh->slot_expect, sh->S, sh->S_cap, sh->cfg.hidden, H, me, sh->table,
+  const unsigned int* my_cnt = reinterpret_cast<const unsigned int*>(sh->buf[me] + 128) + half * 8 * sh->n_blk;
+  launch_shard_reduce(my_slots, my_cnt, sh->n_blk, sh->S, sh->S_cap, sh->cfg.hidden, H, me, sh->table,
                       (long long)(half * sh->S_cap * sh->cfg.hidden), sh->limit_ns, sh->status, st);
   return check_launch();
 }
@@ -981,8 +994,9 @@ static foe_status shard_finish(foe_shard* sh, float* dst_f32, bf16* dst_bf16, cu
   if (sh->S == 0) return FOE_OK;
   const int me = sh->cfg.rank;
   const bf16* my_gather = sh->table.gather[me] + size_t(sh->epoch & 1) * sh->S_cap * sh->cfg.hidden;
+  unsigned int* my_cnt = reinterpret_cast<unsigned int*>(sh->buf[me] + 128) + size_t(sh->epoch & 1) * 8 * sh->n_blk;
   launch_shard_gather(my_gather, sh->table.gather_cnt[me], sh->gather_expect, sh->S, sh->cfg.hidden, sh->cfg.n_ranks,
-                      dst_f32, dst_bf16, sh->limit_ns, sh->status, st);
+                      dst_f32, dst_bf16, my_cnt, 8 * sh->n_blk, sh->limit_ns, sh->status, st);
   return check_launch();
 }
 

@@ -28,6 +28,9 @@ enum GemmEpilogue : int {
 // needs the full 256-wide tile (128 gate columns, 128 up columns).
 constexpr int gemm_tile_rows_b(int epi, int N) { return (epi == kEpiSwiGLU ? kBN : gemm_tile_cols(N)) / 2; }
 
+// rows per arrival counter of a cluster-per-GPU exchange (= the row tile of the O-projection GEMM that pushes)
+constexpr int kShardBlockRows = 256;
+
 struct GemmArgs {
   // uniform groups
   int n_groups;
@@ -71,8 +74,9 @@ struct GemmArgs {
   int x_in_out;              // `out` already holds the fp32 sum of the residual streams: out = scale * (C + out)
   // kEpiOProj on one rank of a cluster-per-GPU group (push_span != 0): the scaled tile is not written to `out` but
   // pushed as bf16 to the rank that owns its columns -- columns [o * push_span, (o + 1) * push_span) belong to rank
-  // o -- at push_base[o] + push_slot_off + row * push_span + (column - o * push_span); push_cnt[o] then grows by
-  // the number of elements written (after a system-scope fence), which is what the owner's reduction waits for.
+  // o -- at push_base[o] + push_slot_off + row * push_span + (column - o * push_span); push_cnt[o][row / 256] then grows
+  // by the number of elements written (after a system-scope fence), which is what the owner's reduction of those rows
+  // waits for.
   // The pointers are this rank's mappings of the owners' buffers (peer memory, or plain local memory).
   __nv_bfloat16* push_base[8];
   unsigned int* push_cnt[8];

@@ -86,7 +86,7 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmArgs& args, uint32_
     if (push_n) {
       __threadfence_system();                                       // every lane: its stores before the count
       __syncwarp();
-      if (lane == 0) atomicAdd_system(args.push_cnt[push_owner], push_n);
+      if (lane == 0) atomicAdd_system(args.push_cnt[push_owner] + row0 / kShardBlockRows, push_n);   // the tile's row block
       push_n = 0;
     }
   };

@@ -190,6 +190,9 @@ struct DecodeProjArgs {
   const int* context_lens; const int* block_table; int max_pages_per_seq, num_pages, max_context;
   // kEpiOProj
   const bf16* xsum; int x_count; size_t x_stride; float out_scale;
+  // kEpiOProj on one rank of a cluster-per-GPU group (push_span != 0, a multiple of the 128-row weight slab): the scaled
+  // result goes as bf16 to the rank that owns its columns instead of `out` (see GemmArgs)
+  bf16* push_base[8]; unsigned int* push_cnt[8]; int push_span; long long push_slot_off;
 };
 bool decode_proj_supported(int epi, int N, int K, int dh);
 // tmW: the weights [n_groups * N][K] with 64-column boxes of 128 rows; tmX: the activations with 64 x 64 boxes
@@ -197,27 +200,32 @@ void launch_decode_proj(const CUtensorMap& tmW, const CUtensorMap& tmX, DecodePr
 
 // ---- shard.cu  (sync of a cluster-per-GPU group over peer memory)
 // This rank's mappings of every rank's exchange buffer: receive slots ([2][H][S_cap][d/H] bf16), gather buffer
-// ([2][S_cap][d] bf16), arrival counters of the slots ([H], one per source) and of the gather buffer ([H], one per owner).
+// ([2][S_cap][d] bf16), arrival counters of the slots (per exchange parity, source rank and block of kShardBlockRows
+// rows, so that an owner can reduce a block of rows as soon as ITS partials have landed) and of the gather buffer ([H],
+// one per owner, only ever growing).
 struct ShardPeerTable {
   bf16* slots[8];
   bf16* gather[8];
-  unsigned int* slot_cnt[8];      // slot_cnt[o]: the counter on rank o that counts THIS rank's pushes
+  unsigned int* slot_cnt[8];      // slot_cnt[o]: on rank o, the counters [n_blocks] of THIS rank's pushes (parity 0; the
+                                  // other parity's lie 8 * n_blocks further)
   unsigned int* gather_cnt[8];    // gather_cnt[p]: rank p's array of H counters (indexed by owner)
 };
 // src ([S][d] bf16 or fp32) * scale -> bf16 into this rank's slot on every owner; slot_off = element offset of that
-// slot ((parity * H + rank) * S_cap * (d/H)).  Adds S * d/H to every slot_cnt[o].
+// slot ((parity * H + rank) * S_cap * (d/H)); cnt_off = parity * 8 * n_blocks.  Adds rows * d/H to the counter of every
+// block of rows on every owner.
 void launch_shard_push(const void* src, int src_is_f32, float scale, int S, int d, int H, const ShardPeerTable& t,
-                       long long slot_off, cudaStream_t st);
-// waits until my_slot_cnt[0..H) reached `expect`, sums the H slots (my_slots = this parity's [H][S_cap][d/H]) and
-// writes the bf16 result to gather[p] + gather_off + row * d + rank * d/H of every rank p; adds S * d/H to
-// gather_cnt[p][rank].
-void launch_shard_reduce(const bf16* my_slots, const unsigned int* my_slot_cnt, unsigned int expect, int S, size_t S_cap,
+                       long long slot_off, int cnt_off, cudaStream_t st);
+// every block of 16 rows waits until the H counters of its row block (my_slot_cnt[h * n_blocks + block], this parity's)
+// hold that block's rows * d/H, sums the H slots (my_slots = this parity's [H][S_cap][d/H]) and writes the bf16 result
+// to gather[p] + gather_off + row * d + rank * d/H of every rank p; adds rows * d/H to gather_cnt[p][rank].
+void launch_shard_reduce(const bf16* my_slots, const unsigned int* my_slot_cnt, int n_blocks, int S, size_t S_cap,
                          int d, int H, int rank, const ShardPeerTable& t, long long gather_off,
                          unsigned long long limit_ns, int* status, cudaStream_t st);
 // waits until my_gather_cnt[0..H) reached `expect` and copies the [S][d] gathered tensor (my_gather = this parity's
-// half) to dst_f32 and / or dst_bf16 (either may be null)
+// half) to dst_f32 and / or dst_bf16 (either may be null); zeroes this rank's own slot counters of the exchange
+// (zero_cnt[0 .. zero_n)), which nobody reads any more and which the exchange after the next will count up again
 void launch_shard_gather(const bf16* my_gather, const unsigned int* my_gather_cnt, unsigned int expect, int S, int d,
-                         int H, float* dst_f32, bf16* dst_bf16, unsigned long long limit_ns, int* status,
-                         cudaStream_t st);
+                         int H, float* dst_f32, bf16* dst_bf16, unsigned int* zero_cnt, int zero_n,
+                         unsigned long long limit_ns, int* status, cudaStream_t st);
 
 }  // namespace foe

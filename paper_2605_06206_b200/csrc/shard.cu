@@ -3,15 +3,19 @@
 //
 // Each rank h holds one cluster.  r_full = sum_h partial[h] is formed as a two-step exchange over peer memory,
 // with the columns of the [S][d] tensor split evenly between the ranks (rank o owns columns [o*span, (o+1)*span)):
-//   push    every rank writes its partial of owner o's columns into slot h of o's receive buffer (the prefill
-//           O-projection does this from its epilogue, tile by tile; shard_push_kernel does it for a tensor that
-//           already sits in memory), then adds the element count to o's arrival counter for source h;
-//   reduce  owner o waits until all H counters reached the expected total, adds the H slots in rank order in
-//           fp32, rounds to bf16 and writes the result into the gather buffer of every rank, then adds to their
-//           counters for owner o;
-//   gather  every rank waits for the H owners' counters and reads its own gather buffer.
-// Counters only ever grow (the expected totals are kept by the host), buffers alternate between two halves by the
-// parity of the exchange number, and all waits are bounded by a wall-clock limit after which the kernel records
+//   push    every rank writes its partial of owner o's columns into slot h of o's receive buffer (the O-projections
+//           do this from their epilogues, tile by tile; shard_push_kernel does it for a tensor that already sits in
+//           memory), then adds the element count to o's arrival counter for (source h, block of 256 rows);
+//   reduce  owner o: every block of 16 rows waits until the H counters of ITS 256-row block hold the block's element
+//           count -- so the reduction of the first rows runs while later tiles are still being pushed --, adds the H
+//           slots in rank order in fp32, rounds to bf16 and writes the result into the gather buffer of every rank,
+//           then adds to their counters for owner o;
+//   gather  every rank waits for the H owners' counters and reads its own gather buffer; it also zeroes its own slot
+//           counters of this exchange (its reduction is over, and a peer's next push with the same parity comes two
+//           exchanges later, after that peer has gathered the exchange in between, which this rank's reduction of
+//           that exchange -- queued behind this kernel -- feeds).
+// The gather counters only ever grow (the expected totals are kept by the host), buffers and slot counters alternate
+// between two halves by the parity of the exchange number, and all waits are bounded by a wall-clock limit after which the kernel records
 // kStatusTimeout and returns.  A rank never waits for something that needs one of its own later kernels, so the
 // three kernels of one rank can be queued back to back on a stream; ranks emulated on ONE device must run all
 // pushes before the first reduce and all reduces before the first gather, so that no wait ever spins.
@@ -23,7 +27,7 @@ namespace foe {
 namespace {
 
 constexpr int kShardThreads = 256;
-constexpr int kShardRows = 16;       // rows of one block's share
+constexpr int kShardRows = 16;       // rows of one block's share (divides kShardBlockRows)
 
 __device__ __forceinline__ unsigned int ld_acquire_sys(const unsigned int* p) {
   unsigned int v;
@@ -52,7 +56,7 @@ __device__ __forceinline__ bool wait_count(const unsigned int* cnt, unsigned int
 // bf16 into slot `rank` of o's receive buffer
 __global__ void __launch_bounds__(kShardThreads)
 shard_push_kernel(const void* __restrict__ src, int src_is_f32, float scale, int S, int d, int span, ShardPeerTable t,
-                  long long slot_off) {
+                  long long slot_off, int cnt_off) {
   const int o = blockIdx.y;
   const int r0 = blockIdx.x * kShardRows;
   const int rows = min(kShardRows, S - r0);
@@ -78,20 +82,25 @@ shard_push_kernel(const void* __restrict__ src, int src_is_f32, float scale, int
   }
   __threadfence_system();
   __syncthreads();
-  if (threadIdx.x == 0) atomicAdd_system(t.slot_cnt[o], unsigned(rows) * unsigned(span));
+  if (threadIdx.x == 0) atomicAdd_system(t.slot_cnt[o] + cnt_off + r0 / kShardBlockRows, unsigned(rows) * unsigned(span));
 }
 
 // owner side: block rb reduces rows [rb*16, +16) of this rank's columns over the H slots and hands the result to
 // every rank's gather buffer
 __global__ void __launch_bounds__(kShardThreads)
-shard_reduce_kernel(const bf16* __restrict__ my_slots, const unsigned int* my_slot_cnt, unsigned int expect, int S,
+shard_reduce_kernel(const bf16* __restrict__ my_slots, const unsigned int* my_slot_cnt, int n_blocks, int S,
                     size_t S_cap, int d, int span, int H, int rank, ShardPeerTable t, long long gather_off,
                     unsigned long long limit_ns, int* status) {
   __shared__ int s_ok;
   if (threadIdx.x == 0) s_ok = 1;
   __syncthreads();
-  if (threadIdx.x < H) {
-    if (!wait_count(my_slot_cnt + threadIdx.x, expect, limit_ns)) s_ok = 0;
+  {
+    // only the partials of this block's rows have to be there
+    const int blk = blockIdx.x * kShardRows / kShardBlockRows;
+    const unsigned int expect = unsigned(min(kShardBlockRows, S - blk * kShardBlockRows)) * unsigned(span);
+    if (threadIdx.x < H) {
+      if (!wait_count(my_slot_cnt + threadIdx.x * n_blocks + blk, expect, limit_ns)) s_ok = 0;
+    }
   }
   __syncthreads();
   if (!s_ok) {
@@ -124,9 +133,12 @@ shard_reduce_kernel(const bf16* __restrict__ my_slots, const unsigned int* my_sl
 // gather buffer (to fp32 and / or bf16)
 __global__ void __launch_bounds__(kShardThreads)
 shard_gather_kernel(const bf16* __restrict__ my_gather, const unsigned int* my_gather_cnt, unsigned int expect, int S,
-                    int d, int span, float* dst_f32, bf16* dst_bf16, unsigned long long limit_ns, int* status) {
+                    int d, int span, float* dst_f32, bf16* dst_bf16, unsigned int* zero_cnt, int zero_n,
+                    unsigned long long limit_ns, int* status) {
   __shared__ int s_ok;
   const int o = blockIdx.y;
+  if (blockIdx.x == 0 && o == 0)
+    for (int i = threadIdx.x; i < zero_n; i += kShardThreads) zero_cnt[i] = 0u;
   if (threadIdx.x == 0) s_ok = wait_count(my_gather_cnt + o, expect, limit_ns) ? 1 : 0;
   __syncthreads();
   if (!s_ok) {
@@ -152,24 +164,24 @@ shard_gather_kernel(const bf16* __restrict__ my_gather, const unsigned int* my_g
 }  // namespace
 
 void launch_shard_push(const void* src, int src_is_f32, float scale, int S, int d, int H, const ShardPeerTable& t,
-                       long long slot_off, cudaStream_t st) {
+                       long long slot_off, int cnt_off, cudaStream_t st) {
   const dim3 grid((S + kShardRows - 1) / kShardRows, H);
-  shard_push_kernel<<<grid, kShardThreads, 0, st>>>(src, src_is_f32, scale, S, d, d / H, t, slot_off);
+  shard_push_kernel<<<grid, kShardThreads, 0, st>>>(src, src_is_f32, scale, S, d, d / H, t, slot_off, cnt_off);
 }
 
-void launch_shard_reduce(const bf16* my_slots, const unsigned int* my_slot_cnt, unsigned int expect, int S, size_t S_cap,
+void launch_shard_reduce(const bf16* my_slots, const unsigned int* my_slot_cnt, int n_blocks, int S, size_t S_cap,
                          int d, int H, int rank, const ShardPeerTable& t, long long gather_off,
                          unsigned long long limit_ns, int* status, cudaStream_t st) {
   shard_reduce_kernel<<<(S + kShardRows - 1) / kShardRows, kShardThreads, 0, st>>>(
-      my_slots, my_slot_cnt, expect, S, S_cap, d, d / H, H, rank, t, gather_off, limit_ns, status);
+      my_slots, my_slot_cnt, n_blocks, S, S_cap, d, d / H, H, rank, t, gather_off, limit_ns, status);
 }
 
 void launch_shard_gather(const bf16* my_gather, const unsigned int* my_gather_cnt, unsigned int expect, int S, int d,
-                         int H, float* dst_f32, bf16* dst_bf16, unsigned long long limit_ns, int* status,
-                         cudaStream_t st) {
+                         int H, float* dst_f32, bf16* dst_bf16, unsigned int* zero_cnt, int zero_n,
+                         unsigned long long limit_ns, int* status, cudaStream_t st) {
   const dim3 grid((S + kShardRows - 1) / kShardRows, H);
   shard_gather_kernel<<<grid, kShardThreads, 0, st>>>(my_gather, my_gather_cnt, expect, S, d, d / H, dst_f32, dst_bf16,
-                                                      limit_ns, status);
+                                                      zero_cnt, zero_n, limit_ns, status);
 }
 
 }  // namespace foe

@@ -82,6 +82,18 @@ def test_group_decode(position):
     assert all(n == 10 for n in res["launches"])
 
 
+def test_group_decode_pushes_from_the_projection_epilogue_when_the_owner_span_allows():
+    """hidden 1024 over 4 ranks: 256 columns per owner, a whole number of the decode O-projection's 128-row weight slabs,
+    so the projection stores its result straight into the owners' slots (no push launch: nine launches per rank), over
+    several row blocks' worth of exchanges of different sizes (a prefill first, then decode steps on what it cached)."""
+    s = synth.LayerShape(1024, 8, 4, 4, 128, 4, 2, 128)
+    res = run_group(s, 17, [1] * 70, [3 + 7 * i for i in range(70)], decode=True, also_one_device=True)
+    assert all(n == 9 for n in res["launches"])
+    run_group(s, 18, [300, 41], [0, 0])
+    res = run_group(s, 19, [1] * 3, [64, 5, 600], decode=True)
+    assert all(n == 9 for n in res["launches"])
+
+
 def test_group_several_tiles_ragged_tail_head_dim_128():
     # 8 clusters x (2 query heads, 1 KV head) of width 128, hidden 2048: 256 columns per owner, rows spanning three
     # 256-row tile pairs with a ragged tail
