@@ -37,8 +37,11 @@ def test_description_checks_and_buffer_size(lib):
     from paper_2605_06206_b200 import shard
     assert ctypes.sizeof(shard.FoeShardConfig) == 20
     ok = shard.FoeShardConfig(2, 8, 4096, 16384, 0)
-    # 1 KB of counters + slots [2][8][16384][512] + gather [2][16384][4096], bf16
-    assert lib.foe_shard_buffer_bytes(ctypes.byref(ok)) == 1024 + 2 * (2 * 16384 * 4096 * 2)
+    # header (8 gather counters, then slot counters [2 parities][8 sources][64 blocks of 256 rows], rounded up to 1 KB)
+    # + slots [2][8][16384][512] + gather [2][16384][4096], bf16
+    header = -(-(128 + 2 * 8 * (16384 // 256) * 4) // 1024) * 1024
+    assert header == 5120
+    assert lib.foe_shard_buffer_bytes(ctypes.byref(ok)) == header + 2 * (2 * 16384 * 4096 * 2)
     for bad in [shard.FoeShardConfig(8, 8, 4096, 16, 0),      # rank out of range
                 shard.FoeShardConfig(0, 9, 4608, 16, 0),      # more than 8 ranks
                 shard.FoeShardConfig(0, 8, 4096 + 128, 16, 0),  # hidden not a multiple of 32 * ranks
