@@ -118,8 +118,8 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   uint64_t* s_full = kv_empty + kAtStages; // 2 tiles: the tile's scores are in tensor memory
   uint64_t* s_free = s_full + 2;           // 2 tiles: the step's four softmax warps hold the scores in registers
   uint64_t* p_ready = s_free + 2;          // 2
-  uint64_t* o_full = p_ready + 2;          // 2 tiles: phase j = the P V product of step j has completed
-  uint64_t* o_done = o_full + 2;           // 2 tiles: every product of the block has completed (one phase)
+  uint64_t* o_full = p_ready + 2;          // 2 tiles x 2 step parities: phase i of [t][b] = the P V product of step 2 i + b has completed
+  uint64_t* o_done = o_full + 4;           // 2 tiles: every product of the block has completed (one phase)
   uint64_t* hand = o_done + 2;             // 2 tiles x 4 lane quarters: phase j = step j's reference maximum is published
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(hand + 8);
 
@@ -152,7 +152,8 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     mbar_init(q_full, 1);
     for (int s = 0; s < kAtStages; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], n_tiles_q); }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(&s_full[t], 1); mbar_init(&s_free[t], 4); mbar_init(&p_ready[t], 4); mbar_init(&o_full[t], 1);
+      mbar_init(&s_full[t], 1); mbar_init(&s_free[t], 4); mbar_init(&p_ready[t], 4);
+      mbar_init(&o_full[2 * t], 1); mbar_init(&o_full[2 * t + 1], 1);
       mbar_init(&o_done[t], 1);
       for (int q = 0; q < 4; ++q) mbar_init(&hand[4 * t + q], 1);
     }
@@ -220,7 +221,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         for (int kk = 0; kk < kAtKeys / 16; ++kk)
           umma_bf16_ts(tmem_base + 256 + t * DH, p_tmem + kk * 8,
                        desc_mnmajor(vb_ + kk * (16 * 128), kAtKeys * 128, 1024), idesc_o, (j | kk) != 0);
-        umma_commit(&o_full[t]);
+        umma_commit(&o_full[2 * t + (j & 1)]);
       };
       if (ok && n_tiles > 0) {
         ok = mbar_wait(&kv_full[0], 0);
@@ -229,19 +230,33 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           issue_s(t, 0);
         }
       }
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const uint32_t ph = j & 1;
-        // scores of the next step first, as soon as this step's have been read out of their buffer
-        if (j + 1 < n_tiles) {
-          if (!mbar_wait(&kv_full[(j + 1) % kAtStages], ((j + 1) / kAtStages) & 1)) { ok = false; break; }
-          if (!mbar_wait(&s_free[t], ph)) { ok = false; break; }
+      // Two streams of work, each in its own order: Q K^T of step q as soon as its K/V page has landed and the scores of
+      // step q-1 have been read out of the buffer; P V of step p as soon as its probabilities are in place.  Whichever is
+      // ready is issued (the scores of step j+2 are not held back by the probabilities of step j: the thread that
+      // will need them is the one that is finishing step j).
+      int q = 1, p = 0;                                                 // next Q K^T, next P V
+      unsigned long long t0 = 0;
+      for (uint32_t spin = 0; p < n_tiles && ok;) {
+        bool did = false;
+        if (q < n_tiles && mbar_test(&kv_full[q % kAtStages], (q / kAtStages) & 1) && mbar_test(&s_free[t], (q - 1) & 1)) {
           tc_fence_after();
-          issue_s(t, j + 1);
+          issue_s(t, q);
+          ++q;
+          did = true;
         }
-        if (!mbar_wait(&p_ready[t], ph)) { ok = false; break; }         // P_t(j) is in tensor memory
-        tc_fence_after();
-        issue_o(t, j);
-        umma_commit(&kv_empty[j % kAtStages]);                          // stage j reusable once both tiles' products retire
+        if (mbar_test(&p_ready[t], p & 1)) {                            // P_t(p) is in tensor memory
+          tc_fence_after();
+          issue_o(t, p);
+          umma_commit(&kv_empty[p % kAtStages]);                        // stage p reusable once both tiles' products retire
+          ++p;
+          did = true;
+        }
+        if (did) { spin = 0; t0 = 0; continue; }
+        if ((++spin & 0x3ff) == 0) {                                    // bounded like every other wait
+          const unsigned long long now = globaltimer_ns();
+          if (t0 == 0) t0 = now;
+          else if (now - t0 > kWaitLimitNs) ok = false;
+        }
       }
       umma_commit(&o_done[t]);                                          // (also after a timeout: nobody waits in vain)
       if (!ok) atomicExch(a.status, kStatusTimeout);
@@ -327,7 +342,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         if (move) {
           const float alpha = (m_ref == -INFINITY) ? 0.f : fast_exp2(m_ref - m_new);
           if (j > 0) {
-            if (!mbar_wait(&o_full[t], ph ^ 1)) { ok = false; break; }      // every P V product so far has landed
+            if (!mbar_wait(&o_full[2 * t + (ph ^ 1)], ((j - 1) >> 1) & 1)) { ok = false; break; }   // every P V product so far has landed
             o_seen = true;
             tc_fence_after();
             // eight columns at a time: this path is rare, and a wider chunk here would raise the register demand of
@@ -351,6 +366,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         // scores at a time: scalings (packed, two values per instruction), exponentials back to back, sums and packing.
         // P of step j-2 sat in this buffer; its product has completed (see above).
         const uint32_t p_addr = p_base + (j & 1) * 32;
+        if (j >= 2 && !mbar_wait(&o_full[2 * t + ph], ((j - 2) >> 1) & 1)) { ok = false; break; }   // P V of step j-2 has read this buffer
         uint64_t rs2[4] = {0ull, 0ull, 0ull, 0ull};           // four independent chains of (even, odd) partial sums
         const uint64_t sc2 = pack_f32x2(a.scale_log2, a.scale_log2), nm2 = pack_f32x2(-m_use, -m_use);
 #pragma unroll
@@ -379,7 +395,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         l_run += (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
         // (before this warp's arrival below: P V of step j cannot have been issued yet, so the barrier is at most one
         // phase ahead of what is waited for)
-        if (!o_seen && !mbar_wait(&o_full[t], ph ^ 1)) { ok = false; break; }
+        if (!o_seen && !mbar_wait(&o_full[2 * t + (ph ^ 1)], ((j - 1) >> 1) & 1)) { ok = false; break; }
         tmem_st_wait();                                      // P is in tensor memory
         tc_fence_before();
         __syncwarp();
