@@ -195,6 +195,19 @@ def test_mixed_batch_of_prefill_chunks_and_decode_tokens():
     run_block_parity(shape, 18, [1, 200, 1, 64, 1], [300, 0, 1000, 64, 63], wscale=4.0)
 
 
+@pytest.mark.parametrize("dh,group", [(128, 2), (64, 4), (128, 1), (64, 3)])
+def test_prefill_attention_step_counts_and_mask_positions(dh, group):
+    """The prefill attention hands the 64-key steps of a query block alternately to two threads per row, so the cases
+    that matter are the number of steps of a block (one, two, odd, even), where the causal mask starts (an even or an
+    odd step, at a page boundary or inside a page) and a last block with few rows: new-token counts around 64, 128 and
+    192 on cached contexts around the page size.  One or two query heads per CTA (odd group sizes take one)."""
+    n_kv = 2
+    shape = synth.LayerShape(512, n_kv * group, n_kv, 2, dh, 4, 2, 128)
+    q_lens = [1, 63, 64, 65, 127, 128, 129, 191, 192, 193, 257, 5]
+    ctx = [0, 1, 64, 63, 130, 0, 62, 65, 128, 1, 191, 700]
+    run_block_parity(shape, 60 + dh + group, q_lens, ctx, wscale=2.0)
+
+
 def test_empty_and_single_token_calls():
     shape = shape_small()
     W = synth.make_weights(shape, 16, "cuda")
