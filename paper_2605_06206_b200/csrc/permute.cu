@@ -11,6 +11,7 @@
 // from which each selection reads its rank inside the block; (2) one block scans block counts and
 // expert totals and writes the m-tile table the grouped GEMMs walk; (3) every selection computes its
 // slot.
+#include <climits>
 #include "common.cuh"
 #include "kernels.h"
 
@@ -214,28 +215,47 @@ permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, 
         }
       }
     }
-    for (int task = in_regs ? n_tokens * H : t; task < n_tokens * H; task += 1024) {
+    // any other E_c (up to 128): one warp per (token, cluster), the scores in registers (lane l holds experts l, l + 32,
+    // ...), one shuffle arg-max per selection; selection j is kept by lane j % 32 and written once
+    for (int task = in_regs ? n_tokens * H : (t >> 5); task < n_tokens * H; task += 32) {
+      const int lane = t & 31;
       const int i = task / H, h = task - i * H;
       const size_t o = size_t(i) * E + size_t(h) * Ec;
-      uint32_t taken[4] = {0u, 0u, 0u, 0u};                 // E_c <= 128
+      float cand[4];
+      bool taken[4];
+#pragma unroll
+      for (int s = 0; s < 4; ++s) {
+        const int e = lane + 32 * s;
+        taken[s] = e >= Ec;
+        cand[s] = taken[s] ? 0.f : tk.logits_out[o + e];
+      }
       float m = 0.f, sum = 0.f;
       const size_t oo = size_t(task) * kc;
       for (int j = 0; j < kc; ++j) {
         float bv = 0.f;
-        int bi = -1;
-        for (int e = 0; e < Ec; ++e) {
-          if ((taken[e >> 5] >> (e & 31)) & 1u) continue;
-          const float v = tk.logits_out[o + e];
-          if (bi < 0 || v > bv) { bv = v; bi = e; }         // ascending e: first wins ties
+        int bi = INT_MAX;                                   // INT_MAX: nothing left in this lane
+#pragma unroll
+        for (int s = 0; s < 4; ++s)
+          if (!taken[s] && (bi == INT_MAX || cand[s] > bv)) { bv = cand[s]; bi = lane + 32 * s; }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+          const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+          const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+          if (oi != INT_MAX && (bi == INT_MAX || ov > bv || (ov == bv && oi < bi))) { bv = ov; bi = oi; }
         }
-        taken[bi >> 5] |= 1u << (bi & 31);
+        if ((bi & 31) == lane) {
+#pragma unroll
+          for (int s = 0; s < 4; ++s) taken[s] = taken[s] || (bi >> 5) == s;
+        }
         if (j == 0) m = bv;
-        const float ex = expf(bv - m);
+        const float ex = expf(bv - m);                      // the same value in every lane
         sum += ex;
-        tk.idx_out[oo + j] = h * Ec + bi;
-        tk.w_out[oo + j] = ex;
+        if ((j & 31) == lane) {
+          tk.idx_out[oo + j] = h * Ec + bi;
+          tk.w_out[oo + j] = ex;
+        }
       }
-      for (int j = 0; j < kc; ++j) tk.w_out[oo + j] = tk.w_out[oo + j] / sum;
+      for (int j = lane; j < kc; j += 32) tk.w_out[oo + j] = tk.w_out[oo + j] / sum;   // lane j % 32 wrote entry j
     }
     __threadfence_block();
     __syncthreads();                            // idx (== tk.idx_out) is read below by other threads of this block

@@ -100,6 +100,45 @@ def test_route_bit_exact_where_split_k_partials_would_outgrow_their_buffer(wl, n
     check_maps(shape, aux, idx.cpu().numpy())
 
 
+@pytest.mark.parametrize("H,Ec,kc,n_tok,ties", [(1, 128, 16, 2, False), (1, 128, 32, 200, False), (2, 100, 31, 33, False),
+                                                (4, 24, 24, 256, False), (8, 64, 7, 65, False), (1, 3, 3, 5, False),
+                                                (2, 96, 20, 40, True), (1, 33, 32, 3, True)])
+def test_route_of_a_decode_step_with_wide_or_odd_expert_sets(H, Ec, kc, n_tok, ties):
+    """Calls of at most 256 tokens select inside the map kernel; cluster sizes other than 4, 8, 16 and 32 take its
+    one-warp-per-(token, cluster) selection.  With `ties` the router weights are zero and the bias repeats each value
+    four times, so that every selection is decided by the lower-expert-id rule."""
+    shape = synth.LayerShape(512, 2 * H, H, H, 64, Ec, kc, 128)
+    seed = 1300 + Ec + kc
+    W = dict(ffn_norm_g=synth.normal_bf16(seed, synth.TID["ffn_norm_g"], (shape.hidden,), 0.02, 1.0, "cuda"),
+             router_w=synth.normal_bf16(seed, synth.TID["router_w"], (shape.n_experts, shape.hidden), 0.02, 0.0, "cuda").float())
+    full = _route_only_weights(shape, W)
+    if ties:
+        W["router_w"] = torch.zeros_like(W["router_w"])
+        full["router_w"] = W["router_w"]
+        b = torch.tensor([float((7 * (e // 4)) % 11) for e in range(shape.n_experts)], dtype=torch.float32, device="cuda")
+        W["router_b"] = full["router_b"] = b
+    h = synth.normal_bf16(seed, 77, (n_tok, shape.hidden), 1.5, 0.0, "cuda")
+    layer = binding.FoeLayer(shape, full, max_tokens=256, max_seqs=1, max_context=64)
+    idx, w = layer.route(h)
+    assert layer.poll_status() == 0
+    aux = layer.aux()
+    layer.close()
+    cfg = adapter.cfg_from_shape(shape)
+    Wn = {k: adapter.to_np(W[k]) for k in ("ffn_norm_g", "router_w")}
+    Wn["router_b"] = adapter.to_np(W["router_b"]) if ties else None
+    rt = orc.route(cfg, Wn, adapter.to_np(h))
+    idx_g, w_g = idx.cpu().numpy(), w.cpu().numpy().astype(np.float64)
+    if ties:
+        assert np.array_equal(idx_g.reshape(rt["idx"].shape), rt["idx"])            # exact scores: no exemptions
+        assert np.abs(w_g.reshape(rt["w"].shape) - rt["w"]).max() <= 1e-6
+    else:
+        exempt = check_routing(shape, idx_g, w_g, rt["logits"], rt["idx"], rt["w"])
+        assert exempt <= 2
+        lg = np.take_along_axis(rt["logits"], idx_g.reshape(n_tok, -1).astype(np.int64), 1).reshape(idx_g.shape)
+        assert (np.diff(lg, axis=-1) <= 1e-5).all()
+    check_maps(shape, aux, idx_g)
+
+
 def _route_only_weights(shape, W):
     """A full weight set for foe_layer_create in which everything but the router and the FFN-norm gain is a small
     shared zero buffer of the right size class (routing reads nothing else)."""
