@@ -140,6 +140,10 @@ foe_status foe_layer_create_shared(const foe_config* config, const foe_weights* 
 /* Frees everything the handle owns.  NULL is accepted. */
 foe_status foe_layer_destroy(foe_layer* layer);
 
+/* Alignment, all calls: device pointers to bf16 or fp32 tensors (weights, x, out, work buffers, K/V pages, h) must be
+ * 16-byte aligned, int32 and per-expert fp32 arrays (block_table, context_lens, q_lens, router_b, topk_idx, topk_w)
+ * 4-byte aligned.  A misaligned pointer is refused with FOE_ERR_SHAPE before anything is launched. */
+
 /* Table 2 (all four rows) for S = kv->n_tokens new tokens of kv->n_seqs sequences: attention over the
  * paged cache plus the new tokens (causal), sync, routing, experts, combine.  x: [H][S][hidden] bf16
  * ([S][hidden] on a first layer); out likewise ([S][hidden] on a last layer); out must not alias x.

@@ -308,6 +308,7 @@ void launch_combine(const float* r_full, const bf16* y, const float* w, const in
   if (threads > 256) threads = 256;
   if (threads < 32) threads = 32;
   if (n_tokens <= 1024) {
+    if (d / 8 >= 512) threads = 512;          // one pass over the row: the kernel is a chain of round trips, not a stream
     launch_pdl(combine_small_kernel, dim3(n_tokens), dim3(threads), 0, st, r_full, y, w, inv, out, n_tokens, d, H, kc, last_mean);
     return;
   }

@@ -440,8 +440,15 @@ foe_status run_block(foe_layer* L, const void* x, const foe_kv_cache* kv, void* 
 }
 
 // argument checks shared by foe_prefill / foe_decode and foe_shard_attend (x and out are checked by the callers)
+bool misaligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
+
 foe_status check_call(const foe_layer* L, const foe_kv_cache* kv, bool decode) {
   if (!kv->k_pages || !kv->v_pages || !kv->block_table || !kv->context_lens) return FOE_ERR_NULL;
+  // pages are read through tensor maps and 16-byte accesses, the integer arrays element by element: a misaligned view
+  // is refused here, before any launch, rather than found by the device
+  if (misaligned(kv->k_pages, 16) || misaligned(kv->v_pages, 16) || misaligned(kv->block_table, 4) ||
+      misaligned(kv->context_lens, 4) || (kv->q_lens && misaligned(kv->q_lens, 4)))
+    return FOE_ERR_SHAPE;
   if (decode) {
     if (kv->n_seqs > L->cfg.max_seqs || kv->max_pages_per_seq <= 0 || kv->num_pages <= 0) return FOE_ERR_SHAPE;
     return FOE_OK;
@@ -493,6 +500,10 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
   if (!w->attn_norm_g || !w->wq || !w->wk || !w->wv || !w->wo || !w->ffn_norm_g || !w->w_gate || !w->w_up ||
       !w->w_down || !w->router_w)
     return FOE_ERR_NULL;
+  if (misaligned(w->attn_norm_g, 16) || misaligned(w->wq, 16) || misaligned(w->wk, 16) || misaligned(w->wv, 16) ||
+      misaligned(w->wo, 16) || misaligned(w->ffn_norm_g, 16) || misaligned(w->w_gate, 16) || misaligned(w->w_up, 16) ||
+      misaligned(w->w_down, 16) || misaligned(w->router_w, 16) || (w->router_b && misaligned(w->router_b, 4)))
+    return FOE_ERR_SHAPE;
   int dev = 0, n_dev = 0;
   if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0) { cudaGetLastError(); return FOE_ERR_CUDA; }
   if (cudaGetDevice(&dev) != cudaSuccess) return FOE_ERR_CUDA;
@@ -660,6 +671,7 @@ foe_status foe_prefill(foe_layer* L, const void* x, const foe_kv_cache* kv, void
   if (!x || !out) return FOE_ERR_NULL;
   const foe_status c = check_call(L, kv, false);
   if (c != FOE_OK) return c;
+  if (misaligned(x, 16) || misaligned(out, 16)) return FOE_ERR_SHAPE;
   if (x == out) return FOE_ERR_UNSUPPORTED;
   return run_block(L, x, kv, out, static_cast<cudaStream_t>(stream), false);
 }
@@ -671,6 +683,7 @@ foe_status foe_decode(foe_layer* L, const void* x, const foe_kv_cache* kv, void*
   if (!x || !out) return FOE_ERR_NULL;
   const foe_status c = check_call(L, kv, true);
   if (c != FOE_OK) return c;
+  if (misaligned(x, 16) || misaligned(out, 16)) return FOE_ERR_SHAPE;
   if (x == out) return FOE_ERR_UNSUPPORTED;
   return run_block(L, x, kv, out, static_cast<cudaStream_t>(stream), true);
 }
@@ -700,6 +713,7 @@ foe_status foe_stack_forward(foe_layer* const* layers, int n_layers, const void*
   }
   const int S = decode ? kvs[0].n_seqs : kvs[0].n_tokens;
   if (S > 0 && (!x || !out)) return FOE_ERR_NULL;
+  if (misaligned(x, 16) || misaligned(out, 16) || misaligned(work0, 16) || misaligned(work1, 16)) return FOE_ERR_SHAPE;
   if (S > 0 && x == out) return FOE_ERR_UNSUPPORTED;
   void* bufs[2] = {work0, work1};
   const void* in = x;
@@ -724,6 +738,7 @@ foe_status foe_context_advance(int* context_lens, int n_seqs, int by, void* stre
 foe_status foe_route(foe_layer* L, const void* h, int n_tokens, int* topk_idx, float* topk_w, void* stream) {
   if (!L || !h || !topk_idx || !topk_w) return FOE_ERR_NULL;
   if (n_tokens < 0 || n_tokens > L->S_max) return FOE_ERR_SHAPE;
+  if (misaligned(h, 16) || misaligned(topk_idx, 4) || misaligned(topk_w, 4)) return FOE_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   L->last_stream = st;
   L->launches = 0;
@@ -752,7 +767,6 @@ foe_status foe_route_noalloc(int hidden, int n_clusters, int experts_per_cluster
   if (n_tokens < 0) return FOE_ERR_SHAPE;
   // the kernels read h and router_w 16 bytes at a time, the gain 8, the outputs 4: a misaligned view is refused here
   // instead of faulting on the device
-  auto misaligned = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; };
   if (misaligned(h, 16) || misaligned(router_w, 16) || misaligned(ffn_norm_g, 8) || misaligned(topk_idx, 4) ||
       misaligned(topk_w, 4) || (router_b && misaligned(router_b, 4)))
     return FOE_ERR_SHAPE;
@@ -949,6 +963,7 @@ foe_status foe_shard_attend(foe_layer* L, foe_shard* sh, const void* x, const fo
     if (!x) return FOE_ERR_NULL;
     const foe_status c = check_call(L, kv, decode != 0);
     if (c != FOE_OK) return c;
+    if (misaligned(x, 16)) return FOE_ERR_SHAPE;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const foe_status b = shard_begin(sh, S, st);
@@ -961,6 +976,7 @@ foe_status foe_shard_attend(foe_layer* L, foe_shard* sh, const void* x, const fo
 foe_status foe_shard_push(foe_shard* sh, const void* src, int n_tokens, float scale, void* stream) {
   if (!sh) return FOE_ERR_NULL;
   if (n_tokens > 0 && !src) return FOE_ERR_NULL;
+  if (misaligned(src, 16)) return FOE_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const foe_status b = shard_begin(sh, n_tokens, st);
   if (b != FOE_OK) return b;
@@ -1004,6 +1020,7 @@ foe_status foe_shard_ffn(foe_layer* L, foe_shard* sh, void* out, void* stream) {
   if (!L || !sh) return FOE_ERR_NULL;
   if (L->shard_stage != 1 || L->last_tokens != sh->S) return FOE_ERR_UNSUPPORTED;
   if (sh->S > 0 && !out) return FOE_ERR_NULL;
+  if (misaligned(out, 16)) return FOE_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   g_overlap_launches = false;             // (the exchange kernels are launched the ordinary way)
   const foe_status f = shard_finish(sh, L->ws->r_full, nullptr, st);      // r_full of the whole group, as fp32
@@ -1018,6 +1035,7 @@ foe_status foe_shard_ffn(foe_layer* L, foe_shard* sh, void* out, void* stream) {
 foe_status foe_shard_gather(foe_shard* sh, void* dst, void* stream) {
   if (!sh) return FOE_ERR_NULL;
   if (sh->S > 0 && !dst) return FOE_ERR_NULL;
+  if (misaligned(dst, 16)) return FOE_ERR_SHAPE;
   return shard_finish(sh, nullptr, static_cast<bf16*>(dst), static_cast<cudaStream_t>(stream));
 }
 

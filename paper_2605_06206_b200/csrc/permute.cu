@@ -174,11 +174,12 @@ __device__ __forceinline__ void topk_small_regs(const TopkSmall& tk, int task) {
 }
 
 __global__ void __launch_bounds__(1024)
-permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, const PermuteBuffers pb,
-                     int* __restrict__ status, const TopkSmall tk) {
+permute_small_kernel(const int* idx, int n_tokens, int sel, int E, const PermuteBuffers pb,
+                     int* __restrict__ status, const TopkSmall tk, int idx_in_smem) {
   pdl_wait();
   pdl_launch_dependents();
-  extern __shared__ uint32_t bm[];            // [E][8]
+  extern __shared__ uint32_t bm[];            // [E][8], then (idx_in_smem) a copy of idx: [n_tokens][sel]
+  int* s_idx = reinterpret_cast<int*>(bm + E * 8);
   __shared__ int s_a[1024], s_b[1024], s_off[1024];
   int* counts = pb.counts;
   int* offsets = pb.offsets;
@@ -261,6 +262,12 @@ permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, 
     __syncthreads();                            // idx (== tk.idx_out) is read below by other threads of this block
   }
   for (int q = t; q < E * 8; q += 1024) bm[q] = 0u;
+  // the selections are read twice below, token by token; one coalesced pass brings them next to the bitmap when they fit
+  // (a thread walking its token's list in global memory pays one round trip to L2 per selection)
+  if (idx_in_smem) {
+    for (int q = t; q < n_tokens * sel; q += 1024) s_idx[q] = idx[q];
+    idx = s_idx;
+  }
   __syncthreads();
   if (t < n_tokens) {
     for (int s = 0; s < sel; ++s) {
@@ -310,13 +317,22 @@ permute_small_kernel(const int* __restrict__ idx, int n_tokens, int sel, int E, 
   }
 }
 
+// Bytes of the selections' copy in shared memory, or 0 when it does not fit beside the bitmap and the 12 KB of static
+// arrays within the 48 KB a kernel gets without opting in.
+static size_t small_idx_bytes(int n_tokens, int sel, int E) {
+  const size_t want = size_t(n_tokens) * sel * sizeof(int);
+  return size_t(E) * 32 + want <= 34 * 1024 ? want : 0;
+}
+
 int launch_permute(const int* idx, const PermuteBuffers& pb, int n_tokens, int sel, int E, int* status,
                    cudaStream_t st) {
   if (n_tokens <= 0) return 0;
   if (n_tokens <= kPB) {
     TopkSmall none;
     none.scores = nullptr;
-    launch_pdl(permute_small_kernel, dim3(1), dim3(1024), size_t(E) * 32, st, idx, n_tokens, sel, E, pb, status, none);
+    const size_t copy = small_idx_bytes(n_tokens, sel, E);
+    launch_pdl(permute_small_kernel, dim3(1), dim3(1024), size_t(E) * 32 + copy, st, idx, n_tokens, sel, E, pb, status, none,
+               copy ? 1 : 0);
     return 1;
   }
   const int n_blocks = (n_tokens + kPB - 1) / kPB;
@@ -335,7 +351,9 @@ int launch_topk_permute_small(const float* scores, int k_splits, const float* bi
   TopkSmall tk;
   tk.scores = scores; tk.k_splits = k_splits; tk.bias = bias; tk.logits_out = logits; tk.idx_out = idx; tk.w_out = w; tk.H = H; tk.Ec = Ec; tk.kc = kc;
   const int E = H * Ec;
-  launch_pdl(permute_small_kernel, dim3(1), dim3(1024), size_t(E) * 32, st, idx, n_tokens, H * kc, E, pb, status, tk);
+  const size_t copy = small_idx_bytes(n_tokens, H * kc, E);
+  launch_pdl(permute_small_kernel, dim3(1), dim3(1024), size_t(E) * 32 + copy, st, idx, n_tokens, H * kc, E, pb, status, tk,
+             copy ? 1 : 0);
   return 1;
 }
 

@@ -289,41 +289,70 @@ __global__ void __launch_bounds__(kRsThreads)
 route_scores_small_kernel(const void* __restrict__ r_in, int r_is_bf16, const bf16* __restrict__ gain,
                           const float* __restrict__ wr, bf16* __restrict__ u_out, float* __restrict__ scores,
                           int n_tokens, int d, int E, float eps, int k_per_split) {
-  pdl_wait();
-  pdl_launch_dependents();
   __shared__ float w_s[kRsK][kRsExp + 1];
   __shared__ float u_s[kRsTok][kRsK];
   __shared__ float red[kRsTok][2];
   const int tid = threadIdx.x, el = tid & 63, tq = tid >> 6;
   const int tok = min(blockIdx.x * kRsTok + tq, n_tokens - 1);          // rows past the end repeat the last one
   const int e0 = blockIdx.y * kRsExp;
-  auto load_r = [&](int k) -> float {
-    return r_is_bf16 ? __bfloat162float(static_cast<const bf16*>(r_in)[size_t(tok) * d + k])
-                     : static_cast<const float*>(r_in)[size_t(tok) * d + k];
-  };
-  // 1/rms of this thread's token: 64 threads per token
-  float ss = 0.f;
-  for (int k = el; k < d; k += 64) { const float v = load_r(k); ss += v * v; }
-  ss = warp_sum(ss);
-  if ((tid & 31) == 0) red[tq][(tid >> 5) & 1] = ss;
-  __syncthreads();
-  const float inv = rsqrtf((red[tq][0] + red[tq][1]) / float(d) + eps);
-
+  const int kbeg = blockIdx.z * k_per_split, kend = min(d, kbeg + k_per_split);   // this CTA's slice of K
   // loader roles for the weight tile: float4 (row = i >> 4, column group = i & 15), i = tid + 256 j
   float4 wq[4];
   float uq;
-  auto fetch = [&](int k0) {
+  auto fetch_w = [&](int k0) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int i = tid + kRsThreads * j;
       const int e = min(e0 + (i >> 4), E - 1);
       wq[j] = __ldg(reinterpret_cast<const float4*>(wr + size_t(e) * d + k0 + (i & 15) * 4));
     }
+  };
+  // The router weights are older than the kernel before this one: the first tile is requested before the wait for it.
+  fetch_w(kbeg);
+  pdl_wait();
+  pdl_launch_dependents();
+  auto load_r = [&](int k) -> float {
+    return r_is_bf16 ? __bfloat162float(static_cast<const bf16*>(r_in)[size_t(tok) * d + k])
+                     : static_cast<const float*>(r_in)[size_t(tok) * d + k];
+  };
+  // 1/rms of this thread's token: 64 threads per token, eight 16-byte loads in flight per thread (the row sits in L2;
+  // one element per load made this pass a chain of d / 256 round trips)
+  float ss = 0.f;
+  if (!r_is_bf16) {
+    const float4* row = reinterpret_cast<const float4*>(static_cast<const float*>(r_in) + size_t(tok) * d);
+    const int n4 = d >> 2;
+    for (int k4 = el; k4 < n4; k4 += 64 * 8) {
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = k4 + 64 * u < n4 ? row[k4 + 64 * u] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) ss += (v[u].x * v[u].x + v[u].y * v[u].y) + (v[u].z * v[u].z + v[u].w * v[u].w);
+    }
+  } else {
+    const uint2* row = reinterpret_cast<const uint2*>(static_cast<const bf16*>(r_in) + size_t(tok) * d);
+    const int n4 = d >> 2;
+    for (int k4 = el; k4 < n4; k4 += 64 * 8) {
+      uint2 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = k4 + 64 * u < n4 ? row[k4 + 64 * u] : make_uint2(0u, 0u);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float a = bf16_lo(v[u].x), b = bf16_hi(v[u].x), c = bf16_lo(v[u].y), e = bf16_hi(v[u].y);
+        ss += (a * a + b * b) + (c * c + e * e);
+      }
+    }
+  }
+  ss = warp_sum(ss);
+  if ((tid & 31) == 0) red[tq][(tid >> 5) & 1] = ss;
+  __syncthreads();
+  const float inv = rsqrtf((red[tq][0] + red[tq][1]) / float(d) + eps);
+
+  auto fetch = [&](int k0) {
+    fetch_w(k0);
     uq = load_r(k0 + el) * inv * __bfloat162float(gain[k0 + el]);
   };
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  const int kbeg = blockIdx.z * k_per_split, kend = min(d, kbeg + k_per_split);   // this CTA's slice of K
-  fetch(kbeg);
+  uq = load_r(kbeg + el) * inv * __bfloat162float(gain[kbeg + el]);
   for (int k0 = kbeg; k0 < kend; k0 += kRsK) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {

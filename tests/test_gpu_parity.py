@@ -503,6 +503,35 @@ def test_host_side_argument_errors():
     assert layer.poll_status() == -8
     layer.prefill(x8, kv, n_tokens=8, max_q_len=8)                     # and the handle is fine afterwards
     assert layer.poll_status() == 0
+    # views that start 2 bytes off a 16-byte boundary (contiguous, right type): refused before any launch
+    def off_by_one(t):
+        flat = torch.empty(t.numel() + 8, dtype=t.dtype, device=t.device)
+        v = flat[1:1 + t.numel()].view(t.shape)
+        v.copy_(t)
+        assert v.is_contiguous() and v.data_ptr() % 16 != 0
+        return v
+    for call in (lambda: layer.prefill(off_by_one(x8), kv, n_tokens=8, max_q_len=8),
+                 lambda: layer.prefill(x8, kv, n_tokens=8, max_q_len=8, out=off_by_one(torch.empty_like(x8))),
+                 lambda: layer.route(off_by_one(synth.normal_bf16(27, 77, (8, shape.hidden), 1.0, 0.0, "cuda")))):
+        with pytest.raises(binding.FoeError) as e:
+            call()
+        assert e.value.code == -3
+    kv1 = synth.make_paged_cache(shape, 27, [20], [1], "cuda")
+    with pytest.raises(binding.FoeError) as e:
+        layer.decode(off_by_one(synth.make_x(shape, 27, 1, "cuda")), kv1)
+    assert e.value.code == -3
+    kv1.k_pages = off_by_one(kv1.k_pages)
+    with pytest.raises(binding.FoeError) as e:
+        layer.decode(synth.make_x(shape, 27, 1, "cuda"), kv1)
+    assert e.value.code == -3
+    assert layer.poll_status() == 0
+    layer.prefill(x8, kv, n_tokens=8, max_q_len=8)
+    assert layer.poll_status() == 0
+    W2 = dict(W)
+    W2["wq"] = off_by_one(W["wq"])
+    with pytest.raises(binding.FoeError) as e:
+        binding.FoeLayer(shape, W2, 8, 1, 64)
+    assert e.value.code == -3
     layer.close()
 
 
