@@ -79,7 +79,7 @@ struct foe_layer {
   CUtensorMap tm_router;
   float2* rope_tab;
   foe_workspace* ws;
-  int max_splits, pages_per_split;
+  int max_splits;
   // tensor maps of the weights
   CUtensorMap tm_wqkv, tm_wo, tm_wgu, tm_wd;       // weights; box = the rows of B one CTA of a pair stages per k-block
   CUtensorMap tms_wqkv, tms_wo, tms_wgu, tms_wd;   // same weights, boxes sized for the decode kernels
@@ -303,8 +303,9 @@ foe_status run_attend(foe_layer* L, const void* x, const foe_kv_cache* kv, cudaS
   aa.max_pages_per_seq = kv->max_pages_per_seq; aa.num_pages = kv->num_pages; aa.n_tokens = S; aa.n_q = L->n_q; aa.n_kv = L->n_kv;
   aa.dh = dh; aa.max_q_len = decode ? 1 : kv->max_q_len; aa.scale_log2 = float(1.4426950408889634 / sqrt(double(dh)));
   aa.status = L->ws->status; aa.part_o = L->ws->part_o; aa.part_ml = L->ws->part_ml; aa.max_splits = L->max_splits;
-  aa.pages_per_split = L->pages_per_split; aa.split_done = L->ws->split_done;
-  if (decode) { launch_attn_decode(tmK, tmV, aa, st); L->launches += 1; }
+  aa.split_done = L->ws->split_done;
+  aa.max_kv_pages = min(kv->max_pages_per_seq, (L->cfg.max_context + 63) / 64);   // part_o / part_ml were sized for this many
+  if (decode) { launch_attn_decode(tmK, tmV, aa, L->n_sms, st); L->launches += 1; }
   else { launch_attn_prefill_tc(L->ws->tm_qkv, tmK, tmV, aa, st); L->launches += 1; }
 
   // ---- output projection; the cross-cluster sync is its K-reduction plus the sum of x[h] in the epilogue
@@ -539,8 +540,7 @@ foe_status foe_layer_create_shared(const foe_config* cfg, const foe_weights* w, 
   L->n_sms = prop.multiProcessorCount;
   const int H = L->H, d = L->d, dh = L->dh, I = L->I, E = L->E, S = L->S_max, R = L->R_max;
   const int max_pages = (cfg->max_context + 63) / 64;
-  L->pages_per_split = 16;
-  L->max_splits = (max_pages + L->pages_per_split - 1) / L->pages_per_split;
+  L->max_splits = attn_decode_max_segments(max_pages);
   const int n_blocks = (S + kPermuteBlockTokens - 1) / kPermuteBlockTokens;
   const int qkvN = (L->g + 2 * L->c) * dh;
 

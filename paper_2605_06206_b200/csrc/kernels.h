@@ -123,16 +123,17 @@ struct AttnArgs {
   float scale_log2;         // log2(e) / sqrt(dh)
   int* status;
   // decode only
-  float* part_o;            // [n_seqs][n_q][max_splits][dh]
+  float* part_o;            // [n_seqs][n_q][max_splits][dh] partial outputs of the segments of a (sequence, KV head) pair
   float* part_ml;           // [n_seqs][n_q][max_splits][2]
-  int* split_done;          // [n_seqs][n_kv] splits finished so far (zero between calls)
-  int max_splits;
-  int pages_per_split;
+  int* split_done;          // [n_seqs][n_kv] segments finished so far (zero between calls)
+  int max_splits;           // attn_decode_max_segments(max pages per sequence the layer was created for)
+  int max_kv_pages;         // pages of a sequence the decode kernel looks at: min(block-table width, the layer's max_context / 64)
 };
 // tensor-core (tcgen05) prefill attention; tmQ maps the qkv buffer [S][(n_q+2n_kv)*dh] with 128-row boxes
 void launch_attn_prefill_tc(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a,
                             cudaStream_t st);
-void launch_attn_decode(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, cudaStream_t st);
+void launch_attn_decode(const CUtensorMap& tmK, const CUtensorMap& tmV, const AttnArgs& a, int n_sms, cudaStream_t st);
+int attn_decode_max_segments(int max_pages_per_seq);   // per (sequence, KV head): second-to-last extent of part_o / part_ml
 
 // ---- gemm_tcgen05.cu
 void launch_gemm(int epi, const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args, int n_sms,

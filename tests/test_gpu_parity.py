@@ -286,6 +286,24 @@ def test_decode_head_dim_128_many_splits():
     run_block_parity(shape, 22, [1] * 4, [10, 1030, 2100, 5000], decode=True, wscale=4.0)
 
 
+@pytest.mark.parametrize("dh,n_seqs,spread", [(128, 40, 5200), (64, 45, 3000), (128, 33, 9000), (64, 3, 700)])
+def test_decode_attention_page_partition_across_sequences(dh, n_seqs, spread):
+    """The decode attention kernel cuts the list of all (sequence, KV head, page) entries into equal ranges, one per
+    CTA: with a few thousand pages in the call the ranges are longer than the minimum, start and end anywhere inside
+    a pair, and a range may hold the tail of one sequence, whole short sequences and the head of the next.  Contexts
+    on and around page boundaries, one-page sequences, more than 32 sequences (the range search walks them in chunks
+    of 32)."""
+    if dh == 64:
+        shape = shape_small()
+    else:
+        shape = synth.LayerShape(512, 8, 2, 2, 128, 4, 2, 256)
+    ctx = [(613 * i * i + 97 * i) % spread for i in range(n_seqs)]
+    for i, v in enumerate([0, 63, 64, 65, 127, 128, 1, 511, 512]):
+        if 2 * i + 1 < n_seqs:
+            ctx[2 * i + 1] = v
+    run_block_parity(shape, 31, [1] * n_seqs, ctx, decode=True, wscale=4.0)
+
+
 @pytest.mark.parametrize("dh,position,n_seqs", [(64, "middle", 130), (128, "middle", 200), (64, "first", 65), (128, "last", 256)])
 def test_decode_more_sequences_than_one_token_tile(dh, position, n_seqs):
     # the decode projections take 64 tokens per CTA: several token tiles, the last one ragged (or exactly full)
