@@ -452,6 +452,9 @@ foe_status check_call(const foe_layer* L, const foe_kv_cache* kv, bool decode) {
     return FOE_ERR_SHAPE;
   if (decode) {
     if (kv->n_seqs > L->cfg.max_seqs || kv->max_pages_per_seq <= 0 || kv->num_pages <= 0) return FOE_ERR_SHAPE;
+    // the decode attention kernel numbers the pages of all (sequence, KV head) pairs with 32-bit integers
+    const long long pages = (long long)kv->n_seqs * L->n_kv * min(kv->max_pages_per_seq, (L->cfg.max_context + 63) / 64);
+    if (pages >= (1LL << 30)) return FOE_ERR_SHAPE;
     return FOE_OK;
   }
   if (!kv->q_lens) return FOE_ERR_NULL;
