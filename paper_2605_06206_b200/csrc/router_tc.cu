@@ -7,14 +7,16 @@
 // is not enough.  Both operands are split into three bf16 terms, x = x1 + x2 + x3, which together hold all 24
 // significant bits of a float; the six products of weight 1, 2^-8 and 2^-16 (x1 w1, x1 w2, x2 w1, x2 w2, x1 w3,
 // x3 w1) are issued as bf16 MMAs with fp32 accumulation -- every product of two bf16 values is exact in fp32 -- and
-// the three dropped ones are below 2^-24.  Eight accumulators take the k-blocks in turn and are summed in fp32 by the
-// epilogue, so that no tensor-core accumulation chain is longer than 96 steps.
+// the three dropped ones are below 2^-24.  Eight (64 experts per CTA) or four (128) accumulators take the k-blocks in
+// turn and are summed in fp32 by the epilogue, which keeps the tensor-core accumulation chains short (96 steps for a
+// hidden size of 2048 with eight accumulators).
 //
 // The weights are split when the layer is created (gain folded in); the residual r is split on the fly: sixteen
 // converter warps read a 128 x 64 fp32 tile per k-block straight from global memory (coalesced, 512 bytes per warp
 // instruction), split it in registers and store the three bf16 tiles in the 128-byte-swizzled operand layout, then
-// cross to the async proxy and arrive on the stage's barrier.  r is read exactly once and the kernel runs at the rate
-// r streams in.  One CTA per 128 tokens x 64 experts.
+// cross to the async proxy and arrive on the stage's barrier.  The kernel runs at the rate of this conversion.  One CTA
+// per 128 tokens x 64 experts, or x 128 experts when the (padded) expert count is a multiple of 128: every token tile
+// is then converted once per 128 experts.
 //
 // Warp roles: 0 TMA producer (weight planes), 1 MMA issuer, 2-5 epilogue, 6-21 converters.  All waits are bounded.
 #include "common.cuh"
@@ -22,15 +24,21 @@
 
 namespace foe {
 
-constexpr int kRtRows = 128, kRtChunk = kRouterChunk, kRtBK = 64, kRtStages = 3;
+constexpr int kRtRows = 128, kRtBK = 64;
 constexpr int kRtATile = kRtRows * kRtBK * 2;       // 16 KB: one bf16 term of the A tile
-constexpr int kRtBTile = kRtChunk * kRtBK * 2;      // 8 KB: one bf16 term of the B tile
-constexpr int kRtStageBytes = 3 * kRtATile + 3 * kRtBTile;   // 72 KB
+// A CTA takes CHUNK = 64 or 128 experts.  The kernel runs at the rate its converters split the residual, so a layer
+// with 128 experts or more converts every token tile once per 128 experts instead of once per 64;
+// the price is a ring of two stages instead of three and accumulation chains twice as long.
+template <int CHUNK> struct RtCfg {
+  static constexpr int kBTile = CHUNK * kRtBK * 2;                 // 8 or 16 KB: one bf16 term of the B tile
+  static constexpr int kStageBytes = 3 * kRtATile + 3 * kBTile;    // 72 or 96 KB
+  static constexpr int kStages = CHUNK == 64 ? 3 : 2;
+  static constexpr int kAccs = 512 / CHUNK;                        // accumulators of CHUNK columns: all 512 TMEM columns
+  static constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 + 256;
+};
 constexpr int kRtConvWarps = 16;
 constexpr int kRtThreads = (6 + kRtConvWarps) * 32;
 constexpr int kRtRowsPerLane = kRtRows / (2 * kRtConvWarps);   // tile rows one converter lane handles per k-block
-constexpr int kRtAccs = 8;                          // accumulators of 64 columns: all 512 TMEM columns
-constexpr size_t kRtSmemBytes = size_t(kRtStages) * kRtStageBytes + 1024 + 256;
 
 // split two floats into three packed bf16 pairs (x = hi + mid + lo up to 2^-24 |x|)
 __device__ __forceinline__ void split3(float x, float y, uint32_t& hi, uint32_t& mid, uint32_t& lo) {
@@ -61,12 +69,16 @@ __global__ void split_router_weights_kernel(const float* __restrict__ wr, const 
   out[2 * plane + idx] = lo;
 }
 
+template <int CHUNK>
 __global__ void __launch_bounds__(kRtThreads, 1)
 router_tc_kernel(const __grid_constant__ CUtensorMap tmW, const void* __restrict__ r_in, int r_is_bf16,
                  const float* __restrict__ inv_rms, float* __restrict__ part, int n_tokens, int d, int E, int E_pad,
                  int* __restrict__ status) {
   pdl_wait();
   pdl_launch_dependents();
+  using Cfg = RtCfg<CHUNK>;
+  constexpr int kRtChunk = CHUNK, kRtBTile = Cfg::kBTile, kRtStageBytes = Cfg::kStageBytes, kRtStages = Cfg::kStages,
+                kRtAccs = Cfg::kAccs;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kRtStages * kRtStageBytes);
@@ -99,7 +111,11 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmW, const void* __restrict
         if (!mbar_wait(&empty_bar[s], ((kb / kRtStages) & 1) ^ 1)) { ok = false; break; }
         uint8_t* sb = smem + s * kRtStageBytes + 3 * kRtATile;
         mbar_expect_tx(&full_bar[s], 3 * kRtBTile);
-        for (int p = 0; p < 3; ++p) tma_load_2d(sb + p * kRtBTile, &tmW, &full_bar[s], kb * kRtBK, p * E_pad + chunk * kRtChunk);
+        for (int p = 0; p < 3; ++p)
+#pragma unroll
+          for (int hb = 0; hb < kRtChunk / kRouterChunk; ++hb)          // the tensor map's box is 64 rows
+            tma_load_2d(sb + p * kRtBTile + hb * (kRouterChunk * kRtBK * 2), &tmW, &full_bar[s], kb * kRtBK,
+                        p * E_pad + chunk * kRtChunk + hb * kRouterChunk);
       }
       if (!ok) atomicExch(status, kStatusTimeout);
     }
@@ -197,7 +213,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmW, const void* __restrict
       const int n_acc = kblocks < kRtAccs ? kblocks : kRtAccs;
       const float inv = row < n_tokens ? inv_rms[row] : 0.f;
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
+      for (int hf = 0; hf < kRtChunk / 32; ++hf) {
         float sum[32];
 #pragma unroll
         for (int c = 0; c < 32; ++c) sum[c] = 0.f;
@@ -242,14 +258,22 @@ void launch_split_router_weights(const float* wr, const bf16* gain, bf16* planes
 }
 
 cudaError_t router_tc_configure() {
-  return cudaFuncSetAttribute(router_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kRtSmemBytes));
+  cudaError_t e = cudaFuncSetAttribute(router_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(RtCfg<64>::kSmemBytes));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(router_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(RtCfg<128>::kSmemBytes));
 }
 
 void launch_router_tc(const CUtensorMap& tmW, const void* r, int r_is_bf16, const float* inv_rms, float* part,
                       int n_tokens, int d, int E, int* status, cudaStream_t st) {
   const int E_pad = router_padded_experts(E);
-  dim3 grid((n_tokens + kRtRows - 1) / kRtRows, E_pad / kRtChunk);
-  launch_pdl(router_tc_kernel, grid, dim3(kRtThreads), kRtSmemBytes, st, tmW, r, r_is_bf16, inv_rms, part, n_tokens, d, E, E_pad, status);
+  const int tiles = (n_tokens + kRtRows - 1) / kRtRows;
+  if (E_pad % 128 == 0) {
+    launch_pdl(router_tc_kernel<128>, dim3(tiles, E_pad / 128), dim3(kRtThreads), RtCfg<128>::kSmemBytes, st, tmW, r, r_is_bf16, inv_rms,
+               part, n_tokens, d, E, E_pad, status);
+  } else {
+    launch_pdl(router_tc_kernel<64>, dim3(tiles, E_pad / 64), dim3(kRtThreads), RtCfg<64>::kSmemBytes, st, tmW, r, r_is_bf16, inv_rms,
+               part, n_tokens, d, E, E_pad, status);
+  }
 }
 
 }  // namespace foe
