@@ -104,13 +104,46 @@ __global__ void cu_q_kernel(const int* __restrict__ q_lens, int n_seqs, int* __r
   }
 }
 
-__global__ void token_map_kernel(const int* __restrict__ cu_q, int* __restrict__ cu_q_out, int has_q_lens, const int* __restrict__ context_lens,
+// With `q_lens` given (at most kMapScanSeqs sequences) every block first builds the prefix sums of the sequences'
+// new-token counts in shared memory -- one warp, 32 consecutive sequences per lane -- and block 0 also writes them to
+// cu_q_out for the attention kernel: no separate one-thread prefix kernel in front of this one.
+constexpr int kMapScanSeqs = 1024;
+
+__global__ void token_map_kernel(const int* cu_q_in, int* cu_q_out, int has_q_lens,
+                                 const int* __restrict__ q_lens, const int* __restrict__ context_lens,
                                  const int* __restrict__ block_table, int n_seqs, int max_pages_per_seq,
                                  int num_pages, int page_size, int n_tokens, int max_context, int max_q_len,
                                  int* __restrict__ tok_seq, int* __restrict__ tok_pos, int* __restrict__ tok_slot,
                                  int* __restrict__ status) {
+  __shared__ int s_cu[kMapScanSeqs + 1];
   pdl_wait();
   pdl_launch_dependents();
+  const int* cu_q = cu_q_in;
+  if (q_lens) {                               // (n_seqs <= kMapScanSeqs: the launcher's choice)
+    for (int b = threadIdx.x; b < n_seqs; b += blockDim.x) s_cu[b + 1] = q_lens[b];
+    if (threadIdx.x == 0) s_cu[0] = 0;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      const int lane = threadIdx.x;
+      const int b0 = lane * 32;               // this lane's sequences: b0 .. b0 + 31
+      int sum = 0;
+      for (int k = 0; k < 32; ++k)
+        if (b0 + k < n_seqs) sum += s_cu[b0 + k + 1];
+      int incl = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      int run = incl - sum;                   // tokens of the sequences before b0
+      for (int k = 0; k < 32; ++k)
+        if (b0 + k < n_seqs) { run += s_cu[b0 + k + 1]; s_cu[b0 + k + 1] = run; }
+    }
+    __syncthreads();
+    if (blockIdx.x == 0)
+      for (int b = threadIdx.x; b <= n_seqs; b += blockDim.x) cu_q_out[b] = s_cu[b];
+    cu_q = s_cu;
+  }
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_tokens) return;
   int b;
@@ -149,11 +182,12 @@ int launch_token_map(const int* q_lens, const int* context_lens, const int* bloc
                       int max_pages_per_seq, int num_pages, int page_size, int n_tokens, int max_context, int max_q_len,
                       int* cu_q, int* tok_seq, int* tok_pos, int* tok_slot, int* status, cudaStream_t st) {
   int launches = 0;
-  if (q_lens) { launch_pdl(cu_q_kernel, dim3(1), dim3(32), 0, st, q_lens, n_seqs, cu_q); ++launches; }
+  const bool scan_in_block = q_lens && n_seqs <= kMapScanSeqs && n_tokens > 0;
+  if (q_lens && !scan_in_block) { launch_pdl(cu_q_kernel, dim3(1), dim3(32), 0, st, q_lens, n_seqs, cu_q); ++launches; }
   if (n_tokens <= 0) return launches;
-  launch_pdl(token_map_kernel, dim3((n_tokens + 255) / 256), dim3(256), 0, st, cu_q, cu_q, q_lens != nullptr, context_lens, block_table, n_seqs,
-                                                         max_pages_per_seq, num_pages, page_size, n_tokens,
-                                                         max_context, max_q_len, tok_seq, tok_pos, tok_slot, status);
+  launch_pdl(token_map_kernel, dim3((n_tokens + 255) / 256), dim3(256), 0, st, cu_q, cu_q, q_lens != nullptr,
+             scan_in_block ? q_lens : static_cast<const int*>(nullptr), context_lens, block_table, n_seqs,
+             max_pages_per_seq, num_pages, page_size, n_tokens, max_context, max_q_len, tok_seq, tok_pos, tok_slot, status);
   return launches + 1;
 }
 

@@ -227,6 +227,16 @@ def test_chunked_prefill_over_cached_context():
     run_block_parity(shape, 15, [40, 17, 130], [100, 64, 1], wscale=4.0)
 
 
+def test_prefill_call_with_more_sequences_than_the_token_map_scans_in_one_block():
+    """Up to 1024 sequences the token-map kernel builds the prefix sums of q_lens itself, beyond that a separate kernel
+    does; 1030 sequences of one or two tokens (and, in the same test, 1024 exactly) over short cached contexts."""
+    shape = shape_small()
+    for n in (1030, 1024):
+        q = [1 + (i % 3 == 0) for i in range(n)]
+        ctx = [(7 * i) % 40 for i in range(n)]
+        run_block_parity(shape, 33, q, ctx, decode=False, wscale=4.0)
+
+
 def test_mixed_batch_of_prefill_chunks_and_decode_tokens():
     """One prefill call carrying fresh prompts, a chunk of a longer prompt and single decode tokens of running
     sequences (q_len 1 over a long cached context): the serving batch shape of Section 4's engine."""
