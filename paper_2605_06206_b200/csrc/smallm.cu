@@ -298,6 +298,15 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
     // epilogue: c[nt][0..1] = (weight row A, tokens 2*t4, 2*t4+1), c[nt][2..3] = (weight row B, same tokens)
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
+      // QKV: 1/rms of token row nt*8 + 2*t4 + e sits in the quad whose g equals that row index.  Fetched here by ALL
+      // lanes: below, lanes whose row lies past the end of a ragged chunk skip the row, and a full-mask shuffle that
+      // some lanes never reach leaves the others waiting for them -- forever once the skipping lanes have run on into
+      // the next task's __syncwarp (a CTA with a second task and a last chunk of fewer than 16 tokens hung).
+      float sc_e[2] = {1.f, 1.f};
+      if (EPI == kEpiQKV) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) sc_e[e] = __shfl_sync(0xffffffffu, ssq[nt], (t4 * 2 + e) * 4);
+      }
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
         const int r = m0 + nt * 8 + t4 * 2 + e;              // logical row inside the group
@@ -312,8 +321,7 @@ smallm_kernel(const __grid_constant__ CUtensorMap tmW, const SmallMArgs a) {
           o[n_a] = __float2bfloat16_rn(va);
           o[n_b] = __float2bfloat16_rn(vb);
         } else if (EPI == kEpiQKV) {
-          // 1/rms of token row nt*8 + 2*t4 + e sits in the quad whose g equals that row index
-          const float sc = __shfl_sync(0xffffffffu, ssq[nt], (t4 * 2 + e) * 4);
+          const float sc = sc_e[e];
           const int tok = out_row0 + r;
           // packed columns n_a = 2i and n_a + 1 of a head are its natural columns i and i + dh/2: one rotary pair
           const int i = (n_a % a.dh) >> 1, half = a.dh >> 1;

@@ -50,6 +50,19 @@ def test_random_shape_and_batch(case):
     run_block_parity(shape, 7000 + case, q_lens, ctx_lens, decode=decode)
 
 
+@pytest.mark.timeout(300)
+@pytest.mark.parametrize("case", range(20100, 20148))
+def test_random_shape_and_batch_second_series(case):
+    """A second series of draws with decode steps as likely as prefill calls.  Draw 20122 (head width 96, five
+    clusters, 150 sequences) is the one that found the weight-streaming QKV kernel waiting forever in a CTA's second
+    task: a full-mask shuffle sat behind a row test that the lanes of a ragged last chunk fail."""
+    rng = random.Random(case)
+    shape = draw_shape(rng)
+    decode = rng.random() < 0.5
+    q_lens, ctx_lens = draw_batch(rng, decode)
+    run_block_parity(shape, case, q_lens, ctx_lens, decode=decode)
+
+
 @pytest.mark.parametrize("case", range(16))
 def test_random_shape_and_batch_one_cluster_per_rank(case):
     rng = random.Random(9000 + case)

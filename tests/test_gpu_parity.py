@@ -325,6 +325,17 @@ def test_decode_more_sequences_than_one_token_tile(dh, position, n_seqs):
     run_block_parity(shape, 29, [1] * n_seqs, ctx, decode=True, wscale=4.0)
 
 
+@pytest.mark.timeout(300)
+@pytest.mark.parametrize("H,n_seqs", [(5, 150), (4, 150), (8, 250)])
+def test_decode_head_dim_96_with_more_projection_tasks_than_resident_ctas(H, n_seqs):
+    """Heads of width 96 take the weight-streaming QKV projection; with 150 and more sequences it has more
+    (cluster, slab, 16-token chunk) tasks than the 2 x 148 CTAs of its grid, so CTAs run a second task, and the last
+    chunk of every cluster is ragged (150 = 9 x 16 + 6)."""
+    shape = synth.LayerShape(1024, 4 * H, H, H, 96, 2, 1, 256, position="single")
+    ctx = [(37 * i) % 300 for i in range(n_seqs)]
+    run_block_parity(shape, 34, [1] * n_seqs, ctx, decode=True)
+
+
 @pytest.mark.parametrize("position", ["first", "last"])
 def test_decode_boundary_layers(position):
     shape = shape_small(position=position)
