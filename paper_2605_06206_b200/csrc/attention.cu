@@ -44,7 +44,9 @@ __device__ __forceinline__ void tma_load_page(uint8_t* k_dst, uint8_t* v_dst, co
 // consecutive CTAs, numbered in CTA order.  Every segment leaves a partial (m, l, o) in global memory and takes a ticket
 // on its pair; whichever CTA takes the last ticket merges the pair's segments in segment order (so the result does not
 // depend on which one that is).  A pair that lies inside one segment is finished without either.  The partition is a
-// function of the call's context lengths and the grid only: the same call gives the same bits.
+// function of the call's context lengths and the grid only: the same call gives the same bits.  Where a sequence's pages
+// are cut depends on the other sequences of the call, so its output can differ in the last bits (the rounding of the
+// merge) between two batches it is part of.
 constexpr int kDcConsumers = 4;
 constexpr int kDcThreads = (kDcConsumers + 1) * 32;
 constexpr int kDcStages = 3;
@@ -63,8 +65,8 @@ struct DcSmem {
   static constexpr int kMoOff = kQOff + kQBytes;
   static constexpr int kMmOff = kMoOff + kMoBytes;               // [4][16] running maxima, then [4][16] running sums
   static constexpr int kBarOff = kMmOff + 2 * 4 * 16 * 4;        // full[stages], empty[stages]
-  static constexpr int kMiscOff = kBarOff + 2 * kDcStages * 8;   // tickets
-  static constexpr size_t kBytes = size_t(kMiscOff) + 16 + 1024; // (two tickets) + alignment slack
+  static constexpr int kMiscOff = kBarOff + 2 * kDcStages * 8;   // ticket
+  static constexpr size_t kBytes = size_t(kMiscOff) + 16 + 1024; // + alignment slack
 };
 
 // position inside the list of pages
