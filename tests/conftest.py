@@ -10,6 +10,8 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
+    # (registered by pytest-timeout where it is installed; named here so that the tests also collect without it)
+    config.addinivalue_line("markers", "timeout(seconds): limit for one test, enforced by pytest-timeout")
 
 
 def pytest_collection_modifyitems(config, items):
