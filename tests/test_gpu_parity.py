@@ -74,6 +74,32 @@ def test_route_bit_exact_tensor_core_scores_odd_k_blocks():
     check_maps(shape, aux, idx.cpu().numpy())
 
 
+@pytest.mark.parametrize("H,Ec,kc", [(1, 100, 8), (2, 96, 4), (5, 64, 2), (2, 128, 16), (4, 24, 3)])
+def test_route_tensor_core_scores_with_padded_expert_counts(H, Ec, kc):
+    """The tensor-core score kernel pads the expert count to a multiple of 64 and gives a CTA 128 experts when the
+    padded count is a multiple of 128, 64 otherwise: 100 -> 128 (one CTA column of 128, 28 of them padding),
+    192 and 320 (columns of 64), 256 (two columns of 128), 96 -> 128."""
+    shape = synth.LayerShape(512, 2 * H, H, H, 64, Ec, kc, 128)
+    seed = 1500 + H * Ec
+    W = dict(ffn_norm_g=synth.normal_bf16(seed, synth.TID["ffn_norm_g"], (shape.hidden,), 0.02, 1.0, "cuda"),
+             router_w=synth.normal_bf16(seed, synth.TID["router_w"], (shape.n_experts, shape.hidden), 0.02, 0.0, "cuda").float())
+    n_tok = 2100
+    h = synth.normal_bf16(seed, 77, (n_tok, shape.hidden), 1.5, 0.0, "cuda")
+    layer = binding.FoeLayer(shape, _route_only_weights(shape, W), max_tokens=n_tok, max_seqs=1, max_context=64)
+    idx, w = layer.route(h)
+    assert layer.poll_status() == 0
+    aux = layer.aux()
+    layer.close()
+    cfg = adapter.cfg_from_shape(shape)
+    Wn = {k: adapter.to_np(W[k]) for k in ("ffn_norm_g", "router_w")}
+    Wn["router_b"] = None
+    rt = orc.route(cfg, Wn, adapter.to_np(h))
+    exempt = check_routing(shape, idx.cpu().numpy(), w.cpu().numpy().astype(np.float64), rt["logits"], rt["idx"], rt["w"])
+    assert exempt <= max(2, n_tok // 200)
+    assert np.abs(adapter.to_np(aux["logits"]) - rt["logits"]).max() <= 2e-5 * max(1.0, np.abs(rt["logits"]).max())
+    check_maps(shape, aux, idx.cpu().numpy())
+
+
 @pytest.mark.parametrize("wl,n_tok,max_tokens", [(5, 1088, 1088), (5, 1100, 16384), (4, 560, 8192), (4, 1152, 4096)])
 def test_route_bit_exact_where_split_k_partials_would_outgrow_their_buffer(wl, n_tok, max_tokens):
     """Call sizes at which the fp32 score kernel would like 16 slices of the hidden dimension while the partial-score
