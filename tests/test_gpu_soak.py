@@ -1,5 +1,5 @@
 """Opt-in soak: the seeded generators of the fuzz tests (and three wider ones) with OTHER seeds than the committed
-cases.  Skipped unless FOE_SOAK=<draws per generator> is set; FOE_SOAK_BASE moves the seed range.
+cases, on one device (the one-cluster-per-rank generator runs its ranks one after the other there).  Skipped unless FOE_SOAK=<draws per generator> is set; FOE_SOAK_BASE moves the seed range.
 
     FOE_SOAK=300 FOE_SOAK_BASE=70000 python -m pytest tests/test_gpu_soak.py -m gpu -q
 
@@ -13,6 +13,7 @@ import pytest
 from paper_2605_06206_b200 import synth
 
 from parity import run_block_parity
+from test_gpu_shard import run_group
 import test_gpu_fuzz as fuzz
 
 pytestmark = [pytest.mark.gpu, pytest.mark.timeout(3600)]
@@ -84,3 +85,45 @@ def test_soak_wide_groups_and_odd_cluster_counts():
         q = [rng.choice([1, 65, 257, 600]) for _ in range(rng.randint(1, 3))]
         return shape, q, [rng.choice([0, 64, 191]) for _ in q], False
     _run("wide-groups", make)
+
+
+@needs_soak
+def test_soak_wide_expert_sets_with_skewed_routing():
+    for seed in range(BASE, BASE + DRAWS):
+        rng = random.Random(seed)
+        H = rng.choice([1, 2, 4, 8])
+        Ec = rng.choice([32, 64, 128, 24, 100])
+        k = min(rng.choice([1, 2, 4, 8, 16]), Ec)
+        hidden = 128 * rng.choice([2, 4, 8])
+        shape = synth.LayerShape(hidden, 2 * H, H, H, rng.choice([64, 128]), Ec, k, 128 * rng.choice([1, 2]),
+                                 position=rng.choice(["middle", "first", "last"]) if H > 1 else "single")
+        bias = synth.zipf_router_bias(shape, seed, 1.0, 1.2, dead_per_cluster=rng.choice([0, 5])) if seed % 2 else None
+        decode = rng.random() < 0.5
+        if decode:
+            n = rng.choice([3, 64, 200, 256, 257])
+            q_lens, ctx_lens = [1] * n, [rng.choice([0, 63, 64, 300]) for _ in range(n)]
+        else:
+            q_lens = [rng.choice([20, 257, 700, 1500]) for _ in range(rng.randint(1, 2))]
+            ctx_lens = [rng.choice([0, 64, 100]) for _ in q_lens]
+        try:
+            run_block_parity(shape, seed, q_lens, ctx_lens, decode=decode, wscale=4.0 if hidden <= 512 else 2.0,
+                             router_bias=bias)
+        except Exception as e:
+            raise AssertionError(f"wide-experts draw {seed}: {shape} decode={decode} q_lens={q_lens}") from e
+
+
+@needs_soak
+def test_soak_one_cluster_per_rank():
+    for seed in range(BASE, BASE + DRAWS):
+        rng = random.Random(seed)
+        while True:
+            shape = fuzz.draw_shape(rng)
+            if (shape.n_clusters > 1 and shape.hidden % (32 * shape.n_clusters) == 0
+                    and (shape.q_per_cluster * shape.head_dim) % 128 == 0):
+                break
+        decode = rng.random() < 0.5
+        q_lens, ctx_lens = fuzz.draw_batch(rng, decode)
+        try:
+            run_group(shape, seed, q_lens, ctx_lens, decode=decode)
+        except Exception as e:
+            raise AssertionError(f"group draw {seed}: {shape} decode={decode} q_lens={q_lens} ctx={ctx_lens}") from e
